@@ -1,0 +1,180 @@
+/*
+ * csd.h - C ABI of the continuous speculative decoding (CSD) hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, for a batch of independent token rows, what one round of Algorithm 1
+ * ("ContinuousSpeculativeDecodingStep") of "Continuous Speculative Decoding for Autoregressive
+ * Image Generation" needs from the per-token diffusion heads, with the AR transformer backbones
+ * left to the caller: their output vectors z, the Gaussian noise, the uniforms, the noise schedule
+ * and the head weights are all inputs.
+ *
+ * Conventions
+ *   B sequences, gamma draft tokens per sequence, R = B*gamma token rows, row r = b*gamma + i.
+ *   cfg = 1 doubles the head rows for classifier-free guidance (Appendix "Classifier-Free
+ *   Guidance"): z has 2R rows, [conditional rows | unconditional rows]; both halves see the
+ *   same x_t and eps_hat = eps_u + cfg_scale * (eps_c - eps_u).
+ *   C token dim, W head width, L residual blocks, Dz condition dim, F timestep-feature dim, T steps.
+ *   Every array is dense row-major.  "device" = pointer to GPU global memory of the context's
+ *   device, "host" = ordinary host memory.  The library never frees or keeps caller memory
+ *   beyond the call (host arrays are copied before the call returns; device arrays are read by
+ *   the kernels the call enqueues and must stay valid until those have run).
+ *   All work is enqueued on the stream given to csd_create(); calls return without
+ *   synchronising unless stated.  Device-side error flags (for instance a bounded wait that ran
+ *   out) are reported by csd_sync().
+ *
+ * Head evaluated per head row and step t (eps-prediction network of Eq. 3; the layout below is
+ * this library's specification, the paper does not describe the head's inside):
+ *   cz = Wz z + bz ;  te_t = Wt2 SiLU(Wt1 tfeat_t + bt1) + bt2 ;  s = SiLU(cz + te_t)
+ *   h = Win x_t + bin
+ *   for k < L: (shift|scale|gate) = Wada_k s + bada_k ; u = LN(h)(1+scale)+shift ;
+ *              h = h + gate * (W2_k SiLU(W1_k u + b1_k) + b2_k)
+ *   (shift|scale) = Wfada s + bfada ;  eps_hat = Wout (LN(h)(1+scale)+shift) + bout
+ *   LN: no affine, eps 1e-6, biased variance over W.
+ *
+ * Errors: every function returns CSD_OK (0) or a negative code; nothing aborts, throws or traps.
+ * csd_last_error() returns a description of the most recent failure on that context.
+ */
+#ifndef CSD_H_
+#define CSD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct csd_ctx csd_ctx;
+typedef struct csd_head csd_head;
+
+enum {
+  CSD_OK = 0,
+  CSD_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, bad enum                         */
+  CSD_ERR_SHAPE = -2,       /* dims of heads / schedules / calls do not agree                    */
+  CSD_ERR_UNSUPPORTED = -3, /* e.g. W not a multiple of 128 on the bf16 path, gamma > 32, C > 32 */
+  CSD_ERR_WORKSPACE = -4,   /* device memory for the workspace or weights could not be had      */
+  CSD_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                                 */
+  CSD_ERR_TIMEOUT = -6      /* a bounded device-side wait gave up (reported by csd_sync)         */
+};
+
+enum { CSD_F32 = 0, CSD_BF16 = 1 };
+
+/* Shape and arithmetic of one head.  CSD_F32: fp32 weights and activations on plain FMA units.
+ * CSD_BF16: bf16 weights and bf16 GEMM inputs on tcgen05 tensor cores with fp32 accumulation;
+ * residual stream, LayerNorm statistics, x_t and mu stay fp32. */
+typedef struct {
+  int C, W, L, Dz, F;
+  int dtype; /* CSD_F32 | CSD_BF16 */
+} csd_head_desc;
+
+/* HOST pointers to fp32 parameters, each matrix row-major [out, in]:
+ * Wz[W,Dz] bz[W] Wt1[W,F] bt1[W] Wt2[W,W] bt2[W] Win[W,C] bin[W] Wada[L,3W,W] bada[L,3W]
+ * W1[L,W,W] b1[L,W] W2[L,W,W] b2[L,W] Wfada[2W,W] bfada[2W] Wout[C,W] bout[C].
+ * For CSD_BF16 heads the matrices are converted to bf16 (round to nearest even); callers that
+ * want bit-defined results pass values that are already bf16-representable. */
+typedef struct {
+  const float *Wz, *bz, *Wt1, *bt1, *Wt2, *bt2, *Win, *bin;
+  const float *Wada, *bada, *W1, *b1, *W2, *b2, *Wfada, *bfada, *Wout, *bout;
+} csd_head_weights;
+
+/* Reverse-process coefficients of a T-step sampler whose transition is the Gaussian of Eq. 3
+ * with isotropic variance: mu_t = a[t-1] x_t - b[t-1] eps_hat, x_{t-1} = mu_t + sigma[t-1] eps_t.
+ * sigma already includes the sampling temperature (Appendix "Temperature").
+ * a, b, sigma: HOST arrays [T].  tfeat: DEVICE array [T, F], row t-1 = features of timestep t. */
+typedef struct {
+  int T;
+  const float *a, *b, *sigma;
+  const float *tfeat;
+} csd_schedule;
+
+/* Context: owns a growable device workspace and the stream association.  `cuda_stream` is a
+ * cudaStream_t (NULL = legacy default stream).  csd_destroy synchronises the stream and frees. */
+int csd_create(csd_ctx **out, int device, void *cuda_stream);
+int csd_destroy(csd_ctx *ctx);
+const char *csd_last_error(const csd_ctx *ctx);
+/* Waits for the context's stream and returns CSD_ERR_TIMEOUT / CSD_ERR_CUDA if any kernel of an
+ * earlier call raised its error flag, else CSD_OK.  Clears the flag. */
+int csd_sync(csd_ctx *ctx);
+/* Number of kernels this context has launched so far (bookkeeping for benchmarks). */
+int64_t csd_launch_count(const csd_ctx *ctx);
+
+/* Copies and repacks the weights into device memory owned by the head (synchronous; the caller
+ * may free `w` afterwards).  A head belongs to the context it was created with. */
+int csd_head_create(csd_ctx *ctx, const csd_head_desc *desc, const csd_head_weights *w, csd_head **out);
+int csd_head_destroy(csd_head *head);
+
+/* Draft trajectories (Alg. 1 "x_i ~ q_i"; Eq. 1, Eq. 3; reparameterised sampling of Sec. 3.2):
+ * for each of R token rows run t = T..1 of the head given, adding sigma_t eps_t at EVERY step
+ * including t = 1, so that x0 = mu1 + sigma_1 eps_1 is a draw from the final-step Gaussian
+ * q(x_0 | x_1).  Given the target head this call is also the target-only pre-fill of
+ * Sec. 3.2 ("Inconsistency in Autoregressive Process").
+ *   z    device [R*(1+cfg), Dz] fp32        x_T  device [R, C]      eps  device [T, R, C]
+ *   x0   device [R, C] out                  mu1  device [R, C] out  (mean of the last step)
+ *   x1   device [R, C] out or NULL          (state before the last step) */
+int csd_draft_denoise(csd_ctx *ctx, const csd_head *head, const csd_schedule *sched, int R, int cfg,
+                      float cfg_scale, const float *z, const float *x_T, const float *eps,
+                      float *x0, float *mu1, float *x1);
+
+/* Verification (Alg. 1: target run with the draft's noise, Sigma, ratios, accepted count).
+ * Runs the target head on the SAME x_T and eps as the draft call (denoising trajectory
+ * alignment, Theorem 1) for t = T..1 without sampling x_0, then per row
+ *   logratio = log Sigma + log N(x0; mu1_p, sigma_p,1^2 I) - log N(x0; mu1_q, sigma_q,1^2 I)
+ * (Eq. 8) with log Sigma = C * sum_{t=2..T} (log sigma_q,t - log sigma_p,t) (Eq. 7), accepts
+ * position i iff log u[b,i] <= logratio[b,i] and returns n_accept[b] = number of leading accepts.
+ *   sched_p: full schedule of the target; sched_q: only T and sigma are read.
+ *   z_p device [B*gamma*(1+cfg), Dz_p]; x_T, eps, x0_q, mu1_q device as in the draft call;
+ *   u device [B, gamma] in (0,1];  logratio device [B, gamma] out;  n_accept device int32 [B] out;
+ *   accept_mask device uint32 [B] out or NULL (bit i = position i accepted);
+ *   mu1_p device [B*gamma, C] out. */
+int csd_verify(csd_ctx *ctx, const csd_head *head_p, const csd_schedule *sched_p,
+               const csd_schedule *sched_q, int B, int gamma, int cfg, float cfg_scale,
+               const float *z_p, const float *x_T, const float *eps, const float *x0_q,
+               const float *mu1_q, const float *u, float *logratio, int32_t *n_accept,
+               uint32_t *accept_mask, float *mu1_p);
+
+/* Only the ratio / accept / prefix part of csd_verify, for callers that already hold mu1_p
+ * (no head is evaluated).  log_sigma_term = log Sigma of Eq. 7 (host double). */
+int csd_accept_scan(csd_ctx *ctx, int B, int gamma, int C, double log_sigma_term, float sigma1_p,
+                    float sigma1_q, const float *x0_q, const float *mu1_q, const float *mu1_p,
+                    const float *u, float *logratio, int32_t *n_accept, uint32_t *accept_mask);
+
+/* Resampling from the modified distribution max(0, p - q)/Z (Eq. 5) by acceptance-rejection with
+ * the bound M = 1/Z (Eq. 9-11) in the inference-free form of Corollary 1.  For each sequence with
+ * n_accept[b] < gamma, row j = b*gamma + n_accept[b]: for k = 0..cap-1
+ *   x' = mu1_p[j] + sigma1_p * xi[b,k];
+ *   alpha_s = max(0, 1 - q(x'|x_1^q) / (Sigma p(x'|x_1^p)));   accept iff v[b,k] <= alpha_s.
+ * The loop of Alg. 1 is unbounded; here it stops after `cap` proposals, returns the last one and
+ * sets bit 1 of flags[b].
+ *   n_accept device int32 [B]; mu1_p, mu1_q device [B*gamma, C]; xi device [B, cap, C] ~ N(0,1);
+ *   v device [B, cap] in (0,1);  x_new device [B, C] out (untouched where n_accept == gamma);
+ *   n_prop device int32 [B] out (0 where nothing was resampled);
+ *   flags device uint32 [B] out: bit0 resampled, bit1 cap hit;  cap_hits device int32 [1] out. */
+int csd_resample(csd_ctx *ctx, int B, int gamma, int C, int cap, double log_sigma_term,
+                 float sigma1_p, float sigma1_q, const int32_t *n_accept, const float *mu1_p,
+                 const float *mu1_q, const float *xi, const float *v, float *x_new,
+                 int32_t *n_prop, uint32_t *flags, int32_t *cap_hits);
+
+/* One whole round of Alg. 1 = csd_draft_denoise + csd_verify + csd_resample with bit-identical
+ * results; the two heads' chains run concurrently on internal streams (they are independent
+ * until the final-step densities, Eq. 4) and are joined on the context's stream before return
+ * of control to that stream.  Argument meaning as in the three calls. */
+int csd_round(csd_ctx *ctx, const csd_head *head_q, const csd_head *head_p,
+              const csd_schedule *sched_q, const csd_schedule *sched_p, int B, int gamma, int cfg,
+              float cfg_scale, int cap, const float *z_q, const float *z_p, const float *x_T,
+              const float *eps, const float *u, const float *xi, const float *v, float *x0,
+              float *mu1_q, float *mu1_p, float *logratio, int32_t *n_accept,
+              uint32_t *accept_mask, float *x_new, int32_t *n_prop, uint32_t *flags,
+              int32_t *cap_hits);
+
+/* Same computation as csd_round, but every array is a HOST pointer: the call copies the inputs
+ * to the device, runs the round, copies the outputs back and synchronises before returning. */
+int csd_round_host(csd_ctx *ctx, const csd_head *head_q, const csd_head *head_p,
+                   const csd_schedule *sched_q, const csd_schedule *sched_p, int B, int gamma,
+                   int cfg, float cfg_scale, int cap, const float *z_q, const float *z_p,
+                   const float *x_T, const float *eps, const float *u, const float *xi,
+                   const float *v, float *x0, float *mu1_q, float *mu1_p, float *logratio,
+                   int32_t *n_accept, uint32_t *accept_mask, float *x_new, int32_t *n_prop,
+                   uint32_t *flags, int32_t *cap_hits);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSD_H_ */

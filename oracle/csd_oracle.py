@@ -1,0 +1,296 @@
+"""Float64 CPU checker for continuous speculative decoding (CSD).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of what the
+method computes, written from the paper; the CUDA library never imports it and
+shares no code with it.  Only the test-suite, the smoke check and the
+benchmark's CPU-baseline leg may call it.
+
+Everything is numpy float64, vectorised over independent token rows and
+otherwise in the paper's order: no blocking, fusion or reordering.
+
+What pins each function (see tests/test_oracle_pins.py):
+
+  ddpm_schedule            textbook special case (N(0,1) data: mu_t = sqrt(alpha_t) x_t)
+  denoise / run_pair       Theorem 1 pathwise identity and its Monte-Carlo form
+  log_sigma_term, log_ratio_*   long form (Eq. 4) == closed form (Eq. 7, 8);
+                           identical heads give exactly 0; 1-D Gaussian toy
+                           head matches an independently composed affine map
+  accept_prefix            brute force over all accept masks (Alg. 1)
+  resample                 KS test against the numerically integrated
+                           max(0, Sigma*p - q) (Eq. 5, Eq. 11, Cor. 1); textbook
+                           total-variation acceptance rate
+  silu, layer_norm, timestep MLP   library routines (torch float64)
+  head_eps (architecture)  PARITY UNPINNED by the paper: the paper does not
+                           describe the diffusion head; its layout is this
+                           project's own specification.  Only structural
+                           special cases are pinned.
+"""
+from __future__ import annotations
+
+from typing import Callable, Dict, Optional, Tuple
+
+import numpy as np
+
+f64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# Noise schedule: the Gaussian transition of Eq. 3, N(x_{t-1}; mu, Sigma), with
+# the epsilon-prediction mean of the DDPM work the paper cites for Eq. 3 and a
+# fixed isotropic variance sigma_t^2 = tau^2 * beta_t (temperature, Appendix
+# "Temperature").
+# --------------------------------------------------------------------------
+def ddpm_schedule(beta: np.ndarray, tau: float = 1.0) -> Dict[str, np.ndarray]:
+    beta = np.asarray(beta, dtype=f64)
+    alpha = 1.0 - beta
+    alphabar = np.cumprod(alpha)
+    a = 1.0 / np.sqrt(alpha)                              # mu_t = a_t x_t - b_t eps_hat
+    b = beta / (np.sqrt(alpha) * np.sqrt(1.0 - alphabar))
+    sigma = tau * np.sqrt(beta)
+    return {"a": a, "b": b, "sigma": sigma, "alphabar": alphabar, "beta": beta}
+
+
+# --------------------------------------------------------------------------
+# The per-token diffusion head eps_hat = head(x_t, t, z) (the "diffusion loss"
+# module of Sec. "Implementation Details"; architecture = project spec).
+# --------------------------------------------------------------------------
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def layer_norm(h: np.ndarray, eps: float = 1e-6) -> np.ndarray:
+    """No affine parameters, biased variance over the last axis."""
+    m = h.mean(axis=-1, keepdims=True)
+    v = ((h - m) ** 2).mean(axis=-1, keepdims=True)
+    return (h - m) / np.sqrt(v + eps)
+
+
+def timestep_embedding(w: Dict[str, np.ndarray], tfeat_t: np.ndarray) -> np.ndarray:
+    """te_t = Wt2 SiLU(Wt1 tfeat_t + bt1) + bt2, one vector of width W."""
+    hid = silu(w["Wt1"].astype(f64) @ tfeat_t.astype(f64) + w["bt1"].astype(f64))
+    return w["Wt2"].astype(f64) @ hid + w["bt2"].astype(f64)
+
+
+def head_eps(w: Dict[str, np.ndarray], x_t: np.ndarray, tfeat_t: np.ndarray, z: np.ndarray,
+             trace: Optional[dict] = None) -> np.ndarray:
+    """eps_hat for a batch of head rows.  x_t [N,C], z [N,Dz], tfeat_t [F]."""
+    W64 = {k: v.astype(f64) for k, v in w.items()}
+    x_t = x_t.astype(f64)
+    cz = z.astype(f64) @ W64["Wz"].T + W64["bz"]
+    te = timestep_embedding(w, tfeat_t)
+    s = silu(cz + te[None, :])
+    h = x_t @ W64["Win"].T + W64["bin"]
+    L = W64["W1"].shape[0]
+    Wd = W64["W1"].shape[1]
+    if trace is not None:
+        trace["s"] = s.copy(); trace["h_in"] = h.copy(); trace["h"] = []
+    for k in range(L):
+        mod = s @ W64["Wada"][k].T + W64["bada"][k]
+        shift, scale, gate = mod[:, :Wd], mod[:, Wd:2 * Wd], mod[:, 2 * Wd:]
+        u = layer_norm(h) * (1.0 + scale) + shift
+        u = silu(u @ W64["W1"][k].T + W64["b1"][k])
+        u = u @ W64["W2"][k].T + W64["b2"][k]
+        h = h + gate * u
+        if trace is not None:
+            trace["h"].append(h.copy())
+    mod = s @ W64["Wfada"].T + W64["bfada"]
+    shift, scale = mod[:, :Wd], mod[:, Wd:]
+    uf = layer_norm(h) * (1.0 + scale) + shift
+    return uf @ W64["Wout"].T + W64["bout"]
+
+
+def make_mlp_head(w: Dict[str, np.ndarray], z: np.ndarray, tfeat: np.ndarray,
+                  cfg: bool, cfg_scale: float) -> Callable[[np.ndarray, int], np.ndarray]:
+    """Return eps_fn(x_t [R,C], t) with classifier-free guidance folded in:
+    rows [0,R) of z are conditional, rows [R,2R) unconditional, both halves see
+    the same x_t, and eps = eps_u + scale*(eps_c - eps_u) (Appendix
+    "Classifier-Free Guidance")."""
+    def eps_fn(x_t: np.ndarray, t: int) -> np.ndarray:
+        R = x_t.shape[0]
+        if cfg:
+            e = head_eps(w, np.concatenate([x_t, x_t], axis=0), tfeat[t - 1], z)
+            e_c, e_u = e[:R], e[R:]
+            return e_u + cfg_scale * (e_c - e_u)
+        return head_eps(w, x_t, tfeat[t - 1], z)
+    return eps_fn
+
+
+def make_gaussian_toy_head(m: float, s: float, alphabar: np.ndarray
+                           ) -> Callable[[np.ndarray, int], np.ndarray]:
+    """Analytic eps-predictor when the data are N(m, s^2) per coordinate:
+    x_t ~ N(sqrt(ab) m, ab s^2 + 1 - ab) and
+    E[eps | x_t] = sqrt(1-ab) (x_t - sqrt(ab) m) / (ab s^2 + 1 - ab)."""
+    def eps_fn(x_t: np.ndarray, t: int) -> np.ndarray:
+        ab = alphabar[t - 1]
+        return np.sqrt(1.0 - ab) * (x_t - np.sqrt(ab) * m) / (ab * s * s + 1.0 - ab)
+    return eps_fn
+
+
+# --------------------------------------------------------------------------
+# Denoising trajectories (Eq. 1, Eq. 3; reparameterised sampling
+# x_{t-1} = sqrt(Sigma) eps_t + mu, Sec. 3.2 / Appendix A.2)
+# --------------------------------------------------------------------------
+def denoise(eps_fn: Callable[[np.ndarray, int], np.ndarray], sched: Dict[str, np.ndarray],
+            x_T: np.ndarray, noise: np.ndarray, sample_last: bool = True,
+            keep: bool = False) -> Dict[str, np.ndarray]:
+    """Run t = T..1.  noise[t-1] is the N(0,I) draw of step t.  Noise is added at
+    every step including t=1, because p(x_0|x_1) must be a proper Gaussian to take
+    ratios of (Eq. 8) and to propose from (Cor. 1).  With sample_last=False the
+    last step only yields mu_1 (the target never samples x_0: it evaluates the
+    density of the draft's x_0, Appendix A.2 after the ratio derivation)."""
+    T = len(sched["a"])
+    x = x_T.astype(f64)
+    xs = [x.copy()] if keep else None       # xs[j] = x_{T-j}
+    mus = [] if keep else None              # mus[j] = mu_{T-j}
+    x1 = mu1 = x0 = None
+    for t in range(T, 0, -1):
+        e_hat = eps_fn(x, t)
+        mu = sched["a"][t - 1] * x - sched["b"][t - 1] * e_hat
+        if t == 1:
+            x1, mu1 = x, mu
+        if t > 1 or sample_last:
+            x = mu + sched["sigma"][t - 1] * noise[t - 1].astype(f64)
+            if t == 1:
+                x0 = x
+        if keep:
+            mus.append(mu.copy())
+            if t > 1 or sample_last:
+                xs.append(x.copy())
+    out = {"x1": x1, "mu1": mu1, "x0": x0}
+    if keep:
+        out["xs"], out["mus"] = xs, mus
+    return out
+
+
+def run_pair(eps_q, eps_p, sched_q, sched_p, x_T, noise, noise_p=None, keep=False):
+    """Draft and target trajectories from the same x_T (Eq. 8 assumes
+    p(x_T^p) = q(x_T^q)).  Denoising trajectory alignment = both use the same
+    noise; pass noise_p to break the alignment (ablation of Table 6)."""
+    dq = denoise(eps_q, sched_q, x_T, noise, sample_last=True, keep=keep)
+    dp = denoise(eps_p, sched_p, x_T, noise if noise_p is None else noise_p,
+                 sample_last=False, keep=keep)
+    return dq, dp
+
+
+# --------------------------------------------------------------------------
+# Ratio of joint path densities (Eq. 4), its alignment simplification (Eq. 7, 8)
+# --------------------------------------------------------------------------
+def gaussian_logpdf_iso(x: np.ndarray, mu: np.ndarray, sigma: float) -> np.ndarray:
+    """log N(x; mu, sigma^2 I) over the last axis (standard form, with the minus
+    sign the paper's printed density dropped)."""
+    C = x.shape[-1]
+    d = x - mu
+    return (-0.5 * C * np.log(2.0 * np.pi) - C * np.log(sigma)
+            - 0.5 * np.sum(d * d, axis=-1) / (sigma * sigma))
+
+
+def log_sigma_term(sigma_q: np.ndarray, sigma_p: np.ndarray, C: int) -> float:
+    """log of Sigma = prod_{t=2..T} sqrt|Sigma_q,t| / sqrt|Sigma_p,t| (Eq. 7) for
+    isotropic variances: C * sum_{t>=2} (log sigma_q,t - log sigma_p,t)."""
+    return float(C * np.sum(np.log(sigma_q[1:]) - np.log(sigma_p[1:])))
+
+
+def log_ratio_closed(x0, mu1_q, mu1_p, sigma1_q, sigma1_p, log_sigma) -> np.ndarray:
+    """log [ Sigma * p(x_0 | x_1^p) / q(x_0 | x_1^q) ]  (Eq. 8)."""
+    return (log_sigma + gaussian_logpdf_iso(x0, mu1_p, sigma1_p)
+            - gaussian_logpdf_iso(x0, mu1_q, sigma1_q))
+
+
+def log_ratio_long(dq: dict, dp: dict, sched_q, sched_p) -> np.ndarray:
+    """log p(Y_p)/q(Y_q) as the full product over t = 1..T of per-step Gaussian
+    ratios (Eq. 4) with x_0^p := x_0^q, p(x_T) = q(x_T).  Needs keep=True runs."""
+    T = len(sched_q["a"])
+    total = 0.0
+    for j in range(T):                       # j-th step handles t = T-j
+        t = T - j
+        xq_next = dq["xs"][j + 1]
+        xp_next = dp["xs"][j + 1] if t > 1 else dq["xs"][j + 1]
+        total = total + gaussian_logpdf_iso(xp_next, dp["mus"][j], sched_p["sigma"][t - 1]) \
+                      - gaussian_logpdf_iso(xq_next, dq["mus"][j], sched_q["sigma"][t - 1])
+    return total
+
+
+# --------------------------------------------------------------------------
+# Verification (Alg. 1: draw r_i, accept while r_i <= ratio, n = first reject)
+# --------------------------------------------------------------------------
+def accept_prefix(log_ratio: np.ndarray, u: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """log_ratio, u: [B, gamma].  Position i is rejected iff u > p/q (so it is
+    accepted iff log u <= log ratio); n[b] = number of leading accepts."""
+    acc = np.log(u.astype(f64)) <= log_ratio
+    B, g = acc.shape
+    n = np.full(B, g, dtype=np.int32)
+    for b in range(B):
+        for i in range(g):
+            if not acc[b, i]:
+                n[b] = i
+                break
+    return n, acc
+
+
+# --------------------------------------------------------------------------
+# Resampling from the modified distribution max(0, p - q)/Z (Eq. 5) by
+# acceptance-rejection with bound M = 1/Z (Eq. 9-11) in the form of Corollary 1:
+# propose x' ~ p(x_0 | x_1^p), accept with
+#   alpha_s = max(0, Sigma p(x'|x_1^p) - q(x'|x_1^q)) / (Sigma p(x'|x_1^p)).
+# --------------------------------------------------------------------------
+def resample(n_accept, mu1_p, mu1_q, sigma1_p, sigma1_q, log_sigma, xi, v, gamma, cap):
+    B = len(n_accept)
+    C = mu1_p.shape[-1]
+    x_new = np.zeros((B, C), dtype=f64)
+    n_prop = np.zeros(B, dtype=np.int32)
+    flags = np.zeros(B, dtype=np.uint32)
+    alpha_first = np.full(B, np.nan)
+    for b in range(B):
+        n = int(n_accept[b])
+        if n >= gamma:
+            continue                          # all accepted: nothing to resample
+        j = b * gamma + n                     # first rejected position
+        flags[b] |= 1
+        done = False
+        for k in range(cap):
+            xp = mu1_p[j] + sigma1_p * xi[b, k].astype(f64)
+            lp = gaussian_logpdf_iso(xp, mu1_p[j], sigma1_p)
+            lq = gaussian_logpdf_iso(xp, mu1_q[j], sigma1_q)
+            # alpha_s = max(0, 1 - q/(Sigma p)), evaluated in the log domain
+            alpha_s = max(0.0, -np.expm1(min(0.0, lq - log_sigma - lp)))
+            if k == 0:
+                alpha_first[b] = alpha_s
+            x_new[b] = xp
+            n_prop[b] = k + 1
+            if float(v[b, k]) <= alpha_s:
+                done = True
+                break
+        if not done:
+            flags[b] |= 2                     # cap hit: last proposal is returned
+    return {"x_new": x_new, "n_prop": n_prop, "flags": flags,
+            "cap_hits": int(np.sum((flags & 2) != 0)), "alpha_first": alpha_first}
+
+
+# --------------------------------------------------------------------------
+# One full speculative round (Alg. 1 without the AR backbones)
+# --------------------------------------------------------------------------
+def csd_round(eps_q, eps_p, sched_q, sched_p, x_T, noise, u, xi, v, B, gamma, cap,
+              keep=False) -> Dict[str, np.ndarray]:
+    C = x_T.shape[-1]
+    dq, dp = run_pair(eps_q, eps_p, sched_q, sched_p, x_T, noise, keep=keep)
+    ls = log_sigma_term(sched_q["sigma"], sched_p["sigma"], C)
+    s1q, s1p = sched_q["sigma"][0], sched_p["sigma"][0]
+    logr = log_ratio_closed(dq["x0"], dq["mu1"], dp["mu1"], s1q, s1p, ls)
+    n, acc = accept_prefix(logr.reshape(B, gamma), u)
+    rs = resample(n, dp["mu1"], dq["mu1"], s1p, s1q, ls, xi, v, gamma, cap)
+    out = {"x0": dq["x0"], "mu1_q": dq["mu1"], "x1_q": dq["x1"], "mu1_p": dp["mu1"],
+           "x1_p": dp["x1"], "log_sigma": ls, "logratio": logr.reshape(B, gamma),
+           "n_accept": n, "accept": acc, **rs}
+    if keep:
+        out["dq"], out["dp"] = dq, dp
+    return out
+
+
+def round_from_inputs(inp, keep: bool = False) -> Dict[str, np.ndarray]:
+    """Run csd_round on a RoundInputs bundle (MLP heads, linear-beta schedule)."""
+    wl = inp.wl
+    sched = ddpm_schedule(inp.beta, wl.tau)
+    eq = make_mlp_head(inp.w_q, inp.z_q, inp.tfeat, wl.cfg, wl.cfg_scale)
+    ep = make_mlp_head(inp.w_p, inp.z_p, inp.tfeat, wl.cfg, wl.cfg_scale)
+    return csd_round(eq, ep, sched, sched, inp.x_T, inp.eps, inp.u, inp.xi, inp.v,
+                     wl.B, wl.gamma, wl.cap, keep=keep)
