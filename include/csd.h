@@ -49,27 +49,34 @@ enum {
   CSD_OK = 0,
   CSD_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, bad enum                         */
   CSD_ERR_SHAPE = -2,       /* dims of heads / schedules / calls do not agree                    */
-  CSD_ERR_UNSUPPORTED = -3, /* e.g. W not a multiple of 128 on the bf16 path, gamma > 32, C > 32 */
+  CSD_ERR_UNSUPPORTED = -3, /* e.g. W not a multiple of 128, gamma > 32, C > 16, not an sm_100 GPU */
   CSD_ERR_WORKSPACE = -4,   /* device memory for the workspace or weights could not be had      */
   CSD_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                                 */
   CSD_ERR_TIMEOUT = -6      /* a bounded device-side wait gave up (reported by csd_sync)         */
 };
 
-enum { CSD_F32 = 0, CSD_BF16 = 1 };
+enum { CSD_F32 = 0, CSD_BF16 = 1, CSD_F16 = 2 };
 
-/* Shape and arithmetic of one head.  CSD_F32: fp32 weights and activations on plain FMA units.
- * CSD_BF16: bf16 weights and bf16 GEMM inputs on tcgen05 tensor cores with fp32 accumulation;
- * residual stream, LayerNorm statistics, x_t and mu stay fp32. */
+/* Shape and arithmetic of one head.
+ * CSD_F32 : fp32 weights and activations on plain FMA units.
+ * CSD_BF16: tcgen05 tensor cores, both GEMM operands bf16 (weights and activations rounded to
+ *           bf16), fp32 accumulation in TMEM.
+ * CSD_F16 : the same kernels with both operands IEEE fp16.  Meant for weights whose VALUES are
+ *           bf16-representable: such a value is exact in fp16 when |w| >= 2^-17 (else it is off
+ *           by at most 2^-25), and activations keep 11 significant bits instead of 8, which the
+ *           long, error-amplifying T-step trajectories need (a tensor-core instruction takes
+ *           both operands in one 16-bit format).  Activations must stay below 65504 in magnitude.
+ * In all three the residual stream, LayerNorm statistics, x_t, mu and the densities are fp32. */
 typedef struct {
   int C, W, L, Dz, F;
-  int dtype; /* CSD_F32 | CSD_BF16 */
+  int dtype; /* CSD_F32 | CSD_BF16 | CSD_F16 */
 } csd_head_desc;
 
 /* HOST pointers to fp32 parameters, each matrix row-major [out, in]:
  * Wz[W,Dz] bz[W] Wt1[W,F] bt1[W] Wt2[W,W] bt2[W] Win[W,C] bin[W] Wada[L,3W,W] bada[L,3W]
  * W1[L,W,W] b1[L,W] W2[L,W,W] b2[L,W] Wfada[2W,W] bfada[2W] Wout[C,W] bout[C].
- * For CSD_BF16 heads the matrices are converted to bf16 (round to nearest even); callers that
- * want bit-defined results pass values that are already bf16-representable. */
+ * For CSD_BF16 / CSD_F16 heads the matrices are converted to that format (round to nearest
+ * even); callers that want bit-defined results pass values that are already representable. */
 typedef struct {
   const float *Wz, *bz, *Wt1, *bt1, *Wt2, *bt2, *Win, *bin;
   const float *Wada, *bada, *W1, *b1, *W2, *b2, *Wfada, *bfada, *Wout, *bout;

@@ -1,0 +1,215 @@
+"""ctypes binding of libcsd.so: argument marshalling only.
+
+Every step of the hot path runs inside the CUDA library; this module passes
+pointers and sizes.  torch is used for device memory and streams.  There is no
+CPU path: importing this module raises if the library is missing.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+_c_float_p = C.POINTER(C.c_float)
+
+ERRORS = {0: "CSD_OK", -1: "CSD_ERR_INVALID_ARG", -2: "CSD_ERR_SHAPE", -3: "CSD_ERR_UNSUPPORTED",
+          -4: "CSD_ERR_WORKSPACE", -5: "CSD_ERR_CUDA", -6: "CSD_ERR_TIMEOUT"}
+CSD_F32, CSD_BF16, CSD_F16 = 0, 1, 2
+DTYPES = {"f32": CSD_F32, "bf16": CSD_BF16, "f16": CSD_F16}
+
+EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launch_count",
+           "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_verify",
+           "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host")
+
+WEIGHT_FIELDS = ("Wz", "bz", "Wt1", "bt1", "Wt2", "bt2", "Win", "bin", "Wada", "bada",
+                 "W1", "b1", "W2", "b2", "Wfada", "bfada", "Wout", "bout")
+
+
+class CsdError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"{ERRORS.get(code, code)}: {msg}")
+        self.code = code
+
+
+class _HeadDesc(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("C", "W", "L", "Dz", "F", "dtype")]
+
+
+class _HeadWeights(C.Structure):
+    _fields_ = [(n, _c_float_p) for n in WEIGHT_FIELDS]
+
+
+class _Schedule(C.Structure):
+    _fields_ = [("T", C.c_int), ("a", _c_float_p), ("b", _c_float_p), ("sigma", _c_float_p),
+                ("tfeat", C.c_void_p)]
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    path = path or _build.LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: run `python -m paper_2411_11925_b200.build` "
+                          "(or __graft_entry__.build()); there is no CPU fallback")
+    lib = C.CDLL(path)
+    vp, i32, f32, f64 = C.c_void_p, C.c_int, C.c_float, C.c_double
+    lib.csd_create.argtypes = [C.POINTER(vp), i32, vp]
+    lib.csd_destroy.argtypes = [vp]
+    lib.csd_last_error.argtypes = [vp]; lib.csd_last_error.restype = C.c_char_p
+    lib.csd_sync.argtypes = [vp]
+    lib.csd_launch_count.argtypes = [vp]; lib.csd_launch_count.restype = C.c_int64
+    lib.csd_head_create.argtypes = [vp, C.POINTER(_HeadDesc), C.POINTER(_HeadWeights), C.POINTER(vp)]
+    lib.csd_head_destroy.argtypes = [vp]
+    lib.csd_draft_denoise.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, f32] + [vp] * 6
+    lib.csd_verify.argtypes = [vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32] + [vp] * 10
+    lib.csd_accept_scan.argtypes = [vp, i32, i32, i32, f64, f32, f32] + [vp] * 7
+    lib.csd_resample.argtypes = [vp, i32, i32, i32, i32, f64, f32, f32] + [vp] * 9
+    round_args = [vp, vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32, i32] + [vp] * 17
+    lib.csd_round.argtypes = round_args
+    lib.csd_round_host.argtypes = round_args
+    for name in EXPORTS:
+        if name not in ("csd_last_error", "csd_launch_count"):
+            getattr(lib, name).restype = C.c_int
+    return lib
+
+
+_LIB = load_library()
+
+
+def ddpm_coefficients(beta: np.ndarray, tau: float = 1.0) -> Dict[str, np.ndarray]:
+    """Host helper: reverse-process coefficients of a DDPM with fixed variance
+    sigma_t^2 = tau^2 beta_t (Eq. 3): mu_t = a_t x_t - b_t eps_hat."""
+    beta = np.asarray(beta, dtype=np.float64)
+    alpha = 1.0 - beta
+    abar = np.cumprod(alpha)
+    return {"a": (alpha ** -0.5).astype(np.float32),
+            "b": (beta / np.sqrt(alpha * (1.0 - abar))).astype(np.float32),
+            "sigma": (tau * np.sqrt(beta)).astype(np.float32)}
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        assert t.is_contiguous(), "tensor must be contiguous"
+        return t.data_ptr()
+    if isinstance(t, np.ndarray):
+        assert t.flags["C_CONTIGUOUS"], "array must be contiguous"
+        return t.ctypes.data
+    raise TypeError(type(t))
+
+
+class Schedule:
+    """Keeps the host coefficient arrays and the device feature table alive."""
+
+    def __init__(self, a, b, sigma, tfeat: torch.Tensor):
+        self.a = np.ascontiguousarray(a, dtype=np.float32)
+        self.b = np.ascontiguousarray(b, dtype=np.float32)
+        self.sigma = np.ascontiguousarray(sigma, dtype=np.float32)
+        assert tfeat.is_cuda and tfeat.dtype == torch.float32 and tfeat.is_contiguous()
+        self.tfeat = tfeat
+        self.T = int(self.sigma.shape[0])
+        self.c = _Schedule(self.T, self.a.ctypes.data_as(_c_float_p), self.b.ctypes.data_as(_c_float_p),
+                           self.sigma.ctypes.data_as(_c_float_p), tfeat.data_ptr())
+
+    def log_sigma_term(self, other_p: "Schedule", Cdim: int) -> float:
+        """log Sigma of Eq. 7 for (self = draft, other_p = target), as the library computes it."""
+        return float(Cdim * np.sum(np.log(self.sigma[1:].astype(np.float64))
+                                   - np.log(other_p.sigma[1:].astype(np.float64))))
+
+
+class Context:
+    def __init__(self, device: int = 0, stream: Optional[torch.cuda.Stream] = None):
+        self._h = C.c_void_p()
+        self.device = device
+        self.stream = stream
+        sp = stream.cuda_stream if stream is not None else None
+        rc = _LIB.csd_create(C.byref(self._h), device, sp)
+        if rc != 0:
+            raise CsdError(rc, "csd_create failed")
+        self._heads = []
+
+    def _check(self, rc: int):
+        if rc != 0:
+            raise CsdError(rc, _LIB.csd_last_error(self._h).decode())
+
+    def sync(self):
+        self._check(_LIB.csd_sync(self._h))
+
+    def launch_count(self) -> int:
+        return int(_LIB.csd_launch_count(self._h))
+
+    def close(self):
+        for h in list(self._heads):
+            h.close()
+        if self._h:
+            _LIB.csd_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- calls, named as in the C ABI ------------------------------------------------------
+    def csd_draft_denoise(self, head: "Head", sched: Schedule, R, cfg, cfg_scale, z, x_T, eps, x0, mu1, x1=None):
+        self._check(_LIB.csd_draft_denoise(self._h, head._h, C.byref(sched.c), R, int(cfg), cfg_scale,
+                                           _ptr(z), _ptr(x_T), _ptr(eps), _ptr(x0), _ptr(mu1), _ptr(x1)))
+
+    def csd_verify(self, head_p: "Head", sched_p: Schedule, sched_q: Schedule, B, gamma, cfg, cfg_scale,
+                   z_p, x_T, eps, x0_q, mu1_q, u, logratio, n_accept, accept_mask, mu1_p):
+        self._check(_LIB.csd_verify(self._h, head_p._h, C.byref(sched_p.c), C.byref(sched_q.c), B, gamma, int(cfg),
+                                    cfg_scale, _ptr(z_p), _ptr(x_T), _ptr(eps), _ptr(x0_q), _ptr(mu1_q), _ptr(u),
+                                    _ptr(logratio), _ptr(n_accept), _ptr(accept_mask), _ptr(mu1_p)))
+
+    def csd_accept_scan(self, B, gamma, Cdim, log_sigma, sigma1_p, sigma1_q, x0_q, mu1_q, mu1_p, u, logratio,
+                        n_accept, accept_mask=None):
+        self._check(_LIB.csd_accept_scan(self._h, B, gamma, Cdim, log_sigma, sigma1_p, sigma1_q, _ptr(x0_q),
+                                         _ptr(mu1_q), _ptr(mu1_p), _ptr(u), _ptr(logratio), _ptr(n_accept),
+                                         _ptr(accept_mask)))
+
+    def csd_resample(self, B, gamma, Cdim, cap, log_sigma, sigma1_p, sigma1_q, n_accept, mu1_p, mu1_q, xi, v,
+                     x_new, n_prop, flags, cap_hits):
+        self._check(_LIB.csd_resample(self._h, B, gamma, Cdim, cap, log_sigma, sigma1_p, sigma1_q, _ptr(n_accept),
+                                      _ptr(mu1_p), _ptr(mu1_q), _ptr(xi), _ptr(v), _ptr(x_new), _ptr(n_prop),
+                                      _ptr(flags), _ptr(cap_hits)))
+
+    def _round(self, fn, head_q, head_p, sched_q, sched_p, B, gamma, cfg, cfg_scale, cap, z_q, z_p, x_T, eps, u,
+               xi, v, x0, mu1_q, mu1_p, logratio, n_accept, accept_mask, x_new, n_prop, flags, cap_hits):
+        self._check(fn(self._h, head_q._h, head_p._h, C.byref(sched_q.c), C.byref(sched_p.c), B, gamma, int(cfg),
+                       cfg_scale, cap, *[_ptr(t) for t in (z_q, z_p, x_T, eps, u, xi, v, x0, mu1_q, mu1_p, logratio,
+                                                           n_accept, accept_mask, x_new, n_prop, flags, cap_hits)]))
+
+    def csd_round(self, *args):
+        self._round(_LIB.csd_round, *args)
+
+    def csd_round_host(self, *args):
+        self._round(_LIB.csd_round_host, *args)
+
+
+class Head:
+    def __init__(self, ctx: Context, weights: Dict[str, np.ndarray], operand: str):
+        """operand: "f32", "bf16" or "f16" = the GEMM operand format (see csd_head_desc)."""
+        Wd, Dz = weights["Wz"].shape
+        Cdim = weights["Wout"].shape[0]
+        L = weights["W1"].shape[0]
+        F = weights["Wt1"].shape[1]
+        self.desc = _HeadDesc(Cdim, Wd, L, Dz, F, DTYPES[operand])
+        keep = {k: np.ascontiguousarray(weights[k], dtype=np.float32) for k in WEIGHT_FIELDS}
+        hw = _HeadWeights(*[keep[k].ctypes.data_as(_c_float_p) for k in WEIGHT_FIELDS])
+        self._h = C.c_void_p()
+        self.ctx = ctx
+        rc = _LIB.csd_head_create(ctx._h, C.byref(self.desc), C.byref(hw), C.byref(self._h))
+        ctx._check(rc)
+        ctx._heads.append(self)
+
+    def close(self):
+        if self._h:
+            _LIB.csd_head_destroy(self._h)
+            self._h = C.c_void_p()
+            if self in self.ctx._heads:
+                self.ctx._heads.remove(self)

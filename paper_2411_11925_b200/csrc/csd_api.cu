@@ -1,0 +1,688 @@
+// C ABI of the continuous speculative decoding hot path (see include/csd.h for the contract).
+// Host side: argument checks, weight packing, workspace, launch sequencing.  Every arithmetic step
+// runs in the kernels of gemm.cuh / rowops.cuh.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <type_traits>
+#include <vector>
+
+#include "../../include/csd.h"
+#include "gemm.cuh"
+#include "rowops.cuh"
+
+using namespace csd;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct ChainWs {
+  void* base = nullptr;
+  size_t cap = 0;
+  // carved per call
+  void *zc, *s, *u, *v;
+  float *cz, *te, *h, *stats, *epart, *x;
+};
+
+struct HostIo {  // device mirrors for csd_round_host
+  void* base = nullptr;
+  size_t cap = 0;
+};
+
+}  // namespace
+
+struct csd_ctx {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  cudaStream_t side[2] = {nullptr, nullptr};
+  cudaEvent_t ev_fork = nullptr, ev_done[2] = {nullptr, nullptr};
+  int* d_err = nullptr;
+  int64_t launches = 0;
+  EncodeTiledFn encode = nullptr;
+  ChainWs ws[2];
+  HostIo io;
+  char err[512] = {0};
+};
+
+struct csd_head {
+  csd_ctx* ctx = nullptr;
+  csd_head_desc d{};
+  void* wblob = nullptr;   // GEMM weights (bf16 or fp32)
+  float* fblob = nullptr;  // fp32 side parameters
+  size_t esz = 4;
+  // GEMM weights
+  void* Wz = nullptr;
+  std::vector<void*> Wss, Wg, W1, W2;
+  void* Wfss = nullptr;
+  // fp32 parameters
+  float *bz, *Wt1, *bt1, *Wt2, *bt2, *win, *bin, *bfsh, *bfsc, *wout_t, *bout;
+  std::vector<float*> bsh, bsc, bg, b1, b2;
+  // tensor maps of the weights (bf16 heads)
+  CUtensorMap tmWz{};
+  std::vector<CUtensorMap> tmWss, tmWg, tmW1, tmW2;
+  CUtensorMap tmWfss{};
+};
+
+namespace {
+
+int fail(csd_ctx* ctx, int code, const char* fmt, ...) {
+  if (ctx) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+#define CSD_CUDA(ctx, call)                                                                          \
+  do {                                                                                               \
+    cudaError_t e_ = (call);                                                                         \
+    if (e_ != cudaSuccess)                                                                           \
+      return fail(ctx, CSD_ERR_CUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), __FILE__, \
+                  __LINE__);                                                                         \
+  } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+uint16_t f32_to_bf16_bits(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<uint16_t>((u >> 16) | 0x40);  // NaN
+  const uint32_t bias = ((u >> 16) & 1u) + 0x7fffu;
+  return static_cast<uint16_t>((u + bias) >> 16);
+}
+
+int make_tmap(csd_ctx* ctx, CUtensorMap* m, int dtype, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld,
+              uint32_t box_rows) {
+  const cuuint64_t gdim[2] = {cols, rows};
+  const cuuint64_t gstride[1] = {ld * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = ctx->encode(m, dtype == CSD_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box,
+                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, CSD_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return CSD_OK;
+}
+
+int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, int T) {
+  const size_t asz = d.dtype == CSD_F32 ? 4 : 2;
+  const size_t W = d.W;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+  const size_t o_zc = take(static_cast<size_t>(Rh) * d.Dz * asz);
+  const size_t o_s = take(Rh * W * asz), o_u = take(Rh * W * asz), o_v = take(Rh * W * asz);
+  const size_t o_cz = take(Rh * W * 4), o_te = take(static_cast<size_t>(T) * W * 4), o_h = take(Rh * W * 4);
+  const size_t o_st = take(Rh * (W / kChunk) * 8);
+  const size_t o_ep = take(Rh * (W / kTileN) * kCPad * 4);
+  const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
+  if (off > ws.cap) {
+    CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamSynchronize(ctx->side[i]));
+    if (ws.base) CSD_CUDA(ctx, cudaFree(ws.base));
+    ws.base = nullptr;
+    ws.cap = 0;
+    if (cudaMalloc(&ws.base, off) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes of workspace", off);
+    }
+    ws.cap = off;
+  }
+  char* b = static_cast<char*>(ws.base);
+  ws.zc = b + o_zc; ws.s = b + o_s; ws.u = b + o_u; ws.v = b + o_v;
+  ws.cz = reinterpret_cast<float*>(b + o_cz); ws.te = reinterpret_cast<float*>(b + o_te);
+  ws.h = reinterpret_cast<float*>(b + o_h); ws.stats = reinterpret_cast<float*>(b + o_st);
+  ws.epart = reinterpret_cast<float*>(b + o_ep); ws.x = reinterpret_cast<float*>(b + o_x);
+  return CSD_OK;
+}
+
+template <int EPI, int NSEG, int MMA_N, typename ACT>
+int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0, const CUtensorMap& a1,
+                const CUtensorMap& b1, int K0, int K1, int N, const EpiParams& ep) {
+  auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, std::is_same<ACT, __half>::value ? 0 : 1>;
+  static bool attr_done = false;
+  constexpr int smem = TcCfg<MMA_N>::kSmemBytes;
+  if (!attr_done) {
+    CSD_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_done = true;
+  }
+  dim3 grid(N / kTileN, (ep.M + kTileM - 1) / kTileM);
+  kern<<<grid, kTcThreads, smem, st>>>(a0, b0, a1, b1, K0 / kBlockK, K1 / kBlockK, ep, ctx->d_err);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+template <int EPI, int NSEG, int MMA_N>
+int launch_tc(csd_ctx* ctx, int dtype, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0,
+              const CUtensorMap& a1, const CUtensorMap& b1, int K0, int K1, int N, const EpiParams& ep) {
+  if (dtype == CSD_F16) return launch_tc_t<EPI, NSEG, MMA_N, __half>(ctx, st, a0, b0, a1, b1, K0, K1, N, ep);
+  return launch_tc_t<EPI, NSEG, MMA_N, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, K0, K1, N, ep);
+}
+
+template <int EPI, int NSEG, int MMA_N>
+int launch_simt(csd_ctx* ctx, cudaStream_t st, const float* A0, int lda0, const float* B0, int K0, const float* A1,
+                int lda1, const float* B1, int K1, int N, const EpiParams& ep) {
+  dim3 grid(N / kTileN, (ep.M + kSimtRows - 1) / kSimtRows);
+  gemm_simt_kernel<EPI, NSEG, MMA_N><<<grid, 128, 0, st>>>(A0, lda0, B0, K0, K0, A1, lda1, B1, K1, K1, ep);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+int check_sched(csd_ctx* ctx, const csd_schedule* s, bool full) {
+  if (!s) return fail(ctx, CSD_ERR_INVALID_ARG, "schedule is null");
+  if (s->T < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "schedule T = %d must be >= 1", s->T);
+  if (!s->sigma) return fail(ctx, CSD_ERR_INVALID_ARG, "schedule sigma is null");
+  if (full && (!s->a || !s->b || !s->tfeat)) return fail(ctx, CSD_ERR_INVALID_ARG, "schedule a/b/tfeat is null");
+  for (int t = 0; t < s->T; ++t)
+    if (!(s->sigma[t] > 0.0f)) return fail(ctx, CSD_ERR_INVALID_ARG, "schedule sigma[%d] must be > 0", t);
+  return CSD_OK;
+}
+
+// Runs t = T..1 of one head for R token rows on stream `st` with workspace slot `slot`.
+int run_chain(csd_ctx* ctx, int slot, cudaStream_t st, const csd_head* hd, const csd_schedule* sc, int R, int cfg,
+              float cfg_scale, const float* z, const float* x_T, const float* eps, int sample_last, float* x0,
+              float* mu1, float* x1) {
+  const csd_head_desc& d = hd->d;
+  const int Rh = R * (cfg ? 2 : 1), W = d.W, L = d.L, T = sc->T, NT = W / kTileN;
+  const bool tc = d.dtype != CSD_F32;
+  ChainWs& ws = ctx->ws[slot];
+  int rc = ensure_ws(ctx, ws, d, Rh, R, T);
+  if (rc) return rc;
+
+  timestep_embed_kernel<<<T, 256, (d.F + W) * sizeof(float), st>>>(sc->tfeat, hd->Wt1, hd->bt1, hd->Wt2, hd->bt2, W,
+                                                                  d.F, ws.te);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+
+  CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{};
+  EpiParams ep{};
+  ep.M = Rh; ep.ldo = W;
+  if (tc) {
+    const size_t nz = static_cast<size_t>(Rh) * d.Dz;
+    const unsigned nblk = static_cast<unsigned>((nz + 255) / 256);
+    if (d.dtype == CSD_F16) convert_act_kernel<__half><<<nblk, 256, 0, st>>>(z, static_cast<__half*>(ws.zc), nz);
+    else convert_act_kernel<__nv_bfloat16><<<nblk, 256, 0, st>>>(z, static_cast<__nv_bfloat16*>(ws.zc), nz);
+    ctx->launches++;
+    if ((rc = make_tmap(ctx, &tm_z, d.dtype, ws.zc, Rh, d.Dz, d.Dz, kTileM))) return rc;
+    if ((rc = make_tmap(ctx, &tm_s, d.dtype, ws.s, Rh, W, W, kTileM))) return rc;
+    if ((rc = make_tmap(ctx, &tm_u, d.dtype, ws.u, Rh, W, W, kTileM))) return rc;
+    if ((rc = make_tmap(ctx, &tm_v, d.dtype, ws.v, Rh, W, W, kTileM))) return rc;
+  }
+  // S0: cz = z Wz^T + bz
+  ep.bias0 = hd->bz; ep.out_f32 = ws.cz;
+  if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 128>(ctx, d.dtype, st, tm_z, hd->tmWz, tm_z, hd->tmWz, d.Dz, 0, W, ep);
+  else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
+                                              nullptr, 0, W, ep);
+  if (rc) return rc;
+
+  StepParams sp{};
+  sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = NT; sp.cfg_scale = cfg_scale;
+  sp.sample_last = sample_last; sp.epart = ws.epart; sp.bout = hd->bout; sp.x_src = x_T; sp.x = ws.x;
+  sp.x0 = x0; sp.mu1 = mu1; sp.x1 = x1; sp.win = hd->win; sp.bin = hd->bin; sp.cz = ws.cz; sp.h = ws.h;
+  sp.stats = ws.stats; sp.s = ws.s;
+  auto launch_step = [&](int mode) -> int {
+    if (d.dtype == CSD_F16) step_kernel<__half><<<R, 256, 0, st>>>(sp, mode);
+    else if (d.dtype == CSD_BF16) step_kernel<__nv_bfloat16><<<R, 256, 0, st>>>(sp, mode);
+    else step_kernel<float><<<R, 256, 0, st>>>(sp, mode);
+    ctx->launches++;
+    CSD_CUDA(ctx, cudaGetLastError());
+    return CSD_OK;
+  };
+  sp.te_next = ws.te + static_cast<size_t>(T - 1) * W;
+  sp.eps_t = eps;
+  if ((rc = launch_step(STEP_INIT))) return rc;
+
+  const float* sf = static_cast<const float*>(ws.s);
+  const float* uf = static_cast<const float*>(ws.u);
+  const float* vf = static_cast<const float*>(ws.v);
+  for (int t = T; t >= 1; --t) {
+    for (int k = 0; k < L; ++k) {
+      EpiParams e = ep;
+      e.h = ws.h; e.stats = ws.stats;
+      // u = LN(h)(1 + scale) + shift
+      e.bias0 = hd->bsh[k]; e.bias1 = hd->bsc[k]; e.out_act = ws.u;
+      if (tc) rc = launch_tc<EPI_MOD, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWss[k], tm_s, hd->tmWss[k], W, 0, W, e);
+      else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
+                                             nullptr, 0, W, e);
+      if (rc) return rc;
+      // v = SiLU(W1 u + b1)
+      e.bias0 = hd->b1[k]; e.bias1 = nullptr; e.out_act = ws.v;
+      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 128>(ctx, d.dtype, st, tm_u, hd->tmW1[k], tm_u, hd->tmW1[k], W, 0, W, e);
+      else rc = launch_simt<EPI_SILU_ACT, 1, 128>(ctx, st, uf, W, static_cast<const float*>(hd->W1[k]), W, nullptr, 0,
+                                                  nullptr, 0, W, e);
+      if (rc) return rc;
+      // h += gate * (W2 v + b2)
+      e.bias0 = hd->b2[k]; e.bias1 = hd->bg[k]; e.out_act = nullptr;
+      if (tc) rc = launch_tc<EPI_GATE_RES, 2, 128>(ctx, d.dtype, st, tm_v, hd->tmW2[k], tm_s, hd->tmWg[k], W, W, W, e);
+      else rc = launch_simt<EPI_GATE_RES, 2, 128>(ctx, st, vf, W, static_cast<const float*>(hd->W2[k]), W, sf, W,
+                                                  static_cast<const float*>(hd->Wg[k]), W, W, e);
+      if (rc) return rc;
+    }
+    EpiParams e = ep;
+    e.h = ws.h; e.stats = ws.stats; e.bias0 = hd->bfsh; e.bias1 = hd->bfsc; e.wout_t = hd->wout_t; e.epart = ws.epart;
+    if (tc) rc = launch_tc<EPI_MODF, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWfss, tm_s, hd->tmWfss, W, 0, W, e);
+    else rc = launch_simt<EPI_MODF, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
+                                            0, W, e);
+    if (rc) return rc;
+    sp.a = sc->a[t - 1]; sp.b = sc->b[t - 1]; sp.sigma = sc->sigma[t - 1];
+    sp.eps_t = eps + static_cast<size_t>(t - 1) * R * d.C;
+    if (t > 1) sp.te_next = ws.te + static_cast<size_t>(t - 2) * W;
+    if ((rc = launch_step(t > 1 ? STEP_MID : STEP_LAST))) return rc;
+  }
+  return CSD_OK;
+}
+
+int check_chain_args(csd_ctx* ctx, const csd_head* hd, const csd_schedule* sc, int R, int cfg, const void* z,
+                     const void* x_T, const void* eps) {
+  if (!hd) return fail(ctx, CSD_ERR_INVALID_ARG, "head is null");
+  if (hd->ctx != ctx) return fail(ctx, CSD_ERR_INVALID_ARG, "head belongs to another context");
+  int rc = check_sched(ctx, sc, true);
+  if (rc) return rc;
+  if (R < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "row count %d must be >= 1", R);
+  if (cfg != 0 && cfg != 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cfg must be 0 or 1");
+  if (!z || !x_T || !eps) return fail(ctx, CSD_ERR_INVALID_ARG, "z / x_T / eps is null");
+  return CSD_OK;
+}
+
+double log_sigma_term(const csd_schedule* q, const csd_schedule* p, int C) {
+  double acc = 0.0;
+  for (int t = 1; t < q->T; ++t) acc += std::log(static_cast<double>(q->sigma[t])) - std::log(static_cast<double>(p->sigma[t]));
+  return C * acc;
+}
+
+int accept_scan(csd_ctx* ctx, cudaStream_t st, int B, int gamma, int C, double log_sigma, float sp1, float sq1,
+                const float* x0, const float* mu_q, const float* mu_p, const float* u, float* logratio,
+                int32_t* n_accept, uint32_t* mask) {
+  const double lc = log_sigma + C * (std::log(static_cast<double>(sq1)) - std::log(static_cast<double>(sp1)));
+  const float inv2vp = static_cast<float>(0.5 / (static_cast<double>(sp1) * sp1));
+  const float inv2vq = static_cast<float>(0.5 / (static_cast<double>(sq1) * sq1));
+  accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, gamma, C, static_cast<float>(lc), inv2vp, inv2vq, x0, mu_q, mu_p, u,
+                                                  logratio, n_accept, mask);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+int resample(csd_ctx* ctx, cudaStream_t st, int B, int gamma, int C, int cap, double log_sigma, float sp1, float sq1,
+             const int32_t* n_accept, const float* mu_p, const float* mu_q, const float* xi, const float* v,
+             float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  CSD_CUDA(ctx, cudaMemsetAsync(cap_hits, 0, sizeof(int32_t), st));
+  resample_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, gamma, C, cap, static_cast<float>(log_sigma), sp1, sq1,
+                                               static_cast<float>(std::log(static_cast<double>(sp1))),
+                                               static_cast<float>(std::log(static_cast<double>(sq1))), n_accept, mu_p,
+                                               mu_q, xi, v, x_new, n_prop, flags, cap_hits);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+int check_verify_dims(csd_ctx* ctx, int B, int gamma, int C) {
+  if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
+  if (gamma > 32) return fail(ctx, CSD_ERR_UNSUPPORTED, "gamma = %d exceeds 32", gamma);
+  if (C < 1 || C > kCPad) return fail(ctx, CSD_ERR_UNSUPPORTED, "token dim C = %d must be in [1, 16]", C);
+  return CSD_OK;
+}
+
+}  // namespace
+
+// ================================================================================== C ABI
+extern "C" {
+
+int csd_create(csd_ctx** out, int device, void* cuda_stream) {
+  if (!out) return CSD_ERR_INVALID_ARG;
+  *out = nullptr;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+    cudaGetLastError();
+    return CSD_ERR_CUDA;
+  }
+  if (cudaSetDevice(device) != cudaSuccess) return CSD_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return CSD_ERR_CUDA;
+  if (prop.major != 10) return CSD_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
+  csd_ctx* c = new (std::nothrow) csd_ctx();
+  if (!c) return CSD_ERR_WORKSPACE;
+  c->device = device;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  bool ok = true;
+  for (int i = 0; i < 2; ++i) {
+    ok = ok && cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+  }
+  ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_err, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_err, 0, sizeof(int)) == cudaSuccess;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  ok = ok && cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+       qres == cudaDriverEntryPointSuccess && fn != nullptr;
+  if (!ok) {
+    cudaGetLastError();
+    csd_destroy(c);
+    return CSD_ERR_CUDA;
+  }
+  c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  *out = c;
+  return CSD_OK;
+}
+
+int csd_destroy(csd_ctx* c) {
+  if (!c) return CSD_ERR_INVALID_ARG;
+  cudaSetDevice(c->device);
+  cudaStreamSynchronize(c->stream);
+  for (int i = 0; i < 2; ++i) {
+    if (c->side[i]) { cudaStreamSynchronize(c->side[i]); cudaStreamDestroy(c->side[i]); }
+    if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
+    if (c->ws[i].base) cudaFree(c->ws[i].base);
+  }
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->io.base) cudaFree(c->io.base);
+  if (c->d_err) cudaFree(c->d_err);
+  cudaGetLastError();
+  delete c;
+  return CSD_OK;
+}
+
+const char* csd_last_error(const csd_ctx* c) { return c ? c->err : "null context"; }
+
+int64_t csd_launch_count(const csd_ctx* c) { return c ? c->launches : 0; }
+
+int csd_sync(csd_ctx* c) {
+  if (!c) return CSD_ERR_INVALID_ARG;
+  CSD_CUDA(c, cudaStreamSynchronize(c->stream));
+  int e = 0;
+  CSD_CUDA(c, cudaMemcpy(&e, c->d_err, sizeof(int), cudaMemcpyDeviceToHost));
+  if (e != 0) {
+    cudaMemset(c->d_err, 0, sizeof(int));
+    return fail(c, CSD_ERR_TIMEOUT, "a device-side bounded wait gave up (code %d: 1 = TMA producer, 2 = MMA issuer, "
+                "3 = epilogue)", e);
+  }
+  return CSD_OK;
+}
+
+int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weights* w, csd_head** out) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (!desc || !w || !out) return fail(ctx, CSD_ERR_INVALID_ARG, "desc / weights / out is null");
+  *out = nullptr;
+  const csd_head_desc d = *desc;
+  if (d.dtype != CSD_F32 && d.dtype != CSD_BF16 && d.dtype != CSD_F16) return fail(ctx, CSD_ERR_INVALID_ARG, "dtype %d unknown", d.dtype);
+  if (d.C < 1 || d.W < 1 || d.L < 1 || d.Dz < 1 || d.F < 1)
+    return fail(ctx, CSD_ERR_INVALID_ARG, "head dims must be positive (C=%d W=%d L=%d Dz=%d F=%d)", d.C, d.W, d.L, d.Dz, d.F);
+  if (d.C > kCPad) return fail(ctx, CSD_ERR_UNSUPPORTED, "token dim C = %d exceeds 16", d.C);
+  if (d.W % kTileN != 0) return fail(ctx, CSD_ERR_UNSUPPORTED, "width W = %d must be a multiple of 128", d.W);
+  const int kmul = d.dtype != CSD_F32 ? kBlockK : kSimtBK;
+  if (d.Dz % kmul != 0) return fail(ctx, CSD_ERR_UNSUPPORTED, "Dz = %d must be a multiple of %d", d.Dz, kmul);
+  if (static_cast<size_t>(d.F + d.W) * 4 > 40 * 1024)
+    return fail(ctx, CSD_ERR_UNSUPPORTED, "F + W = %d too large for the timestep-embedding kernel", d.F + d.W);
+  const float* const* ptrs = reinterpret_cast<const float* const*>(w);
+  for (size_t i = 0; i < sizeof(csd_head_weights) / sizeof(float*); ++i)
+    if (!ptrs[i]) return fail(ctx, CSD_ERR_INVALID_ARG, "weight pointer #%zu is null", i);
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+
+  csd_head* h = new (std::nothrow) csd_head();
+  if (!h) return fail(ctx, CSD_ERR_WORKSPACE, "out of host memory");
+  h->ctx = ctx; h->d = d; h->esz = d.dtype != CSD_F32 ? 2 : 4;
+  const size_t W = d.W, L = d.L, Dz = d.Dz, F = d.F, C = d.C;
+
+  // ---- GEMM weights, packed: Wz | per block (Wss, Wg, W1, W2) | Wfss
+  const size_t n_gemm = W * Dz + L * (5 * W * W) + 2 * W * W;
+  std::vector<float> stage;
+  try { stage.resize(n_gemm); } catch (...) { delete h; return fail(ctx, CSD_ERR_WORKSPACE, "out of host memory"); }
+  std::vector<size_t> o_wss(L), o_wg(L), o_w1(L), o_w2(L);
+  size_t off = 0;
+  const size_t o_wz = off; memcpy(&stage[off], w->Wz, W * Dz * 4); off += W * Dz;
+  auto interleave = [&](const float* shift_rows, const float* scale_rows, float* dst) {
+    for (size_t j = 0; j < W / kTileN; ++j) {
+      memcpy(dst + (2 * j) * kTileN * W, shift_rows + j * kTileN * W, kTileN * W * 4);
+      memcpy(dst + (2 * j + 1) * kTileN * W, scale_rows + j * kTileN * W, kTileN * W * 4);
+    }
+  };
+  for (size_t k = 0; k < L; ++k) {
+    const float* ada = w->Wada + k * 3 * W * W;
+    o_wss[k] = off; interleave(ada, ada + W * W, &stage[off]); off += 2 * W * W;
+    o_wg[k] = off; memcpy(&stage[off], ada + 2 * W * W, W * W * 4); off += W * W;
+    o_w1[k] = off; memcpy(&stage[off], w->W1 + k * W * W, W * W * 4); off += W * W;
+    o_w2[k] = off; memcpy(&stage[off], w->W2 + k * W * W, W * W * 4); off += W * W;
+  }
+  const size_t o_wfss = off; interleave(w->Wfada, w->Wfada + W * W, &stage[off]); off += 2 * W * W;
+
+  auto bail = [&](int code, const char* what) { csd_head_destroy(h); return fail(ctx, code, "%s", what); };
+  if (cudaMalloc(&h->wblob, n_gemm * h->esz) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the weights"); }
+  if (d.dtype != CSD_F32) {
+    std::vector<uint16_t> hb;
+    try { hb.resize(n_gemm); } catch (...) { return bail(CSD_ERR_WORKSPACE, "out of host memory"); }
+    if (d.dtype == CSD_BF16) {
+      for (size_t i = 0; i < n_gemm; ++i) hb[i] = f32_to_bf16_bits(stage[i]);
+    } else {
+      for (size_t i = 0; i < n_gemm; ++i) { const __half hv = __float2half_rn(stage[i]); memcpy(&hb[i], &hv, 2); }
+    }
+    if (cudaMemcpy(h->wblob, hb.data(), n_gemm * 2, cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "weight upload failed");
+  } else {
+    if (cudaMemcpy(h->wblob, stage.data(), n_gemm * 4, cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "weight upload failed");
+  }
+  auto wp = [&](size_t o) { return static_cast<void*>(static_cast<char*>(h->wblob) + o * h->esz); };
+  h->Wz = wp(o_wz); h->Wfss = wp(o_wfss);
+  h->Wss.resize(L); h->Wg.resize(L); h->W1.resize(L); h->W2.resize(L);
+  for (size_t k = 0; k < L; ++k) { h->Wss[k] = wp(o_wss[k]); h->Wg[k] = wp(o_wg[k]); h->W1[k] = wp(o_w1[k]); h->W2[k] = wp(o_w2[k]); }
+
+  // ---- fp32 side parameters
+  std::vector<float> fs;
+  auto put = [&](const float* src, size_t n) { size_t o = fs.size(); fs.insert(fs.end(), src, src + n); while (fs.size() % 4) fs.push_back(0.0f); return o; };
+  const size_t f_bz = put(w->bz, W), f_wt1 = put(w->Wt1, W * F), f_bt1 = put(w->bt1, W), f_wt2 = put(w->Wt2, W * W),
+               f_bt2 = put(w->bt2, W), f_bin = put(w->bin, W);
+  std::vector<float> win_pad(W * kCPad, 0.0f), wout_t(W * kCPad, 0.0f), bout_pad(kCPad, 0.0f);
+  for (size_t n = 0; n < W; ++n)
+    for (size_t c = 0; c < C; ++c) { win_pad[n * kCPad + c] = w->Win[n * C + c]; wout_t[n * kCPad + c] = w->Wout[c * W + n]; }
+  for (size_t c = 0; c < C; ++c) bout_pad[c] = w->bout[c];
+  const size_t f_win = put(win_pad.data(), win_pad.size()), f_wout = put(wout_t.data(), wout_t.size()),
+               f_bout = put(bout_pad.data(), kCPad);
+  std::vector<size_t> f_bsh(L), f_bsc(L), f_bg(L), f_b1(L), f_b2(L);
+  for (size_t k = 0; k < L; ++k) {
+    f_bsh[k] = put(w->bada + k * 3 * W, W); f_bsc[k] = put(w->bada + k * 3 * W + W, W);
+    f_bg[k] = put(w->bada + k * 3 * W + 2 * W, W);
+    f_b1[k] = put(w->b1 + k * W, W); f_b2[k] = put(w->b2 + k * W, W);
+  }
+  const size_t f_bfsh = put(w->bfada, W), f_bfsc = put(w->bfada + W, W);
+  if (cudaMalloc(&h->fblob, fs.size() * 4) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the parameters"); }
+  if (cudaMemcpy(h->fblob, fs.data(), fs.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "parameter upload failed");
+  float* fb = h->fblob;
+  h->bz = fb + f_bz; h->Wt1 = fb + f_wt1; h->bt1 = fb + f_bt1; h->Wt2 = fb + f_wt2; h->bt2 = fb + f_bt2;
+  h->win = fb + f_win; h->bin = fb + f_bin; h->wout_t = fb + f_wout; h->bout = fb + f_bout;
+  h->bfsh = fb + f_bfsh; h->bfsc = fb + f_bfsc;
+  h->bsh.resize(L); h->bsc.resize(L); h->bg.resize(L); h->b1.resize(L); h->b2.resize(L);
+  for (size_t k = 0; k < L; ++k) { h->bsh[k] = fb + f_bsh[k]; h->bsc[k] = fb + f_bsc[k]; h->bg[k] = fb + f_bg[k]; h->b1[k] = fb + f_b1[k]; h->b2[k] = fb + f_b2[k]; }
+
+  if (d.dtype != CSD_F32) {
+    int rc = make_tmap(ctx, &h->tmWz, d.dtype, h->Wz, W, Dz, Dz, 128);
+    h->tmWss.resize(L); h->tmWg.resize(L); h->tmW1.resize(L); h->tmW2.resize(L);
+    for (size_t k = 0; k < L && !rc; ++k) {
+      rc = make_tmap(ctx, &h->tmWss[k], d.dtype, h->Wss[k], 2 * W, W, W, 256);
+      if (!rc) rc = make_tmap(ctx, &h->tmWg[k], d.dtype, h->Wg[k], W, W, W, 128);
+      if (!rc) rc = make_tmap(ctx, &h->tmW1[k], d.dtype, h->W1[k], W, W, W, 128);
+      if (!rc) rc = make_tmap(ctx, &h->tmW2[k], d.dtype, h->W2[k], W, W, W, 128);
+    }
+    if (!rc) rc = make_tmap(ctx, &h->tmWfss, d.dtype, h->Wfss, 2 * W, W, W, 256);
+    if (rc) { csd_head_destroy(h); return rc; }
+  }
+  *out = h;
+  return CSD_OK;
+}
+
+int csd_head_destroy(csd_head* h) {
+  if (!h) return CSD_ERR_INVALID_ARG;
+  if (h->ctx) {
+    cudaSetDevice(h->ctx->device);
+    cudaStreamSynchronize(h->ctx->stream);
+    for (int i = 0; i < 2; ++i) cudaStreamSynchronize(h->ctx->side[i]);
+  }
+  if (h->wblob) cudaFree(h->wblob);
+  if (h->fblob) cudaFree(h->fblob);
+  cudaGetLastError();
+  delete h;
+  return CSD_OK;
+}
+
+int csd_draft_denoise(csd_ctx* ctx, const csd_head* head, const csd_schedule* sched, int R, int cfg, float cfg_scale,
+                      const float* z, const float* x_T, const float* eps, float* x0, float* mu1, float* x1) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_chain_args(ctx, head, sched, R, cfg, z, x_T, eps);
+  if (rc) return rc;
+  if (!x0 || !mu1) return fail(ctx, CSD_ERR_INVALID_ARG, "x0 / mu1 is null");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  return run_chain(ctx, 0, ctx->stream, head, sched, R, cfg, cfg_scale, z, x_T, eps, 1, x0, mu1, x1);
+}
+
+int csd_accept_scan(csd_ctx* ctx, int B, int gamma, int C, double log_sigma_term_, float sigma1_p, float sigma1_q,
+                    const float* x0_q, const float* mu1_q, const float* mu1_p, const float* u, float* logratio,
+                    int32_t* n_accept, uint32_t* accept_mask) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_verify_dims(ctx, B, gamma, C);
+  if (rc) return rc;
+  if (!x0_q || !mu1_q || !mu1_p || !u || !logratio || !n_accept) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  if (!(sigma1_p > 0.0f) || !(sigma1_q > 0.0f)) return fail(ctx, CSD_ERR_INVALID_ARG, "sigma1 must be > 0");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  return accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term_, sigma1_p, sigma1_q, x0_q, mu1_q, mu1_p, u, logratio,
+                     n_accept, accept_mask);
+}
+
+int csd_verify(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p, const csd_schedule* sched_q, int B,
+               int gamma, int cfg, float cfg_scale, const float* z_p, const float* x_T, const float* eps,
+               const float* x0_q, const float* mu1_q, const float* u, float* logratio, int32_t* n_accept,
+               uint32_t* accept_mask, float* mu1_p) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
+  int rc = check_chain_args(ctx, head_p, sched_p, B * gamma, cfg, z_p, x_T, eps);
+  if (rc) return rc;
+  if ((rc = check_sched(ctx, sched_q, false))) return rc;
+  if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
+  if ((rc = check_verify_dims(ctx, B, gamma, head_p->d.C))) return rc;
+  if (!x0_q || !mu1_q || !u || !logratio || !n_accept || !mu1_p) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  rc = run_chain(ctx, 1, ctx->stream, head_p, sched_p, B * gamma, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr);
+  if (rc) return rc;
+  const int C = head_p->d.C;
+  return accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term(sched_q, sched_p, C), sched_p->sigma[0],
+                     sched_q->sigma[0], x0_q, mu1_q, mu1_p, u, logratio, n_accept, accept_mask);
+}
+
+int csd_resample(csd_ctx* ctx, int B, int gamma, int C, int cap, double log_sigma_term_, float sigma1_p, float sigma1_q,
+                 const int32_t* n_accept, const float* mu1_p, const float* mu1_q, const float* xi, const float* v,
+                 float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_verify_dims(ctx, B, gamma, C);
+  if (rc) return rc;
+  if (cap < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cap = %d must be >= 1", cap);
+  if (!n_accept || !mu1_p || !mu1_q || !xi || !v || !x_new || !n_prop || !flags || !cap_hits)
+    return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  if (!(sigma1_p > 0.0f) || !(sigma1_q > 0.0f)) return fail(ctx, CSD_ERR_INVALID_ARG, "sigma1 must be > 0");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  return resample(ctx, ctx->stream, B, gamma, C, cap, log_sigma_term_, sigma1_p, sigma1_q, n_accept, mu1_p, mu1_q, xi, v,
+                  x_new, n_prop, flags, cap_hits);
+}
+
+int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule* sched_q,
+              const csd_schedule* sched_p, int B, int gamma, int cfg, float cfg_scale, int cap, const float* z_q,
+              const float* z_p, const float* x_T, const float* eps, const float* u, const float* xi, const float* v,
+              float* x0, float* mu1_q, float* mu1_p, float* logratio, int32_t* n_accept, uint32_t* accept_mask,
+              float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
+  const int R = B * gamma;
+  int rc = check_chain_args(ctx, head_q, sched_q, R, cfg, z_q, x_T, eps);
+  if (rc) return rc;
+  if ((rc = check_chain_args(ctx, head_p, sched_p, R, cfg, z_p, x_T, eps))) return rc;
+  if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
+  if (head_q->d.C != head_p->d.C) return fail(ctx, CSD_ERR_SHAPE, "draft C = %d and target C = %d differ", head_q->d.C, head_p->d.C);
+  const int C = head_p->d.C;
+  if ((rc = check_verify_dims(ctx, B, gamma, C))) return rc;
+  if (cap < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cap = %d must be >= 1", cap);
+  if (!u || !xi || !v || !x0 || !mu1_q || !mu1_p || !logratio || !n_accept || !x_new || !n_prop || !flags || !cap_hits)
+    return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  // workspaces first (growing one synchronises), then fork the two chains
+  if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T))) return rc;
+  CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
+  for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
+  rc = run_chain(ctx, 0, ctx->side[0], head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr);
+  int rc2 = run_chain(ctx, 1, ctx->side[1], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr);
+  for (int i = 0; i < 2; ++i) {
+    CSD_CUDA(ctx, cudaEventRecord(ctx->ev_done[i], ctx->side[i]));
+    CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_done[i], 0));
+  }
+  if (rc) return rc;
+  if (rc2) return rc2;
+  const double ls = log_sigma_term(sched_q, sched_p, C);
+  rc = accept_scan(ctx, ctx->stream, B, gamma, C, ls, sched_p->sigma[0], sched_q->sigma[0], x0, mu1_q, mu1_p, u, logratio,
+                   n_accept, accept_mask);
+  if (rc) return rc;
+  return resample(ctx, ctx->stream, B, gamma, C, cap, ls, sched_p->sigma[0], sched_q->sigma[0], n_accept, mu1_p, mu1_q, xi,
+                  v, x_new, n_prop, flags, cap_hits);
+}
+
+int csd_round_host(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule* sched_q,
+                   const csd_schedule* sched_p, int B, int gamma, int cfg, float cfg_scale, int cap, const float* z_q,
+                   const float* z_p, const float* x_T, const float* eps, const float* u, const float* xi,
+                   const float* v, float* x0, float* mu1_q, float* mu1_p, float* logratio, int32_t* n_accept,
+                   uint32_t* accept_mask, float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (!head_q || !head_p || !sched_q || !sched_p) return fail(ctx, CSD_ERR_INVALID_ARG, "head / schedule is null");
+  if (B < 1 || gamma < 1 || cap < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B, gamma, cap must be >= 1");
+  if (!z_q || !z_p || !x_T || !eps || !u || !xi || !v || !x0 || !mu1_q || !mu1_p || !logratio || !n_accept || !x_new ||
+      !n_prop || !flags || !cap_hits)
+    return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  if (sched_q->T < 1 || sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "schedules disagree on T");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  const size_t R = static_cast<size_t>(B) * gamma, Rh = R * (cfg ? 2 : 1), C = head_p->d.C, T = sched_p->T;
+  struct Item { const void* src; void* dst; size_t bytes; size_t off; bool in; };
+  Item items[] = {
+      {z_q, nullptr, Rh * head_q->d.Dz * 4, 0, true}, {z_p, nullptr, Rh * head_p->d.Dz * 4, 0, true},
+      {x_T, nullptr, R * C * 4, 0, true},             {eps, nullptr, T * R * C * 4, 0, true},
+      {u, nullptr, R * 4, 0, true},                   {xi, nullptr, static_cast<size_t>(B) * cap * C * 4, 0, true},
+      {v, nullptr, static_cast<size_t>(B) * cap * 4, 0, true},
+      {nullptr, x0, R * C * 4, 0, false},             {nullptr, mu1_q, R * C * 4, 0, false},
+      {nullptr, mu1_p, R * C * 4, 0, false},          {nullptr, logratio, R * 4, 0, false},
+      {nullptr, n_accept, static_cast<size_t>(B) * 4, 0, false},
+      {nullptr, accept_mask, static_cast<size_t>(B) * 4, 0, false},
+      {nullptr, x_new, static_cast<size_t>(B) * C * 4, 0, false},
+      {nullptr, n_prop, static_cast<size_t>(B) * 4, 0, false}, {nullptr, flags, static_cast<size_t>(B) * 4, 0, false},
+      {nullptr, cap_hits, 4, 0, false}};
+  size_t total = 0;
+  for (Item& it : items) { it.off = total; total = align_up(total + it.bytes, 256); }
+  if (total > ctx->io.cap) {
+    CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (ctx->io.base) CSD_CUDA(ctx, cudaFree(ctx->io.base));
+    ctx->io.base = nullptr; ctx->io.cap = 0;
+    if (cudaMalloc(&ctx->io.base, total) != cudaSuccess) { cudaGetLastError(); return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes for the host-call mirrors", total); }
+    ctx->io.cap = total;
+  }
+  char* base = static_cast<char*>(ctx->io.base);
+  auto dp = [&](int i) { return base + items[i].off; };
+  for (int i = 0; i < 7; ++i) CSD_CUDA(ctx, cudaMemcpyAsync(dp(i), items[i].src, items[i].bytes, cudaMemcpyHostToDevice, ctx->stream));
+  CSD_CUDA(ctx, cudaMemsetAsync(dp(13), 0, items[13].bytes, ctx->stream));  // x_new: rows that are not resampled read 0
+  int rc = csd_round(ctx, head_q, head_p, sched_q, sched_p, B, gamma, cfg, cfg_scale, cap, (const float*)dp(0),
+                     (const float*)dp(1), (const float*)dp(2), (const float*)dp(3), (const float*)dp(4),
+                     (const float*)dp(5), (const float*)dp(6), (float*)dp(7), (float*)dp(8), (float*)dp(9), (float*)dp(10),
+                     (int32_t*)dp(11), (uint32_t*)dp(12), (float*)dp(13), (int32_t*)dp(14), (uint32_t*)dp(15),
+                     (int32_t*)dp(16));
+  if (rc) return rc;
+  for (int i = 7; i < 17; ++i)
+    if (items[i].dst) CSD_CUDA(ctx, cudaMemcpyAsync(items[i].dst, dp(i), items[i].bytes, cudaMemcpyDeviceToHost, ctx->stream));
+  return csd_sync(ctx);
+}
+
+}  // extern "C"

@@ -1,0 +1,192 @@
+// Fused epilogues of the head's GEMMs.  One thread owns one output row and walks its 128-column
+// output tile in chunks of 32 columns; the same code serves the tcgen05 kernel (chunks read from
+// TMEM) and the fp32 FMA kernel (chunks held in registers).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace csd {
+
+constexpr int kTileM = 128;   // rows per tensor-core tile
+constexpr int kTileN = 128;   // output columns per tile
+constexpr int kChunk = 32;    // columns per epilogue chunk and per LayerNorm partial
+constexpr int kCPad = 16;     // token dim is padded to 16 in Wout^T and the eps partials
+
+enum Epi : int {
+  EPI_BIAS_F32 = 0,  // out_f32 = acc0 + bias0                                   (condition projection)
+  EPI_SILU_ACT = 1,  // out_act = SiLU(acc0 + bias0)                             (block MLP, first layer)
+  EPI_MOD = 2,       // out_act = LN(h)(1 + acc1 + bias1) + acc0 + bias0         (AdaLN modulate)
+  EPI_GATE_RES = 3,  // h += (acc1 + bias1) * (acc0 + bias0); LayerNorm partials (second layer + gate)
+  EPI_MODF = 4       // eps partial = Wout^T-tile . [LN(h)(1 + acc1 + bias1) + acc0 + bias0]
+};
+
+struct EpiParams {
+  int M;                 // valid rows
+  int ldo;               // leading dimension (elements) of out / h  (= W or N)
+  const float* bias0;    // [N]
+  const float* bias1;    // [N]
+  float* out_f32;        // EPI_BIAS_F32
+  void* out_act;         // EPI_SILU_ACT, EPI_MOD
+  float* h;              // EPI_MOD / EPI_MODF (read), EPI_GATE_RES (read-modify-write)
+  float* stats;          // [M, ldo/32, 2] (mean, M2) per 32-column group of h
+  const float* wout_t;   // [N, 16] fp32, Wout transposed and zero padded (EPI_MODF)
+  float* epart;          // [M, N/128, 16] (EPI_MODF)
+};
+
+__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
+
+template <typename T> __device__ __forceinline__ T to_act(float v);
+template <> __device__ __forceinline__ float to_act<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 to_act<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ __half to_act<__half>(float v) { return __float2half_rn(v); }
+
+template <typename T> __device__ __forceinline__ void store_chunk(T* dst, const float* v);
+template <> __device__ __forceinline__ void store_chunk<float>(float* dst, const float* v) {
+  float4* d = reinterpret_cast<float4*>(dst);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) d[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+}
+template <> __device__ __forceinline__ void store_chunk<__nv_bfloat16>(__nv_bfloat16* dst, const float* v) {
+  uint4* d = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    __nv_bfloat162 p0 = __floats2bfloat162_rn(v[8 * j + 0], v[8 * j + 1]);
+    __nv_bfloat162 p1 = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+    __nv_bfloat162 p2 = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
+    __nv_bfloat162 p3 = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+    uint4 q;
+    q.x = *reinterpret_cast<uint32_t*>(&p0); q.y = *reinterpret_cast<uint32_t*>(&p1);
+    q.z = *reinterpret_cast<uint32_t*>(&p2); q.w = *reinterpret_cast<uint32_t*>(&p3);
+    d[j] = q;
+  }
+}
+
+template <> __device__ __forceinline__ void store_chunk<__half>(__half* dst, const float* v) {
+  uint4* d = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    __half2 p0 = __floats2half2_rn(v[8 * j + 0], v[8 * j + 1]);
+    __half2 p1 = __floats2half2_rn(v[8 * j + 2], v[8 * j + 3]);
+    __half2 p2 = __floats2half2_rn(v[8 * j + 4], v[8 * j + 5]);
+    __half2 p3 = __floats2half2_rn(v[8 * j + 6], v[8 * j + 7]);
+    uint4 q;
+    q.x = *reinterpret_cast<uint32_t*>(&p0); q.y = *reinterpret_cast<uint32_t*>(&p1);
+    q.z = *reinterpret_cast<uint32_t*>(&p2); q.w = *reinterpret_cast<uint32_t*>(&p3);
+    d[j] = q;
+  }
+}
+
+__device__ __forceinline__ void load_chunk_f32(const float* src, float* v) {
+  const float4* s = reinterpret_cast<const float4*>(src);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    float4 q = s[j];
+    v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+  }
+}
+
+// Per-row state carried across the chunks of one tile.
+struct RowState {
+  float mean, rstd;
+  float eacc[kCPad];
+};
+
+// Merge the per-32-column (mean, M2) partials of row m in a fixed order (Chan et al.), so the
+// LayerNorm statistics do not depend on which CTA computes them.
+__device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
+  const int G = W / kChunk;
+  const float2* p = reinterpret_cast<const float2*>(stats) + static_cast<size_t>(m) * G;
+  float2 a = p[0];
+  float na = static_cast<float>(kChunk);
+  for (int g = 1; g < G; ++g) {
+    const float2 b = p[g];
+    const float nb = static_cast<float>(kChunk);
+    const float n = na + nb;
+    const float d = b.x - a.x;
+    a.x += d * (nb / n);
+    a.y += b.y + d * d * (na * nb / n);
+    na = n;
+  }
+  mean = a.x;
+  rstd = 1.0f / sqrtf(a.y / static_cast<float>(W) + 1e-6f);
+}
+
+template <int EPI>
+__device__ __forceinline__ void epi_row_begin(const EpiParams& ep, int m, RowState& rs) {
+  if constexpr (EPI == EPI_MOD || EPI == EPI_MODF) row_stats(ep.stats, m, ep.ldo, rs.mean, rs.rstd);
+  if constexpr (EPI == EPI_MODF) {
+#pragma unroll
+    for (int c = 0; c < kCPad; ++c) rs.eacc[c] = 0.0f;
+  }
+}
+
+// a0 / a1: accumulator chunk (32 columns) of the first / second accumulator; n0 = first global
+// output column of the chunk; wout_s: this tile's [128][16] slice of Wout^T in shared memory.
+template <int EPI, typename ACT>
+__device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, int chunk, float* a0,
+                                          const float* a1, RowState& rs, const float* wout_s) {
+  const size_t off = static_cast<size_t>(m) * ep.ldo + n0;
+  if constexpr (EPI == EPI_BIAS_F32) {
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) a0[j] += __ldg(ep.bias0 + n0 + j);
+    store_chunk<float>(ep.out_f32 + off, a0);
+  } else if constexpr (EPI == EPI_SILU_ACT) {
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) a0[j] = silu_f(a0[j] + __ldg(ep.bias0 + n0 + j));
+    store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
+  } else if constexpr (EPI == EPI_MOD || EPI == EPI_MODF) {
+    float hv[kChunk];
+    load_chunk_f32(ep.h + off, hv);
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) {
+      const float shift = a0[j] + __ldg(ep.bias0 + n0 + j);
+      const float scale = a1[j] + __ldg(ep.bias1 + n0 + j);
+      a0[j] = (hv[j] - rs.mean) * rs.rstd * (1.0f + scale) + shift;
+    }
+    if constexpr (EPI == EPI_MOD) {
+      store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
+    } else {
+      const float* w = wout_s + chunk * kChunk * kCPad;
+#pragma unroll
+      for (int j = 0; j < kChunk; ++j) {
+#pragma unroll
+        for (int c = 0; c < kCPad; ++c) rs.eacc[c] = fmaf(a0[j], w[j * kCPad + c], rs.eacc[c]);
+      }
+    }
+  } else if constexpr (EPI == EPI_GATE_RES) {
+    float hv[kChunk];
+    load_chunk_f32(ep.h + off, hv);
+    float sum = 0.0f;
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) {
+      const float y = a0[j] + __ldg(ep.bias0 + n0 + j);
+      const float g = a1[j] + __ldg(ep.bias1 + n0 + j);
+      hv[j] = fmaf(g, y, hv[j]);
+      sum += hv[j];
+    }
+    store_chunk<float>(ep.h + off, hv);
+    const float mean = sum * (1.0f / kChunk);
+    float m2 = 0.0f;
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) {
+      const float d = hv[j] - mean;
+      m2 = fmaf(d, d, m2);
+    }
+    reinterpret_cast<float2*>(ep.stats)[static_cast<size_t>(m) * (ep.ldo / kChunk) + n0 / kChunk] =
+        make_float2(mean, m2);
+  }
+}
+
+template <int EPI>
+__device__ __forceinline__ void epi_row_end(const EpiParams& ep, int m, int tile_n, const RowState& rs) {
+  if constexpr (EPI == EPI_MODF) {
+    float4* d = reinterpret_cast<float4*>(ep.epart + (static_cast<size_t>(m) * (ep.ldo / kTileN) + tile_n) * kCPad);
+#pragma unroll
+    for (int c = 0; c < kCPad / 4; ++c)
+      d[c] = make_float4(rs.eacc[4 * c], rs.eacc[4 * c + 1], rs.eacc[4 * c + 2], rs.eacc[4 * c + 3]);
+  }
+}
+
+}  // namespace csd

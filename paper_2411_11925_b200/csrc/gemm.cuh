@@ -1,0 +1,235 @@
+// GEMM kernels of the head: out-tile[128 x 128] = epilogue(A[M,K] * B[N,K]^T ...).
+//   gemm_tc_kernel   : bf16 operands on tcgen05 tensor cores, TMA-fed shared-memory ring,
+//                      fp32 accumulators in TMEM, warp-specialised (TMA / MMA / 4 epilogue warps).
+//   gemm_simt_kernel : fp32 operands on plain FMA units (CSD_F32 heads).
+// Accumulator layout (both kernels), by template parameters:
+//   NSEG=1, MMA_N=128 : acc0 = A0 * B0[tile rows]^T
+//   NSEG=1, MMA_N=256 : B0 is packed so that rows [256 j, 256 j+128) and [256 j+128, 256 j+256) are
+//                       the two weight slices that pair up column by column (AdaLN shift | scale):
+//                       acc0 = first half, acc1 = second half, one shared A.
+//   NSEG=2, MMA_N=128 : acc0 = A0 * B0^T, acc1 = A1 * B1^T (second MLP layer | AdaLN gate).
+#pragma once
+#include "epilogue.cuh"
+#include "ptx.cuh"
+
+namespace csd {
+
+constexpr int kBlockK = 64;  // bf16 elements per TMA box row = 128 bytes = one swizzle row
+constexpr int kTcThreads = 192;
+
+enum DevErr : int { DEV_OK = 0, DEV_ERR_TMA_WAIT = 1, DEV_ERR_MMA_WAIT = 2, DEV_ERR_EPI_WAIT = 3 };
+
+template <int MMA_N> struct TcCfg {
+  static constexpr int kStages = (MMA_N == 256) ? 4 : 6;
+  static constexpr int kABytes = kTileM * kBlockK * 2;
+  static constexpr int kBBytes = MMA_N * kBlockK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kWoutBytes = kTileN * kCPad * 4;
+  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kWoutBytes + 256;
+};
+
+template <int EPI, typename ACT, int NSEG, int MMA_N, int AB_FMT>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+               const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
+               int nkb0, int nkb1, EpiParams ep, int* err) {
+  using Cfg = TcCfg<MMA_N>;
+  constexpr int S = Cfg::kStages;
+  constexpr uint32_t kTmemCols = NSEG * MMA_N;  // 128 or 256: a power of two >= 32
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* stage_base = smem;
+  float* wout_s = reinterpret_cast<float*>(smem + S * Cfg::kStageBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStageBytes + Cfg::kWoutBytes);
+  uint64_t* empty_bar = full_bar + S;
+  uint64_t* tmem_full_bar = empty_bar + S;
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_full_bar + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile_n = blockIdx.x, tile_m = blockIdx.y;
+  const int total_kb = nkb0 + (NSEG == 2 ? nkb1 : 0);
+
+  // Once any kernel of this context has raised the error flag, later launches return at once
+  // (block-uniform decision) so that a failure costs one bounded wait, not one per launch.
+  __shared__ int s_abort;
+  if (threadIdx.x == 0) s_abort = *reinterpret_cast<volatile int*>(err);
+  __syncthreads();
+  if (s_abort != 0) return;
+
+  if (warp == 0 && lane == 0) {
+    tma_prefetch_desc(&tmA0);
+    tma_prefetch_desc(&tmB0);
+    if (NSEG == 2) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
+    for (int s = 0; s < S; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(tmem_full_bar, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_base_s, kTmemCols);
+    tmem_relinquish();
+  }
+  if (EPI == EPI_MODF && warp >= 2) {
+    const float* src = ep.wout_t + static_cast<size_t>(tile_n) * kTileN * kCPad;
+    for (int i = threadIdx.x - 64; i < kTileN * kCPad; i += kTcThreads - 64) wout_s[i] = src[i];
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_base_s;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kb = 0; kb < total_kb; ++kb) {
+        const int s = kb % S;
+        const uint32_t ph = (kb / S) & 1;
+        if (!mbar_wait(&empty_bar[s], ph ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); break; }
+        mbar_arrive_expect_tx(&full_bar[s], Cfg::kStageBytes);
+        const bool second = (NSEG == 2) && (kb >= nkb0);
+        const int kk = second ? kb - nkb0 : kb;
+        uint8_t* sa = stage_base + s * Cfg::kStageBytes;
+        tma_load_2d(sa, second ? &tmA1 : &tmA0, &full_bar[s], kk * kBlockK, tile_m * kTileM);
+        tma_load_2d(sa + Cfg::kABytes, second ? &tmB1 : &tmB0, &full_bar[s], kk * kBlockK, tile_n * MMA_N);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_f16(MMA_N, AB_FMT);
+      bool ok = true;
+      for (int kb = 0; kb < total_kb; ++kb) {
+        const int s = kb % S;
+        const uint32_t ph = (kb / S) & 1;
+        if (!mbar_wait(&full_bar[s], ph)) { atomicExch(err, DEV_ERR_MMA_WAIT); ok = false; break; }
+        tc_fence_after_sync();
+        const bool second = (NSEG == 2) && (kb >= nkb0);
+        const int kk = second ? kb - nkb0 : kb;
+        const uint32_t sa = smem_u32(stage_base + s * Cfg::kStageBytes);
+        const uint64_t da = umma_smem_desc_sw128(sa);
+        const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes);
+        const uint32_t d = tmem_base + (second ? MMA_N : 0);
+#pragma unroll
+        for (int k = 0; k < kBlockK / 16; ++k)  // UMMA_K = 16 bf16 = 32 bytes = 2 descriptor units
+          umma_f16(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
+        umma_commit(&empty_bar[s]);
+      }
+      if (ok) umma_commit(tmem_full_bar);
+    }
+    __syncwarp();
+  } else {
+    // Epilogue: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32).
+    const int q = warp & 3;
+    const int m = tile_m * kTileM + q * 32 + lane;
+    const bool valid = m < ep.M;
+    bool ok = mbar_wait(tmem_full_bar, 0);
+    if (!ok) atomicExch(err, DEV_ERR_EPI_WAIT);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after_sync();
+      RowState rs;
+      if (valid) epi_row_begin<EPI>(ep, m, rs);
+      const uint32_t trow = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < kTileN / kChunk; ++c) {
+        float a0[kChunk], a1[kChunk];
+        tmem_ld32(trow + c * kChunk, a0);
+        if (NSEG * MMA_N == 256) tmem_ld32(trow + kTileN + c * kChunk, a1);
+        tmem_ld_wait();
+        if (valid) epi_chunk<EPI, ACT>(ep, m, tile_n * kTileN + c * kChunk, c, a0, a1, rs, wout_s);
+      }
+      if (valid) epi_row_end<EPI>(ep, m, tile_n, rs);
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ------------------------------------------------------------------ fp32 FMA path
+constexpr int kSimtRows = 32;
+constexpr int kSimtBK = 32;
+
+template <int EPI, int NSEG, int MMA_N>
+__global__ void __launch_bounds__(128)
+gemm_simt_kernel(const float* __restrict__ A0, int lda0, const float* __restrict__ B0, int ldb0, int K0,
+                 const float* __restrict__ A1, int lda1, const float* __restrict__ B1, int ldb1, int K1,
+                 EpiParams ep) {
+  __shared__ float As[kSimtRows][kSimtBK + 1];
+  __shared__ float Bs[MMA_N][kSimtBK + 1];
+  __shared__ float wout_s[(EPI == EPI_MODF) ? kTileN * kCPad : 1];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int tile_n = blockIdx.x, m0 = blockIdx.y * kSimtRows;
+  const int m = m0 + lane;
+  if (EPI == EPI_MODF) {
+    const float* src = ep.wout_t + static_cast<size_t>(tile_n) * kTileN * kCPad;
+    for (int i = threadIdx.x; i < kTileN * kCPad; i += 128) wout_s[i] = src[i];
+  }
+  float acc0[kChunk], acc1[kChunk];
+#pragma unroll
+  for (int j = 0; j < kChunk; ++j) { acc0[j] = 0.0f; acc1[j] = 0.0f; }
+#pragma unroll 1
+  for (int seg = 0; seg < NSEG; ++seg) {
+    const float* A = seg ? A1 : A0;
+    const float* B = seg ? B1 : B0;
+    const int lda = seg ? lda1 : lda0, ldb = seg ? ldb1 : ldb0, K = seg ? K1 : K0;
+    const int brow0 = tile_n * MMA_N;
+#pragma unroll 1
+    for (int k0 = 0; k0 < K; k0 += kSimtBK) {
+      for (int i = threadIdx.x; i < kSimtRows * kSimtBK; i += 128) {
+        const int r = i / kSimtBK, c = i % kSimtBK;
+        As[r][c] = (m0 + r < ep.M) ? A[static_cast<size_t>(m0 + r) * lda + k0 + c] : 0.0f;
+      }
+      for (int i = threadIdx.x; i < MMA_N * kSimtBK; i += 128) {
+        const int r = i / kSimtBK, c = i % kSimtBK;
+        Bs[r][c] = B[static_cast<size_t>(brow0 + r) * ldb + k0 + c];
+      }
+      __syncthreads();
+#pragma unroll 4
+      for (int k = 0; k < kSimtBK; ++k) {
+        const float a = As[lane][k];
+        if constexpr (MMA_N == 256) {
+#pragma unroll
+          for (int j = 0; j < kChunk; ++j) {
+            acc0[j] = fmaf(a, Bs[warp * kChunk + j][k], acc0[j]);
+            acc1[j] = fmaf(a, Bs[128 + warp * kChunk + j][k], acc1[j]);
+          }
+        } else {
+          if (seg == 0) {
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) acc0[j] = fmaf(a, Bs[warp * kChunk + j][k], acc0[j]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) acc1[j] = fmaf(a, Bs[warp * kChunk + j][k], acc1[j]);
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  // This thread owns chunk `warp` of the tile only; EPI_MODF partials are therefore per chunk
+  // and summed below through shared memory in chunk order.
+  RowState rs;
+  if (m < ep.M) {
+    epi_row_begin<EPI>(ep, m, rs);
+    epi_chunk<EPI, float>(ep, m, tile_n * kTileN + warp * kChunk, warp, acc0, acc1, rs, wout_s);
+  }
+  if constexpr (EPI == EPI_MODF) {
+    float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][16]
+    __syncthreads();
+    if (m < ep.M) {
+#pragma unroll
+      for (int c = 0; c < kCPad; ++c) scr[(warp * kSimtRows + lane) * kCPad + c] = rs.eacc[c];
+    }
+    __syncthreads();
+    if (warp == 0 && m < ep.M) {
+#pragma unroll
+      for (int c = 0; c < kCPad; ++c) {
+        float v = 0.0f;
+        for (int w = 0; w < 4; ++w) v += scr[(w * kSimtRows + lane) * kCPad + c];
+        rs.eacc[c] = v;
+      }
+      epi_row_end<EPI>(ep, m, tile_n, rs);
+    }
+  }
+}
+
+}  // namespace csd

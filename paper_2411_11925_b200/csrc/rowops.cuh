@@ -1,0 +1,228 @@
+// Row-parallel kernels around the GEMM chain: timestep embedding, the per-step boundary kernel
+// (eps_hat reduction, classifier-free guidance, DDPM update, input projection, LayerNorm partials,
+// condition vector s), and the verification / resampling kernels.
+#pragma once
+#include "epilogue.cuh"
+
+namespace csd {
+
+// te[t, n] = Wt2[n, :] . SiLU(Wt1 tfeat_t + bt1) + bt2[n]   (one block per timestep)
+__global__ void __launch_bounds__(256)
+timestep_embed_kernel(const float* __restrict__ tfeat, const float* __restrict__ Wt1,
+                      const float* __restrict__ bt1, const float* __restrict__ Wt2,
+                      const float* __restrict__ bt2, int W, int F, float* __restrict__ te) {
+  extern __shared__ float sm[];  // tf[F] | hid[W]
+  float* tf = sm;
+  float* hid = sm + F;
+  const int t = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  for (int i = threadIdx.x; i < F; i += blockDim.x) tf[i] = tfeat[static_cast<size_t>(t) * F + i];
+  __syncthreads();
+  for (int n = warp; n < W; n += nwarp) {
+    float acc = 0.0f;
+    for (int k = lane; k < F; k += 32) acc = fmaf(Wt1[static_cast<size_t>(n) * F + k], tf[k], acc);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) hid[n] = silu_f(acc + bt1[n]);
+  }
+  __syncthreads();
+  for (int n = warp; n < W; n += nwarp) {
+    float acc = 0.0f;
+    for (int k = lane; k < W; k += 32) acc = fmaf(Wt2[static_cast<size_t>(n) * W + k], hid[k], acc);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) te[static_cast<size_t>(t) * W + n] = acc + bt2[n];
+  }
+}
+
+template <typename ACT>
+__global__ void convert_act_kernel(const float* __restrict__ src, ACT* __restrict__ dst, size_t n) {
+  const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = to_act<ACT>(src[i]);
+}
+
+enum StepMode : int { STEP_INIT = 0, STEP_MID = 1, STEP_LAST = 2 };
+
+struct StepParams {
+  int R, cfg, C, W, NT;          // token rows, guidance flag, token dim, width, W/128
+  float cfg_scale, a, b, sigma;  // coefficients of the step being finished (t)
+  int sample_last;               // STEP_LAST: also draw x0 = mu1 + sigma eps
+  const float* epart;            // [Rh, NT, 16] eps_hat partial sums of step t
+  const float* bout;             // [16] (zero padded)
+  const float* eps_t;            // [R, C] noise of step t
+  const float* x_src;            // STEP_INIT: x_T
+  float* x;                      // [R, C] current state (in/out)
+  float *x0, *mu1, *x1;          // STEP_LAST outputs (x0, x1 may be null)
+  const float* win;              // [W, 16] (zero padded), bin [W]
+  const float* bin;
+  const float* cz;               // [Rh, W]
+  const float* te_next;          // [W] embedding of the step being prepared
+  float* h;                      // [Rh, W]
+  float* stats;                  // [Rh, W/32, 2]
+  void* s;                       // [Rh, W] activations
+};
+
+// One block per token row.  Finishes step t (unless STEP_INIT) and prepares the next one:
+//   eps_hat = sum of tile partials + bout; guidance; mu = a x - b eps_hat; x <- mu + sigma eps_t
+//   h = Win x + bin (same for both guidance rows), LayerNorm partials per 32 columns,
+//   s = SiLU(cz + te_next).
+template <typename ACT>
+__global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
+  __shared__ float xs[kCPad];
+  __shared__ float eh[2][kCPad];
+  const int r = blockIdx.x, tid = threadIdx.x;
+  const int nrep = p.cfg ? 2 : 1;
+  if (mode == STEP_INIT) {
+    if (tid < kCPad) xs[tid] = (tid < p.C) ? p.x_src[static_cast<size_t>(r) * p.C + tid] : 0.0f;
+    if (tid < p.C) p.x[static_cast<size_t>(r) * p.C + tid] = p.x_src[static_cast<size_t>(r) * p.C + tid];
+    __syncthreads();
+  } else {
+    if (tid < nrep * kCPad) {
+      const int rep = tid / kCPad, c = tid % kCPad;
+      const float* e = p.epart + (static_cast<size_t>(r + rep * p.R) * p.NT) * kCPad + c;
+      float acc = 0.0f;
+      for (int nt = 0; nt < p.NT; ++nt) acc += e[nt * kCPad];
+      eh[rep][c] = acc + p.bout[c];
+    }
+    __syncthreads();
+    if (tid < kCPad) {
+      float xn = 0.0f;
+      if (tid < p.C) {
+        const size_t o = static_cast<size_t>(r) * p.C + tid;
+        float e = eh[0][tid];
+        if (p.cfg) e = eh[1][tid] + p.cfg_scale * (eh[0][tid] - eh[1][tid]);
+        const float xo = p.x[o];
+        const float mu = p.a * xo - p.b * e;
+        xn = mu + p.sigma * p.eps_t[o];
+        if (mode == STEP_LAST) {
+          p.mu1[o] = mu;
+          if (p.x1) p.x1[o] = xo;
+          if (p.sample_last && p.x0) p.x0[o] = xn;
+        } else {
+          p.x[o] = xn;
+        }
+      }
+      xs[tid] = xn;
+    }
+    if (mode == STEP_LAST) return;
+    __syncthreads();
+  }
+  // prepare: each warp handles 32 consecutive columns at a time (lane = column)
+  const int lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
+  ACT* s = reinterpret_cast<ACT*>(p.s);
+  for (int g = warp; g < p.W / kChunk; g += nwarp) {
+    const int n = g * kChunk + lane;
+    const float4* w4 = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(n) * kCPad);
+    float acc = p.bin[n];
+#pragma unroll
+    for (int c4 = 0; c4 < kCPad / 4; ++c4) {
+      const float4 w = w4[c4];
+      acc = fmaf(w.x, xs[4 * c4], acc); acc = fmaf(w.y, xs[4 * c4 + 1], acc);
+      acc = fmaf(w.z, xs[4 * c4 + 2], acc); acc = fmaf(w.w, xs[4 * c4 + 3], acc);
+    }
+    float sum = acc;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float mean = sum * (1.0f / kChunk);
+    const float d = acc - mean;
+    float m2 = d * d;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
+    const float te = p.te_next[n];
+    for (int rep = 0; rep < nrep; ++rep) {
+      const size_t row = static_cast<size_t>(r) + static_cast<size_t>(rep) * p.R;
+      p.h[row * p.W + n] = acc;
+      if (lane == 0)
+        reinterpret_cast<float2*>(p.stats)[row * (p.W / kChunk) + g] = make_float2(mean, m2);
+      s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + te));
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Verification: one warp per sequence, lane i = draft position i (gamma <= 32).
+//   logratio = log_sigma + C (log sq1 - log sp1) - |x0 - mu_p|^2 / (2 sp1^2) + |x0 - mu_q|^2 / (2 sq1^2)
+//   accept iff log u <= logratio;  n_accept = number of leading accepts (ballot + find-first-set).
+__global__ void __launch_bounds__(128)
+accept_scan_kernel(int B, int gamma, int C, float log_const, float inv2vp, float inv2vq,
+                   const float* __restrict__ x0, const float* __restrict__ mu_q,
+                   const float* __restrict__ mu_p, const float* __restrict__ u,
+                   float* __restrict__ logratio, int32_t* __restrict__ n_accept,
+                   uint32_t* __restrict__ accept_mask) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  bool acc = true;  // lanes beyond gamma do not reject
+  if (lane < gamma) {
+    const size_t row = static_cast<size_t>(b) * gamma + lane;
+    float dp = 0.0f, dq = 0.0f;
+    for (int c = 0; c < C; ++c) {
+      const float x = x0[row * C + c];
+      const float ep = x - mu_p[row * C + c];
+      const float eq = x - mu_q[row * C + c];
+      dp = fmaf(ep, ep, dp);
+      dq = fmaf(eq, eq, dq);
+    }
+    // Both products are rounded separately (no FMA contraction), so that identical draft and target
+    // means give a difference of exactly zero.
+    const float lr = log_const + __fsub_rn(__fmul_rn(dq, inv2vq), __fmul_rn(dp, inv2vp));
+    logratio[row] = lr;
+    acc = logf(u[row]) <= lr;
+  }
+  const uint32_t ballot = __ballot_sync(0xffffffffu, acc);
+  if (lane == 0) {
+    const uint32_t rej = ~ballot;
+    int n = rej ? (__ffs(rej) - 1) : gamma;
+    if (n > gamma) n = gamma;
+    n_accept[b] = n;
+    if (accept_mask) accept_mask[b] = (gamma >= 32) ? ballot : (ballot & ((1u << gamma) - 1u));
+  }
+}
+
+// Resampling: one warp per sequence, lane c < C = coordinate.  Proposals are consumed in order.
+__global__ void __launch_bounds__(128)
+resample_kernel(int B, int gamma, int C, int cap, float log_sigma, float sp1, float sq1,
+                float log_sp1, float log_sq1, const int32_t* __restrict__ n_accept,
+                const float* __restrict__ mu_p, const float* __restrict__ mu_q,
+                const float* __restrict__ xi, const float* __restrict__ v,
+                float* __restrict__ x_new, int32_t* __restrict__ n_prop,
+                uint32_t* __restrict__ flags, int32_t* __restrict__ cap_hits) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  const int n = n_accept[b];
+  if (n >= gamma) {
+    if (lane == 0) { n_prop[b] = 0; flags[b] = 0u; }
+    return;
+  }
+  const size_t row = static_cast<size_t>(b) * gamma + n;
+  const float mp = (lane < C) ? mu_p[row * C + lane] : 0.0f;
+  const float mq = (lane < C) ? mu_q[row * C + lane] : 0.0f;
+  const float inv2vp = 0.5f / (sp1 * sp1), inv2vq = 0.5f / (sq1 * sq1);
+  float xp = 0.0f;
+  int k = 0;
+  bool done = false;
+  for (; k < cap && !done; ++k) {
+    const float z = (lane < C) ? xi[(static_cast<size_t>(b) * cap + k) * C + lane] : 0.0f;
+    xp = mp + sp1 * z;
+    float ep = (lane < C) ? (xp - mp) : 0.0f;
+    float eq = (lane < C) ? (xp - mq) : 0.0f;
+    ep *= ep; eq *= eq;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      ep += __shfl_xor_sync(0xffffffffu, ep, o);
+      eq += __shfl_xor_sync(0xffffffffu, eq, o);
+    }
+    const float lp = -C * log_sp1 - ep * inv2vp;
+    const float lq = -C * log_sq1 - eq * inv2vq;
+    const float alpha = fmaxf(0.0f, -expm1f(fminf(0.0f, lq - log_sigma - lp)));
+    done = v[static_cast<size_t>(b) * cap + k] <= alpha;
+  }
+  if (lane < C) x_new[static_cast<size_t>(b) * C + lane] = xp;
+  if (lane == 0) {
+    n_prop[b] = k;
+    flags[b] = 1u | (done ? 0u : 2u);
+    if (!done) atomicAdd(cap_hits, 1);
+  }
+}
+
+}  // namespace csd

@@ -79,6 +79,13 @@ class Workload:
     tokens: int = 256
     prefill: int = 0
     perturb_std: float = 0.0   # >0: draft = target weights + N(0, std^2)
+    operand: str = ""          # GEMM operand format: "f32" | "bf16" | "f16"; "" = "f16" if bf16 else "f32"
+
+    @property
+    def operand_format(self) -> str:
+        """bf16=True means the weight and z VALUES are bf16-representable; by default such a
+        workload runs with fp16 tensor-core operands (those values are exact in fp16)."""
+        return self.operand or ("f16" if self.bf16 else "f32")
 
     @property
     def R(self) -> int:

@@ -1,0 +1,220 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 checker on the
+same seeded inputs (element by element at sizes the checker finishes in seconds; sampled
+sequences at the full benchmark size)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import csd_oracle as orc
+from paper_2411_11925_b200 import inputs as gen
+
+from _parity import compare_round
+
+pytestmark = pytest.mark.gpu
+
+
+def _wl(base="tiny_fp32", **kw):
+    return gen.Workload(**{**gen.WORKLOADS[base].__dict__, **kw})
+
+
+def _run(inp, fused=False, **kw):
+    from paper_2411_11925_b200.runner import DeviceRound
+    dr = DeviceRound(inp, **kw)
+    dr.fused_round() if fused else dr.three_calls()
+    out = dr.results()
+    return dr, out
+
+
+def _ref(inp, tau_q=None, tau_p=None):
+    wl = inp.wl
+    sq = orc.ddpm_schedule(inp.beta, wl.tau if tau_q is None else tau_q)
+    sp = orc.ddpm_schedule(inp.beta, wl.tau if tau_p is None else tau_p)
+    eq = orc.make_mlp_head(inp.w_q, inp.z_q, inp.tfeat, wl.cfg, wl.cfg_scale)
+    ep = orc.make_mlp_head(inp.w_p, inp.z_p, inp.tfeat, wl.cfg, wl.cfg_scale)
+    ref = orc.csd_round(eq, ep, sq, sp, inp.x_T, inp.eps, inp.u, inp.xi, inp.v, wl.B, wl.gamma, wl.cap)
+    return ref, sq["sigma"][0], sp["sigma"][0]
+
+
+def _check(inp, label, fused=False, tau_q=None, tau_p=None):
+    dr, out = _run(inp, fused=fused, tau_q=tau_q, tau_p=tau_p)
+    ref, s1q, s1p = _ref(inp, tau_q, tau_p)
+    st = compare_round(out, ref, inp.wl, s1q, s1p, inp.u, inp.v, label)
+    print(label, st)
+    dr.ctx.close()
+    return st, out, ref
+
+
+def test_tiny_fp32_workload_matches_checker():
+    inp = gen.make_round_inputs(gen.WORKLOADS["tiny_fp32"])
+    st, out, ref = _check(inp, "tiny_fp32")
+    np.testing.assert_allclose(out["x1_q"], ref["x1_q"], atol=1e-4)
+
+
+def test_fused_round_is_bit_identical_to_three_calls():
+    for base, kw in (("tiny_fp32", dict(B=3, cfg=True, cfg_scale=2.0)),
+                     ("tiny_fp32", dict(B=5, gamma=7, T=6, bf16=True, cfg=True, cfg_scale=3.0)),
+                     ("tiny_fp32", dict(B=5, gamma=7, T=6, bf16=True, operand="bf16", cfg=True, cfg_scale=3.0))):
+        inp = gen.make_round_inputs(_wl(base, **kw))
+        dr, a = _run(inp, fused=False)
+        dr.fused_round()
+        b = dr.results()
+        for k in ("x0", "mu1_q", "mu1_p", "logratio", "n_accept", "accept_mask", "x_new", "n_prop", "flags"):
+            np.testing.assert_array_equal(a[k], b[k], err_msg=k)
+        dr.ctx.close()
+
+
+OPERANDS = ["f32", "bf16", "f16"]
+
+
+@pytest.mark.parametrize("op", OPERANDS)
+def test_identical_heads_give_zero_logratio_and_accept_all(op):
+    wl = _wl(B=6, gamma=5, T=8, bf16=op != "f32", operand=op, cfg=True, cfg_scale=3.0, draft=gen.HeadSpec(2, 256, 256))
+    inp = gen.make_round_inputs(wl)
+    inp.w_q, inp.z_q = inp.w_p, inp.z_p
+    dr, out = _run(inp)
+    assert np.all(out["logratio"] == 0.0)
+    assert np.all(out["n_accept"] == wl.gamma) and np.all(out["flags"] == 0) and np.all(out["n_prop"] == 0)
+    np.testing.assert_array_equal(out["mu1_q"], out["mu1_p"])
+    dr.ctx.close()
+
+
+@pytest.mark.parametrize("op", OPERANDS)
+def test_ragged_rows_guidance_and_several_tiles(op):
+    # Rh = 2*B*gamma = 2*23*7 = 322 rows: three 128-row tensor-core tiles with a ragged tail (66 rows),
+    # eleven 32-row tiles on the fp32 path with a 2-row tail; W = 384 gives three column tiles.
+    wl = _wl(B=23, gamma=7, T=6, bf16=op != "f32", operand=op, cfg=True, cfg_scale=3.0,
+             draft=gen.HeadSpec(1, 256, 128), target=gen.HeadSpec(2, 384, 192))
+    _check(gen.make_round_inputs(wl), f"ragged {op}")
+
+
+@pytest.mark.parametrize("op", OPERANDS)
+def test_close_heads_exercise_accepts_rejects_and_resampling(op):
+    # draft = target + small perturbation: log-ratios are O(1), so accepts, rejects and multi-proposal
+    # resampling all occur and the 5e-2 tolerance is the binding one.
+    wl = _wl(B=48, gamma=8, T=10, bf16=op != "f32", operand=op, cfg=False, perturb_std=1e-4,
+             draft=gen.HeadSpec(2, 256, 256), target=gen.HeadSpec(2, 256, 256))
+    inp = gen.make_round_inputs(wl)
+    inp.z_q = inp.z_p                      # same condition vector: only the weights differ
+    st, out, ref = _check(inp, f"close heads {op}", fused=True)
+    assert 0.05 < st["accept_rate"] < 0.98, st
+    assert st["resampled"] >= 5 and st["n_prop_max"] >= 2, st
+
+
+def test_different_variances_exercise_the_sigma_term():
+    # tau_q != tau_p: Sigma of Eq. 7 is not 1 and sigma_q,1 != sigma_p,1 (general form of Eq. 8)
+    wl = _wl(B=16, gamma=4, T=10, perturb_std=1e-4, draft=gen.HeadSpec(2, 256, 256))
+    inp = gen.make_round_inputs(wl)
+    inp.z_q = inp.z_p
+    st, out, ref = _check(inp, "sigma term", tau_q=1.0, tau_p=0.97)
+    assert abs(ref["log_sigma"]) > 1.0
+
+
+def test_accept_scan_kernel_all_masks_and_edge_cases():
+    from paper_2411_11925_b200 import api
+    dev = torch.device("cuda", 0)
+    ctx = api.Context(0)
+    rng = np.random.default_rng(5)
+    for gamma in (1, 5, 8, 32):
+        B, C = (2 ** gamma if gamma <= 8 else 300), 16
+        R = B * gamma
+        x0 = rng.standard_normal((R, C)).astype(np.float32)
+        mu_q = (x0 + 0.01 * rng.standard_normal((R, C))).astype(np.float32)
+        mu_p = (x0 + 0.012 * rng.standard_normal((R, C))).astype(np.float32)
+        sp1, sq1, ls = 0.011, 0.01, 0.3
+        lr = orc.log_ratio_closed(x0.astype(np.float64), mu_q.astype(np.float64), mu_p.astype(np.float64), sq1, sp1, ls)
+        lr = lr.reshape(B, gamma)
+        if gamma <= 8:      # every accept mask once: u just below / above the ratio
+            bits = ((np.arange(B)[:, None] >> np.arange(gamma)[None, :]) & 1).astype(bool)
+            u = np.where(bits, np.exp(lr - 0.5), np.exp(lr + 0.5))
+            u = np.clip(u, 1e-30, None).astype(np.float32)
+        else:
+            u = rng.random((B, gamma)).astype(np.float32).clip(1e-7, 1)
+        t = lambda a: torch.from_numpy(a).to(dev)
+        d_lr = torch.zeros(B, gamma, device=dev); d_n = torch.zeros(B, dtype=torch.int32, device=dev)
+        d_m = torch.zeros(B, dtype=torch.int32, device=dev)
+        ctx.csd_accept_scan(B, gamma, C, ls, sp1, sq1, t(x0), t(mu_q), t(mu_p), t(u), d_lr, d_n, d_m)
+        ctx.sync()
+        g_lr = d_lr.cpu().numpy()
+        np.testing.assert_allclose(g_lr, lr, atol=2e-3 + 1e-5 * np.abs(lr).max())
+        n_ref, acc_ref = orc.accept_prefix(lr, u)
+        near = np.abs(lr - np.log(u.astype(np.float64))) < 5e-2
+        assert not near.any() or gamma > 8
+        ok_rows = ~near.any(axis=1)
+        np.testing.assert_array_equal(d_n.cpu().numpy()[ok_rows], n_ref[ok_rows])
+        gm = d_m.cpu().numpy().astype(np.int64) & 0xFFFFFFFF
+        accg = ((gm[:, None] >> np.arange(gamma)[None, :]) & 1).astype(bool)
+        np.testing.assert_array_equal(accg[ok_rows], acc_ref[ok_rows])
+    ctx.close()
+
+
+def test_resample_kernel_matches_checker_including_cap_hits():
+    from paper_2411_11925_b200 import api
+    dev = torch.device("cuda", 0)
+    ctx = api.Context(0)
+    rng = np.random.default_rng(6)
+    B, gamma, C, cap = 500, 6, 16, 8
+    R = B * gamma
+    mu_p = rng.standard_normal((R, C)).astype(np.float32)
+    mu_q = (mu_p + 0.002 * rng.standard_normal((R, C))).astype(np.float32)   # low acceptance -> cap hits
+    n_acc = rng.integers(0, gamma + 1, B).astype(np.int32)
+    xi = rng.standard_normal((B, cap, C)).astype(np.float32)
+    v = rng.random((B, cap)).astype(np.float32).clip(1e-7, 1 - 1e-7)
+    sp1, sq1, ls = 0.01, 0.0105, -0.2
+    ref = orc.resample(n_acc, mu_p.astype(np.float64), mu_q.astype(np.float64), sp1, sq1, ls, xi, v, gamma, cap)
+    t = lambda a: torch.from_numpy(a).to(dev)
+    x_new = torch.full((B, C), 7.0, device=dev)
+    n_prop = torch.zeros(B, dtype=torch.int32, device=dev); flags = torch.zeros(B, dtype=torch.int32, device=dev)
+    hits = torch.full((1,), 99, dtype=torch.int32, device=dev)
+    for _ in range(2):       # second call: the cap-hit counter must restart from zero
+        ctx.csd_resample(B, gamma, C, cap, ls, sp1, sq1, t(n_acc), t(mu_p), t(mu_q), t(xi), t(v), x_new, n_prop, flags, hits)
+    ctx.sync()
+    g_prop, g_flags, g_x = n_prop.cpu().numpy(), flags.cpu().numpy(), x_new.cpu().numpy()
+    same = g_prop == ref["n_prop"]
+    assert same.mean() > 0.97, same.mean()          # thresholds within rounding of v may flip a proposal
+    np.testing.assert_array_equal(g_flags[same], ref["flags"][same])
+    res = same & (n_acc < gamma)
+    np.testing.assert_allclose(g_x[res], ref["x_new"][res], atol=1e-6)
+    assert np.all(g_x[n_acc == gamma] == 7.0) and np.all(g_prop[n_acc == gamma] == 0)   # untouched
+    assert ref["cap_hits"] > 10 and abs(int(hits.item()) - ref["cap_hits"]) <= (~same).sum()
+    ctx.close()
+
+
+def test_argument_errors_are_reported_not_raised_by_the_device():
+    from paper_2411_11925_b200 import api
+    ctx = api.Context(0)
+    wl = _wl(B=2)
+    inp = gen.make_round_inputs(wl)
+    w_bad = dict(inp.w_p); w_bad["Wz"] = np.zeros((200, 256), np.float32)   # W = 200 not a multiple of 128
+    with pytest.raises(api.CsdError) as e:
+        api.Head(ctx, {**w_bad, "bz": np.zeros(200, np.float32)}, "f32")
+    assert e.value.code == -3
+    dev = torch.device("cuda", 0)
+    z = torch.zeros(4, device=dev)
+    with pytest.raises(api.CsdError) as e:
+        ctx.csd_accept_scan(2, 33, 16, 0.0, 0.01, 0.01, z, z, z, z, z, z.int())
+    assert e.value.code == -3 and "gamma" in str(e.value)
+    with pytest.raises(api.CsdError) as e:
+        ctx.csd_resample(2, 4, 16, 0, 0.0, 0.01, 0.01, z.int(), z, z, z, z, z, z.int(), z.int(), z.int())
+    assert e.value.code == -1
+    with pytest.raises(api.CsdError) as e:
+        ctx.csd_accept_scan(2, 4, 16, 0.0, 0.01, 0.01, None, z, z, z, z, z.int())
+    assert e.value.code == -1
+    ctx.sync()
+    ctx.close()
+
+
+def test_mar256_full_size_sampled_sequences():
+    # The benchmark's launch configuration (B=64, gamma=8, T=100, guidance, bf16) on the GPU; the checker
+    # evaluates four sequences: first, last and both sides of the 128-row tile boundary.
+    wl = gen.WORKLOADS["mar256"]
+    inp = gen.make_round_inputs(wl)
+    dr, out = _run(inp, fused=True)
+    seqs = [0, 15, 16, 63]
+    sub = gen.select_sequences(inp, seqs)
+    ref, s1q, s1p = _ref(sub)
+    rows = sub.extras["rows"]
+    gsub = {k: (out[k][rows] if out[k].shape[0] == wl.R else out[k][seqs]) for k in out if k != "cap_hits"}
+    gsub["cap_hits"] = out["cap_hits"]
+    st = compare_round(gsub, ref, sub.wl, s1q, s1p, sub.u, sub.v, "mar256 sampled")
+    print("mar256 sampled", st)
+    dr.ctx.close()

@@ -1,0 +1,103 @@
+"""CPU-side checks: the C-ABI library loads and exports what include/csd.h declares, the binding's
+host helpers agree with the float64 checker, the input generators behave."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import torch
+
+from oracle import csd_oracle as orc
+from paper_2411_11925_b200 import build, inputs as gen
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    src = open(os.path.join(ROOT, "include", "csd.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(csd_[a-z_]+)\s*\(", src)))
+
+
+def test_library_builds_loads_and_exports_every_declared_symbol():
+    path = build.build_library()
+    lib = ctypes.CDLL(path)
+    names = _declared()
+    assert len(names) >= 12
+    missing = [n for n in names if not hasattr(lib, n)]
+    assert not missing, missing
+
+
+def test_binding_covers_the_header():
+    from paper_2411_11925_b200 import api
+    assert sorted(api.EXPORTS) == _declared()
+    # struct layouts mirror the header
+    assert [f[0] for f in api._HeadDesc._fields_] == ["C", "W", "L", "Dz", "F", "dtype"]
+    hdr = open(os.path.join(ROOT, "include", "csd.h")).read()
+    block = hdr[hdr.index("typedef struct {\n  const float *Wz"):hdr.index("} csd_head_weights;")]
+    assert re.findall(r"\*(\w+)", block) == list(api.WEIGHT_FIELDS)
+
+
+def test_null_context_calls_return_invalid_arg_without_a_gpu():
+    lib = ctypes.CDLL(build.build_library())
+    assert lib.csd_sync(None) == -1
+    assert lib.csd_destroy(None) == -1
+    assert lib.csd_head_destroy(None) == -1
+    assert lib.csd_create(None, 0, None) == -1
+
+
+def test_ddpm_coefficients_match_the_checker_schedule():
+    from paper_2411_11925_b200 import api
+    for T, tau in ((10, 1.0), (100, 0.9)):
+        beta = gen.beta_linear(T)
+        c, s = api.ddpm_coefficients(beta, tau), orc.ddpm_schedule(beta, tau)
+        for k in ("a", "b", "sigma"):
+            np.testing.assert_allclose(c[k], s[k], rtol=1e-7)
+
+
+def test_round_to_bf16_matches_torch_and_is_idempotent():
+    rng = np.random.default_rng(0)
+    a = (rng.standard_normal(10000) * 10.0 ** rng.integers(-6, 3, 10000)).astype(np.float32)
+    want = torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
+    got = gen.round_to_bf16(a)
+    np.testing.assert_array_equal(got, want)
+    np.testing.assert_array_equal(gen.round_to_bf16(got), got)
+
+
+def test_inputs_are_seeded_shaped_and_in_range():
+    wl = gen.WORKLOADS["tiny_fp32"]
+    a, b = gen.make_round_inputs(wl), gen.make_round_inputs(wl)
+    for k in gen.WEIGHT_NAMES:
+        np.testing.assert_array_equal(a.w_p[k], b.w_p[k])
+    np.testing.assert_array_equal(a.eps, b.eps)
+    assert a.eps.shape == (wl.T, wl.R, 16) and a.z_q.shape == (wl.Rh, 256) and a.u.shape == (1, 4)
+    assert np.all((a.u > 0) & (a.u < 1)) and np.all((a.v > 0) & (a.v < 1))
+    c = gen.make_round_inputs(wl, seed_offset=7)
+    assert not np.array_equal(a.eps, c.eps)
+    assert abs(float(np.abs(a.w_p["Wada"]).max()) - np.sqrt(6.0 / (4 * 256))) < 1e-3   # Xavier bound
+    assert wl.target.n_params() == sum(v.size for v in a.w_p.values())
+
+
+def test_workload_table_matches_the_stated_sizes():
+    w = gen.WORKLOADS
+    assert (w["mar256"].R, w["mar256"].Rh) == (512, 1024)
+    assert (w["large_target"].R, w["large_target"].Rh) == (2048, 4096)
+    assert (w["mar512"].R, w["mar512"].Rh) == (1024, 2048)
+    assert (w["ar_stress"].R, w["ar_stress"].Rh) == (4096, 4096)
+    assert abs(w["mar256"].target.flops_per_row_step() / 1e6 - 67.2) < 0.1
+    assert abs(w["mar256"].draft.flops_per_row_step() / 1e6 - 35.7) < 0.1
+    assert abs(w["mar256"].flops_per_round() / 1e12 - 10.54) < 0.01
+    assert abs(w["large_target"].flops_per_round() / 1e12 - 147.4) < 0.1
+
+
+def test_select_sequences_slices_rows_consistently():
+    wl = gen.Workload(**{**gen.WORKLOADS["tiny_fp32"].__dict__, "B": 3, "cfg": True, "cfg_scale": 2.0})
+    inp = gen.make_round_inputs(wl)
+    sub = gen.select_sequences(inp, [2, 0])
+    g = wl.gamma
+    np.testing.assert_array_equal(sub.x_T[:g], inp.x_T[2 * g:3 * g])
+    np.testing.assert_array_equal(sub.z_p[sub.wl.R:sub.wl.R + g], inp.z_p[wl.R + 2 * g: wl.R + 3 * g])
+    np.testing.assert_array_equal(sub.eps[:, g:], inp.eps[:, :g])
+    full, part = orc.round_from_inputs(inp), orc.round_from_inputs(sub)
+    np.testing.assert_allclose(part["logratio"], full["logratio"][[2, 0]], rtol=1e-9)
+    np.testing.assert_allclose(part["x0"][:g], full["x0"][2 * g:3 * g], atol=1e-12)
