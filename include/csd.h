@@ -103,6 +103,18 @@ int csd_sync(csd_ctx *ctx);
 /* Number of kernels this context has launched so far (bookkeeping for benchmarks). */
 int64_t csd_launch_count(const csd_ctx *ctx);
 
+/* Optional per-launch timing for benchmarks.  csd_profile(ctx, 1) synchronises, clears the records
+ * and makes every later GEMM-chain launch of this context be bracketed by CUDA events on the
+ * stream it runs on (this costs a little time per launch, so throughput is measured with it
+ * off); csd_profile(ctx, 0) switches it off.  csd_profile_read synchronises and sums, for one
+ * kernel class, the launches recorded since: their count, device time (ms) and algorithmic FLOPs
+ * (2*M*N*K per GEMM).  Classes: 0 condition projection, 1 block MLP first layer (+SiLU),
+ * 2 AdaLN modulate (shift|scale), 3 block MLP second layer + gate + residual, 4 final modulate +
+ * output projection, 5 per-step boundary kernel. */
+int csd_profile(csd_ctx *ctx, int enable);
+int csd_profile_read(csd_ctx *ctx, int kernel_class, int64_t *launches, double *total_ms,
+                     double *total_flops);
+
 /* Copies and repacks the weights into device memory owned by the head (synchronous; the caller
  * may free `w` afterwards).  A head belongs to the context it was created with. */
 int csd_head_create(csd_ctx *ctx, const csd_head_desc *desc, const csd_head_weights *w, csd_head **out);

@@ -23,6 +23,7 @@ CSD_F32, CSD_BF16, CSD_F16 = 0, 1, 2
 DTYPES = {"f32": CSD_F32, "bf16": CSD_BF16, "f16": CSD_F16}
 
 EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launch_count",
+           "csd_profile", "csd_profile_read",
            "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_verify",
            "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host")
 
@@ -61,6 +62,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_last_error.argtypes = [vp]; lib.csd_last_error.restype = C.c_char_p
     lib.csd_sync.argtypes = [vp]
     lib.csd_launch_count.argtypes = [vp]; lib.csd_launch_count.restype = C.c_int64
+    lib.csd_profile.argtypes = [vp, i32]
+    lib.csd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_int64), C.POINTER(f64), C.POINTER(f64)]
     lib.csd_head_create.argtypes = [vp, C.POINTER(_HeadDesc), C.POINTER(_HeadWeights), C.POINTER(vp)]
     lib.csd_head_destroy.argtypes = [vp]
     lib.csd_draft_denoise.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, f32] + [vp] * 6
@@ -141,6 +144,19 @@ class Context:
 
     def launch_count(self) -> int:
         return int(_LIB.csd_launch_count(self._h))
+
+    KERNEL_CLASSES = ("cond_proj", "mlp1_silu", "adaln_modulate", "mlp2_gate_residual", "final_mod_outproj", "step")
+
+    def profile(self, enable: bool):
+        self._check(_LIB.csd_profile(self._h, int(enable)))
+
+    def profile_read(self) -> dict:
+        out = {}
+        for i, name in enumerate(self.KERNEL_CLASSES):
+            n, ms, fl = C.c_int64(), C.c_double(), C.c_double()
+            self._check(_LIB.csd_profile_read(self._h, i, C.byref(n), C.byref(ms), C.byref(fl)))
+            out[name] = {"launches": n.value, "ms": ms.value, "flops": fl.value}
+        return out
 
     def close(self):
         for h in list(self._heads):

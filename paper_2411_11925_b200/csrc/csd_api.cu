@@ -35,6 +35,8 @@ struct ChainWs {
   float *cz, *te, *h, *stats, *epart, *x;
 };
 
+struct ProfRec { cudaEvent_t a, b; int cls; double flops; };
+
 struct HostIo {  // device mirrors for csd_round_host
   void* base = nullptr;
   size_t cap = 0;
@@ -53,6 +55,11 @@ struct csd_ctx {
   ChainWs ws[2];
   HostIo io;
   char err[512] = {0};
+  // optional per-launch timing (csd_profile)
+  bool prof_on = false;
+  std::vector<ProfRec> prof;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used = 0;
 };
 
 struct csd_head {
@@ -93,6 +100,25 @@ int fail(csd_ctx* ctx, int code, const char* fmt, ...) {
       return fail(ctx, CSD_ERR_CUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), __FILE__, \
                   __LINE__);                                                                         \
   } while (0)
+
+cudaEvent_t prof_event(csd_ctx* ctx) {
+  if (ctx->ev_used == ctx->ev_pool.size()) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    ctx->ev_pool.push_back(e);
+  }
+  return ctx->ev_pool[ctx->ev_used++];
+}
+// Brackets one launch with events on its own stream when profiling is on.
+struct ProfScope {
+  csd_ctx* ctx; cudaStream_t st; cudaEvent_t a = nullptr, b = nullptr; int cls; double flops;
+  ProfScope(csd_ctx* c, cudaStream_t s, int cls_, double fl) : ctx(c), st(s), cls(cls_), flops(fl) {
+    if (ctx->prof_on && (a = prof_event(ctx)) && (b = prof_event(ctx))) cudaEventRecord(a, st);
+  }
+  ~ProfScope() {
+    if (a && b) { cudaEventRecord(b, st); ctx->prof.push_back({a, b, cls, flops}); }
+  }
+};
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -159,6 +185,7 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
     attr_done = true;
   }
   dim3 grid(N / kTileN, (ep.M + kTileM - 1) / kTileM);
+  ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * ((NSEG == 1 && MMA_N == 256) ? 2.0 : 1.0));
   kern<<<grid, kTcThreads, smem, st>>>(a0, b0, a1, b1, K0 / kBlockK, K1 / kBlockK, ep, ctx->d_err);
   ctx->launches++;
   CSD_CUDA(ctx, cudaGetLastError());
@@ -176,6 +203,7 @@ template <int EPI, int NSEG, int MMA_N>
 int launch_simt(csd_ctx* ctx, cudaStream_t st, const float* A0, int lda0, const float* B0, int K0, const float* A1,
                 int lda1, const float* B1, int K1, int N, const EpiParams& ep) {
   dim3 grid(N / kTileN, (ep.M + kSimtRows - 1) / kSimtRows);
+  ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * ((NSEG == 1 && MMA_N == 256) ? 2.0 : 1.0));
   gemm_simt_kernel<EPI, NSEG, MMA_N><<<grid, 128, 0, st>>>(A0, lda0, B0, K0, K0, A1, lda1, B1, K1, K1, ep);
   ctx->launches++;
   CSD_CUDA(ctx, cudaGetLastError());
@@ -192,64 +220,75 @@ int check_sched(csd_ctx* ctx, const csd_schedule* s, bool full) {
   return CSD_OK;
 }
 
-// Runs t = T..1 of one head for R token rows on stream `st` with workspace slot `slot`.
-int run_chain(csd_ctx* ctx, int slot, cudaStream_t st, const csd_head* hd, const csd_schedule* sc, int R, int cfg,
-              float cfg_scale, const float* z, const float* x_T, const float* eps, int sample_last, float* x0,
-              float* mu1, float* x1) {
-  const csd_head_desc& d = hd->d;
-  const int Rh = R * (cfg ? 2 : 1), W = d.W, L = d.L, T = sc->T, NT = W / kTileN;
-  const bool tc = d.dtype != CSD_F32;
-  ChainWs& ws = ctx->ws[slot];
-  int rc = ensure_ws(ctx, ws, d, Rh, R, T);
-  if (rc) return rc;
-
-  timestep_embed_kernel<<<T, 256, (d.F + W) * sizeof(float), st>>>(sc->tfeat, hd->Wt1, hd->bt1, hd->Wt2, hd->bt2, W,
-                                                                  d.F, ws.te);
-  ctx->launches++;
-  CSD_CUDA(ctx, cudaGetLastError());
-
+// One head's denoising chain for R token rows on stream `st` with workspace slot `slot`:
+// begin() enqueues the per-call work (timestep embedding, condition projection, first boundary
+// kernel), step(t) enqueues the kernels of step t.  Two chains can be interleaved launch by launch.
+struct Chain {
+  csd_ctx* ctx; int slot; cudaStream_t st; const csd_head* hd; const csd_schedule* sc;
+  int R, cfg; float cfg_scale; const float *z, *x_T, *eps; int sample_last; float *x0, *mu1, *x1;
+  int Rh = 0, W = 0, L = 0, T = 0;
+  bool tc = false;
   CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{};
   EpiParams ep{};
-  ep.M = Rh; ep.ldo = W;
-  if (tc) {
-    const size_t nz = static_cast<size_t>(Rh) * d.Dz;
-    const unsigned nblk = static_cast<unsigned>((nz + 255) / 256);
-    if (d.dtype == CSD_F16) convert_act_kernel<__half><<<nblk, 256, 0, st>>>(z, static_cast<__half*>(ws.zc), nz);
-    else convert_act_kernel<__nv_bfloat16><<<nblk, 256, 0, st>>>(z, static_cast<__nv_bfloat16*>(ws.zc), nz);
-    ctx->launches++;
-    if ((rc = make_tmap(ctx, &tm_z, d.dtype, ws.zc, Rh, d.Dz, d.Dz, kTileM))) return rc;
-    if ((rc = make_tmap(ctx, &tm_s, d.dtype, ws.s, Rh, W, W, kTileM))) return rc;
-    if ((rc = make_tmap(ctx, &tm_u, d.dtype, ws.u, Rh, W, W, kTileM))) return rc;
-    if ((rc = make_tmap(ctx, &tm_v, d.dtype, ws.v, Rh, W, W, kTileM))) return rc;
-  }
-  // S0: cz = z Wz^T + bz
-  ep.bias0 = hd->bz; ep.out_f32 = ws.cz;
-  if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 128>(ctx, d.dtype, st, tm_z, hd->tmWz, tm_z, hd->tmWz, d.Dz, 0, W, ep);
-  else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
-                                              nullptr, 0, W, ep);
-  if (rc) return rc;
-
   StepParams sp{};
-  sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = NT; sp.cfg_scale = cfg_scale;
-  sp.sample_last = sample_last; sp.epart = ws.epart; sp.bout = hd->bout; sp.x_src = x_T; sp.x = ws.x;
-  sp.x0 = x0; sp.mu1 = mu1; sp.x1 = x1; sp.win = hd->win; sp.bin = hd->bin; sp.cz = ws.cz; sp.h = ws.h;
-  sp.stats = ws.stats; sp.s = ws.s;
-  auto launch_step = [&](int mode) -> int {
+
+  int launch_step(int mode) {
+    const csd_head_desc& d = hd->d;
+    ProfScope ps(ctx, st, 5, 2.0 * Rh * static_cast<double>(W) * d.C);
     if (d.dtype == CSD_F16) step_kernel<__half><<<R, 256, 0, st>>>(sp, mode);
     else if (d.dtype == CSD_BF16) step_kernel<__nv_bfloat16><<<R, 256, 0, st>>>(sp, mode);
     else step_kernel<float><<<R, 256, 0, st>>>(sp, mode);
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
     return CSD_OK;
-  };
-  sp.te_next = ws.te + static_cast<size_t>(T - 1) * W;
-  sp.eps_t = eps;
-  if ((rc = launch_step(STEP_INIT))) return rc;
+  }
 
-  const float* sf = static_cast<const float*>(ws.s);
-  const float* uf = static_cast<const float*>(ws.u);
-  const float* vf = static_cast<const float*>(ws.v);
-  for (int t = T; t >= 1; --t) {
+  int begin() {
+    const csd_head_desc& d = hd->d;
+    Rh = R * (cfg ? 2 : 1); W = d.W; L = d.L; T = sc->T;
+    tc = d.dtype != CSD_F32;
+    ChainWs& ws = ctx->ws[slot];
+    int rc = ensure_ws(ctx, ws, d, Rh, R, T);
+    if (rc) return rc;
+    timestep_embed_kernel<<<T, 256, (d.F + W) * sizeof(float), st>>>(sc->tfeat, hd->Wt1, hd->bt1, hd->Wt2, hd->bt2, W,
+                                                                    d.F, ws.te);
+    ctx->launches++;
+    CSD_CUDA(ctx, cudaGetLastError());
+    ep.M = Rh; ep.ldo = W;
+    if (tc) {
+      const size_t nz = static_cast<size_t>(Rh) * d.Dz;
+      const unsigned nblk = static_cast<unsigned>((nz + 255) / 256);
+      if (d.dtype == CSD_F16) convert_act_kernel<__half><<<nblk, 256, 0, st>>>(z, static_cast<__half*>(ws.zc), nz);
+      else convert_act_kernel<__nv_bfloat16><<<nblk, 256, 0, st>>>(z, static_cast<__nv_bfloat16*>(ws.zc), nz);
+      ctx->launches++;
+      if ((rc = make_tmap(ctx, &tm_z, d.dtype, ws.zc, Rh, d.Dz, d.Dz, kTileM))) return rc;
+      if ((rc = make_tmap(ctx, &tm_s, d.dtype, ws.s, Rh, W, W, kTileM))) return rc;
+      if ((rc = make_tmap(ctx, &tm_u, d.dtype, ws.u, Rh, W, W, kTileM))) return rc;
+      if ((rc = make_tmap(ctx, &tm_v, d.dtype, ws.v, Rh, W, W, kTileM))) return rc;
+    }
+    // cz = z Wz^T + bz
+    EpiParams e = ep;
+    e.bias0 = hd->bz; e.out_f32 = ws.cz;
+    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 128>(ctx, d.dtype, st, tm_z, hd->tmWz, tm_z, hd->tmWz, d.Dz, 0, W, e);
+    else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
+                                                nullptr, 0, W, e);
+    if (rc) return rc;
+    sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = W / kTileN; sp.cfg_scale = cfg_scale;
+    sp.sample_last = sample_last; sp.epart = ws.epart; sp.bout = hd->bout; sp.x_src = x_T; sp.x = ws.x;
+    sp.x0 = x0; sp.mu1 = mu1; sp.x1 = x1; sp.win = hd->win; sp.bin = hd->bin; sp.cz = ws.cz; sp.h = ws.h;
+    sp.stats = ws.stats; sp.s = ws.s;
+    sp.te_next = ws.te + static_cast<size_t>(T - 1) * W;
+    sp.eps_t = eps;
+    return launch_step(STEP_INIT);
+  }
+
+  int step(int t) {
+    const csd_head_desc& d = hd->d;
+    ChainWs& ws = ctx->ws[slot];
+    const float* sf = static_cast<const float*>(ws.s);
+    const float* uf = static_cast<const float*>(ws.u);
+    const float* vf = static_cast<const float*>(ws.v);
+    int rc = CSD_OK;
     for (int k = 0; k < L; ++k) {
       EpiParams e = ep;
       e.h = ws.h; e.stats = ws.stats;
@@ -281,9 +320,17 @@ int run_chain(csd_ctx* ctx, int slot, cudaStream_t st, const csd_head* hd, const
     sp.a = sc->a[t - 1]; sp.b = sc->b[t - 1]; sp.sigma = sc->sigma[t - 1];
     sp.eps_t = eps + static_cast<size_t>(t - 1) * R * d.C;
     if (t > 1) sp.te_next = ws.te + static_cast<size_t>(t - 2) * W;
-    if ((rc = launch_step(t > 1 ? STEP_MID : STEP_LAST))) return rc;
+    return launch_step(t > 1 ? STEP_MID : STEP_LAST);
   }
-  return CSD_OK;
+};
+
+int run_chain(csd_ctx* ctx, int slot, cudaStream_t st, const csd_head* hd, const csd_schedule* sc, int R, int cfg,
+              float cfg_scale, const float* z, const float* x_T, const float* eps, int sample_last, float* x0,
+              float* mu1, float* x1) {
+  Chain c{ctx, slot, st, hd, sc, R, cfg, cfg_scale, z, x_T, eps, sample_last, x0, mu1, x1};
+  int rc = c.begin();
+  for (int t = sc->T; t >= 1 && !rc; --t) rc = c.step(t);
+  return rc;
 }
 
 int check_chain_args(csd_ctx* ctx, const csd_head* hd, const csd_schedule* sc, int R, int cfg, const void* z,
@@ -389,6 +436,7 @@ int csd_destroy(csd_ctx* c) {
     if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
     if (c->ws[i].base) cudaFree(c->ws[i].base);
   }
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->io.base) cudaFree(c->io.base);
   if (c->d_err) cudaFree(c->d_err);
@@ -410,6 +458,31 @@ int csd_sync(csd_ctx* c) {
     cudaMemset(c->d_err, 0, sizeof(int));
     return fail(c, CSD_ERR_TIMEOUT, "a device-side bounded wait gave up (code %d: 1 = TMA producer, 2 = MMA issuer, "
                 "3 = epilogue)", e);
+  }
+  return CSD_OK;
+}
+
+int csd_profile(csd_ctx* c, int enable) {
+  if (!c) return CSD_ERR_INVALID_ARG;
+  CSD_CUDA(c, cudaStreamSynchronize(c->stream));
+  c->prof_on = enable != 0;
+  c->prof.clear();
+  c->ev_used = 0;
+  return CSD_OK;
+}
+
+int csd_profile_read(csd_ctx* c, int kernel_class, int64_t* launches, double* total_ms, double* total_flops) {
+  if (!c) return CSD_ERR_INVALID_ARG;
+  if (!launches || !total_ms || !total_flops) return fail(c, CSD_ERR_INVALID_ARG, "null output pointer");
+  if (kernel_class < 0 || kernel_class > 5) return fail(c, CSD_ERR_INVALID_ARG, "kernel class %d not in [0, 5]", kernel_class);
+  CSD_CUDA(c, cudaStreamSynchronize(c->stream));
+  for (int i = 0; i < 2; ++i) CSD_CUDA(c, cudaStreamSynchronize(c->side[i]));
+  *launches = 0; *total_ms = 0.0; *total_flops = 0.0;
+  for (const ProfRec& r : c->prof) {
+    if (r.cls != kernel_class) continue;
+    float ms = 0.0f;
+    CSD_CUDA(c, cudaEventElapsedTime(&ms, r.a, r.b));
+    *launches += 1; *total_ms += ms; *total_flops += r.flops;
   }
   return CSD_OK;
 }
@@ -618,8 +691,15 @@ int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, cons
   if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T))) return rc;
   CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
   for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
-  rc = run_chain(ctx, 0, ctx->side[0], head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr);
-  int rc2 = run_chain(ctx, 1, ctx->side[1], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr);
+  // the two chains' launches are interleaved step by step so that neither stream starves
+  Chain cq{ctx, 0, ctx->side[0], head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr};
+  Chain cp{ctx, 1, ctx->side[1], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr};
+  rc = cp.begin();
+  int rc2 = cq.begin();
+  for (int t = sched_p->T; t >= 1 && !rc && !rc2; --t) {
+    rc = cp.step(t);
+    if (!rc) rc2 = cq.step(t);
+  }
   for (int i = 0; i < 2; ++i) {
     CSD_CUDA(ctx, cudaEventRecord(ctx->ev_done[i], ctx->side[i]));
     CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_done[i], 0));

@@ -36,6 +36,9 @@ struct EpiParams {
 };
 
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
+// Fast variant for the tensor-core path (its result is rounded to a 16-bit operand anyway).
+__device__ __forceinline__ float silu_fast(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
+template <bool FAST> __device__ __forceinline__ float silu_t(float x) { return FAST ? silu_fast(x) : silu_f(x); }
 
 template <typename T> __device__ __forceinline__ T to_act(float v);
 template <> __device__ __forceinline__ float to_act<float>(float v) { return v; }
@@ -94,20 +97,27 @@ struct RowState {
 };
 
 // Merge the per-32-column (mean, M2) partials of row m in a fixed order (Chan et al.), so the
-// LayerNorm statistics do not depend on which CTA computes them.
+// LayerNorm statistics do not depend on which CTA computes them.  Loads are issued eight at a time.
 __device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
   const int G = W / kChunk;
   const float2* p = reinterpret_cast<const float2*>(stats) + static_cast<size_t>(m) * G;
-  float2 a = p[0];
-  float na = static_cast<float>(kChunk);
-  for (int g = 1; g < G; ++g) {
-    const float2 b = p[g];
-    const float nb = static_cast<float>(kChunk);
-    const float n = na + nb;
-    const float d = b.x - a.x;
-    a.x += d * (nb / n);
-    a.y += b.y + d * d * (na * nb / n);
-    na = n;
+  float2 a = make_float2(0.0f, 0.0f);
+  float na = 0.0f;
+  for (int g0 = 0; g0 < G; g0 += 8) {
+    float2 b[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) b[j] = (g0 + j < G) ? p[g0 + j] : make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (g0 + j < G) {
+        const float nb = static_cast<float>(kChunk);
+        const float n = na + nb;
+        const float d = b[j].x - a.x;
+        a.x += d * (nb / n);
+        a.y += b[j].y + d * d * (na * nb / n);
+        na = n;
+      }
+    }
   }
   mean = a.x;
   rstd = 1.0f / sqrtf(a.y / static_cast<float>(W) + 1e-6f);
@@ -122,47 +132,54 @@ __device__ __forceinline__ void epi_row_begin(const EpiParams& ep, int m, RowSta
   }
 }
 
+template <int EPI> __host__ __device__ constexpr bool epi_reads_h() { return EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES; }
+
 // a0 / a1: accumulator chunk (32 columns) of the first / second accumulator; n0 = first global
-// output column of the chunk; wout_s: this tile's [128][16] slice of Wout^T in shared memory.
-template <int EPI, typename ACT>
-__device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, int chunk, float* a0,
-                                          const float* a1, RowState& rs, const float* wout_s) {
+// output column of the chunk; b0 / b1: the chunk's 32 biases (shared or global memory); hv: the
+// chunk's 32 values of h, already loaded (EPI_MOD, EPI_MODF, EPI_GATE_RES); wout_c: the chunk's
+// [32][16] slice of Wout^T in shared memory (EPI_MODF).
+template <int EPI, typename ACT, bool FAST>
+__device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, float* a0, const float* a1,
+                                          const float* b0, const float* b1, float* hv, RowState& rs,
+                                          const float* wout_c) {
   const size_t off = static_cast<size_t>(m) * ep.ldo + n0;
   if constexpr (EPI == EPI_BIAS_F32) {
 #pragma unroll
-    for (int j = 0; j < kChunk; ++j) a0[j] += __ldg(ep.bias0 + n0 + j);
+    for (int j = 0; j < kChunk; ++j) a0[j] += b0[j];
     store_chunk<float>(ep.out_f32 + off, a0);
   } else if constexpr (EPI == EPI_SILU_ACT) {
 #pragma unroll
-    for (int j = 0; j < kChunk; ++j) a0[j] = silu_f(a0[j] + __ldg(ep.bias0 + n0 + j));
+    for (int j = 0; j < kChunk; ++j) a0[j] = silu_t<FAST>(a0[j] + b0[j]);
     store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
   } else if constexpr (EPI == EPI_MOD || EPI == EPI_MODF) {
-    float hv[kChunk];
-    load_chunk_f32(ep.h + off, hv);
 #pragma unroll
     for (int j = 0; j < kChunk; ++j) {
-      const float shift = a0[j] + __ldg(ep.bias0 + n0 + j);
-      const float scale = a1[j] + __ldg(ep.bias1 + n0 + j);
+      const float shift = a0[j] + b0[j];
+      const float scale = a1[j] + b1[j];
       a0[j] = (hv[j] - rs.mean) * rs.rstd * (1.0f + scale) + shift;
     }
     if constexpr (EPI == EPI_MOD) {
       store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
     } else {
-      const float* w = wout_s + chunk * kChunk * kCPad;
 #pragma unroll
       for (int j = 0; j < kChunk; ++j) {
+        const float4* w4 = reinterpret_cast<const float4*>(wout_c + j * kCPad);
 #pragma unroll
-        for (int c = 0; c < kCPad; ++c) rs.eacc[c] = fmaf(a0[j], w[j * kCPad + c], rs.eacc[c]);
+        for (int c4 = 0; c4 < kCPad / 4; ++c4) {
+          const float4 w = w4[c4];
+          rs.eacc[4 * c4 + 0] = fmaf(a0[j], w.x, rs.eacc[4 * c4 + 0]);
+          rs.eacc[4 * c4 + 1] = fmaf(a0[j], w.y, rs.eacc[4 * c4 + 1]);
+          rs.eacc[4 * c4 + 2] = fmaf(a0[j], w.z, rs.eacc[4 * c4 + 2]);
+          rs.eacc[4 * c4 + 3] = fmaf(a0[j], w.w, rs.eacc[4 * c4 + 3]);
+        }
       }
     }
   } else if constexpr (EPI == EPI_GATE_RES) {
-    float hv[kChunk];
-    load_chunk_f32(ep.h + off, hv);
     float sum = 0.0f;
 #pragma unroll
     for (int j = 0; j < kChunk; ++j) {
-      const float y = a0[j] + __ldg(ep.bias0 + n0 + j);
-      const float g = a1[j] + __ldg(ep.bias1 + n0 + j);
+      const float y = a0[j] + b0[j];
+      const float g = a1[j] + b1[j];
       hv[j] = fmaf(g, y, hv[j]);
       sum += hv[j];
     }

@@ -15,7 +15,8 @@
 namespace csd {
 
 constexpr int kBlockK = 64;  // bf16 elements per TMA box row = 128 bytes = one swizzle row
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int kEpiThreads = 256;
 
 enum DevErr : int { DEV_OK = 0, DEV_ERR_TMA_WAIT = 1, DEV_ERR_MMA_WAIT = 2, DEV_ERR_EPI_WAIT = 3 };
 
@@ -24,8 +25,9 @@ template <int MMA_N> struct TcCfg {
   static constexpr int kABytes = kTileM * kBlockK * 2;
   static constexpr int kBBytes = MMA_N * kBlockK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kWoutBytes = kTileN * kCPad * 4;
-  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kWoutBytes + 256;
+  static constexpr int kWoutBytes = kTileN * kCPad * 4;      // Wout^T tile, reused for the eps partials
+  static constexpr int kBiasBytes = 2 * kTileN * 4;
+  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kWoutBytes + kBiasBytes + 256;
 };
 
 template <int EPI, typename ACT, int NSEG, int MMA_N, int AB_FMT>
@@ -40,7 +42,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stage_base = smem;
   float* wout_s = reinterpret_cast<float*>(smem + S * Cfg::kStageBytes);
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStageBytes + Cfg::kWoutBytes);
+  float* bias_s = reinterpret_cast<float*>(smem + S * Cfg::kStageBytes + Cfg::kWoutBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStageBytes + Cfg::kWoutBytes + Cfg::kBiasBytes);
   uint64_t* empty_bar = full_bar + S;
   uint64_t* tmem_full_bar = empty_bar + S;
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_full_bar + 1);
@@ -67,10 +70,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   if (warp == 1) {
     tmem_alloc(tmem_base_s, kTmemCols);
     tmem_relinquish();
-  }
-  if (EPI == EPI_MODF && warp >= 2) {
-    const float* src = ep.wout_t + static_cast<size_t>(tile_n) * kTileN * kCPad;
-    for (int i = threadIdx.x - 64; i < kTileN * kCPad; i += kTcThreads - 64) wout_s[i] = src[i];
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -116,27 +115,66 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     }
     __syncwarp();
   } else {
-    // Epilogue: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32).
-    const int q = warp & 3;
+    // Epilogue, 8 warps: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32); warps 2..5 take
+    // column chunks 0 and 1 of the tile, warps 6..9 chunks 2 and 3.  Everything that does not need
+    // the accumulators (biases, Wout^T tile, LayerNorm statistics, h) is fetched while the MMAs run.
+    const int et = threadIdx.x - 64;
+    const int q = warp & 3, half = (warp - 2) >> 2;
     const int m = tile_m * kTileM + q * 32 + lane;
     const bool valid = m < ep.M;
+    if (et < kTileN) {
+      bias_s[et] = ep.bias0[tile_n * kTileN + et];
+      bias_s[kTileN + et] = ep.bias1 ? ep.bias1[tile_n * kTileN + et] : 0.0f;
+    }
+    if (EPI == EPI_MODF) {
+      const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * kTileN * kCPad);
+      float4* dst = reinterpret_cast<float4*>(wout_s);
+#pragma unroll
+      for (int i = 0; i < kTileN * kCPad / 4 / kEpiThreads; ++i) dst[et + i * kEpiThreads] = src[et + i * kEpiThreads];
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    RowState rs;
+    float hv[2][kChunk];
+    if (valid) {
+      epi_row_begin<EPI>(ep, m, rs);
+      if (epi_reads_h<EPI>()) {
+#pragma unroll
+        for (int ci = 0; ci < 2; ++ci)
+          load_chunk_f32(ep.h + static_cast<size_t>(m) * ep.ldo + tile_n * kTileN + (2 * half + ci) * kChunk, hv[ci]);
+      }
+    }
     bool ok = mbar_wait(tmem_full_bar, 0);
     if (!ok) atomicExch(err, DEV_ERR_EPI_WAIT);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after_sync();
-      RowState rs;
-      if (valid) epi_row_begin<EPI>(ep, m, rs);
       const uint32_t trow = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-#pragma unroll 1
-      for (int c = 0; c < kTileN / kChunk; ++c) {
+#pragma unroll
+      for (int ci = 0; ci < 2; ++ci) {
+        const int c = 2 * half + ci;
         float a0[kChunk], a1[kChunk];
         tmem_ld32(trow + c * kChunk, a0);
         if (NSEG * MMA_N == 256) tmem_ld32(trow + kTileN + c * kChunk, a1);
         tmem_ld_wait();
-        if (valid) epi_chunk<EPI, ACT>(ep, m, tile_n * kTileN + c * kChunk, c, a0, a1, rs, wout_s);
+        if (valid)
+          epi_chunk<EPI, ACT, true>(ep, m, tile_n * kTileN + c * kChunk, a0, a1, bias_s + c * kChunk,
+                                    bias_s + kTileN + c * kChunk, hv[ci], rs, wout_s + c * kChunk * kCPad);
       }
-      if (valid) epi_row_end<EPI>(ep, m, tile_n, rs);
+    }
+    if (EPI == EPI_MODF) {
+      // combine the two column halves of each row in a fixed order: (chunks 0,1) + (chunks 2,3)
+      asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread is done reading the Wout^T tile
+      float* part = wout_s;                            // [128 rows][16]
+      if (half == 1 && ok) {
+#pragma unroll
+        for (int c = 0; c < kCPad; ++c) part[(q * 32 + lane) * kCPad + c] = rs.eacc[c];
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (half == 0 && ok && valid) {
+#pragma unroll
+        for (int c = 0; c < kCPad; ++c) rs.eacc[c] += part[(q * 32 + lane) * kCPad + c];
+        epi_row_end<EPI>(ep, m, tile_n, rs);
+      }
     }
   }
   tc_fence_before_sync();
@@ -209,8 +247,12 @@ gemm_simt_kernel(const float* __restrict__ A0, int lda0, const float* __restrict
   // and summed below through shared memory in chunk order.
   RowState rs;
   if (m < ep.M) {
+    const int n0 = tile_n * kTileN + warp * kChunk;
+    float hv[kChunk];
     epi_row_begin<EPI>(ep, m, rs);
-    epi_chunk<EPI, float>(ep, m, tile_n * kTileN + warp * kChunk, warp, acc0, acc1, rs, wout_s);
+    if (epi_reads_h<EPI>()) load_chunk_f32(ep.h + static_cast<size_t>(m) * ep.ldo + n0, hv);
+    epi_chunk<EPI, float, false>(ep, m, n0, acc0, acc1, ep.bias0 + n0, ep.bias1 ? ep.bias1 + n0 : ep.bias0 + n0, hv, rs,
+                                 wout_s + warp * kChunk * kCPad);
   }
   if constexpr (EPI == EPI_MODF) {
     float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][16]

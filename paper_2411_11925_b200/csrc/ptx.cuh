@@ -11,12 +11,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
-__device__ __forceinline__ uint64_t global_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred = 0;
   asm volatile(
@@ -55,16 +49,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after `limit_ns` of wall time (default 2 s) and returns false.
+// Bounded wait: polls the barrier and gives up (returns false) after about `limit_cycles` SM
+// clock cycles (default 4e9, roughly two seconds).  The clock is read only once per 1024 failed
+// polls: a timer read on every wait would sit on the pipeline's critical path.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
-                                          uint64_t limit_ns = 2000000000ull) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
+                                          long long limit_cycles = 4000000000ll) {
+  long long t0 = 0;
+  uint32_t spins = 0;
   for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (global_timer_ns() - t0 > limit_ns) return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 1023u) == 0u) {
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > limit_cycles) return false;
+    }
   }
 }
 
