@@ -254,3 +254,12 @@ def select_sequences(inp: RoundInputs, seqs) -> RoundInputs:
     return RoundInputs(sub, inp.w_q, inp.w_p, inp.z_q[hrows], inp.z_p[hrows], inp.x_T[rows],
                        inp.eps[:, rows], inp.u[seqs], inp.xi[seqs], inp.v[seqs],
                        inp.beta, inp.tfeat, {"rows": rows, "seqs": seqs})
+
+
+def shard_sequences(B: int, world: int, rank: int) -> range:
+    """Contiguous block of sequence indices owned by `rank` when B sequences are split over
+    `world` ranks (the first B % world ranks get one more).  Rows of different sequences never
+    interact, so a sharded round needs no exchange."""
+    base, extra = divmod(B, world)
+    start = rank * base + min(rank, extra)
+    return range(start, start + base + (1 if rank < extra else 0))
