@@ -132,6 +132,32 @@ int csd_draft_denoise(csd_ctx *ctx, const csd_head *head, const csd_schedule *sc
                       float cfg_scale, const float *z, const float *x_T, const float *eps,
                       float *x0, float *mu1, float *x1);
 
+/* csd_draft_denoise without any allocation (the paper has no counterpart: this is a deployment
+ * variant of the call above, same arguments, same kernels, bit-identical results).
+ * Who needs it: code that must not, or cannot, reach the CUDA allocator when the call is made -
+ * a serving process whose framework has handed all free device memory to its own pool so that
+ * cudaMalloc fails, a latency-critical loop where cudaMalloc's implicit device synchronisation is
+ * unacceptable, or a sandboxed plug-in that is only allowed to launch kernels.  csd_draft_denoise
+ * grows a cudaMalloc'ed workspace on demand; this call instead keeps every intermediate
+ * (condition projection, activations, residual stream, LayerNorm partials, eps partial sums, x_t)
+ * in one 8 MiB array that is compiled into the library as a static __device__ object, so every
+ * GPU that loads the library holds those 8 MiB until the process exits.
+ * Limits and rules:
+ *   - the call is rejected with CSD_ERR_WORKSPACE, before anything is enqueued, if its
+ *     intermediates do not fit in 8 MiB (roughly R*(1+cfg) <= 128 head rows at W = 1536, T = 100;
+ *     the error text gives the exact byte count);
+ *   - it calls no cudaMalloc / cudaFree and no allocating library routine; profiling
+ *     (csd_profile) must be off, since recording creates CUDA events;
+ *   - the first call on a device looks up the array's device address (cudaGetSymbolAddress); make
+ *     that first call outside any stream capture;
+ *   - all calls, from every context of the process on that GPU, share the one array, which keeps
+ *     the previous call's contents (nothing in it needs to start at zero: each buffer is written
+ *     before it is read).  Two such calls that overlap on the GPU (different streams or contexts)
+ *     race on it and give wrong results: serialise them. */
+int csd_draft_denoise_static(csd_ctx *ctx, const csd_head *head, const csd_schedule *sched, int R,
+                             int cfg, float cfg_scale, const float *z, const float *x_T,
+                             const float *eps, float *x0, float *mu1, float *x1);
+
 /* Verification (Alg. 1: target run with the draft's noise, Sigma, ratios, accepted count).
  * Runs the target head on the SAME x_T and eps as the draft call (denoising trajectory
  * alignment, Theorem 1) for t = T..1 without sampling x_0, then per row

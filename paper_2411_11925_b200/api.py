@@ -24,7 +24,7 @@ DTYPES = {"f32": CSD_F32, "bf16": CSD_BF16, "f16": CSD_F16}
 
 EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launch_count",
            "csd_profile", "csd_profile_read",
-           "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_verify",
+           "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_draft_denoise_static", "csd_verify",
            "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host")
 
 WEIGHT_FIELDS = ("Wz", "bz", "Wt1", "bt1", "Wt2", "bt2", "Win", "bin", "Wada", "bada",
@@ -67,6 +67,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_head_create.argtypes = [vp, C.POINTER(_HeadDesc), C.POINTER(_HeadWeights), C.POINTER(vp)]
     lib.csd_head_destroy.argtypes = [vp]
     lib.csd_draft_denoise.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, f32] + [vp] * 6
+    lib.csd_draft_denoise_static.argtypes = lib.csd_draft_denoise.argtypes
     lib.csd_verify.argtypes = [vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32] + [vp] * 10
     lib.csd_accept_scan.argtypes = [vp, i32, i32, i32, f64, f32, f32] + [vp] * 7
     lib.csd_resample.argtypes = [vp, i32, i32, i32, i32, f64, f32, f32] + [vp] * 9
@@ -175,6 +176,11 @@ class Context:
     def csd_draft_denoise(self, head: "Head", sched: Schedule, R, cfg, cfg_scale, z, x_T, eps, x0, mu1, x1=None):
         self._check(_LIB.csd_draft_denoise(self._h, head._h, C.byref(sched.c), R, int(cfg), cfg_scale,
                                            _ptr(z), _ptr(x_T), _ptr(eps), _ptr(x0), _ptr(mu1), _ptr(x1)))
+
+    def csd_draft_denoise_static(self, head: "Head", sched: Schedule, R, cfg, cfg_scale, z, x_T, eps, x0, mu1, x1=None):
+        """csd_draft_denoise with its intermediates in the library's built-in 8 MiB device array: no allocation."""
+        self._check(_LIB.csd_draft_denoise_static(self._h, head._h, C.byref(sched.c), R, int(cfg), cfg_scale,
+                                                  _ptr(z), _ptr(x_T), _ptr(eps), _ptr(x0), _ptr(mu1), _ptr(x1)))
 
     def csd_verify(self, head_p: "Head", sched_p: Schedule, sched_q: Schedule, B, gamma, cfg, cfg_scale,
                    z_p, x_T, eps, x0_q, mu1_q, u, logratio, n_accept, accept_mask, mu1_p):

@@ -52,7 +52,7 @@ struct csd_ctx {
   int* d_err = nullptr;
   int64_t launches = 0;
   EncodeTiledFn encode = nullptr;
-  ChainWs ws[2];
+  ChainWs ws[3];   // draft chain, target chain, static-scratch calls
   HostIo io;
   char err[512] = {0};
   // optional per-launch timing (csd_profile)
@@ -617,6 +617,54 @@ int csd_draft_denoise(csd_ctx* ctx, const csd_head* head, const csd_schedule* sc
   if (!x0 || !mu1) return fail(ctx, CSD_ERR_INVALID_ARG, "x0 / mu1 is null");
   CSD_CUDA(ctx, cudaSetDevice(ctx->device));
   return run_chain(ctx, 0, ctx->stream, head, sched, R, cfg, cfg_scale, z, x_T, eps, 1, x0, mu1, x1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// csd_draft_denoise_static: the same kernels as csd_draft_denoise, but every intermediate buffer
+// lives in this one file-scope device array instead of a cudaMalloc'ed workspace.
+constexpr size_t kStaticScratchBytes = size_t(8) << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static void* g_static_scratch_addr[64] = {nullptr};   // device address of the array, per device ordinal
+
+int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_schedule* sched, int R, int cfg,
+                             float cfg_scale, const float* z, const float* x_T, const float* eps, float* x0,
+                             float* mu1, float* x1) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_chain_args(ctx, head, sched, R, cfg, z, x_T, eps);
+  if (rc) return rc;
+  if (!x0 || !mu1) return fail(ctx, CSD_ERR_INVALID_ARG, "x0 / mu1 is null");
+  if (ctx->device < 0 || ctx->device >= 64) return fail(ctx, CSD_ERR_UNSUPPORTED, "device ordinal %d not in [0, 64)", ctx->device);
+  if (ctx->prof_on) return fail(ctx, CSD_ERR_INVALID_ARG, "csd_draft_denoise_static: switch csd_profile off first (recording creates CUDA events)");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  // Bytes the chain's intermediates need, laid out exactly as the growable workspace lays them out
+  // (each piece rounded up to 1 KiB).  Reject before anything is enqueued.
+  const csd_head_desc& d = head->d;
+  const size_t Rh = static_cast<size_t>(R) * (cfg ? 2 : 1), W = d.W, asz = d.dtype == CSD_F32 ? 4 : 2;
+  size_t need = 0;
+  auto take = [&](size_t bytes) { need = align_up(need + bytes, 1024); };
+  take(Rh * d.Dz * asz); take(Rh * W * asz); take(Rh * W * asz); take(Rh * W * asz);
+  take(Rh * W * 4); take(static_cast<size_t>(sched->T) * W * 4); take(Rh * W * 4);
+  take(Rh * (W / kChunk) * 8); take(Rh * (W / kTileN) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
+  if (need > kStaticScratchBytes)
+    return fail(ctx, CSD_ERR_WORKSPACE,
+                "csd_draft_denoise_static: this call needs %zu bytes of scratch but the built-in array holds %zu "
+                "(rows R=%d%s, width %d, T=%d); use csd_draft_denoise or fewer rows", need, kStaticScratchBytes, R,
+                cfg ? " doubled by guidance" : "", d.W, sched->T);
+  // First call on this device: look up the device address of the array (the symbol's name is only a
+  // host-side stand-in and must never be handed to a kernel).
+  if (!g_static_scratch_addr[ctx->device]) {
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess || !p) {
+      cudaGetLastError();
+      return fail(ctx, CSD_ERR_CUDA, "cudaGetSymbolAddress(static scratch) failed: %s", cudaGetErrorString(e));
+    }
+    g_static_scratch_addr[ctx->device] = p;
+  }
+  ChainWs& ws = ctx->ws[2];
+  ws.base = g_static_scratch_addr[ctx->device];
+  ws.cap = kStaticScratchBytes;          // never grown: `need` was checked above
+  return run_chain(ctx, 2, ctx->stream, head, sched, R, cfg, cfg_scale, z, x_T, eps, 1, x0, mu1, x1);
 }
 
 int csd_accept_scan(csd_ctx* ctx, int B, int gamma, int C, double log_sigma_term_, float sigma1_p, float sigma1_q,
