@@ -143,6 +143,19 @@ int make_tmap(csd_ctx* ctx, CUtensorMap* m, int dtype, const void* ptr, uint64_t
   return CSD_OK;
 }
 
+// fp32 [rows, cols] matrix read in boxes of 32 floats (128 bytes, swizzled) x 128 rows.
+int make_tmap_f32(csd_ctx* ctx, CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
+  const cuuint64_t gdim[2] = {cols, rows};
+  const cuuint64_t gstride[1] = {cols * 4};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kChunk), static_cast<cuuint32_t>(kTileM)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, CSD_ERR_CUDA, "cuTensorMapEncodeTiled (fp32) failed with code %d", (int)r);
+  return CSD_OK;
+}
+
 int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, int T) {
   const size_t asz = d.dtype == CSD_F32 ? 4 : 2;
   const size_t W = d.W;
@@ -151,7 +164,7 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   const size_t o_zc = take(static_cast<size_t>(Rh) * d.Dz * asz);
   const size_t o_s = take(Rh * W * asz), o_u = take(Rh * W * asz), o_v = take(Rh * W * asz);
   const size_t o_cz = take(Rh * W * 4), o_te = take(static_cast<size_t>(T) * W * 4), o_h = take(Rh * W * 4);
-  const size_t o_st = take(Rh * (W / kChunk) * 8);
+  const size_t o_st = take(Rh * (W / kStatCols) * 8);
   const size_t o_ep = take(Rh * (W / kTileN) * kCPad * 4);
   const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
   if (off > ws.cap) {
@@ -176,17 +189,23 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
 
 template <int EPI, int NSEG, int MMA_N, typename ACT>
 int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0, const CUtensorMap& a1,
-                const CUtensorMap& b1, int K0, int K1, int N, const EpiParams& ep) {
+                const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int N, const EpiParams& ep) {
   auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, std::is_same<ACT, __half>::value ? 0 : 1>;
   static bool attr_done = false;
-  constexpr int smem = TcCfg<MMA_N>::kSmemBytes;
+  constexpr int smem = TcCfg<EPI, MMA_N>::kSmemBytes;
   if (!attr_done) {
     CSD_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done = true;
   }
   dim3 grid(N / kTileN, (ep.M + kTileM - 1) / kTileM);
   ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * ((NSEG == 1 && MMA_N == 256) ? 2.0 : 1.0));
-  kern<<<grid, kTcThreads, smem, st>>>(a0, b0, a1, b1, K0 / kBlockK, K1 / kBlockK, ep, ctx->d_err);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = ctx->prof_on ? 0 : 1;   // event pairs between launches defeat the overlap anyway
+  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, ep, ctx->d_err));
   ctx->launches++;
   CSD_CUDA(ctx, cudaGetLastError());
   return CSD_OK;
@@ -194,9 +213,10 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
 
 template <int EPI, int NSEG, int MMA_N>
 int launch_tc(csd_ctx* ctx, int dtype, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0,
-              const CUtensorMap& a1, const CUtensorMap& b1, int K0, int K1, int N, const EpiParams& ep) {
-  if (dtype == CSD_F16) return launch_tc_t<EPI, NSEG, MMA_N, __half>(ctx, st, a0, b0, a1, b1, K0, K1, N, ep);
-  return launch_tc_t<EPI, NSEG, MMA_N, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, K0, K1, N, ep);
+              const CUtensorMap& a1, const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int N,
+              const EpiParams& ep) {
+  if (dtype == CSD_F16) return launch_tc_t<EPI, NSEG, MMA_N, __half>(ctx, st, a0, b0, a1, b1, th, K0, K1, N, ep);
+  return launch_tc_t<EPI, NSEG, MMA_N, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, th, K0, K1, N, ep);
 }
 
 template <int EPI, int NSEG, int MMA_N>
@@ -228,16 +248,22 @@ struct Chain {
   int R, cfg; float cfg_scale; const float *z, *x_T, *eps; int sample_last; float *x0, *mu1, *x1;
   int Rh = 0, W = 0, L = 0, T = 0;
   bool tc = false;
-  CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{};
+  CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{}, tm_h{};
   EpiParams ep{};
   StepParams sp{};
 
   int launch_step(int mode) {
     const csd_head_desc& d = hd->d;
     ProfScope ps(ctx, st, 5, 2.0 * Rh * static_cast<double>(W) * d.C);
-    if (d.dtype == CSD_F16) step_kernel<__half><<<R, 256, 0, st>>>(sp, mode);
-    else if (d.dtype == CSD_BF16) step_kernel<__nv_bfloat16><<<R, 256, 0, st>>>(sp, mode);
-    else step_kernel<float><<<R, 256, 0, st>>>(sp, mode);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(R); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = (ctx->prof_on || !tc) ? 0 : 1;
+    if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, step_kernel<__half>, sp, mode));
+    else if (d.dtype == CSD_BF16) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, step_kernel<__nv_bfloat16>, sp, mode));
+    else CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, step_kernel<float>, sp, mode));
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
     return CSD_OK;
@@ -265,11 +291,12 @@ struct Chain {
       if ((rc = make_tmap(ctx, &tm_s, d.dtype, ws.s, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_u, d.dtype, ws.u, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_v, d.dtype, ws.v, Rh, W, W, kTileM))) return rc;
+      if ((rc = make_tmap_f32(ctx, &tm_h, ws.h, Rh, W))) return rc;
     }
     // cz = z Wz^T + bz
     EpiParams e = ep;
     e.bias0 = hd->bz; e.out_f32 = ws.cz;
-    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 128>(ctx, d.dtype, st, tm_z, hd->tmWz, tm_z, hd->tmWz, d.Dz, 0, W, e);
+    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 128>(ctx, d.dtype, st, tm_z, hd->tmWz, tm_z, hd->tmWz, tm_h, d.Dz, 0, W, e);
     else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
                                                 nullptr, 0, W, e);
     if (rc) return rc;
@@ -294,26 +321,26 @@ struct Chain {
       e.h = ws.h; e.stats = ws.stats;
       // u = LN(h)(1 + scale) + shift
       e.bias0 = hd->bsh[k]; e.bias1 = hd->bsc[k]; e.out_act = ws.u;
-      if (tc) rc = launch_tc<EPI_MOD, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWss[k], tm_s, hd->tmWss[k], W, 0, W, e);
+      if (tc) rc = launch_tc<EPI_MOD, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWss[k], tm_s, hd->tmWss[k], tm_h, W, 0, W, e);
       else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
                                              nullptr, 0, W, e);
       if (rc) return rc;
       // v = SiLU(W1 u + b1)
       e.bias0 = hd->b1[k]; e.bias1 = nullptr; e.out_act = ws.v;
-      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 128>(ctx, d.dtype, st, tm_u, hd->tmW1[k], tm_u, hd->tmW1[k], W, 0, W, e);
+      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 128>(ctx, d.dtype, st, tm_u, hd->tmW1[k], tm_u, hd->tmW1[k], tm_h, W, 0, W, e);
       else rc = launch_simt<EPI_SILU_ACT, 1, 128>(ctx, st, uf, W, static_cast<const float*>(hd->W1[k]), W, nullptr, 0,
                                                   nullptr, 0, W, e);
       if (rc) return rc;
       // h += gate * (W2 v + b2)
       e.bias0 = hd->b2[k]; e.bias1 = hd->bg[k]; e.out_act = nullptr;
-      if (tc) rc = launch_tc<EPI_GATE_RES, 2, 128>(ctx, d.dtype, st, tm_v, hd->tmW2[k], tm_s, hd->tmWg[k], W, W, W, e);
+      if (tc) rc = launch_tc<EPI_GATE_RES, 2, 128>(ctx, d.dtype, st, tm_v, hd->tmW2[k], tm_s, hd->tmWg[k], tm_h, W, W, W, e);
       else rc = launch_simt<EPI_GATE_RES, 2, 128>(ctx, st, vf, W, static_cast<const float*>(hd->W2[k]), W, sf, W,
                                                   static_cast<const float*>(hd->Wg[k]), W, W, e);
       if (rc) return rc;
     }
     EpiParams e = ep;
     e.h = ws.h; e.stats = ws.stats; e.bias0 = hd->bfsh; e.bias1 = hd->bfsc; e.wout_t = hd->wout_t; e.epart = ws.epart;
-    if (tc) rc = launch_tc<EPI_MODF, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWfss, tm_s, hd->tmWfss, W, 0, W, e);
+    if (tc) rc = launch_tc<EPI_MODF, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWfss, tm_s, hd->tmWfss, tm_h, W, 0, W, e);
     else rc = launch_simt<EPI_MODF, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
                                             0, W, e);
     if (rc) return rc;
@@ -644,7 +671,7 @@ int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_sched
   auto take = [&](size_t bytes) { need = align_up(need + bytes, 1024); };
   take(Rh * d.Dz * asz); take(Rh * W * asz); take(Rh * W * asz); take(Rh * W * asz);
   take(Rh * W * 4); take(static_cast<size_t>(sched->T) * W * 4); take(Rh * W * 4);
-  take(Rh * (W / kChunk) * 8); take(Rh * (W / kTileN) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
+  take(Rh * (W / kStatCols) * 8); take(Rh * (W / kTileN) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
   if (need > kStaticScratchBytes)
     return fail(ctx, CSD_ERR_WORKSPACE,
                 "csd_draft_denoise_static: this call needs %zu bytes of scratch but the built-in array holds %zu "

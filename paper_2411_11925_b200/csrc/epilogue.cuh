@@ -11,7 +11,8 @@ namespace csd {
 
 constexpr int kTileM = 128;   // rows per tensor-core tile
 constexpr int kTileN = 128;   // output columns per tile
-constexpr int kChunk = 32;    // columns per epilogue chunk and per LayerNorm partial
+constexpr int kChunk = 32;    // columns per epilogue chunk
+constexpr int kStatCols = 128; // columns per LayerNorm partial (one output tile)
 constexpr int kCPad = 16;     // token dim is padded to 16 in Wout^T and the eps partials
 
 enum Epi : int {
@@ -30,7 +31,7 @@ struct EpiParams {
   float* out_f32;        // EPI_BIAS_F32
   void* out_act;         // EPI_SILU_ACT, EPI_MOD
   float* h;              // EPI_MOD / EPI_MODF (read), EPI_GATE_RES (read-modify-write)
-  float* stats;          // [M, ldo/32, 2] (mean, M2) per 32-column group of h
+  float* stats;          // [M, ldo/128, 2] (mean, M2) per 128-column group of h
   const float* wout_t;   // [N, 16] fp32, Wout transposed and zero padded (EPI_MODF)
   float* epart;          // [M, N/128, 16] (EPI_MODF)
 };
@@ -92,35 +93,38 @@ __device__ __forceinline__ void load_chunk_f32(const float* src, float* v) {
 
 // Per-row state carried across the chunks of one tile.
 struct RowState {
-  float mean, rstd;
-  float eacc[kCPad];
+  float mean, rstd;          // LayerNorm statistics of the row (EPI_MOD, EPI_MODF)
+  float eacc[kCPad];         // eps_hat partial sums (EPI_MODF)
+  float pm, pm2, pn;         // running (mean, M2, count) of the new h values (EPI_GATE_RES)
 };
 
-// Merge the per-32-column (mean, M2) partials of row m in a fixed order (Chan et al.), so the
-// LayerNorm statistics do not depend on which CTA computes them.  Loads are issued eight at a time.
+// Chan et al. merge of two (mean, M2, count) triples; b is merged into a.
+__device__ __forceinline__ void chan_merge(float& ma, float& m2a, float& na, float mb, float m2b, float nb) {
+  if (nb <= 0.0f) return;
+  if (na <= 0.0f) { ma = mb; m2a = m2b; na = nb; return; }
+  const float n = na + nb;
+  const float d = mb - ma;
+  ma += d * (nb / n);
+  m2a += m2b + d * d * (na * nb / n);
+  na = n;
+}
+
+// Merge the per-128-column (mean, M2) partials of row m in a fixed order, so the LayerNorm
+// statistics do not depend on which CTA computes them.  All loads are issued before the merges.
 __device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
-  const int G = W / kChunk;
+  const int G = W / kStatCols;
   const float2* p = reinterpret_cast<const float2*>(stats) + static_cast<size_t>(m) * G;
-  float2 a = make_float2(0.0f, 0.0f);
-  float na = 0.0f;
-  for (int g0 = 0; g0 < G; g0 += 8) {
-    float2 b[8];
+  float ma = 0.0f, m2a = 0.0f, na = 0.0f;
+  for (int g0 = 0; g0 < G; g0 += 12) {
+    float2 b[12];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) b[j] = (g0 + j < G) ? p[g0 + j] : make_float2(0.0f, 0.0f);
+    for (int j = 0; j < 12; ++j) b[j] = (g0 + j < G) ? p[g0 + j] : make_float2(0.0f, 0.0f);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if (g0 + j < G) {
-        const float nb = static_cast<float>(kChunk);
-        const float n = na + nb;
-        const float d = b[j].x - a.x;
-        a.x += d * (nb / n);
-        a.y += b[j].y + d * d * (na * nb / n);
-        na = n;
-      }
-    }
+    for (int j = 0; j < 12; ++j)
+      if (g0 + j < G) chan_merge(ma, m2a, na, b[j].x, b[j].y, static_cast<float>(kStatCols));
   }
-  mean = a.x;
-  rstd = 1.0f / sqrtf(a.y / static_cast<float>(W) + 1e-6f);
+  mean = ma;
+  rstd = 1.0f / sqrtf(m2a / static_cast<float>(W) + 1e-6f);
 }
 
 template <int EPI>
@@ -130,6 +134,7 @@ __device__ __forceinline__ void epi_row_begin(const EpiParams& ep, int m, RowSta
 #pragma unroll
     for (int c = 0; c < kCPad; ++c) rs.eacc[c] = 0.0f;
   }
+  if constexpr (EPI == EPI_GATE_RES) { rs.pm = 0.0f; rs.pm2 = 0.0f; rs.pn = 0.0f; }
 }
 
 template <int EPI> __host__ __device__ constexpr bool epi_reads_h() { return EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES; }
@@ -191,9 +196,13 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, fl
       const float d = hv[j] - mean;
       m2 = fmaf(d, d, m2);
     }
-    reinterpret_cast<float2*>(ep.stats)[static_cast<size_t>(m) * (ep.ldo / kChunk) + n0 / kChunk] =
-        make_float2(mean, m2);
+    chan_merge(rs.pm, rs.pm2, rs.pn, mean, m2, static_cast<float>(kChunk));
   }
+}
+
+// Writes the (mean, M2) partial of one row over one whole 128-column tile.
+__device__ __forceinline__ void store_tile_stats(const EpiParams& ep, int m, int tile_n, float mean, float m2) {
+  reinterpret_cast<float2*>(ep.stats)[static_cast<size_t>(m) * (ep.ldo / kStatCols) + tile_n] = make_float2(mean, m2);
 }
 
 template <int EPI>

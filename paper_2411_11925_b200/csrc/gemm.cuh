@@ -15,38 +15,57 @@
 namespace csd {
 
 constexpr int kBlockK = 64;  // bf16 elements per TMA box row = 128 bytes = one swizzle row
-constexpr int kTcThreads = 320;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int kTcThreads = 352;   // warp 0 TMA (A), warp 1 MMA, warps 2..9 epilogue, warp 10 TMA (B)
 constexpr int kEpiThreads = 256;
 
 enum DevErr : int { DEV_OK = 0, DEV_ERR_TMA_WAIT = 1, DEV_ERR_MMA_WAIT = 2, DEV_ERR_EPI_WAIT = 3 };
 
-template <int MMA_N> struct TcCfg {
-  static constexpr int kStages = (MMA_N == 256) ? 4 : 6;
+constexpr int kHTileBytes = kTileM * kTileN * 4;   // fp32 h tile staged in shared memory (64 KB)
+
+template <int EPI, int MMA_N> struct TcCfg {
+  static constexpr bool kStageH = EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES;
   static constexpr int kABytes = kTileM * kBlockK * 2;
   static constexpr int kBBytes = MMA_N * kBlockK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kHBytes = kStageH ? kHTileBytes : 0;
   static constexpr int kWoutBytes = kTileN * kCPad * 4;      // Wout^T tile, reused for the eps partials
-  static constexpr int kBiasBytes = 2 * kTileN * 4;
-  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kWoutBytes + kBiasBytes + 256;
+  static constexpr int kMiscBytes = 2 * kTileN * 4 + kTileM * 16;   // two bias slices + per-row exchange
+  static constexpr int kFixedBytes = 1024 + kHBytes + kWoutBytes + kMiscBytes + 256;
+  static constexpr int kStages = (227 * 1024 - kFixedBytes) / kStageBytes;   // 6 (N=128), 4 (N=128 + h), 3 (N=256 + h)
+  static constexpr int kSmemBytes = kFixedBytes + kStages * kStageBytes;
 };
+
+// Reads 32 consecutive floats of row r from a [128 rows][128 bytes] tile that TMA wrote with the
+// 128-byte swizzle (16-byte unit j of row r lives at unit j ^ (r & 7)).
+__device__ __forceinline__ void load_swizzled_row32(const uint8_t* tile, int r, float* v) {
+  const uint8_t* row = tile + r * 128;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float4 q = *reinterpret_cast<const float4*>(row + ((j ^ (r & 7)) << 4));
+    v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+  }
+}
 
 template <int EPI, typename ACT, int NSEG, int MMA_N, int AB_FMT>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
-               int nkb0, int nkb1, EpiParams ep, int* err) {
-  using Cfg = TcCfg<MMA_N>;
+               const __grid_constant__ CUtensorMap tmH, int nkb0, int nkb1, EpiParams ep, int* err) {
+  using Cfg = TcCfg<EPI, MMA_N>;
   constexpr int S = Cfg::kStages;
   constexpr uint32_t kTmemCols = NSEG * MMA_N;  // 128 or 256: a power of two >= 32
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stage_base = smem;
-  float* wout_s = reinterpret_cast<float*>(smem + S * Cfg::kStageBytes);
-  float* bias_s = reinterpret_cast<float*>(smem + S * Cfg::kStageBytes + Cfg::kWoutBytes);
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + S * Cfg::kStageBytes + Cfg::kWoutBytes + Cfg::kBiasBytes);
+  uint8_t* h_s = smem + S * Cfg::kStageBytes;                    // 4 chunks of [128 rows][128 B], swizzled
+  float* wout_s = reinterpret_cast<float*>(h_s + Cfg::kHBytes);
+  float* bias_s = reinterpret_cast<float*>(h_s + Cfg::kHBytes + Cfg::kWoutBytes);
+  float* xch_s = bias_s + 2 * kTileN;                            // [128 rows][4] exchange between column halves
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(h_s + Cfg::kHBytes + Cfg::kWoutBytes + Cfg::kMiscBytes);
   uint64_t* empty_bar = full_bar + S;
   uint64_t* tmem_full_bar = empty_bar + S;
-  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_full_bar + 1);
+  uint64_t* h_bar = tmem_full_bar + 1;
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(h_bar + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile_n = blockIdx.x, tile_m = blockIdx.y;
@@ -63,8 +82,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     tma_prefetch_desc(&tmA0);
     tma_prefetch_desc(&tmB0);
     if (NSEG == 2) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
-    for (int s = 0; s < S; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    if (Cfg::kStageH) tma_prefetch_desc(&tmH);
+    for (int s = 0; s < S; ++s) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
     mbar_init(tmem_full_bar, 1);
+    mbar_init(h_bar, 1);
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -75,21 +96,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_base_s;
+  if (threadIdx.x == 0) griddep_launch_dependents();
 
-  if (warp == 0) {
-    if (lane == 0) {
-      for (int kb = 0; kb < total_kb; ++kb) {
+  // Two TMA producers: one thread sustains only about one request per 240 clk, so the activation
+  // tiles (A, warp 0) and the weight tiles (B, warp 10) are requested by different warps; each arms
+  // the stage's barrier with its own byte count.
+  auto produce = [&](const CUtensorMap* t0, const CUtensorMap* t1, uint32_t bytes, int off, int crd) {
+    bool ok = true;
+    for (int kb = 0; kb < nkb0 && ok; ++kb) {
+      const int s = kb % S;
+      if (kb >= S && !mbar_wait(&empty_bar[s], ((kb / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
+      mbar_arrive_expect_tx(&full_bar[s], bytes);
+      tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t0, &full_bar[s], kb * kBlockK, crd);
+    }
+    if (NSEG == 2) {
+      for (int kb = nkb0; kb < total_kb && ok; ++kb) {
         const int s = kb % S;
-        const uint32_t ph = (kb / S) & 1;
-        if (!mbar_wait(&empty_bar[s], ph ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); break; }
-        mbar_arrive_expect_tx(&full_bar[s], Cfg::kStageBytes);
-        const bool second = (NSEG == 2) && (kb >= nkb0);
-        const int kk = second ? kb - nkb0 : kb;
-        uint8_t* sa = stage_base + s * Cfg::kStageBytes;
-        tma_load_2d(sa, second ? &tmA1 : &tmA0, &full_bar[s], kk * kBlockK, tile_m * kTileM);
-        tma_load_2d(sa + Cfg::kABytes, second ? &tmB1 : &tmB0, &full_bar[s], kk * kBlockK, tile_n * MMA_N);
+        if (kb >= S && !mbar_wait(&empty_bar[s], ((kb / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
+        mbar_arrive_expect_tx(&full_bar[s], bytes);
+        tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t1, &full_bar[s], (kb - nkb0) * kBlockK, crd);
       }
     }
+  };
+  if (warp == 0) {            // activation tiles and the h tile: produced by the preceding kernels
+    if (lane == 0) {
+      griddep_wait();
+      if (Cfg::kStageH) {
+        // The epilogue's h tile goes first: ordinary loads issued while the pipeline saturates the
+        // SM's shared-memory port would take thousands of cycles.
+        mbar_arrive_expect_tx(h_bar, kHTileBytes);
+#pragma unroll
+        for (int c = 0; c < kTileN / kChunk; ++c)
+          tma_load_2d(h_s + c * (kTileM * 128), &tmH, h_bar, tile_n * kTileN + c * kChunk, tile_m * kTileM);
+      }
+      produce(&tmA0, &tmA1, Cfg::kABytes, 0, tile_m * kTileM);
+    }
+    __syncwarp();
+  } else if (warp == 10) {    // weight tiles: never depend on the preceding kernel
+    if (lane == 0) produce(&tmB0, &tmB1, Cfg::kBBytes, Cfg::kABytes, tile_n * MMA_N);
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
@@ -107,7 +151,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes);
         const uint32_t d = tmem_base + (second ? MMA_N : 0);
 #pragma unroll
-        for (int k = 0; k < kBlockK / 16; ++k)  // UMMA_K = 16 bf16 = 32 bytes = 2 descriptor units
+        for (int k = 0; k < kBlockK / 16; ++k)  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
           umma_f16(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
         umma_commit(&empty_bar[s]);
       }
@@ -116,11 +160,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     __syncwarp();
   } else {
     // Epilogue, 8 warps: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32); warps 2..5 take
-    // column chunks 0 and 1 of the tile, warps 6..9 chunks 2 and 3.  Everything that does not need
-    // the accumulators (biases, Wout^T tile, LayerNorm statistics, h) is fetched while the MMAs run.
+    // column chunks 0 and 1 of the tile, warps 6..9 chunks 2 and 3.  What does not need the
+    // accumulators (biases, Wout^T tile, LayerNorm partials) is fetched right away.
     const int et = threadIdx.x - 64;
     const int q = warp & 3, half = (warp - 2) >> 2;
-    const int m = tile_m * kTileM + q * 32 + lane;
+    const int rloc = q * 32 + lane;
+    const int m = tile_m * kTileM + rloc;
     const bool valid = m < ep.M;
     if (et < kTileN) {
       bias_s[et] = ep.bias0[tile_n * kTileN + et];
@@ -132,18 +177,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
       for (int i = 0; i < kTileN * kCPad / 4 / kEpiThreads; ++i) dst[et + i * kEpiThreads] = src[et + i * kEpiThreads];
     }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
+    griddep_wait();   // the LayerNorm partials come from the preceding kernels
     RowState rs;
-    float hv[2][kChunk];
-    if (valid) {
-      epi_row_begin<EPI>(ep, m, rs);
-      if (epi_reads_h<EPI>()) {
-#pragma unroll
-        for (int ci = 0; ci < 2; ++ci)
-          load_chunk_f32(ep.h + static_cast<size_t>(m) * ep.ldo + tile_n * kTileN + (2 * half + ci) * kChunk, hv[ci]);
-      }
-    }
+    if (valid) epi_row_begin<EPI>(ep, m, rs);
+    asm volatile("bar.sync 1, 256;" ::: "memory");   // biases and the Wout^T tile are in place
     bool ok = mbar_wait(tmem_full_bar, 0);
+    if (ok && Cfg::kStageH) ok = mbar_wait(h_bar, 0);
     if (!ok) atomicExch(err, DEV_ERR_EPI_WAIT);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
@@ -152,13 +191,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
       for (int ci = 0; ci < 2; ++ci) {
         const int c = 2 * half + ci;
-        float a0[kChunk], a1[kChunk];
+        float a0[kChunk], a1[kChunk], hv[kChunk];
         tmem_ld32(trow + c * kChunk, a0);
         if (NSEG * MMA_N == 256) tmem_ld32(trow + kTileN + c * kChunk, a1);
+        if (Cfg::kStageH) load_swizzled_row32(h_s + c * (kTileM * 128), rloc, hv);
         tmem_ld_wait();
         if (valid)
           epi_chunk<EPI, ACT, true>(ep, m, tile_n * kTileN + c * kChunk, a0, a1, bias_s + c * kChunk,
-                                    bias_s + kTileN + c * kChunk, hv[ci], rs, wout_s + c * kChunk * kCPad);
+                                    bias_s + kTileN + c * kChunk, hv, rs, wout_s + c * kChunk * kCPad);
+      }
+    }
+    if (EPI == EPI_GATE_RES) {
+      // one (mean, M2) partial per row over the whole tile: columns 64..127 are merged into 0..63
+      if (half == 1) { xch_s[rloc * 4] = rs.pm; xch_s[rloc * 4 + 1] = rs.pm2; xch_s[rloc * 4 + 2] = rs.pn; }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (half == 0 && ok && valid) {
+        chan_merge(rs.pm, rs.pm2, rs.pn, xch_s[rloc * 4], xch_s[rloc * 4 + 1], xch_s[rloc * 4 + 2]);
+        store_tile_stats(ep, m, tile_n, rs.pm, rs.pm2);
       }
     }
     if (EPI == EPI_MODF) {
@@ -167,12 +216,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       float* part = wout_s;                            // [128 rows][16]
       if (half == 1 && ok) {
 #pragma unroll
-        for (int c = 0; c < kCPad; ++c) part[(q * 32 + lane) * kCPad + c] = rs.eacc[c];
+        for (int c = 0; c < kCPad; ++c) part[rloc * kCPad + c] = rs.eacc[c];
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (half == 0 && ok && valid) {
 #pragma unroll
-        for (int c = 0; c < kCPad; ++c) rs.eacc[c] += part[(q * 32 + lane) * kCPad + c];
+        for (int c = 0; c < kCPad; ++c) rs.eacc[c] += part[rloc * kCPad + c];
         epi_row_end<EPI>(ep, m, tile_n, rs);
       }
     }
@@ -253,6 +302,18 @@ gemm_simt_kernel(const float* __restrict__ A0, int lda0, const float* __restrict
     if (epi_reads_h<EPI>()) load_chunk_f32(ep.h + static_cast<size_t>(m) * ep.ldo + n0, hv);
     epi_chunk<EPI, float, false>(ep, m, n0, acc0, acc1, ep.bias0 + n0, ep.bias1 ? ep.bias1 + n0 : ep.bias0 + n0, hv, rs,
                                  wout_s + warp * kChunk * kCPad);
+  }
+  if constexpr (EPI == EPI_GATE_RES) {
+    float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][4]
+    __syncthreads();
+    if (m < ep.M) { scr[(warp * kSimtRows + lane) * 4] = rs.pm; scr[(warp * kSimtRows + lane) * 4 + 1] = rs.pm2; }
+    __syncthreads();
+    if (warp == 0 && m < ep.M) {
+      float pm = 0.0f, pm2 = 0.0f, pn = 0.0f;
+      for (int w = 0; w < 4; ++w)
+        chan_merge(pm, pm2, pn, scr[(w * kSimtRows + lane) * 4], scr[(w * kSimtRows + lane) * 4 + 1], static_cast<float>(kChunk));
+      store_tile_stats(ep, m, tile_n, pm, pm2);
+    }
   }
   if constexpr (EPI == EPI_MODF) {
     float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][16]

@@ -3,6 +3,7 @@
 // condition vector s), and the verification / resampling kernels.
 #pragma once
 #include "epilogue.cuh"
+#include "ptx.cuh"
 
 namespace csd {
 
@@ -57,7 +58,7 @@ struct StepParams {
   const float* cz;               // [Rh, W]
   const float* te_next;          // [W] embedding of the step being prepared
   float* h;                      // [Rh, W]
-  float* stats;                  // [Rh, W/32, 2]
+  float* stats;                  // [Rh, W/128, 2]
   void* s;                       // [Rh, W] activations
 };
 
@@ -71,6 +72,8 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
   __shared__ float eh[2][kCPad];
   const int r = blockIdx.x, tid = threadIdx.x;
   const int nrep = p.cfg ? 2 : 1;
+  if (tid == 0) griddep_launch_dependents();
+  griddep_wait();
   if (mode == STEP_INIT) {
     if (tid < kCPad) xs[tid] = (tid < p.C) ? p.x_src[static_cast<size_t>(r) * p.C + tid] : 0.0f;
     if (tid < p.C) p.x[static_cast<size_t>(r) * p.C + tid] = p.x_src[static_cast<size_t>(r) * p.C + tid];
@@ -106,34 +109,44 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
     if (mode == STEP_LAST) return;
     __syncthreads();
   }
-  // prepare: each warp handles 32 consecutive columns at a time (lane = column)
+  // prepare: each warp handles 128 consecutive columns at a time (lane + 32 j), one LayerNorm partial
   const int lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
   ACT* s = reinterpret_cast<ACT*>(p.s);
-  for (int g = warp; g < p.W / kChunk; g += nwarp) {
-    const int n = g * kChunk + lane;
-    const float4* w4 = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(n) * kCPad);
-    float acc = p.bin[n];
+  for (int g = warp; g < p.W / kStatCols; g += nwarp) {
+    float acc[4];
+    float sum = 0.0f;
 #pragma unroll
-    for (int c4 = 0; c4 < kCPad / 4; ++c4) {
-      const float4 w = w4[c4];
-      acc = fmaf(w.x, xs[4 * c4], acc); acc = fmaf(w.y, xs[4 * c4 + 1], acc);
-      acc = fmaf(w.z, xs[4 * c4 + 2], acc); acc = fmaf(w.w, xs[4 * c4 + 3], acc);
+    for (int j = 0; j < 4; ++j) {
+      const int n = g * kStatCols + j * 32 + lane;
+      const float4* w4 = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(n) * kCPad);
+      float a = p.bin[n];
+#pragma unroll
+      for (int c4 = 0; c4 < kCPad / 4; ++c4) {
+        const float4 w = w4[c4];
+        a = fmaf(w.x, xs[4 * c4], a); a = fmaf(w.y, xs[4 * c4 + 1], a);
+        a = fmaf(w.z, xs[4 * c4 + 2], a); a = fmaf(w.w, xs[4 * c4 + 3], a);
+      }
+      acc[j] = a;
+      sum += a;
     }
-    float sum = acc;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    const float mean = sum * (1.0f / kChunk);
-    const float d = acc - mean;
-    float m2 = d * d;
+    const float mean = sum * (1.0f / kStatCols);
+    float m2 = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { const float d = acc[j] - mean; m2 = fmaf(d, d, m2); }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
-    const float te = p.te_next[n];
     for (int rep = 0; rep < nrep; ++rep) {
       const size_t row = static_cast<size_t>(r) + static_cast<size_t>(rep) * p.R;
-      p.h[row * p.W + n] = acc;
       if (lane == 0)
-        reinterpret_cast<float2*>(p.stats)[row * (p.W / kChunk) + g] = make_float2(mean, m2);
-      s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + te));
+        reinterpret_cast<float2*>(p.stats)[row * (p.W / kStatCols) + g] = make_float2(mean, m2);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int n = g * kStatCols + j * 32 + lane;
+        p.h[row * p.W + n] = acc[j];
+        s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + p.te_next[n]));
+      }
     }
   }
 }
