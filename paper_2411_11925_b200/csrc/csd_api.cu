@@ -189,7 +189,7 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
 
 template <int EPI, int NSEG, int MMA_N, typename ACT>
 int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0, const CUtensorMap& a1,
-                const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int N, const EpiParams& ep) {
+                const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k, int N, const EpiParams& ep) {
   auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, std::is_same<ACT, __half>::value ? 0 : 1>;
   static bool attr_done = false;
   constexpr int smem = TcCfg<EPI, MMA_N>::kSmemBytes;
@@ -200,12 +200,12 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
   dim3 grid(N / kTileN, (ep.M + kTileM - 1) / kTileM);
   ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * ((NSEG == 1 && MMA_N == 256) ? 2.0 : 1.0));
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = grid; cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cfg.gridDim = grid; cfg.blockDim = dim3(TcWarps<EPI>::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at; cfg.numAttrs = ctx->prof_on ? 0 : 1;   // event pairs between launches defeat the overlap anyway
-  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, ep, ctx->d_err));
+  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, ep, ctx->d_err));
   ctx->launches++;
   CSD_CUDA(ctx, cudaGetLastError());
   return CSD_OK;
@@ -213,10 +213,11 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
 
 template <int EPI, int NSEG, int MMA_N>
 int launch_tc(csd_ctx* ctx, int dtype, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0,
-              const CUtensorMap& a1, const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int N,
-              const EpiParams& ep) {
-  if (dtype == CSD_F16) return launch_tc_t<EPI, NSEG, MMA_N, __half>(ctx, st, a0, b0, a1, b1, th, K0, K1, N, ep);
-  return launch_tc_t<EPI, NSEG, MMA_N, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, th, K0, K1, N, ep);
+              const CUtensorMap& a1, const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k,
+              int N, const EpiParams& ep) {
+  // dep_k: first K index (over both segments) whose A operand is written by the preceding kernel
+  if (dtype == CSD_F16) return launch_tc_t<EPI, NSEG, MMA_N, __half>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+  return launch_tc_t<EPI, NSEG, MMA_N, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
 }
 
 template <int EPI, int NSEG, int MMA_N>
@@ -296,7 +297,7 @@ struct Chain {
     // cz = z Wz^T + bz
     EpiParams e = ep;
     e.bias0 = hd->bz; e.out_f32 = ws.cz;
-    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 128>(ctx, d.dtype, st, tm_z, hd->tmWz, tm_z, hd->tmWz, tm_h, d.Dz, 0, W, e);
+    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 128>(ctx, d.dtype, st, tm_z, hd->tmWz, tm_z, hd->tmWz, tm_h, d.Dz, 0, 0, W, e);
     else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
                                                 nullptr, 0, W, e);
     if (rc) return rc;
@@ -321,26 +322,31 @@ struct Chain {
       e.h = ws.h; e.stats = ws.stats;
       // u = LN(h)(1 + scale) + shift
       e.bias0 = hd->bsh[k]; e.bias1 = hd->bsc[k]; e.out_act = ws.u;
-      if (tc) rc = launch_tc<EPI_MOD, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWss[k], tm_s, hd->tmWss[k], tm_h, W, 0, W, e);
+      if (tc) rc = launch_tc<EPI_MOD, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWss[k], tm_s, hd->tmWss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
       else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
                                              nullptr, 0, W, e);
       if (rc) return rc;
       // v = SiLU(W1 u + b1)
       e.bias0 = hd->b1[k]; e.bias1 = nullptr; e.out_act = ws.v;
-      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 128>(ctx, d.dtype, st, tm_u, hd->tmW1[k], tm_u, hd->tmW1[k], tm_h, W, 0, W, e);
+      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 128>(ctx, d.dtype, st, tm_u, hd->tmW1[k], tm_u, hd->tmW1[k], tm_h, W, 0, 0, W, e);
       else rc = launch_simt<EPI_SILU_ACT, 1, 128>(ctx, st, uf, W, static_cast<const float*>(hd->W1[k]), W, nullptr, 0,
                                                   nullptr, 0, W, e);
       if (rc) return rc;
-      // h += gate * (W2 v + b2)
+      // h += gate * (W2 v + b2).  On the tensor-core path the gate product s Wg^T comes first: it does
+      // not depend on the preceding kernel (which writes v) and overlaps with it.
       e.bias0 = hd->b2[k]; e.bias1 = hd->bg[k]; e.out_act = nullptr;
-      if (tc) rc = launch_tc<EPI_GATE_RES, 2, 128>(ctx, d.dtype, st, tm_v, hd->tmW2[k], tm_s, hd->tmWg[k], tm_h, W, W, W, e);
+      if (tc) {
+        EpiParams g = e;
+        g.bias0 = hd->bg[k]; g.bias1 = hd->b2[k];
+        rc = launch_tc<EPI_GATE_RES, 2, 128>(ctx, d.dtype, st, tm_s, hd->tmWg[k], tm_v, hd->tmW2[k], tm_h, W, W, W, W, g);
+      }
       else rc = launch_simt<EPI_GATE_RES, 2, 128>(ctx, st, vf, W, static_cast<const float*>(hd->W2[k]), W, sf, W,
                                                   static_cast<const float*>(hd->Wg[k]), W, W, e);
       if (rc) return rc;
     }
     EpiParams e = ep;
     e.h = ws.h; e.stats = ws.stats; e.bias0 = hd->bfsh; e.bias1 = hd->bfsc; e.wout_t = hd->wout_t; e.epart = ws.epart;
-    if (tc) rc = launch_tc<EPI_MODF, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWfss, tm_s, hd->tmWfss, tm_h, W, 0, W, e);
+    if (tc) rc = launch_tc<EPI_MODF, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWfss, tm_s, hd->tmWfss, tm_h, W, 0, W, W, e);
     else rc = launch_simt<EPI_MODF, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
                                             0, W, e);
     if (rc) return rc;

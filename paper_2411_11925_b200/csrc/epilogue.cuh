@@ -109,6 +109,13 @@ __device__ __forceinline__ void chan_merge(float& ma, float& m2a, float& na, flo
   na = n;
 }
 
+// Same for two partials of equal count n (no division): mean = (ma + mb)/2, M2 = M2a + M2b + d^2 n/2.
+__device__ __forceinline__ void chan_merge_equal(float& ma, float& m2a, float mb, float m2b, float n) {
+  const float d = mb - ma;
+  ma = fmaf(d, 0.5f, ma);
+  m2a += m2b + d * d * (0.5f * n);
+}
+
 // Merge the per-128-column (mean, M2) partials of row m in a fixed order, so the LayerNorm
 // statistics do not depend on which CTA computes them.  All loads are issued before the merges.
 __device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
@@ -196,7 +203,10 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, fl
       const float d = hv[j] - mean;
       m2 = fmaf(d, d, m2);
     }
-    chan_merge(rs.pm, rs.pm2, rs.pn, mean, m2, static_cast<float>(kChunk));
+    // a thread owns one or two chunks of the tile: the second is merged with equal counts
+    if (rs.pn <= 0.0f) { rs.pm = mean; rs.pm2 = m2; }
+    else chan_merge_equal(rs.pm, rs.pm2, mean, m2, static_cast<float>(kChunk));
+    rs.pn += static_cast<float>(kChunk);
   }
 }
 

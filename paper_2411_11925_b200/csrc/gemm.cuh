@@ -15,8 +15,13 @@
 namespace csd {
 
 constexpr int kBlockK = 64;  // bf16 elements per TMA box row = 128 bytes = one swizzle row
-constexpr int kTcThreads = 352;   // warp 0 TMA (A), warp 1 MMA, warps 2..9 epilogue, warp 10 TMA (B)
-constexpr int kEpiThreads = 256;
+// Warp roles: warp 0 TMA (A), warp 1 MMA, then the epilogue warps, last warp TMA (B).  The cheap
+// epilogues run 16 warps (one 32-column chunk per thread), the register-heavy ones 8 (two chunks).
+template <int EPI> struct TcWarps {
+  static constexpr int kEpi = (EPI == EPI_SILU_ACT || EPI == EPI_BIAS_F32) ? 16 : 8;
+  static constexpr int kThreads = (kEpi + 3) * 32;
+  static constexpr int kChunksPerThread = 16 / kEpi;   // 4 chunks x 4 lane quarters over kEpi warps
+};
 
 enum DevErr : int { DEV_OK = 0, DEV_ERR_TMA_WAIT = 1, DEV_ERR_MMA_WAIT = 2, DEV_ERR_EPI_WAIT = 3 };
 
@@ -47,12 +52,13 @@ __device__ __forceinline__ void load_swizzled_row32(const uint8_t* tile, int r, 
 }
 
 template <int EPI, typename ACT, int NSEG, int MMA_N, int AB_FMT>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(TcWarps<EPI>::kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
-               const __grid_constant__ CUtensorMap tmH, int nkb0, int nkb1, EpiParams ep, int* err) {
+               const __grid_constant__ CUtensorMap tmH, int nkb0, int nkb1, int dep_kb, EpiParams ep, int* err) {
   using Cfg = TcCfg<EPI, MMA_N>;
   constexpr int S = Cfg::kStages;
+  constexpr int EW = TcWarps<EPI>::kEpi, CPT = TcWarps<EPI>::kChunksPerThread, kEpiThreads = EW * 32;
   constexpr uint32_t kTmemCols = NSEG * MMA_N;  // 128 or 256: a power of two >= 32
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -96,15 +102,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_base_s;
-  if (threadIdx.x == 0) griddep_launch_dependents();
 
   // Two TMA producers: one thread sustains only about one request per 240 clk, so the activation
   // tiles (A, warp 0) and the weight tiles (B, warp 10) are requested by different warps; each arms
-  // the stage's barrier with its own byte count.
-  auto produce = [&](const CUtensorMap* t0, const CUtensorMap* t1, uint32_t bytes, int off, int crd) {
+  // the stage's barrier with its own byte count.  Weights never depend on the preceding kernel; of
+  // the activations only k-blocks >= dep_kb do (the A producer waits for it there), so the part of
+  // the product that is independent of the preceding kernel overlaps with that kernel.
+  auto produce = [&](const CUtensorMap* t0, const CUtensorMap* t1, uint32_t bytes, int off, int crd, int wait_kb) {
     bool ok = true;
     for (int kb = 0; kb < nkb0 && ok; ++kb) {
       const int s = kb % S;
+      if (kb == wait_kb) griddep_wait();
       if (kb >= S && !mbar_wait(&empty_bar[s], ((kb / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
       mbar_arrive_expect_tx(&full_bar[s], bytes);
       tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t0, &full_bar[s], kb * kBlockK, crd);
@@ -112,28 +120,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (NSEG == 2) {
       for (int kb = nkb0; kb < total_kb && ok; ++kb) {
         const int s = kb % S;
+        if (kb == wait_kb) griddep_wait();
         if (kb >= S && !mbar_wait(&empty_bar[s], ((kb / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
         mbar_arrive_expect_tx(&full_bar[s], bytes);
         tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t1, &full_bar[s], (kb - nkb0) * kBlockK, crd);
       }
     }
   };
-  if (warp == 0) {            // activation tiles and the h tile: produced by the preceding kernels
-    if (lane == 0) {
-      griddep_wait();
-      if (Cfg::kStageH) {
-        // The epilogue's h tile goes first: ordinary loads issued while the pipeline saturates the
-        // SM's shared-memory port would take thousands of cycles.
-        mbar_arrive_expect_tx(h_bar, kHTileBytes);
-#pragma unroll
-        for (int c = 0; c < kTileN / kChunk; ++c)
-          tma_load_2d(h_s + c * (kTileM * 128), &tmH, h_bar, tile_n * kTileN + c * kChunk, tile_m * kTileM);
-      }
-      produce(&tmA0, &tmA1, Cfg::kABytes, 0, tile_m * kTileM);
-    }
+  if (warp == 0) {            // activation tiles
+    if (lane == 0) produce(&tmA0, &tmA1, Cfg::kABytes, 0, tile_m * kTileM, dep_kb);
     __syncwarp();
-  } else if (warp == 10) {    // weight tiles: never depend on the preceding kernel
-    if (lane == 0) produce(&tmB0, &tmB1, Cfg::kBBytes, Cfg::kABytes, tile_n * MMA_N);
+  } else if (warp == EW + 2) {    // weight tiles
+    if (lane == 0) produce(&tmB0, &tmB1, Cfg::kBBytes, Cfg::kABytes, tile_n * MMA_N, -1);
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
@@ -159,11 +157,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     }
     __syncwarp();
   } else {
-    // Epilogue, 8 warps: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32); warps 2..5 take
-    // column chunks 0 and 1 of the tile, warps 6..9 chunks 2 and 3.  What does not need the
-    // accumulators (biases, Wout^T tile, LayerNorm partials) is fetched right away.
+    // Epilogue: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32).  With 8 warps, warps 2..5
+    // take column chunks 0 and 1 of the tile and warps 6..9 chunks 2 and 3; with 16 warps each group
+    // of four takes one chunk.  What does not need the accumulators (biases, Wout^T tile, LayerNorm
+    // partials) is fetched right away.
     const int et = threadIdx.x - 64;
-    const int q = warp & 3, half = (warp - 2) >> 2;
+    const int q = warp & 3, half = (warp - 2) >> 2;   // half = chunk group
     const int rloc = q * 32 + lane;
     const int m = tile_m * kTileM + rloc;
     const bool valid = m < ep.M;
@@ -177,10 +176,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
       for (int i = 0; i < kTileN * kCPad / 4 / kEpiThreads; ++i) dst[et + i * kEpiThreads] = src[et + i * kEpiThreads];
     }
-    griddep_wait();   // the LayerNorm partials come from the preceding kernels
+    // h, the LayerNorm partials and the right to overwrite this kernel's outputs come with the
+    // completion of the preceding kernel.  Only then may the next kernel start its own early part
+    // (at most one kernel runs ahead), and the h tile is requested before this thread block's
+    // remaining pipeline traffic queues up behind it.
+    griddep_wait();
+    if (et == 0) {
+      griddep_launch_dependents();
+      if (Cfg::kStageH) {
+        mbar_arrive_expect_tx(h_bar, kHTileBytes);
+#pragma unroll
+        for (int c = 0; c < kTileN / kChunk; ++c)
+          tma_load_2d(h_s + c * (kTileM * 128), &tmH, h_bar, tile_n * kTileN + c * kChunk, tile_m * kTileM);
+      }
+    }
     RowState rs;
     if (valid) epi_row_begin<EPI>(ep, m, rs);
-    asm volatile("bar.sync 1, 256;" ::: "memory");   // biases and the Wout^T tile are in place
+    asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // biases and the Wout^T tile are in place
     bool ok = mbar_wait(tmem_full_bar, 0);
     if (ok && Cfg::kStageH) ok = mbar_wait(h_bar, 0);
     if (!ok) atomicExch(err, DEV_ERR_EPI_WAIT);
@@ -189,8 +201,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       tc_fence_after_sync();
       const uint32_t trow = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll
-      for (int ci = 0; ci < 2; ++ci) {
-        const int c = 2 * half + ci;
+      for (int ci = 0; ci < CPT; ++ci) {
+        const int c = CPT * half + ci;
         float a0[kChunk], a1[kChunk], hv[kChunk];
         tmem_ld32(trow + c * kChunk, a0);
         if (NSEG * MMA_N == 256) tmem_ld32(trow + kTileN + c * kChunk, a1);
@@ -203,10 +215,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     }
     if (EPI == EPI_GATE_RES) {
       // one (mean, M2) partial per row over the whole tile: columns 64..127 are merged into 0..63
-      if (half == 1) { xch_s[rloc * 4] = rs.pm; xch_s[rloc * 4 + 1] = rs.pm2; xch_s[rloc * 4 + 2] = rs.pn; }
+      if (half == 1) { xch_s[rloc * 4] = rs.pm; xch_s[rloc * 4 + 1] = rs.pm2; }
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (half == 0 && ok && valid) {
-        chan_merge(rs.pm, rs.pm2, rs.pn, xch_s[rloc * 4], xch_s[rloc * 4 + 1], xch_s[rloc * 4 + 2]);
+        chan_merge_equal(rs.pm, rs.pm2, xch_s[rloc * 4], xch_s[rloc * 4 + 1], 2.0f * kChunk);
         store_tile_stats(ep, m, tile_n, rs.pm, rs.pm2);
       }
     }

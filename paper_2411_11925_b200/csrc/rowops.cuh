@@ -72,8 +72,8 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
   __shared__ float eh[2][kCPad];
   const int r = blockIdx.x, tid = threadIdx.x;
   const int nrep = p.cfg ? 2 : 1;
-  if (tid == 0) griddep_launch_dependents();
   griddep_wait();
+  if (tid == 0) griddep_launch_dependents();
   if (mode == STEP_INIT) {
     if (tid < kCPad) xs[tid] = (tid < p.C) ? p.x_src[static_cast<size_t>(r) * p.C + tid] : 0.0f;
     if (tid < p.C) p.x[static_cast<size_t>(r) * p.C + tid] = p.x_src[static_cast<size_t>(r) * p.C + tid];
