@@ -23,6 +23,11 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
+# dram__bytes_read + dram__bytes_write per launch of a kernel class, from the ncu capture summarised in
+# profiles/mar256_gemm_tc_kernels_ncu_full.md (set to None when the kernel changes after the capture)
+NCU_DRAM_BYTES_PER_LAUNCH = {("mar256", "mlp2_gate_residual"): 12.62e6, ("mar256", "adaln_modulate"): 10.60e6,
+                             ("mar256", "mlp1_silu"): 4.22e6}
+
 METRIC = "draft tokens/s through denoise+verify+resample"
 UNIT = "tokens/s"
 
@@ -263,7 +268,8 @@ def run_ours(args):
             tot_ms = sum(v["ms"] for v in prof.values())
             ach = gemm[top]["flops"] / (gemm[top]["ms"] * 1e-3) / 1e12
             line["roofline"] = {"bound": "tensor", "kernel": top, "achieved": ach, "peak": peaks["tflops_sustained"],
-                                "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "traffic": None,
+                                "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"],
+                                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, top)),
                                 "peak_source": f"{peaks['source']} bf16 sustained (fp16 has the same nominal rate)",
                                 "avg_launch_us": 1e3 * gemm[top]["ms"] / gemm[top]["launches"],
                                 "per_class": {k: {"launches": v["launches"], "ms": round(v["ms"], 3),
