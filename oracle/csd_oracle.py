@@ -67,14 +67,14 @@ def layer_norm(h: np.ndarray, eps: float = 1e-6) -> np.ndarray:
 
 def timestep_embedding(w: Dict[str, np.ndarray], tfeat_t: np.ndarray) -> np.ndarray:
     """te_t = Wt2 SiLU(Wt1 tfeat_t + bt1) + bt2, one vector of width W."""
-    hid = silu(w["Wt1"].astype(f64) @ tfeat_t.astype(f64) + w["bt1"].astype(f64))
-    return w["Wt2"].astype(f64) @ hid + w["bt2"].astype(f64)
+    hid = silu(np.asarray(w["Wt1"], dtype=f64) @ tfeat_t.astype(f64) + np.asarray(w["bt1"], dtype=f64))
+    return np.asarray(w["Wt2"], dtype=f64) @ hid + np.asarray(w["bt2"], dtype=f64)
 
 
 def head_eps(w: Dict[str, np.ndarray], x_t: np.ndarray, tfeat_t: np.ndarray, z: np.ndarray,
              trace: Optional[dict] = None) -> np.ndarray:
     """eps_hat for a batch of head rows.  x_t [N,C], z [N,Dz], tfeat_t [F]."""
-    W64 = {k: v.astype(f64) for k, v in w.items()}
+    W64 = {k: np.asarray(v, dtype=f64) for k, v in w.items()}   # no copy when already float64
     x_t = x_t.astype(f64)
     cz = z.astype(f64) @ W64["Wz"].T + W64["bz"]
     te = timestep_embedding(w, tfeat_t)
@@ -105,6 +105,8 @@ def make_mlp_head(w: Dict[str, np.ndarray], z: np.ndarray, tfeat: np.ndarray,
     rows [0,R) of z are conditional, rows [R,2R) unconditional, both halves see
     the same x_t, and eps = eps_u + scale*(eps_c - eps_u) (Appendix
     "Classifier-Free Guidance")."""
+    w = {k: np.asarray(v, dtype=f64) for k, v in w.items()}   # widen once, not at every step
+
     def eps_fn(x_t: np.ndarray, t: int) -> np.ndarray:
         R = x_t.shape[0]
         if cfg:

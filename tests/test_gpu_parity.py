@@ -203,18 +203,68 @@ def test_argument_errors_are_reported_not_raised_by_the_device():
     ctx.close()
 
 
-def test_mar256_full_size_sampled_sequences():
-    # The benchmark's launch configuration (B=64, gamma=8, T=100, guidance, bf16) on the GPU; the checker
-    # evaluates four sequences: first, last and both sides of the 128-row tile boundary.
-    wl = gen.WORKLOADS["mar256"]
+def _sampled(name, seqs, label):
+    wl = gen.WORKLOADS[name]
     inp = gen.make_round_inputs(wl)
     dr, out = _run(inp, fused=True)
-    seqs = [0, 15, 16, 63]
     sub = gen.select_sequences(inp, seqs)
     ref, s1q, s1p = _ref(sub)
     rows = sub.extras["rows"]
     gsub = {k: (out[k][rows] if out[k].shape[0] == wl.R else out[k][seqs]) for k in out if k != "cap_hits"}
     gsub["cap_hits"] = out["cap_hits"]
-    st = compare_round(gsub, ref, sub.wl, s1q, s1p, sub.u, sub.v, "mar256 sampled")
-    print("mar256 sampled", st)
+    st = compare_round(gsub, ref, sub.wl, s1q, s1p, sub.u, sub.v, label)
+    print(label, st)
+    # properties that hold at any size: n_accept within [0, gamma], resampled exactly where n < gamma
+    assert np.all((out["n_accept"] >= 0) & (out["n_accept"] <= wl.gamma))
+    np.testing.assert_array_equal(out["flags"] & 1, (out["n_accept"] < wl.gamma).astype(out["flags"].dtype))
+    assert np.all(np.isfinite(out["x0"])) and np.all(np.isfinite(out["logratio"]))
+    assert int(out["cap_hits"][0]) == int(((out["flags"] & 2) != 0).sum())
     dr.ctx.close()
+    return st
+
+
+def test_mar256_full_size_sampled_sequences():
+    # The benchmark's launch configuration (B=64, gamma=8, T=100, guidance, bf16-valued weights) on the GPU; the
+    # checker evaluates four sequences: first, last and both sides of the 128-row tile boundary.
+    _sampled("mar256", [0, 15, 16, 63], "mar256 sampled")
+
+
+def test_ar_stress_full_size_sampled_sequences():
+    # B=256, gamma=16, T=50, no guidance, draft = perturbed target: sequences on both sides of a tile boundary
+    _sampled("ar_stress", [7, 8, 255], "ar_stress sampled")
+
+
+def test_mar512_full_size_sampled_sequence():
+    # B=32, gamma=32 (the largest draft length the scan supports), T=100, 12x1536 target head
+    _sampled("mar512", [31], "mar512 sampled")
+
+
+def test_large_target_full_size_sampled_sequence():
+    # B=128, gamma=16, T=100, guidance: 4096 head rows = 32 row tiles, W=1536 = 12 column tiles
+    _sampled("large_target", [64], "large_target sampled")
+
+
+def test_target_only_prefill_rows():
+    # Token pre-filling (Sec. 3.2): the first tokens come from the target head alone, i.e. csd_draft_denoise
+    # given the target head samples x0 at every step including the last.
+    from paper_2411_11925_b200.runner import DeviceRound
+    wl = _wl(B=9, gamma=4, T=12, bf16=True, cfg=True, cfg_scale=3.0, draft=gen.HeadSpec(2, 256, 256))
+    inp = gen.make_round_inputs(wl)
+    dr = DeviceRound(inp)
+    x0 = torch.zeros_like(dr.x0); mu1 = torch.zeros_like(dr.x0)
+    dr.ctx.csd_draft_denoise(dr.head_p, dr.sched_p, wl.R, wl.cfg, wl.cfg_scale, dr.z_p, dr.x_T, dr.eps, x0, mu1, None)
+    dr.ctx.sync()
+    sched = orc.ddpm_schedule(inp.beta, wl.tau)
+    ref = orc.denoise(orc.make_mlp_head(inp.w_p, inp.z_p, inp.tfeat, wl.cfg, wl.cfg_scale), sched, inp.x_T, inp.eps,
+                      sample_last=True)
+    assert float(np.max(np.abs(x0.cpu().numpy() - ref["x0"]))) <= 8e-3
+    assert float(np.max(np.abs(mu1.cpu().numpy() - ref["mu1"]))) <= 8e-3
+    dr.ctx.close()
+
+
+@pytest.mark.parametrize("op", ["f32", "f16"])
+def test_degenerate_sizes_single_row_single_step_widest_scan(op):
+    # R = 1 (one sequence, one position), T = 1 (the chain is a single step), and gamma = 32 (every lane of the scan)
+    for kw in (dict(B=1, gamma=1, T=1), dict(B=2, gamma=32, T=2), dict(B=1, gamma=3, T=3, cfg=True, cfg_scale=1.5)):
+        wl = _wl(bf16=op != "f32", operand=op, draft=gen.HeadSpec(1, 128, 64), target=gen.HeadSpec(1, 128, 128), **kw)
+        _check(gen.make_round_inputs(wl), f"degenerate {op} {kw}")
