@@ -46,6 +46,7 @@ struct HostIo {  // device mirrors for csd_round_host
 
 struct csd_ctx {
   int device = 0;
+  int num_sms = 148;
   cudaStream_t stream = nullptr;
   cudaStream_t side[2] = {nullptr, nullptr};
   cudaEvent_t ev_fork = nullptr, ev_done[2] = {nullptr, nullptr};
@@ -75,10 +76,11 @@ struct csd_head {
   // fp32 parameters
   float *bz, *Wt1, *bt1, *Wt2, *bt2, *win, *bin, *bfsh, *bfsc, *wout_t, *bout;
   std::vector<float*> bsh, bsc, bg, b1, b2;
-  // tensor maps of the weights (bf16 heads)
-  CUtensorMap tmWz{};
-  std::vector<CUtensorMap> tmWss, tmWg, tmW1, tmW2;
-  CUtensorMap tmWfss{};
+  // tensor maps of the weights (16-bit heads), one set per output-tile width: [0] 64, [1] 128 columns
+  struct TmSet {
+    CUtensorMap Wz{}, Wfss{};
+    std::vector<CUtensorMap> Wss, Wg, W1, W2;
+  } tm[2];
 };
 
 namespace {
@@ -165,7 +167,7 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   const size_t o_s = take(Rh * W * asz), o_u = take(Rh * W * asz), o_v = take(Rh * W * asz);
   const size_t o_cz = take(Rh * W * 4), o_te = take(static_cast<size_t>(T) * W * 4), o_h = take(Rh * W * 4);
   const size_t o_st = take(Rh * (W / kStatCols) * 8);
-  const size_t o_ep = take(Rh * (W / kTileN) * kCPad * 4);
+  const size_t o_ep = take(Rh * (W / kStatCols) * kCPad * 4);   // room for 64-wide tiles
   const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
   if (off > ws.cap) {
     CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
@@ -187,37 +189,45 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   return CSD_OK;
 }
 
-template <int EPI, int NSEG, int MMA_N, typename ACT>
+template <int EPI, int NSEG, int NMUL, int TN, typename ACT>
 int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0, const CUtensorMap& a1,
                 const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k, int N, const EpiParams& ep) {
-  auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, std::is_same<ACT, __half>::value ? 0 : 1>;
+  constexpr int MMA_N = NMUL * TN;
+  auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, TN, std::is_same<ACT, __half>::value ? 0 : 1>;
   static bool attr_done = false;
-  constexpr int smem = TcCfg<EPI, MMA_N>::kSmemBytes;
+  constexpr int smem = TcCfg<EPI, MMA_N, TN>::kSmemBytes;
   if (!attr_done) {
     CSD_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done = true;
   }
-  dim3 grid(N / kTileN, (ep.M + kTileM - 1) / kTileM);
-  ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * ((NSEG == 1 && MMA_N == 256) ? 2.0 : 1.0));
+  dim3 grid(N / TN, (ep.M + kTileM - 1) / kTileM);
+  ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * NMUL);
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = grid; cfg.blockDim = dim3(TcWarps<EPI>::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cfg.gridDim = grid; cfg.blockDim = dim3(TcWarps<EPI, TN>::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at; cfg.numAttrs = ctx->prof_on ? 0 : 1;   // event pairs between launches defeat the overlap anyway
-  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, ep, ctx->d_err));
+  EpiParams e = ep;
+  e.nt = N / kStatCols;   // eps partials are per 64-column group for both tile widths
+  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, e, ctx->d_err));
   ctx->launches++;
-  CSD_CUDA(ctx, cudaGetLastError());
   return CSD_OK;
 }
 
-template <int EPI, int NSEG, int MMA_N>
-int launch_tc(csd_ctx* ctx, int dtype, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0,
+// NMUL = 2: B holds the interleaved AdaLN shift | scale rows (two accumulator columns per output column).
+// tn: output columns per CTA, 64 or 128.  dep_k: first K index (over both segments) whose A operand is
+// written by the preceding kernel.
+template <int EPI, int NSEG, int NMUL>
+int launch_tc(csd_ctx* ctx, int dtype, int tn, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0,
               const CUtensorMap& a1, const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k,
               int N, const EpiParams& ep) {
-  // dep_k: first K index (over both segments) whose A operand is written by the preceding kernel
-  if (dtype == CSD_F16) return launch_tc_t<EPI, NSEG, MMA_N, __half>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
-  return launch_tc_t<EPI, NSEG, MMA_N, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+  if (dtype == CSD_F16) {
+    if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __half>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+    return launch_tc_t<EPI, NSEG, NMUL, 128, __half>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+  }
+  if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+  return launch_tc_t<EPI, NSEG, NMUL, 128, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
 }
 
 template <int EPI, int NSEG, int MMA_N>
@@ -225,7 +235,9 @@ int launch_simt(csd_ctx* ctx, cudaStream_t st, const float* A0, int lda0, const 
                 int lda1, const float* B1, int K1, int N, const EpiParams& ep) {
   dim3 grid(N / kTileN, (ep.M + kSimtRows - 1) / kSimtRows);
   ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * ((NSEG == 1 && MMA_N == 256) ? 2.0 : 1.0));
-  gemm_simt_kernel<EPI, NSEG, MMA_N><<<grid, 128, 0, st>>>(A0, lda0, B0, K0, K0, A1, lda1, B1, K1, K1, ep);
+  EpiParams e = ep;
+  e.nt = N / kTileN;
+  gemm_simt_kernel<EPI, NSEG, MMA_N><<<grid, 128, 0, st>>>(A0, lda0, B0, K0, K0, A1, lda1, B1, K1, K1, e);
   ctx->launches++;
   CSD_CUDA(ctx, cudaGetLastError());
   return CSD_OK;
@@ -247,7 +259,8 @@ int check_sched(csd_ctx* ctx, const csd_schedule* s, bool full) {
 struct Chain {
   csd_ctx* ctx; int slot; cudaStream_t st; const csd_head* hd; const csd_schedule* sc;
   int R, cfg; float cfg_scale; const float *z, *x_T, *eps; int sample_last; float *x0, *mu1, *x1;
-  int Rh = 0, W = 0, L = 0, T = 0;
+  int chains = 1;   // chains that run concurrently with this one (itself included)
+  int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
   bool tc = false;
   CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{}, tm_h{};
   EpiParams ep{};
@@ -274,6 +287,9 @@ struct Chain {
     const csd_head_desc& d = hd->d;
     Rh = R * (cfg ? 2 : 1); W = d.W; L = d.L; T = sc->T;
     tc = d.dtype != CSD_F32;
+    // 64-wide output tiles when 128-wide ones (of all chains running side by side) would occupy at most
+    // half of the SMs
+    tn = (tc && chains * (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms / 2) ? 64 : kTileN;
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T);
     if (rc) return rc;
@@ -295,13 +311,14 @@ struct Chain {
       if ((rc = make_tmap_f32(ctx, &tm_h, ws.h, Rh, W))) return rc;
     }
     // cz = z Wz^T + bz
+    const csd_head::TmSet& tmw = hd->tm[tn == 64 ? 0 : 1];
     EpiParams e = ep;
     e.bias0 = hd->bz; e.out_f32 = ws.cz;
-    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 128>(ctx, d.dtype, st, tm_z, hd->tmWz, tm_z, hd->tmWz, tm_h, d.Dz, 0, 0, W, e);
+    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 1>(ctx, d.dtype, tn, st, tm_z, tmw.Wz, tm_z, tmw.Wz, tm_h, d.Dz, 0, 0, W, e);
     else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
                                                 nullptr, 0, W, e);
     if (rc) return rc;
-    sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = W / kTileN; sp.cfg_scale = cfg_scale;
+    sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = tc ? W / kStatCols : W / kTileN; sp.cfg_scale = cfg_scale;
     sp.sample_last = sample_last; sp.epart = ws.epart; sp.bout = hd->bout; sp.x_src = x_T; sp.x = ws.x;
     sp.x0 = x0; sp.mu1 = mu1; sp.x1 = x1; sp.win = hd->win; sp.bin = hd->bin; sp.cz = ws.cz; sp.h = ws.h;
     sp.stats = ws.stats; sp.s = ws.s;
@@ -316,19 +333,20 @@ struct Chain {
     const float* sf = static_cast<const float*>(ws.s);
     const float* uf = static_cast<const float*>(ws.u);
     const float* vf = static_cast<const float*>(ws.v);
+    const csd_head::TmSet& tmw = hd->tm[tn == 64 ? 0 : 1];
     int rc = CSD_OK;
     for (int k = 0; k < L; ++k) {
       EpiParams e = ep;
       e.h = ws.h; e.stats = ws.stats;
       // u = LN(h)(1 + scale) + shift
       e.bias0 = hd->bsh[k]; e.bias1 = hd->bsc[k]; e.out_act = ws.u;
-      if (tc) rc = launch_tc<EPI_MOD, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWss[k], tm_s, hd->tmWss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
+      if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
       else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
                                              nullptr, 0, W, e);
       if (rc) return rc;
       // v = SiLU(W1 u + b1)
       e.bias0 = hd->b1[k]; e.bias1 = nullptr; e.out_act = ws.v;
-      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 128>(ctx, d.dtype, st, tm_u, hd->tmW1[k], tm_u, hd->tmW1[k], tm_h, W, 0, 0, W, e);
+      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 1>(ctx, d.dtype, tn, st, tm_u, tmw.W1[k], tm_u, tmw.W1[k], tm_h, W, 0, 0, W, e);
       else rc = launch_simt<EPI_SILU_ACT, 1, 128>(ctx, st, uf, W, static_cast<const float*>(hd->W1[k]), W, nullptr, 0,
                                                   nullptr, 0, W, e);
       if (rc) return rc;
@@ -338,7 +356,7 @@ struct Chain {
       if (tc) {
         EpiParams g = e;
         g.bias0 = hd->bg[k]; g.bias1 = hd->b2[k];
-        rc = launch_tc<EPI_GATE_RES, 2, 128>(ctx, d.dtype, st, tm_s, hd->tmWg[k], tm_v, hd->tmW2[k], tm_h, W, W, W, W, g);
+        rc = launch_tc<EPI_GATE_RES, 2, 1>(ctx, d.dtype, tn, st, tm_s, tmw.Wg[k], tm_v, tmw.W2[k], tm_h, W, W, W, W, g);
       }
       else rc = launch_simt<EPI_GATE_RES, 2, 128>(ctx, st, vf, W, static_cast<const float*>(hd->W2[k]), W, sf, W,
                                                   static_cast<const float*>(hd->Wg[k]), W, W, e);
@@ -346,7 +364,7 @@ struct Chain {
     }
     EpiParams e = ep;
     e.h = ws.h; e.stats = ws.stats; e.bias0 = hd->bfsh; e.bias1 = hd->bfsc; e.wout_t = hd->wout_t; e.epart = ws.epart;
-    if (tc) rc = launch_tc<EPI_MODF, 1, 256>(ctx, d.dtype, st, tm_s, hd->tmWfss, tm_s, hd->tmWfss, tm_h, W, 0, W, W, e);
+    if (tc) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, tn, st, tm_s, tmw.Wfss, tm_s, tmw.Wfss, tm_h, W, 0, W, W, e);
     else rc = launch_simt<EPI_MODF, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
                                             0, W, e);
     if (rc) return rc;
@@ -437,6 +455,7 @@ int csd_create(csd_ctx** out, int device, void* cuda_stream) {
   csd_ctx* c = new (std::nothrow) csd_ctx();
   if (!c) return CSD_ERR_WORKSPACE;
   c->device = device;
+  c->num_sms = prop.multiProcessorCount;
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   bool ok = true;
   for (int i = 0; i < 2; ++i) {
@@ -551,10 +570,11 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
   std::vector<size_t> o_wss(L), o_wg(L), o_w1(L), o_w2(L);
   size_t off = 0;
   const size_t o_wz = off; memcpy(&stage[off], w->Wz, W * Dz * 4); off += W * Dz;
+  // AdaLN shift and scale rows interleaved in groups of 64: 64 shift rows | 64 scale rows | ...
   auto interleave = [&](const float* shift_rows, const float* scale_rows, float* dst) {
-    for (size_t j = 0; j < W / kTileN; ++j) {
-      memcpy(dst + (2 * j) * kTileN * W, shift_rows + j * kTileN * W, kTileN * W * 4);
-      memcpy(dst + (2 * j + 1) * kTileN * W, scale_rows + j * kTileN * W, kTileN * W * 4);
+    for (size_t j = 0; j < W / kStatCols; ++j) {
+      memcpy(dst + (2 * j) * kStatCols * W, shift_rows + j * kStatCols * W, kStatCols * W * 4);
+      memcpy(dst + (2 * j + 1) * kStatCols * W, scale_rows + j * kStatCols * W, kStatCols * W * 4);
     }
   };
   for (size_t k = 0; k < L; ++k) {
@@ -613,15 +633,20 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
   for (size_t k = 0; k < L; ++k) { h->bsh[k] = fb + f_bsh[k]; h->bsc[k] = fb + f_bsc[k]; h->bg[k] = fb + f_bg[k]; h->b1[k] = fb + f_b1[k]; h->b2[k] = fb + f_b2[k]; }
 
   if (d.dtype != CSD_F32) {
-    int rc = make_tmap(ctx, &h->tmWz, d.dtype, h->Wz, W, Dz, Dz, 128);
-    h->tmWss.resize(L); h->tmWg.resize(L); h->tmW1.resize(L); h->tmW2.resize(L);
-    for (size_t k = 0; k < L && !rc; ++k) {
-      rc = make_tmap(ctx, &h->tmWss[k], d.dtype, h->Wss[k], 2 * W, W, W, 256);
-      if (!rc) rc = make_tmap(ctx, &h->tmWg[k], d.dtype, h->Wg[k], W, W, W, 128);
-      if (!rc) rc = make_tmap(ctx, &h->tmW1[k], d.dtype, h->W1[k], W, W, W, 128);
-      if (!rc) rc = make_tmap(ctx, &h->tmW2[k], d.dtype, h->W2[k], W, W, W, 128);
+    int rc = CSD_OK;
+    for (int i = 0; i < 2 && !rc; ++i) {
+      const uint32_t tn = i == 0 ? 64 : 128;   // B box rows = MMA N: tn, or 2 tn for the interleaved shift | scale rows
+      csd_head::TmSet& tm = h->tm[i];
+      rc = make_tmap(ctx, &tm.Wz, d.dtype, h->Wz, W, Dz, Dz, tn);
+      tm.Wss.resize(L); tm.Wg.resize(L); tm.W1.resize(L); tm.W2.resize(L);
+      for (size_t k = 0; k < L && !rc; ++k) {
+        rc = make_tmap(ctx, &tm.Wss[k], d.dtype, h->Wss[k], 2 * W, W, W, 2 * tn);
+        if (!rc) rc = make_tmap(ctx, &tm.Wg[k], d.dtype, h->Wg[k], W, W, W, tn);
+        if (!rc) rc = make_tmap(ctx, &tm.W1[k], d.dtype, h->W1[k], W, W, W, tn);
+        if (!rc) rc = make_tmap(ctx, &tm.W2[k], d.dtype, h->W2[k], W, W, W, tn);
+      }
+      if (!rc) rc = make_tmap(ctx, &tm.Wfss, d.dtype, h->Wfss, 2 * W, W, W, 2 * tn);
     }
-    if (!rc) rc = make_tmap(ctx, &h->tmWfss, d.dtype, h->Wfss, 2 * W, W, W, 256);
     if (rc) { csd_head_destroy(h); return rc; }
   }
   *out = h;
@@ -677,7 +702,7 @@ int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_sched
   auto take = [&](size_t bytes) { need = align_up(need + bytes, 1024); };
   take(Rh * d.Dz * asz); take(Rh * W * asz); take(Rh * W * asz); take(Rh * W * asz);
   take(Rh * W * 4); take(static_cast<size_t>(sched->T) * W * 4); take(Rh * W * 4);
-  take(Rh * (W / kStatCols) * 8); take(Rh * (W / kTileN) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
+  take(Rh * (W / kStatCols) * 8); take(Rh * (W / kStatCols) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
   if (need > kStaticScratchBytes)
     return fail(ctx, CSD_ERR_WORKSPACE,
                 "csd_draft_denoise_static: this call needs %zu bytes of scratch but the built-in array holds %zu "
@@ -775,6 +800,7 @@ int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, cons
   // the two chains' launches are interleaved step by step so that neither stream starves
   Chain cq{ctx, 0, ctx->side[0], head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr};
   Chain cp{ctx, 1, ctx->side[1], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr};
+  cq.chains = cp.chains = 2;
   rc = cp.begin();
   int rc2 = cq.begin();
   for (int t = sched_p->T; t >= 1 && !rc && !rc2; --t) {

@@ -1,5 +1,5 @@
-// Fused epilogues of the head's GEMMs.  One thread owns one output row and walks its 128-column
-// output tile in chunks of 32 columns; the same code serves the tcgen05 kernel (chunks read from
+// Fused epilogues of the head's GEMMs.  One thread owns one output row and walks its 64- or
+// 128-column output tile in chunks of 32 columns; the same code serves the tcgen05 kernel (chunks read from
 // TMEM) and the fp32 FMA kernel (chunks held in registers).
 #pragma once
 #include <cuda_bf16.h>
@@ -10,9 +10,10 @@
 namespace csd {
 
 constexpr int kTileM = 128;   // rows per tensor-core tile
-constexpr int kTileN = 128;   // output columns per tile
+constexpr int kTileN = 128;   // output columns per tile of the fp32 FMA kernel (the tcgen05 kernel: 64 or 128)
 constexpr int kChunk = 32;    // columns per epilogue chunk
-constexpr int kStatCols = 128; // columns per LayerNorm partial (one output tile)
+constexpr int kStatCols = 64; // columns per LayerNorm partial; also the row granule in which the AdaLN
+                              // shift and scale weight rows are interleaved (64 shift rows | 64 scale rows)
 constexpr int kCPad = 16;     // token dim is padded to 16 in Wout^T and the eps partials
 
 enum Epi : int {
@@ -31,9 +32,10 @@ struct EpiParams {
   float* out_f32;        // EPI_BIAS_F32
   void* out_act;         // EPI_SILU_ACT, EPI_MOD
   float* h;              // EPI_MOD / EPI_MODF (read), EPI_GATE_RES (read-modify-write)
-  float* stats;          // [M, ldo/128, 2] (mean, M2) per 128-column group of h
+  int nt;                // eps partials per row: N/64 (tensor-core kernel), N/128 (FMA kernel)
+  float* stats;          // [M, ldo/64, 2] (mean, M2) per 64-column group of h
   const float* wout_t;   // [N, 16] fp32, Wout transposed and zero padded (EPI_MODF)
-  float* epart;          // [M, N/128, 16] (EPI_MODF)
+  float* epart;          // [M, nt, 16] (EPI_MODF)
 };
 
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
@@ -116,7 +118,7 @@ __device__ __forceinline__ void chan_merge_equal(float& ma, float& m2a, float mb
   m2a += m2b + d * d * (0.5f * n);
 }
 
-// Merge the per-128-column (mean, M2) partials of row m in a fixed order, so the LayerNorm
+// Merge the per-64-column (mean, M2) partials of row m in a fixed order, so the LayerNorm
 // statistics do not depend on which CTA computes them.  All loads are issued before the merges.
 __device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
   const int G = W / kStatCols;
@@ -210,15 +212,15 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, fl
   }
 }
 
-// Writes the (mean, M2) partial of one row over one whole 128-column tile.
-__device__ __forceinline__ void store_tile_stats(const EpiParams& ep, int m, int tile_n, float mean, float m2) {
-  reinterpret_cast<float2*>(ep.stats)[static_cast<size_t>(m) * (ep.ldo / kStatCols) + tile_n] = make_float2(mean, m2);
+// Writes the (mean, M2) partial of one row over 64-column group g.
+__device__ __forceinline__ void store_group_stats(const EpiParams& ep, int m, int g, float mean, float m2) {
+  reinterpret_cast<float2*>(ep.stats)[static_cast<size_t>(m) * (ep.ldo / kStatCols) + g] = make_float2(mean, m2);
 }
 
 template <int EPI>
-__device__ __forceinline__ void epi_row_end(const EpiParams& ep, int m, int tile_n, const RowState& rs) {
+__device__ __forceinline__ void epi_row_end(const EpiParams& ep, int m, int part, const RowState& rs) {
   if constexpr (EPI == EPI_MODF) {
-    float4* d = reinterpret_cast<float4*>(ep.epart + (static_cast<size_t>(m) * (ep.ldo / kTileN) + tile_n) * kCPad);
+    float4* d = reinterpret_cast<float4*>(ep.epart + (static_cast<size_t>(m) * ep.nt + part) * kCPad);
 #pragma unroll
     for (int c = 0; c < kCPad / 4; ++c)
       d[c] = make_float4(rs.eacc[4 * c], rs.eacc[4 * c + 1], rs.eacc[4 * c + 2], rs.eacc[4 * c + 3]);

@@ -1,13 +1,15 @@
-// GEMM kernels of the head: out-tile[128 x 128] = epilogue(A[M,K] * B[N,K]^T ...).
-//   gemm_tc_kernel   : bf16 operands on tcgen05 tensor cores, TMA-fed shared-memory ring,
-//                      fp32 accumulators in TMEM, warp-specialised (TMA / MMA / 4 epilogue warps).
-//   gemm_simt_kernel : fp32 operands on plain FMA units (CSD_F32 heads).
-// Accumulator layout (both kernels), by template parameters:
-//   NSEG=1, MMA_N=128 : acc0 = A0 * B0[tile rows]^T
-//   NSEG=1, MMA_N=256 : B0 is packed so that rows [256 j, 256 j+128) and [256 j+128, 256 j+256) are
-//                       the two weight slices that pair up column by column (AdaLN shift | scale):
-//                       acc0 = first half, acc1 = second half, one shared A.
-//   NSEG=2, MMA_N=128 : acc0 = A0 * B0^T, acc1 = A1 * B1^T (second MLP layer | AdaLN gate).
+// GEMM kernels of the head: out-tile[128 x TN] = epilogue(A[M,K] * B[N,K]^T ...).
+//   gemm_tc_kernel   : 16-bit operands on tcgen05 tensor cores, TMA-fed shared-memory ring, fp32
+//                      accumulators in TMEM, warp-specialised (2 TMA warps / MMA warp / epilogue warps);
+//                      TN = 64 or 128 output columns per CTA (64 when 128 would leave SMs idle).
+//   gemm_simt_kernel : fp32 operands on plain FMA units (CSD_F32 heads), TN = 128.
+// Accumulator layout, by template parameters (NSEG segments, MMA_N rows of B per k-step):
+//   NSEG=1, MMA_N=TN   : acc0 = A0 * B0[tile rows]^T
+//   NSEG=1, MMA_N=2*TN : B0 holds the AdaLN shift and scale rows interleaved in groups of 64
+//                        (64 shift rows | 64 scale rows | next 64 shift rows | ...), one shared A:
+//                        output column c pairs accumulator column (c/64)*128 + c%64 (shift) with
+//                        the one 64 further (scale).
+//   NSEG=2, MMA_N=TN   : acc0 = A0 * B0^T, acc1 = A1 * B1^T (AdaLN gate | second MLP layer).
 #pragma once
 #include "epilogue.cuh"
 #include "ptx.cuh"
@@ -15,28 +17,29 @@
 namespace csd {
 
 constexpr int kBlockK = 64;  // bf16 elements per TMA box row = 128 bytes = one swizzle row
-// Warp roles: warp 0 TMA (A), warp 1 MMA, then the epilogue warps, last warp TMA (B).  The cheap
-// epilogues run 16 warps (one 32-column chunk per thread), the register-heavy ones 8 (two chunks).
-template <int EPI> struct TcWarps {
-  static constexpr int kEpi = (EPI == EPI_SILU_ACT || EPI == EPI_BIAS_F32) ? 16 : 8;
+// Warp roles: warp 0 TMA (A), warp 1 MMA, then the epilogue warps, last warp TMA (B).  A tile has
+// TN/32 column chunks x 4 TMEM lane quarters; the cheap epilogues of 128-wide tiles run 16 warps
+// (one chunk per thread), everything else 8 warps (two chunks per thread, or one when TN = 64).
+template <int EPI, int TN> struct TcWarps {
+  static constexpr int kEpi = (TN == 128 && (EPI == EPI_SILU_ACT || EPI == EPI_BIAS_F32)) ? 16 : 8;
   static constexpr int kThreads = (kEpi + 3) * 32;
-  static constexpr int kChunksPerThread = 16 / kEpi;   // 4 chunks x 4 lane quarters over kEpi warps
+  static constexpr int kChunksPerThread = (TN / kChunk) * 4 / kEpi;
 };
 
 enum DevErr : int { DEV_OK = 0, DEV_ERR_TMA_WAIT = 1, DEV_ERR_MMA_WAIT = 2, DEV_ERR_EPI_WAIT = 3 };
 
-constexpr int kHTileBytes = kTileM * kTileN * 4;   // fp32 h tile staged in shared memory (64 KB)
-
-template <int EPI, int MMA_N> struct TcCfg {
+template <int EPI, int MMA_N, int TN> struct TcCfg {
   static constexpr bool kStageH = EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES;
   static constexpr int kABytes = kTileM * kBlockK * 2;
   static constexpr int kBBytes = MMA_N * kBlockK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kHTileBytes = kTileM * TN * 4;        // fp32 h tile staged in shared memory
   static constexpr int kHBytes = kStageH ? kHTileBytes : 0;
-  static constexpr int kWoutBytes = kTileN * kCPad * 4;      // Wout^T tile, reused for the eps partials
-  static constexpr int kMiscBytes = 2 * kTileN * 4 + kTileM * 16;   // two bias slices + per-row exchange
+  static constexpr int kWoutBytes = kTileM * kCPad * 4;      // Wout^T tile [TN][16], reused for [128 rows][16] eps partials
+  static constexpr int kMiscBytes = 2 * TN * 4 + kTileM * 16;   // two bias slices + per-row exchange
   static constexpr int kFixedBytes = 1024 + kHBytes + kWoutBytes + kMiscBytes + 256;
-  static constexpr int kStages = (227 * 1024 - kFixedBytes) / kStageBytes;   // 6 (N=128), 4 (N=128 + h), 3 (N=256 + h)
+  static constexpr int kStagesMax = (227 * 1024 - kFixedBytes) / kStageBytes;
+  static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
   static constexpr int kSmemBytes = kFixedBytes + kStages * kStageBytes;
 };
 
@@ -51,22 +54,26 @@ __device__ __forceinline__ void load_swizzled_row32(const uint8_t* tile, int r, 
   }
 }
 
-template <int EPI, typename ACT, int NSEG, int MMA_N, int AB_FMT>
-__global__ void __launch_bounds__(TcWarps<EPI>::kThreads, 1)
+template <int EPI, typename ACT, int NSEG, int MMA_N, int TN, int AB_FMT>
+__global__ void __launch_bounds__(TcWarps<EPI, TN>::kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
                const __grid_constant__ CUtensorMap tmH, int nkb0, int nkb1, int dep_kb, EpiParams ep, int* err) {
-  using Cfg = TcCfg<EPI, MMA_N>;
+  using Cfg = TcCfg<EPI, MMA_N, TN>;
   constexpr int S = Cfg::kStages;
-  constexpr int EW = TcWarps<EPI>::kEpi, CPT = TcWarps<EPI>::kChunksPerThread, kEpiThreads = EW * 32;
-  constexpr uint32_t kTmemCols = NSEG * MMA_N;  // 128 or 256: a power of two >= 32
+  constexpr int EW = TcWarps<EPI, TN>::kEpi, CPT = TcWarps<EPI, TN>::kChunksPerThread, kEpiThreads = EW * 32;
+  constexpr int NC = TN / kChunk;               // column chunks per tile
+  constexpr bool kPacked = (NSEG == 1) && (MMA_N == 2 * TN);
+  constexpr bool kTwoAcc = kPacked || NSEG == 2;
+  constexpr uint32_t kTmemCols = NSEG * MMA_N;  // 64, 128 or 256: a power of two >= 32
+  static_assert(MMA_N == TN || kPacked, "MMA_N is TN or 2 TN");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stage_base = smem;
-  uint8_t* h_s = smem + S * Cfg::kStageBytes;                    // 4 chunks of [128 rows][128 B], swizzled
+  uint8_t* h_s = smem + S * Cfg::kStageBytes;                    // NC chunks of [128 rows][128 B], swizzled
   float* wout_s = reinterpret_cast<float*>(h_s + Cfg::kHBytes);
   float* bias_s = reinterpret_cast<float*>(h_s + Cfg::kHBytes + Cfg::kWoutBytes);
-  float* xch_s = bias_s + 2 * kTileN;                            // [128 rows][4] exchange between column halves
+  float* xch_s = bias_s + 2 * TN;                            // [128 rows][4] exchange between column halves
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(h_s + Cfg::kHBytes + Cfg::kWoutBytes + Cfg::kMiscBytes);
   uint64_t* empty_bar = full_bar + S;
   uint64_t* tmem_full_bar = empty_bar + S;
@@ -166,15 +173,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     const int rloc = q * 32 + lane;
     const int m = tile_m * kTileM + rloc;
     const bool valid = m < ep.M;
-    if (et < kTileN) {
-      bias_s[et] = ep.bias0[tile_n * kTileN + et];
-      bias_s[kTileN + et] = ep.bias1 ? ep.bias1[tile_n * kTileN + et] : 0.0f;
+    if (et < TN) {
+      bias_s[et] = ep.bias0[tile_n * TN + et];
+      bias_s[TN + et] = ep.bias1 ? ep.bias1[tile_n * TN + et] : 0.0f;
     }
     if (EPI == EPI_MODF) {
-      const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * kTileN * kCPad);
+      const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * TN * kCPad);
       float4* dst = reinterpret_cast<float4*>(wout_s);
 #pragma unroll
-      for (int i = 0; i < kTileN * kCPad / 4 / kEpiThreads; ++i) dst[et + i * kEpiThreads] = src[et + i * kEpiThreads];
+      for (int i = 0; i < TN * kCPad / 4 / kEpiThreads; ++i) dst[et + i * kEpiThreads] = src[et + i * kEpiThreads];
     }
     // h, the LayerNorm partials and the right to overwrite this kernel's outputs come with the
     // completion of the preceding kernel.  Only then may the next kernel start its own early part
@@ -184,10 +191,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (et == 0) {
       griddep_launch_dependents();
       if (Cfg::kStageH) {
-        mbar_arrive_expect_tx(h_bar, kHTileBytes);
+        mbar_arrive_expect_tx(h_bar, Cfg::kHTileBytes);
 #pragma unroll
-        for (int c = 0; c < kTileN / kChunk; ++c)
-          tma_load_2d(h_s + c * (kTileM * 128), &tmH, h_bar, tile_n * kTileN + c * kChunk, tile_m * kTileM);
+        for (int c = 0; c < NC; ++c)
+          tma_load_2d(h_s + c * (kTileM * 128), &tmH, h_bar, tile_n * TN + c * kChunk, tile_m * kTileM);
       }
     }
     RowState rs;
@@ -204,37 +211,56 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       for (int ci = 0; ci < CPT; ++ci) {
         const int c = CPT * half + ci;
         float a0[kChunk], a1[kChunk], hv[kChunk];
-        tmem_ld32(trow + c * kChunk, a0);
-        if (NSEG * MMA_N == 256) tmem_ld32(trow + kTileN + c * kChunk, a1);
+        const int col0 = kPacked ? (c >> 1) * 128 + (c & 1) * kChunk : c * kChunk;   // first accumulator
+        tmem_ld32(trow + col0, a0);
+        if (kTwoAcc) tmem_ld32(trow + col0 + (kPacked ? kStatCols : TN), a1);
         if (Cfg::kStageH) load_swizzled_row32(h_s + c * (kTileM * 128), rloc, hv);
         tmem_ld_wait();
+        float efirst[kCPad];
+        if (EPI == EPI_MODF && ci == 1) {
+#pragma unroll
+          for (int e = 0; e < kCPad; ++e) { efirst[e] = rs.eacc[e]; rs.eacc[e] = 0.0f; }
+        }
         if (valid)
-          epi_chunk<EPI, ACT, true>(ep, m, tile_n * kTileN + c * kChunk, a0, a1, bias_s + c * kChunk,
-                                    bias_s + kTileN + c * kChunk, hv, rs, wout_s + c * kChunk * kCPad);
+          epi_chunk<EPI, ACT, true>(ep, m, tile_n * TN + c * kChunk, a0, a1, bias_s + c * kChunk,
+                                    bias_s + TN + c * kChunk, hv, rs, wout_s + c * kChunk * kCPad);
+        if (EPI == EPI_MODF && ci == 1) {
+#pragma unroll
+          for (int e = 0; e < kCPad; ++e) rs.eacc[e] = efirst[e] + rs.eacc[e];
+        }
       }
     }
     if (EPI == EPI_GATE_RES) {
-      // one (mean, M2) partial per row over the whole tile: columns 64..127 are merged into 0..63
-      if (half == 1) { xch_s[rloc * 4] = rs.pm; xch_s[rloc * 4 + 1] = rs.pm2; }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (half == 0 && ok && valid) {
-        chan_merge_equal(rs.pm, rs.pm2, xch_s[rloc * 4], xch_s[rloc * 4 + 1], 2.0f * kChunk);
-        store_tile_stats(ep, m, tile_n, rs.pm, rs.pm2);
+      // one (mean, M2) partial per row and 64-column group
+      if (CPT == 2) {            // TN = 128: this thread's two chunks are one group
+        if (ok && valid) store_group_stats(ep, m, tile_n * 2 + half, rs.pm, rs.pm2);
+      } else {                   // TN = 64: chunk 1 (warps 6..9) is merged into chunk 0 (warps 2..5)
+        if (half == 1) { xch_s[rloc * 4] = rs.pm; xch_s[rloc * 4 + 1] = rs.pm2; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (half == 0 && ok && valid) {
+          chan_merge_equal(rs.pm, rs.pm2, xch_s[rloc * 4], xch_s[rloc * 4 + 1], static_cast<float>(kChunk));
+          store_group_stats(ep, m, tile_n, rs.pm, rs.pm2);
+        }
       }
     }
     if (EPI == EPI_MODF) {
-      // combine the two column halves of each row in a fixed order: (chunks 0,1) + (chunks 2,3)
-      asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread is done reading the Wout^T tile
-      float* part = wout_s;                            // [128 rows][16]
-      if (half == 1 && ok) {
+      // one eps partial per row and 64-column group, always formed as (chunk sum) + (next chunk sum) so
+      // that both tile widths give the same bits
+      if (CPT == 2) {            // TN = 128: this thread's two chunks are one group
+        if (ok && valid) epi_row_end<EPI>(ep, m, tile_n * 2 + half, rs);
+      } else {                   // TN = 64: chunk 1 (warps 6..9) is added to chunk 0 (warps 2..5)
+        asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread is done reading the Wout^T tile
+        float* part = wout_s;                            // [128 rows][16]
+        if (half == 1 && ok) {
 #pragma unroll
-        for (int c = 0; c < kCPad; ++c) part[rloc * kCPad + c] = rs.eacc[c];
-      }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (half == 0 && ok && valid) {
+          for (int c = 0; c < kCPad; ++c) part[rloc * kCPad + c] = rs.eacc[c];
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (half == 0 && ok && valid) {
 #pragma unroll
-        for (int c = 0; c < kCPad; ++c) rs.eacc[c] += part[rloc * kCPad + c];
-        epi_row_end<EPI>(ep, m, tile_n, rs);
+          for (int c = 0; c < kCPad; ++c) rs.eacc[c] += part[rloc * kCPad + c];
+          epi_row_end<EPI>(ep, m, tile_n, rs);
+        }
       }
     }
   }
@@ -288,8 +314,8 @@ gemm_simt_kernel(const float* __restrict__ A0, int lda0, const float* __restrict
         if constexpr (MMA_N == 256) {
 #pragma unroll
           for (int j = 0; j < kChunk; ++j) {
-            acc0[j] = fmaf(a, Bs[warp * kChunk + j][k], acc0[j]);
-            acc1[j] = fmaf(a, Bs[128 + warp * kChunk + j][k], acc1[j]);
+            acc0[j] = fmaf(a, Bs[(warp >> 1) * 128 + (warp & 1) * kChunk + j][k], acc0[j]);
+            acc1[j] = fmaf(a, Bs[(warp >> 1) * 128 + (warp & 1) * kChunk + kStatCols + j][k], acc1[j]);
           }
         } else {
           if (seg == 0) {
@@ -316,15 +342,14 @@ gemm_simt_kernel(const float* __restrict__ A0, int lda0, const float* __restrict
                                  wout_s + warp * kChunk * kCPad);
   }
   if constexpr (EPI == EPI_GATE_RES) {
-    float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][4]
+    float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][4]: chunks (0,1) and (2,3) form the 64-column groups
     __syncthreads();
-    if (m < ep.M) { scr[(warp * kSimtRows + lane) * 4] = rs.pm; scr[(warp * kSimtRows + lane) * 4 + 1] = rs.pm2; }
+    if (m < ep.M && (warp & 1)) { scr[(warp * kSimtRows + lane) * 4] = rs.pm; scr[(warp * kSimtRows + lane) * 4 + 1] = rs.pm2; }
     __syncthreads();
-    if (warp == 0 && m < ep.M) {
-      float pm = 0.0f, pm2 = 0.0f, pn = 0.0f;
-      for (int w = 0; w < 4; ++w)
-        chan_merge(pm, pm2, pn, scr[(w * kSimtRows + lane) * 4], scr[(w * kSimtRows + lane) * 4 + 1], static_cast<float>(kChunk));
-      store_tile_stats(ep, m, tile_n, pm, pm2);
+    if (m < ep.M && !(warp & 1)) {
+      chan_merge_equal(rs.pm, rs.pm2, scr[((warp + 1) * kSimtRows + lane) * 4], scr[((warp + 1) * kSimtRows + lane) * 4 + 1],
+                       static_cast<float>(kChunk));
+      store_group_stats(ep, m, tile_n * 2 + (warp >> 1), rs.pm, rs.pm2);
     }
   }
   if constexpr (EPI == EPI_MODF) {

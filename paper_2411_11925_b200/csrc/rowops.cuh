@@ -44,7 +44,7 @@ __global__ void convert_act_kernel(const float* __restrict__ src, ACT* __restric
 enum StepMode : int { STEP_INIT = 0, STEP_MID = 1, STEP_LAST = 2 };
 
 struct StepParams {
-  int R, cfg, C, W, NT;          // token rows, guidance flag, token dim, width, W/128
+  int R, cfg, C, W, NT;          // token rows, guidance flag, token dim, width, number of column tiles
   float cfg_scale, a, b, sigma;  // coefficients of the step being finished (t)
   int sample_last;               // STEP_LAST: also draw x0 = mu1 + sigma eps
   const float* epart;            // [Rh, NT, 16] eps_hat partial sums of step t
@@ -58,7 +58,7 @@ struct StepParams {
   const float* cz;               // [Rh, W]
   const float* te_next;          // [W] embedding of the step being prepared
   float* h;                      // [Rh, W]
-  float* stats;                  // [Rh, W/128, 2]
+  float* stats;                  // [Rh, W/64, 2]
   void* s;                       // [Rh, W] activations
 };
 
@@ -109,14 +109,14 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
     if (mode == STEP_LAST) return;
     __syncthreads();
   }
-  // prepare: each warp handles 128 consecutive columns at a time (lane + 32 j), one LayerNorm partial
+  // prepare: each warp handles 64 consecutive columns at a time (lane, lane + 32): one LayerNorm partial
   const int lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
   ACT* s = reinterpret_cast<ACT*>(p.s);
   for (int g = warp; g < p.W / kStatCols; g += nwarp) {
-    float acc[4];
+    float acc[2];
     float sum = 0.0f;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < 2; ++j) {
       const int n = g * kStatCols + j * 32 + lane;
       const float4* w4 = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(n) * kCPad);
       float a = p.bin[n];
@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
     const float mean = sum * (1.0f / kStatCols);
     float m2 = 0.0f;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) { const float d = acc[j] - mean; m2 = fmaf(d, d, m2); }
+    for (int j = 0; j < 2; ++j) { const float d = acc[j] - mean; m2 = fmaf(d, d, m2); }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
     for (int rep = 0; rep < nrep; ++rep) {
@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
       if (lane == 0)
         reinterpret_cast<float2*>(p.stats)[row * (p.W / kStatCols) + g] = make_float2(mean, m2);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < 2; ++j) {
         const int n = g * kStatCols + j * 32 + lane;
         p.h[row * p.W + n] = acc[j];
         s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + p.te_next[n]));
