@@ -287,9 +287,9 @@ struct Chain {
     const csd_head_desc& d = hd->d;
     Rh = R * (cfg ? 2 : 1); W = d.W; L = d.L; T = sc->T;
     tc = d.dtype != CSD_F32;
-    // 64-wide output tiles when 128-wide ones (of all chains running side by side) would occupy at most
-    // half of the SMs
-    tn = (tc && chains * (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms / 2) ? 64 : kTileN;
+    // 64-wide output tiles when 128-wide ones (of all chains running side by side) would occupy at most a
+    // quarter of the SMs: a kernel and the early part of its successor should both find free SMs
+    tn = (tc && chains * (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms / 4) ? 64 : kTileN;
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T);
     if (rc) return rc;

@@ -54,8 +54,8 @@ def test_fused_round_is_bit_identical_to_three_calls():
     for base, kw in (("tiny_fp32", dict(B=3, cfg=True, cfg_scale=2.0)),
                      ("tiny_fp32", dict(B=5, gamma=7, T=6, bf16=True, cfg=True, cfg_scale=3.0)),
                      ("tiny_fp32", dict(B=5, gamma=7, T=6, bf16=True, operand="bf16", cfg=True, cfg_scale=3.0)),
-                     # 40 tiles of 128 columns per chain: alone a chain runs 64-wide tiles, side by side 128-wide
-                     ("tiny_fp32", dict(B=160, gamma=8, T=3, bf16=True, cfg=True, cfg_scale=3.0,
+                     # 20 tiles of 128 columns per chain: alone a chain runs 64-wide tiles, side by side 128-wide
+                     ("tiny_fp32", dict(B=80, gamma=8, T=3, bf16=True, cfg=True, cfg_scale=3.0,
                                         draft=gen.HeadSpec(1, 256, 128), target=gen.HeadSpec(2, 256, 128)))):
         inp = gen.make_round_inputs(_wl(base, **kw))
         dr, a = _run(inp, fused=False)
