@@ -200,7 +200,8 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
     CSD_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done = true;
   }
-  dim3 grid(N / TN, (ep.M + kTileM - 1) / kTileM);
+  const int tiles_n = N / TN, tiles_total = tiles_n * ((ep.M + kTileM - 1) / kTileM);
+  dim3 grid(tiles_total < ctx->num_sms ? tiles_total : ctx->num_sms);   // persistent: one CTA per SM at most
   ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * NMUL);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid; cfg.blockDim = dim3(TcWarps<EPI, TN>::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
@@ -210,7 +211,7 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
   cfg.attrs = at; cfg.numAttrs = ctx->prof_on ? 0 : 1;   // event pairs between launches defeat the overlap anyway
   EpiParams e = ep;
   e.nt = N / kStatCols;   // eps partials are per 64-column group for both tile widths
-  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, e, ctx->d_err));
+  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, tiles_n, tiles_total, e, ctx->d_err));
   ctx->launches++;
   return CSD_OK;
 }

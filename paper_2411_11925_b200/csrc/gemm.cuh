@@ -54,18 +54,23 @@ __device__ __forceinline__ void load_swizzled_row32(const uint8_t* tile, int r, 
   }
 }
 
+// Persistent over tiles: CTA b handles output tiles b, b + gridDim.x, ... (column tile fastest).  The
+// shared-memory ring runs on across tiles; the accumulators are double-buffered in TMEM, so the
+// epilogue of one tile overlaps the MMAs of the next.
 template <int EPI, typename ACT, int NSEG, int MMA_N, int TN, int AB_FMT>
 __global__ void __launch_bounds__(TcWarps<EPI, TN>::kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
-               const __grid_constant__ CUtensorMap tmH, int nkb0, int nkb1, int dep_kb, EpiParams ep, int* err) {
+               const __grid_constant__ CUtensorMap tmH, int nkb0, int nkb1, int dep_kb, int tiles_n, int tiles_total,
+               EpiParams ep, int* err) {
   using Cfg = TcCfg<EPI, MMA_N, TN>;
   constexpr int S = Cfg::kStages;
   constexpr int EW = TcWarps<EPI, TN>::kEpi, CPT = TcWarps<EPI, TN>::kChunksPerThread, kEpiThreads = EW * 32;
   constexpr int NC = TN / kChunk;               // column chunks per tile
   constexpr bool kPacked = (NSEG == 1) && (MMA_N == 2 * TN);
   constexpr bool kTwoAcc = kPacked || NSEG == 2;
-  constexpr uint32_t kTmemCols = NSEG * MMA_N;  // 64, 128 or 256: a power of two >= 32
+  constexpr uint32_t kAccCols = NSEG * MMA_N;   // 64, 128 or 256 columns per accumulator buffer
+  constexpr uint32_t kTmemCols = 2 * kAccCols;  // two buffers: a power of two in [128, 512]
   static_assert(MMA_N == TN || kPacked, "MMA_N is TN or 2 TN");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -76,13 +81,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   float* xch_s = bias_s + 2 * TN;                            // [128 rows][4] exchange between column halves
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(h_s + Cfg::kHBytes + Cfg::kWoutBytes + Cfg::kMiscBytes);
   uint64_t* empty_bar = full_bar + S;
-  uint64_t* tmem_full_bar = empty_bar + S;
-  uint64_t* h_bar = tmem_full_bar + 1;
+  uint64_t* tmem_full_bar = empty_bar + S;      // [2]
+  uint64_t* tmem_empty_bar = tmem_full_bar + 2; // [2]
+  uint64_t* h_bar = tmem_empty_bar + 2;
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(h_bar + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile_n = blockIdx.x, tile_m = blockIdx.y;
   const int total_kb = nkb0 + (NSEG == 2 ? nkb1 : 0);
+  const int my_tiles = (tiles_total - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
 
   // Once any kernel of this context has raised the error flag, later launches return at once
   // (block-uniform decision) so that a failure costs one bounded wait, not one per launch.
@@ -97,7 +103,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (NSEG == 2) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
     if (Cfg::kStageH) tma_prefetch_desc(&tmH);
     for (int s = 0; s < S; ++s) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
-    mbar_init(tmem_full_bar, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full_bar[i], 1); mbar_init(&tmem_empty_bar[i], 1); }
     mbar_init(h_bar, 1);
     fence_mbar_init();
   }
@@ -111,155 +117,171 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const uint32_t tmem_base = *tmem_base_s;
 
   // Two TMA producers: one thread sustains only about one request per 240 clk, so the activation
-  // tiles (A, warp 0) and the weight tiles (B, warp 10) are requested by different warps; each arms
+  // tiles (A, warp 0) and the weight tiles (B, last warp) are requested by different warps; each arms
   // the stage's barrier with its own byte count.  Weights never depend on the preceding kernel; of
-  // the activations only k-blocks >= dep_kb do (the A producer waits for it there), so the part of
-  // the product that is independent of the preceding kernel overlaps with that kernel.
-  auto produce = [&](const CUtensorMap* t0, const CUtensorMap* t1, uint32_t bytes, int off, int crd, int wait_kb) {
+  // the activations only k-blocks >= dep_kb do (the A producer waits for it there, once), so the part
+  // of the product that is independent of the preceding kernel overlaps with that kernel.
+  auto produce = [&](const CUtensorMap* t0, const CUtensorMap* t1, uint32_t bytes, int off, bool is_a, int wait_kb) {
     bool ok = true;
-    for (int kb = 0; kb < nkb0 && ok; ++kb) {
-      const int s = kb % S;
-      if (kb == wait_kb) griddep_wait();
-      if (kb >= S && !mbar_wait(&empty_bar[s], ((kb / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
-      mbar_arrive_expect_tx(&full_bar[s], bytes);
-      tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t0, &full_bar[s], kb * kBlockK, crd);
-    }
-    if (NSEG == 2) {
-      for (int kb = nkb0; kb < total_kb && ok; ++kb) {
-        const int s = kb % S;
-        if (kb == wait_kb) griddep_wait();
-        if (kb >= S && !mbar_wait(&empty_bar[s], ((kb / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
+    int it = 0;   // k-blocks issued so far over all tiles
+    for (int i = 0; i < my_tiles && ok; ++i) {
+      const int t = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);
+      const int crd = is_a ? (t / tiles_n) * kTileM : (t % tiles_n) * MMA_N;
+      for (int kb = 0; kb < total_kb; ++kb, ++it) {
+        const int s = it % S;
+        if (i == 0 && kb == wait_kb) griddep_wait();
+        if (it >= S && !mbar_wait(&empty_bar[s], ((it / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
         mbar_arrive_expect_tx(&full_bar[s], bytes);
-        tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t1, &full_bar[s], (kb - nkb0) * kBlockK, crd);
+        if (NSEG == 2 && kb >= nkb0)
+          tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t1, &full_bar[s], (kb - nkb0) * kBlockK, crd);
+        else
+          tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t0, &full_bar[s], kb * kBlockK, crd);
       }
     }
   };
   if (warp == 0) {            // activation tiles
-    if (lane == 0) produce(&tmA0, &tmA1, Cfg::kABytes, 0, tile_m * kTileM, dep_kb);
+    if (lane == 0) produce(&tmA0, &tmA1, Cfg::kABytes, 0, true, dep_kb);
     __syncwarp();
   } else if (warp == EW + 2) {    // weight tiles
-    if (lane == 0) produce(&tmB0, &tmB1, Cfg::kBBytes, Cfg::kABytes, tile_n * MMA_N, -1);
+    if (lane == 0) produce(&tmB0, &tmB1, Cfg::kBBytes, Cfg::kABytes, false, -1);
     __syncwarp();
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_f16(MMA_N, AB_FMT);
       bool ok = true;
-      for (int kb = 0; kb < total_kb; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (kb / S) & 1;
-        if (!mbar_wait(&full_bar[s], ph)) { atomicExch(err, DEV_ERR_MMA_WAIT); ok = false; break; }
+      int it = 0;
+      for (int i = 0; i < my_tiles && ok; ++i) {
+        const int ab = i & 1;
+        // the epilogue must have drained this accumulator buffer (tile i - 2)
+        if (i >= 2 && !mbar_wait(&tmem_empty_bar[ab], ((i >> 1) - 1) & 1)) { atomicExch(err, DEV_ERR_MMA_WAIT); ok = false; break; }
         tc_fence_after_sync();
-        const bool second = (NSEG == 2) && (kb >= nkb0);
-        const int kk = second ? kb - nkb0 : kb;
-        const uint32_t sa = smem_u32(stage_base + s * Cfg::kStageBytes);
-        const uint64_t da = umma_smem_desc_sw128(sa);
-        const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes);
-        const uint32_t d = tmem_base + (second ? MMA_N : 0);
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int s = it % S;
+          if (!mbar_wait(&full_bar[s], (it / S) & 1)) { atomicExch(err, DEV_ERR_MMA_WAIT); ok = false; break; }
+          tc_fence_after_sync();
+          const bool second = (NSEG == 2) && (kb >= nkb0);
+          const int kk = second ? kb - nkb0 : kb;
+          const uint32_t sa = smem_u32(stage_base + s * Cfg::kStageBytes);
+          const uint64_t da = umma_smem_desc_sw128(sa);
+          const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes);
+          const uint32_t d = tmem_base + ab * kAccCols + (second ? MMA_N : 0);
 #pragma unroll
-        for (int k = 0; k < kBlockK / 16; ++k)  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
-          umma_f16(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
-        umma_commit(&empty_bar[s]);
+          for (int k = 0; k < kBlockK / 16; ++k)  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
+            umma_f16(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
+          umma_commit(&empty_bar[s]);
+        }
+        if (ok) umma_commit(&tmem_full_bar[ab]);
       }
-      if (ok) umma_commit(tmem_full_bar);
     }
     __syncwarp();
   } else {
     // Epilogue: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32).  With 8 warps, warps 2..5
-    // take column chunks 0 and 1 of the tile and warps 6..9 chunks 2 and 3; with 16 warps each group
-    // of four takes one chunk.  What does not need the accumulators (biases, Wout^T tile, LayerNorm
-    // partials) is fetched right away.
+    // take column chunks 0 and 1 of the tile and warps 6..9 chunks 2 and 3 (one chunk each when the
+    // tile is 64 wide); with 16 warps each group of four takes one chunk.
     const int et = threadIdx.x - 64;
     const int q = warp & 3, half = (warp - 2) >> 2;   // half = chunk group
     const int rloc = q * 32 + lane;
-    const int m = tile_m * kTileM + rloc;
-    const bool valid = m < ep.M;
-    if (et < TN) {
-      bias_s[et] = ep.bias0[tile_n * TN + et];
-      bias_s[TN + et] = ep.bias1 ? ep.bias1[tile_n * TN + et] : 0.0f;
-    }
-    if (EPI == EPI_MODF) {
-      const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * TN * kCPad);
-      float4* dst = reinterpret_cast<float4*>(wout_s);
-#pragma unroll
-      for (int i = 0; i < TN * kCPad / 4 / kEpiThreads; ++i) dst[et + i * kEpiThreads] = src[et + i * kEpiThreads];
-    }
     // h, the LayerNorm partials and the right to overwrite this kernel's outputs come with the
     // completion of the preceding kernel.  Only then may the next kernel start its own early part
-    // (at most one kernel runs ahead), and the h tile is requested before this thread block's
-    // remaining pipeline traffic queues up behind it.
+    // (at most one kernel runs ahead).
     griddep_wait();
-    if (et == 0) {
-      griddep_launch_dependents();
-      if (Cfg::kStageH) {
-        mbar_arrive_expect_tx(h_bar, Cfg::kHTileBytes);
+    if (et == 0) griddep_launch_dependents();
+    bool ok = true;
+    for (int i = 0; i < my_tiles; ++i) {
+      const int t = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);
+      const int tile_n = t % tiles_n, tile_m = t / tiles_n;
+      const int ab = i & 1;
+      const int m = tile_m * kTileM + rloc;
+      const bool valid = m < ep.M;
+      // every epilogue thread is done with the previous tile: its accumulator buffer, the h tile and
+      // the per-tile constants may be replaced
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+      if (et == 0) {
+        if (i >= 1) mbar_arrive(&tmem_empty_bar[ab ^ 1]);
+        if (Cfg::kStageH) {
+          // requested before this thread block's further pipeline traffic queues up behind it: ordinary
+          // loads issued while the pipeline saturates the SM's shared-memory port take thousands of cycles
+          mbar_arrive_expect_tx(h_bar, Cfg::kHTileBytes);
 #pragma unroll
-        for (int c = 0; c < NC; ++c)
-          tma_load_2d(h_s + c * (kTileM * 128), &tmH, h_bar, tile_n * TN + c * kChunk, tile_m * kTileM);
-      }
-    }
-    RowState rs;
-    if (valid) epi_row_begin<EPI>(ep, m, rs);
-    asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // biases and the Wout^T tile are in place
-    bool ok = mbar_wait(tmem_full_bar, 0);
-    if (ok && Cfg::kStageH) ok = mbar_wait(h_bar, 0);
-    if (!ok) atomicExch(err, DEV_ERR_EPI_WAIT);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
-      tc_fence_after_sync();
-      const uint32_t trow = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-#pragma unroll
-      for (int ci = 0; ci < CPT; ++ci) {
-        const int c = CPT * half + ci;
-        float a0[kChunk], a1[kChunk], hv[kChunk];
-        const int col0 = kPacked ? (c >> 1) * 128 + (c & 1) * kChunk : c * kChunk;   // first accumulator
-        tmem_ld32(trow + col0, a0);
-        if (kTwoAcc) tmem_ld32(trow + col0 + (kPacked ? kStatCols : TN), a1);
-        if (Cfg::kStageH) load_swizzled_row32(h_s + c * (kTileM * 128), rloc, hv);
-        tmem_ld_wait();
-        float efirst[kCPad];
-        if (EPI == EPI_MODF && ci == 1) {
-#pragma unroll
-          for (int e = 0; e < kCPad; ++e) { efirst[e] = rs.eacc[e]; rs.eacc[e] = 0.0f; }
-        }
-        if (valid)
-          epi_chunk<EPI, ACT, true>(ep, m, tile_n * TN + c * kChunk, a0, a1, bias_s + c * kChunk,
-                                    bias_s + TN + c * kChunk, hv, rs, wout_s + c * kChunk * kCPad);
-        if (EPI == EPI_MODF && ci == 1) {
-#pragma unroll
-          for (int e = 0; e < kCPad; ++e) rs.eacc[e] = efirst[e] + rs.eacc[e];
+          for (int c = 0; c < NC; ++c)
+            tma_load_2d(h_s + c * (kTileM * 128), &tmH, h_bar, tile_n * TN + c * kChunk, tile_m * kTileM);
         }
       }
-    }
-    if (EPI == EPI_GATE_RES) {
-      // one (mean, M2) partial per row and 64-column group
-      if (CPT == 2) {            // TN = 128: this thread's two chunks are one group
-        if (ok && valid) store_group_stats(ep, m, tile_n * 2 + half, rs.pm, rs.pm2);
-      } else {                   // TN = 64: chunk 1 (warps 6..9) is merged into chunk 0 (warps 2..5)
-        if (half == 1) { xch_s[rloc * 4] = rs.pm; xch_s[rloc * 4 + 1] = rs.pm2; }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (half == 0 && ok && valid) {
-          chan_merge_equal(rs.pm, rs.pm2, xch_s[rloc * 4], xch_s[rloc * 4 + 1], static_cast<float>(kChunk));
-          store_group_stats(ep, m, tile_n, rs.pm, rs.pm2);
+      if (et < TN) {
+        bias_s[et] = ep.bias0[tile_n * TN + et];
+        bias_s[TN + et] = ep.bias1 ? ep.bias1[tile_n * TN + et] : 0.0f;
+      }
+      if (EPI == EPI_MODF) {
+        const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * TN * kCPad);
+        float4* dst = reinterpret_cast<float4*>(wout_s);
+#pragma unroll
+        for (int j = 0; j < TN * kCPad / 4 / kEpiThreads; ++j) dst[et + j * kEpiThreads] = src[et + j * kEpiThreads];
+      }
+      RowState rs;
+      if (valid) epi_row_begin<EPI>(ep, m, rs);
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // biases and the Wout^T tile are in place
+      if (ok) ok = mbar_wait(&tmem_full_bar[ab], (i >> 1) & 1);
+      if (ok && Cfg::kStageH) ok = mbar_wait(h_bar, i & 1);
+      if (!ok) atomicExch(err, DEV_ERR_EPI_WAIT);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        tc_fence_after_sync();
+        const uint32_t trow = tmem_base + ab * kAccCols + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll
+        for (int ci = 0; ci < CPT; ++ci) {
+          const int c = CPT * half + ci;
+          float a0[kChunk], a1[kChunk], hv[kChunk];
+          const int col0 = kPacked ? (c >> 1) * 128 + (c & 1) * kChunk : c * kChunk;   // first accumulator
+          tmem_ld32(trow + col0, a0);
+          if (kTwoAcc) tmem_ld32(trow + col0 + (kPacked ? kStatCols : TN), a1);
+          if (Cfg::kStageH) load_swizzled_row32(h_s + c * (kTileM * 128), rloc, hv);
+          tmem_ld_wait();
+          float efirst[kCPad];
+          if (EPI == EPI_MODF && ci == 1) {
+#pragma unroll
+            for (int e = 0; e < kCPad; ++e) { efirst[e] = rs.eacc[e]; rs.eacc[e] = 0.0f; }
+          }
+          if (valid)
+            epi_chunk<EPI, ACT, true>(ep, m, tile_n * TN + c * kChunk, a0, a1, bias_s + c * kChunk,
+                                      bias_s + TN + c * kChunk, hv, rs, wout_s + c * kChunk * kCPad);
+          if (EPI == EPI_MODF && ci == 1) {
+#pragma unroll
+            for (int e = 0; e < kCPad; ++e) rs.eacc[e] = efirst[e] + rs.eacc[e];
+          }
+        }
+        tc_fence_before_sync();   // orders the TMEM reads before the barrier that releases the buffer
+      }
+      if (EPI == EPI_GATE_RES) {
+        // one (mean, M2) partial per row and 64-column group
+        if (CPT == 2) {            // TN = 128: this thread's two chunks are one group
+          if (ok && valid) store_group_stats(ep, m, tile_n * 2 + half, rs.pm, rs.pm2);
+        } else {                   // TN = 64: chunk 1 (warps 6..9) is merged into chunk 0 (warps 2..5)
+          if (half == 1) { xch_s[rloc * 4] = rs.pm; xch_s[rloc * 4 + 1] = rs.pm2; }
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          if (half == 0 && ok && valid) {
+            chan_merge_equal(rs.pm, rs.pm2, xch_s[rloc * 4], xch_s[rloc * 4 + 1], static_cast<float>(kChunk));
+            store_group_stats(ep, m, tile_n, rs.pm, rs.pm2);
+          }
         }
       }
-    }
-    if (EPI == EPI_MODF) {
-      // one eps partial per row and 64-column group, always formed as (chunk sum) + (next chunk sum) so
-      // that both tile widths give the same bits
-      if (CPT == 2) {            // TN = 128: this thread's two chunks are one group
-        if (ok && valid) epi_row_end<EPI>(ep, m, tile_n * 2 + half, rs);
-      } else {                   // TN = 64: chunk 1 (warps 6..9) is added to chunk 0 (warps 2..5)
-        asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread is done reading the Wout^T tile
-        float* part = wout_s;                            // [128 rows][16]
-        if (half == 1 && ok) {
+      if (EPI == EPI_MODF) {
+        // one eps partial per row and 64-column group, always formed as (chunk sum) + (next chunk sum) so
+        // that both tile widths give the same bits
+        if (CPT == 2) {            // TN = 128: this thread's two chunks are one group
+          if (ok && valid) epi_row_end<EPI>(ep, m, tile_n * 2 + half, rs);
+        } else {                   // TN = 64: chunk 1 (warps 6..9) is added to chunk 0 (warps 2..5)
+          asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread is done reading the Wout^T tile
+          float* part = wout_s;                            // [128 rows][16]
+          if (half == 1 && ok) {
 #pragma unroll
-          for (int c = 0; c < kCPad; ++c) part[rloc * kCPad + c] = rs.eacc[c];
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (half == 0 && ok && valid) {
+            for (int c = 0; c < kCPad; ++c) part[rloc * kCPad + c] = rs.eacc[c];
+          }
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          if (half == 0 && ok && valid) {
 #pragma unroll
-          for (int c = 0; c < kCPad; ++c) rs.eacc[c] += part[rloc * kCPad + c];
-          epi_row_end<EPI>(ep, m, tile_n, rs);
+            for (int c = 0; c < kCPad; ++c) rs.eacc[c] += part[rloc * kCPad + c];
+            epi_row_end<EPI>(ep, m, tile_n, rs);
+          }
         }
       }
     }
