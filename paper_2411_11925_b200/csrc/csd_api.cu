@@ -189,46 +189,62 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   return CSD_OK;
 }
 
-template <int EPI, int NSEG, int NMUL, int TN, typename ACT>
+template <int EPI, int NSEG, int NMUL, int TN, typename ACT, bool PAIR>
 int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0, const CUtensorMap& a1,
                 const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k, int N, const EpiParams& ep) {
   constexpr int MMA_N = NMUL * TN;
-  auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, TN, std::is_same<ACT, __half>::value ? 0 : 1>;
+  auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, TN, std::is_same<ACT, __half>::value ? 0 : 1, PAIR>;
   static bool attr_done = false;
-  constexpr int smem = TcCfg<EPI, MMA_N, TN>::kSmemBytes;
+  constexpr int smem = TcCfg<EPI, MMA_N, TN, PAIR>::kSmemBytes;
   if (!attr_done) {
     CSD_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_done = true;
   }
-  const int tiles_n = N / TN, tiles_total = tiles_n * ((ep.M + kTileM - 1) / kTileM);
-  dim3 grid(tiles_total < ctx->num_sms ? tiles_total : ctx->num_sms);   // persistent: one CTA per SM at most
+  // Work units: output tiles, or pair tiles (two row tiles) for CTA pairs.  Persistent: at most one CTA per SM.
+  const int tiles_n = N / TN, row_tiles = (ep.M + kTileM - 1) / kTileM;
+  const int units = tiles_n * (PAIR ? (row_tiles + 1) / 2 : row_tiles);
+  const int max_units = PAIR ? ctx->num_sms / 2 : ctx->num_sms;
+  dim3 grid((units < max_units ? units : max_units) * (PAIR ? 2 : 1));
   ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * NMUL);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid; cfg.blockDim = dim3(TcWarps<EPI, TN>::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at; cfg.numAttrs = ctx->prof_on ? 0 : 1;   // event pairs between launches defeat the overlap anyway
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (PAIR) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = 2; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  if (!ctx->prof_on) {   // event pairs between launches defeat the overlap anyway
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = at; cfg.numAttrs = na;
   EpiParams e = ep;
   e.nt = N / kStatCols;   // eps partials are per 64-column group for both tile widths
-  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, tiles_n, tiles_total, e, ctx->d_err));
+  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, tiles_n, units, e,
+                                   ctx->d_err));
   ctx->launches++;
   return CSD_OK;
 }
 
 // NMUL = 2: B holds the interleaved AdaLN shift | scale rows (two accumulator columns per output column).
-// tn: output columns per CTA, 64 or 128.  dep_k: first K index (over both segments) whose A operand is
+// tn: output columns per CTA, 64 or 128; pair: two CTAs share each MMA (needs tn = 128; the B tensor maps
+// b0 / b1 then have half-height boxes).  dep_k: first K index (over both segments) whose A operand is
 // written by the preceding kernel.
 template <int EPI, int NSEG, int NMUL>
-int launch_tc(csd_ctx* ctx, int dtype, int tn, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0,
+int launch_tc(csd_ctx* ctx, int dtype, int tn, bool pair, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0,
               const CUtensorMap& a1, const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k,
               int N, const EpiParams& ep) {
   if (dtype == CSD_F16) {
-    if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __half>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
-    return launch_tc_t<EPI, NSEG, NMUL, 128, __half>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+    if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __half, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+    if (pair) return launch_tc_t<EPI, NSEG, NMUL, 128, __half, true>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+    return launch_tc_t<EPI, NSEG, NMUL, 128, __half, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
   }
-  if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
-  return launch_tc_t<EPI, NSEG, NMUL, 128, __nv_bfloat16>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+  if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __nv_bfloat16, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+  if (pair) return launch_tc_t<EPI, NSEG, NMUL, 128, __nv_bfloat16, true>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+  return launch_tc_t<EPI, NSEG, NMUL, 128, __nv_bfloat16, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
 }
 
 template <int EPI, int NSEG, int MMA_N>
@@ -262,7 +278,7 @@ struct Chain {
   int R, cfg; float cfg_scale; const float *z, *x_T, *eps; int sample_last; float *x0, *mu1, *x1;
   int chains = 1;   // chains that run concurrently with this one (itself included)
   int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
-  bool tc = false;
+  bool tc = false, pair = false;
   CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{}, tm_h{};
   EpiParams ep{};
   StepParams sp{};
@@ -291,6 +307,10 @@ struct Chain {
     // 64-wide output tiles when 128-wide ones (of all chains running side by side) would occupy at most a
     // quarter of the SMs: a kernel and the early part of its successor should both find free SMs
     tn = (tc && chains * (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms / 4) ? 64 : kTileN;
+    // CTA pairs (two row tiles per MMA, half of each weight tile per CTA) need 128-wide tiles; they are
+    // used once a kernel has at least two waves of tiles, where L2-to-SM bandwidth is the limit (measured:
+    // a few per cent faster at 384 tiles, slower at 64 and 256)
+    pair = tc && tn == kTileN && (W / kTileN) * ((Rh + kTileM - 1) / kTileM) >= 2 * ctx->num_sms;
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T);
     if (rc) return rc;
@@ -312,10 +332,10 @@ struct Chain {
       if ((rc = make_tmap_f32(ctx, &tm_h, ws.h, Rh, W))) return rc;
     }
     // cz = z Wz^T + bz
-    const csd_head::TmSet& tmw = hd->tm[tn == 64 ? 0 : 1];
+    const csd_head::TmSet& tmw = hd->tm[(tn == 64 || pair) ? 0 : 1];   // pairs load half of each B tile per CTA
     EpiParams e = ep;
     e.bias0 = hd->bz; e.out_f32 = ws.cz;
-    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 1>(ctx, d.dtype, tn, st, tm_z, tmw.Wz, tm_z, tmw.Wz, tm_h, d.Dz, 0, 0, W, e);
+    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 1>(ctx, d.dtype, tn, pair, st, tm_z, tmw.Wz, tm_z, tmw.Wz, tm_h, d.Dz, 0, 0, W, e);
     else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
                                                 nullptr, 0, W, e);
     if (rc) return rc;
@@ -334,20 +354,20 @@ struct Chain {
     const float* sf = static_cast<const float*>(ws.s);
     const float* uf = static_cast<const float*>(ws.u);
     const float* vf = static_cast<const float*>(ws.v);
-    const csd_head::TmSet& tmw = hd->tm[tn == 64 ? 0 : 1];
+    const csd_head::TmSet& tmw = hd->tm[(tn == 64 || pair) ? 0 : 1];   // pairs load half of each B tile per CTA
     int rc = CSD_OK;
     for (int k = 0; k < L; ++k) {
       EpiParams e = ep;
       e.h = ws.h; e.stats = ws.stats;
       // u = LN(h)(1 + scale) + shift
       e.bias0 = hd->bsh[k]; e.bias1 = hd->bsc[k]; e.out_act = ws.u;
-      if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
+      if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
       else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
                                              nullptr, 0, W, e);
       if (rc) return rc;
       // v = SiLU(W1 u + b1)
       e.bias0 = hd->b1[k]; e.bias1 = nullptr; e.out_act = ws.v;
-      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 1>(ctx, d.dtype, tn, st, tm_u, tmw.W1[k], tm_u, tmw.W1[k], tm_h, W, 0, 0, W, e);
+      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 1>(ctx, d.dtype, tn, pair, st, tm_u, tmw.W1[k], tm_u, tmw.W1[k], tm_h, W, 0, 0, W, e);
       else rc = launch_simt<EPI_SILU_ACT, 1, 128>(ctx, st, uf, W, static_cast<const float*>(hd->W1[k]), W, nullptr, 0,
                                                   nullptr, 0, W, e);
       if (rc) return rc;
@@ -357,7 +377,7 @@ struct Chain {
       if (tc) {
         EpiParams g = e;
         g.bias0 = hd->bg[k]; g.bias1 = hd->b2[k];
-        rc = launch_tc<EPI_GATE_RES, 2, 1>(ctx, d.dtype, tn, st, tm_s, tmw.Wg[k], tm_v, tmw.W2[k], tm_h, W, W, W, W, g);
+        rc = launch_tc<EPI_GATE_RES, 2, 1>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wg[k], tm_v, tmw.W2[k], tm_h, W, W, W, W, g);
       }
       else rc = launch_simt<EPI_GATE_RES, 2, 128>(ctx, st, vf, W, static_cast<const float*>(hd->W2[k]), W, sf, W,
                                                   static_cast<const float*>(hd->Wg[k]), W, W, e);
@@ -365,7 +385,7 @@ struct Chain {
     }
     EpiParams e = ep;
     e.h = ws.h; e.stats = ws.stats; e.bias0 = hd->bfsh; e.bias1 = hd->bfsc; e.wout_t = hd->wout_t; e.epart = ws.epart;
-    if (tc) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, tn, st, tm_s, tmw.Wfss, tm_s, tmw.Wfss, tm_h, W, 0, W, W, e);
+    if (tc) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wfss, tm_s, tmw.Wfss, tm_h, W, 0, W, W, e);
     else rc = launch_simt<EPI_MODF, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
                                             0, W, e);
     if (rc) return rc;

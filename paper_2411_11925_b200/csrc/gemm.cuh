@@ -28,10 +28,13 @@ template <int EPI, int TN> struct TcWarps {
 
 enum DevErr : int { DEV_OK = 0, DEV_ERR_TMA_WAIT = 1, DEV_ERR_MMA_WAIT = 2, DEV_ERR_EPI_WAIT = 3 };
 
-template <int EPI, int MMA_N, int TN> struct TcCfg {
+// PAIR: two CTAs of a cluster share one MMA (cta_group::2, M = 256): each holds its own 128 rows of A
+// and half of the B rows, which cuts the shared-memory traffic per CTA and k-block.
+template <int EPI, int MMA_N, int TN, bool PAIR> struct TcCfg {
   static constexpr bool kStageH = EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES;
   static constexpr int kABytes = kTileM * kBlockK * 2;
-  static constexpr int kBBytes = MMA_N * kBlockK * 2;
+  static constexpr int kBRows = PAIR ? MMA_N / 2 : MMA_N;    // rows of the B tile this CTA loads
+  static constexpr int kBBytes = kBRows * kBlockK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kHTileBytes = kTileM * TN * 4;        // fp32 h tile staged in shared memory
   static constexpr int kHBytes = kStageH ? kHTileBytes : 0;
@@ -57,13 +60,13 @@ __device__ __forceinline__ void load_swizzled_row32(const uint8_t* tile, int r, 
 // Persistent over tiles: CTA b handles output tiles b, b + gridDim.x, ... (column tile fastest).  The
 // shared-memory ring runs on across tiles; the accumulators are double-buffered in TMEM, so the
 // epilogue of one tile overlaps the MMAs of the next.
-template <int EPI, typename ACT, int NSEG, int MMA_N, int TN, int AB_FMT>
+template <int EPI, typename ACT, int NSEG, int MMA_N, int TN, int AB_FMT, bool PAIR>
 __global__ void __launch_bounds__(TcWarps<EPI, TN>::kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
                const __grid_constant__ CUtensorMap tmH, int nkb0, int nkb1, int dep_kb, int tiles_n, int tiles_total,
                EpiParams ep, int* err) {
-  using Cfg = TcCfg<EPI, MMA_N, TN>;
+  using Cfg = TcCfg<EPI, MMA_N, TN, PAIR>;
   constexpr int S = Cfg::kStages;
   constexpr int EW = TcWarps<EPI, TN>::kEpi, CPT = TcWarps<EPI, TN>::kChunksPerThread, kEpiThreads = EW * 32;
   constexpr int NC = TN / kChunk;               // column chunks per tile
@@ -88,13 +91,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_kb = nkb0 + (NSEG == 2 ? nkb1 : 0);
-  const int my_tiles = (tiles_total - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+  // Work unit index and count: a CTA, or a pair of CTAs (cluster ranks 0 = leader and 1).  With pairs
+  // tiles_total counts pair tiles (two row tiles each) and the pair's CTAs take row tiles 2p and 2p+1.
+  const int rank = PAIR ? static_cast<int>(cluster_ctarank()) : 0;
+  const int unit = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int nunits = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+  const int my_tiles = (tiles_total - unit + nunits - 1) / nunits;
 
   // Once any kernel of this context has raised the error flag, later launches return at once
-  // (block-uniform decision) so that a failure costs one bounded wait, not one per launch.
+  // (a decision uniform over the block, and over the pair) so that a failure costs one bounded
+  // wait, not one per launch.
   __shared__ int s_abort;
   if (threadIdx.x == 0) s_abort = *reinterpret_cast<volatile int*>(err);
   __syncthreads();
+  if (PAIR) {
+    cluster_arrive(); cluster_wait();               // the peer has published its flag
+    int peer_abort = 0;
+    if (threadIdx.x == 0) {
+      const uint32_t pa = mapa_shared(smem_u32(&s_abort), static_cast<uint32_t>(rank ^ 1));
+      asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(peer_abort) : "r"(pa) : "memory");
+    }
+    cluster_arrive(); cluster_wait();               // both have read before either may overwrite
+    if (threadIdx.x == 0 && peer_abort != 0) s_abort = peer_abort;
+    __syncthreads();
+  }
   if (s_abort != 0) return;
 
   if (warp == 0 && lane == 0) {
@@ -103,16 +123,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (NSEG == 2) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
     if (Cfg::kStageH) tma_prefetch_desc(&tmH);
     for (int s = 0; s < S; ++s) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full_bar[i], 1); mbar_init(&tmem_empty_bar[i], 1); }
+    // a pair's accumulator buffer is released by the epilogues of both CTAs (to the leader's barrier)
+    for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full_bar[i], 1); mbar_init(&tmem_empty_bar[i], PAIR ? 2 : 1); }
     mbar_init(h_bar, 1);
     fence_mbar_init();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_base_s, kTmemCols);
-    tmem_relinquish();
+    if (PAIR) { tmem_alloc_pair(tmem_base_s, kTmemCols); tmem_relinquish_pair(); }
+    else { tmem_alloc(tmem_base_s, kTmemCols); tmem_relinquish(); }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) { cluster_arrive(); cluster_wait(); }   // the peer's barriers exist before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_base_s;
 
@@ -125,17 +147,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     bool ok = true;
     int it = 0;   // k-blocks issued so far over all tiles
     for (int i = 0; i < my_tiles && ok; ++i) {
-      const int t = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);
-      const int crd = is_a ? (t / tiles_n) * kTileM : (t % tiles_n) * MMA_N;
+      const int t = unit + i * nunits;
+      const int tm = PAIR ? 2 * (t / tiles_n) + rank : t / tiles_n;
+      const int crd = is_a ? tm * kTileM : (t % tiles_n) * MMA_N + rank * Cfg::kBRows;
       for (int kb = 0; kb < total_kb; ++kb, ++it) {
         const int s = it % S;
         if (i == 0 && kb == wait_kb) griddep_wait();
         if (it >= S && !mbar_wait(&empty_bar[s], ((it / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
-        mbar_arrive_expect_tx(&full_bar[s], bytes);
-        if (NSEG == 2 && kb >= nkb0)
-          tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t1, &full_bar[s], (kb - nkb0) * kBlockK, crd);
-        else
-          tma_load_2d(stage_base + s * Cfg::kStageBytes + off, t0, &full_bar[s], kb * kBlockK, crd);
+        const CUtensorMap* tmap = (NSEG == 2 && kb >= nkb0) ? t1 : t0;
+        const int kx = ((NSEG == 2 && kb >= nkb0) ? kb - nkb0 : kb) * kBlockK;
+        uint8_t* dst = stage_base + s * Cfg::kStageBytes + off;
+        if (PAIR) {
+          // the leader's barrier counts the bytes of both CTAs; only the leader arms it
+          if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * bytes);
+          tma_load_2d_pair(dst, tmap, mapa_shared(smem_u32(&full_bar[s]), 0), kx, crd);
+        } else {
+          mbar_arrive_expect_tx(&full_bar[s], bytes);
+          tma_load_2d(dst, tmap, &full_bar[s], kx, crd);
+        }
       }
     }
   };
@@ -146,8 +175,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (lane == 0) produce(&tmB0, &tmB1, Cfg::kBBytes, Cfg::kABytes, false, -1);
     __syncwarp();
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_f16(MMA_N, AB_FMT);
+    if (lane == 0 && rank == 0) {     // of a pair only the leader issues MMAs
+      constexpr uint32_t idesc = umma_idesc_f16(MMA_N, AB_FMT, PAIR ? 256 : 128);
       bool ok = true;
       int it = 0;
       for (int i = 0; i < my_tiles && ok; ++i) {
@@ -166,11 +195,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes);
           const uint32_t d = tmem_base + ab * kAccCols + (second ? MMA_N : 0);
 #pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
-            umma_f16(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
-          umma_commit(&empty_bar[s]);
+          for (int k = 0; k < kBlockK / 16; ++k) {  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
+            if (PAIR) umma_f16_pair(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
+            else umma_f16(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
+          }
+          if (PAIR) umma_commit_pair(&empty_bar[s]); else umma_commit(&empty_bar[s]);
         }
-        if (ok) umma_commit(&tmem_full_bar[ab]);
+        if (ok) { if (PAIR) umma_commit_pair(&tmem_full_bar[ab]); else umma_commit(&tmem_full_bar[ab]); }
       }
     }
     __syncwarp();
@@ -188,8 +219,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (et == 0) griddep_launch_dependents();
     bool ok = true;
     for (int i = 0; i < my_tiles; ++i) {
-      const int t = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);
-      const int tile_n = t % tiles_n, tile_m = t / tiles_n;
+      const int t = unit + i * nunits;
+      const int tile_n = t % tiles_n, tile_m = PAIR ? 2 * (t / tiles_n) + rank : t / tiles_n;
       const int ab = i & 1;
       const int m = tile_m * kTileM + rloc;
       const bool valid = m < ep.M;
@@ -197,7 +228,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       // the per-tile constants may be replaced
       asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
       if (et == 0) {
-        if (i >= 1) mbar_arrive(&tmem_empty_bar[ab ^ 1]);
+        if (i >= 1) {
+          if (PAIR) mbar_arrive_cluster(mapa_shared(smem_u32(&tmem_empty_bar[ab ^ 1]), 0));
+          else mbar_arrive(&tmem_empty_bar[ab ^ 1]);
+        }
         if (Cfg::kStageH) {
           // requested before this thread block's further pipeline traffic queues up behind it: ordinary
           // loads issued while the pipeline saturates the SM's shared-memory port take thousands of cycles
@@ -288,7 +322,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+  if (PAIR) { cluster_arrive(); cluster_wait(); }   // neither CTA leaves while the pair's MMAs or signals may touch it
+  if (warp == 1) { if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols); else tmem_dealloc(tmem_base, kTmemCols); }
 }
 
 // ------------------------------------------------------------------ fp32 FMA path
