@@ -32,9 +32,14 @@ enum DevErr : int { DEV_OK = 0, DEV_ERR_TMA_WAIT = 1, DEV_ERR_MMA_WAIT = 2, DEV_
 // and half of the B rows, which cuts the shared-memory traffic per CTA and k-block.
 template <int EPI, int MMA_N, int TN, bool PAIR> struct TcCfg {
   static constexpr bool kStageH = EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES;
-  static constexpr int kABytes = kTileM * kBlockK * 2;
+  // A stage holds kKps k-blocks of 64 elements (one TMA box per operand and k-block).  The kernels whose
+  // MMAs are 128 wide use two: fewer barrier round trips per byte.
+  static constexpr int kKps = (EPI == EPI_SILU_ACT || EPI == EPI_GATE_RES) ? 2 : 1;
+  static constexpr int kABoxBytes = kTileM * kBlockK * 2;
   static constexpr int kBRows = PAIR ? MMA_N / 2 : MMA_N;    // rows of the B tile this CTA loads
-  static constexpr int kBBytes = kBRows * kBlockK * 2;
+  static constexpr int kBBoxBytes = kBRows * kBlockK * 2;
+  static constexpr int kABytes = kKps * kABoxBytes;
+  static constexpr int kBBytes = kKps * kBBoxBytes;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kHTileBytes = kTileM * TN * 4;        // fp32 h tile staged in shared memory
   static constexpr int kHBytes = kStageH ? kHTileBytes : 0;
@@ -90,6 +95,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(h_bar + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int KPS = Cfg::kKps;
+  // from here on nkb0 / nkb1 / dep_kb / total_kb count stages of KPS k-blocks
+  nkb0 /= KPS; nkb1 /= KPS; dep_kb /= KPS;
   const int total_kb = nkb0 + (NSEG == 2 ? nkb1 : 0);
   // Work unit index and count: a CTA, or a pair of CTAs (cluster ranks 0 = leader and 1).  With pairs
   // tiles_total counts pair tiles (two row tiles each) and the pair's CTAs take row tiles 2p and 2p+1.
@@ -155,15 +163,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (i == 0 && kb == wait_kb) griddep_wait();
         if (it >= S && !mbar_wait(&empty_bar[s], ((it / S) & 1) ^ 1)) { atomicExch(err, DEV_ERR_TMA_WAIT); ok = false; break; }
         const CUtensorMap* tmap = (NSEG == 2 && kb >= nkb0) ? t1 : t0;
-        const int kx = ((NSEG == 2 && kb >= nkb0) ? kb - nkb0 : kb) * kBlockK;
+        const int kx = ((NSEG == 2 && kb >= nkb0) ? kb - nkb0 : kb) * KPS * kBlockK;
         uint8_t* dst = stage_base + s * Cfg::kStageBytes + off;
         if (PAIR) {
           // the leader's barrier counts the bytes of both CTAs; only the leader arms it
           if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * bytes);
-          tma_load_2d_pair(dst, tmap, mapa_shared(smem_u32(&full_bar[s]), 0), kx, crd);
+          const uint32_t lb = mapa_shared(smem_u32(&full_bar[s]), 0);
+#pragma unroll
+          for (int j = 0; j < KPS; ++j) tma_load_2d_pair(dst + j * (bytes / KPS), tmap, lb, kx + j * kBlockK, crd);
         } else {
           mbar_arrive_expect_tx(&full_bar[s], bytes);
-          tma_load_2d(dst, tmap, &full_bar[s], kx, crd);
+#pragma unroll
+          for (int j = 0; j < KPS; ++j) tma_load_2d(dst + j * (bytes / KPS), tmap, &full_bar[s], kx + j * kBlockK, crd);
         }
       }
     }
@@ -191,13 +202,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           const bool second = (NSEG == 2) && (kb >= nkb0);
           const int kk = second ? kb - nkb0 : kb;
           const uint32_t sa = smem_u32(stage_base + s * Cfg::kStageBytes);
-          const uint64_t da = umma_smem_desc_sw128(sa);
-          const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes);
           const uint32_t d = tmem_base + ab * kAccCols + (second ? MMA_N : 0);
 #pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k) {  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
-            if (PAIR) umma_f16_pair(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
-            else umma_f16(d, da + 2 * k, db + 2 * k, idesc, (kk > 0 || k > 0) ? 1u : 0u);
+          for (int j = 0; j < KPS; ++j) {
+            const uint64_t da = umma_smem_desc_sw128(sa + j * Cfg::kABoxBytes);
+            const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes + j * Cfg::kBBoxBytes);
+#pragma unroll
+            for (int k = 0; k < kBlockK / 16; ++k) {  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
+              const uint32_t acc = (kk > 0 || j > 0 || k > 0) ? 1u : 0u;
+              if (PAIR) umma_f16_pair(d, da + 2 * k, db + 2 * k, idesc, acc);
+              else umma_f16(d, da + 2 * k, db + 2 * k, idesc, acc);
+            }
           }
           if (PAIR) umma_commit_pair(&empty_bar[s]); else umma_commit(&empty_bar[s]);
         }
