@@ -3,14 +3,15 @@ import math
 
 import numpy as np
 
-# Stated tolerances: trajectories (x0, and mu1 which is a point of the trajectory) 2e-2 max-abs for bf16
-# heads, 1e-4 for fp32 heads; log-ratio 5e-2 abs.  Eq. 8 is ill-conditioned in mu: d logR / d mu =
-# (x0 - mu) / sigma_1^2 with sigma_1 = 0.01, so a per-coordinate error delta_mu in the final-step means moves
-# logR by up to sqrt(2 Q) / sigma_1 * sqrt(C) * delta_mu, Q = |x0 - mu|^2 / (2 sigma_1^2).  The log-ratio
-# tolerance is therefore 5e-2 plus that term, with delta_mu = the accuracy ASSERTED on mu1 below (tighter
-# than the stated trajectory tolerance).
+# Stated tolerances: trajectories 2e-2 max-abs for bf16-valued heads, 1e-4 for fp32 heads; log-ratio 5e-2
+# abs.  mu1 is held to the trajectory tolerance: x0 = mu1 + sigma_1 eps_1 (Eq. 3) with eps_1 an input, so
+# the two carry the same error (for fp32 heads a tighter 2e-5 is asserted).  Eq. 8 is ill-conditioned in
+# mu: d logR / d mu = (x0 - mu) / sigma_1^2 with sigma_1 = 0.01, so a per-coordinate error delta_mu in
+# the final-step means moves logR by up to sqrt(2 Q) / sigma_1 * sqrt(C) * delta_mu, Q = |x0 - mu|^2 /
+# (2 sigma_1^2).  The log-ratio tolerance is therefore 5e-2 plus that term, with delta_mu = the accuracy
+# ASSERTED on mu1 below.
 TOL_X = {"f32": 1e-4, "bf16": 2e-2, "f16": 2e-2}
-TOL_MU = {"f32": 2e-5, "bf16": 1.2e-2, "f16": 1.2e-2}
+TOL_MU = {"f32": 2e-5, "bf16": 2e-2, "f16": 2e-2}
 TOL_LOGR = 5e-2
 
 
