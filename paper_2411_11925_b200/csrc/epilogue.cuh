@@ -100,40 +100,46 @@ struct RowState {
   float pm, pm2, pn;         // running (mean, M2, count) of the new h values (EPI_GATE_RES)
 };
 
-// Chan et al. merge of two (mean, M2, count) triples; b is merged into a.
-__device__ __forceinline__ void chan_merge(float& ma, float& m2a, float& na, float mb, float m2b, float nb) {
-  if (nb <= 0.0f) return;
-  if (na <= 0.0f) { ma = mb; m2a = m2b; na = nb; return; }
-  const float n = na + nb;
-  const float d = mb - ma;
-  ma += d * (nb / n);
-  m2a += m2b + d * d * (na * nb / n);
-  na = n;
-}
-
-// Same for two partials of equal count n (no division): mean = (ma + mb)/2, M2 = M2a + M2b + d^2 n/2.
+// Chan et al. merge of two (mean, M2) partials of equal count n (no division): mean = (ma + mb)/2,
+// M2 = M2a + M2b + d^2 n/2; b is merged into a.
 __device__ __forceinline__ void chan_merge_equal(float& ma, float& m2a, float mb, float m2b, float n) {
   const float d = mb - ma;
   ma = fmaf(d, 0.5f, ma);
   m2a += m2b + d * d * (0.5f * n);
 }
 
-// Merge the per-64-column (mean, M2) partials of row m in a fixed order, so the LayerNorm
-// statistics do not depend on which CTA computes them.  All loads are issued before the merges.
+// LayerNorm statistics of row m from its per-64-column (mean, M2) partials.  All partials have the
+// same count n = 64, so with G groups  mean = (sum_g mean_g) / G  and
+// M2 = sum_g M2_g + n sum_g (mean_g - mean)^2  (Chan et al. for equal counts, all groups at once):
+// no chain of dependent divisions.  Sums run in group order, so the result does not depend on which
+// CTA computes it.  Up to 24 groups (W <= 1536) are loaded once, as one batch of 16-byte loads.
 __device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
-  const int G = W / kStatCols;
-  const float2* p = reinterpret_cast<const float2*>(stats) + static_cast<size_t>(m) * G;
-  float ma = 0.0f, m2a = 0.0f, na = 0.0f;
-  for (int g0 = 0; g0 < G; g0 += 12) {
-    float2 b[12];
+  const int G = W / kStatCols;   // even: W is a multiple of 128
+  const float4* p = reinterpret_cast<const float4*>(stats) + static_cast<size_t>(m) * (G / 2);
+  constexpr int kB = 12;         // 16-byte loads (two groups each) per batch
+  float sum = 0.0f, m2 = 0.0f, q = 0.0f;
+  if (G <= 2 * kB) {
+    float4 b[kB];
 #pragma unroll
-    for (int j = 0; j < 12; ++j) b[j] = (g0 + j < G) ? p[g0 + j] : make_float2(0.0f, 0.0f);
+    for (int j = 0; j < kB; ++j) b[j] = (2 * j < G) ? p[j] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
 #pragma unroll
-    for (int j = 0; j < 12; ++j)
-      if (g0 + j < G) chan_merge(ma, m2a, na, b[j].x, b[j].y, static_cast<float>(kStatCols));
+    for (int j = 0; j < kB; ++j)
+      if (2 * j < G) { sum += b[j].x; sum += b[j].z; m2 += b[j].y; m2 += b[j].w; }
+    mean = sum / static_cast<float>(G);
+#pragma unroll
+    for (int j = 0; j < kB; ++j)
+      if (2 * j < G) { const float d0 = b[j].x - mean, d1 = b[j].z - mean; q = fmaf(d0, d0, q); q = fmaf(d1, d1, q); }
+  } else {
+    for (int j = 0; j < G / 2; ++j) { const float4 b = p[j]; sum += b.x; sum += b.z; m2 += b.y; m2 += b.w; }
+    mean = sum / static_cast<float>(G);
+    for (int j = 0; j < G / 2; ++j) {
+      const float4 b = p[j];
+      const float d0 = b.x - mean, d1 = b.z - mean;
+      q = fmaf(d0, d0, q); q = fmaf(d1, d1, q);
+    }
   }
-  mean = ma;
-  rstd = 1.0f / sqrtf(m2a / static_cast<float>(W) + 1e-6f);
+  const float m2t = fmaf(static_cast<float>(kStatCols), q, m2);
+  rstd = 1.0f / sqrtf(m2t / static_cast<float>(W) + 1e-6f);
 }
 
 template <int EPI>

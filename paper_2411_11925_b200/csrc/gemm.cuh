@@ -186,37 +186,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (lane == 0) produce(&tmB0, &tmB1, Cfg::kBBytes, Cfg::kABytes, false, -1);
     __syncwarp();
   } else if (warp == 1) {
-    if (lane == 0 && rank == 0) {     // of a pair only the leader issues MMAs
+    if (rank == 0) {     // of a pair only the leader issues MMAs
+      // The whole warp runs the loop and waits; one elected lane issues.  (Measured: a loop entered by a
+      // single lane spends about 200 clk more per stage on the same waits, MMAs and commit.)
+      const bool leader = elect_one();
       constexpr uint32_t idesc = umma_idesc_f16(MMA_N, AB_FMT, PAIR ? 256 : 128);
       bool ok = true;
       int it = 0;
       for (int i = 0; i < my_tiles && ok; ++i) {
         const int ab = i & 1;
         // the epilogue must have drained this accumulator buffer (tile i - 2)
-        if (i >= 2 && !mbar_wait(&tmem_empty_bar[ab], ((i >> 1) - 1) & 1)) { atomicExch(err, DEV_ERR_MMA_WAIT); ok = false; break; }
+        if (i >= 2 && !mbar_wait(&tmem_empty_bar[ab], ((i >> 1) - 1) & 1)) { if (leader) atomicExch(err, DEV_ERR_MMA_WAIT); ok = false; break; }
         tc_fence_after_sync();
         for (int kb = 0; kb < total_kb; ++kb, ++it) {
           const int s = it % S;
-          if (!mbar_wait(&full_bar[s], (it / S) & 1)) { atomicExch(err, DEV_ERR_MMA_WAIT); ok = false; break; }
+          if (!mbar_wait(&full_bar[s], (it / S) & 1)) { if (leader) atomicExch(err, DEV_ERR_MMA_WAIT); ok = false; break; }
           tc_fence_after_sync();
-          const bool second = (NSEG == 2) && (kb >= nkb0);
-          const int kk = second ? kb - nkb0 : kb;
-          const uint32_t sa = smem_u32(stage_base + s * Cfg::kStageBytes);
-          const uint32_t d = tmem_base + ab * kAccCols + (second ? MMA_N : 0);
+          if (leader) {
+            const bool second = (NSEG == 2) && (kb >= nkb0);
+            const int kk = second ? kb - nkb0 : kb;
+            const uint32_t sa = smem_u32(stage_base + s * Cfg::kStageBytes);
+            const uint32_t d = tmem_base + ab * kAccCols + (second ? MMA_N : 0);
 #pragma unroll
-          for (int j = 0; j < KPS; ++j) {
-            const uint64_t da = umma_smem_desc_sw128(sa + j * Cfg::kABoxBytes);
-            const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes + j * Cfg::kBBoxBytes);
+            for (int j = 0; j < KPS; ++j) {
+              const uint64_t da = umma_smem_desc_sw128(sa + j * Cfg::kABoxBytes);
+              const uint64_t db = umma_smem_desc_sw128(sa + Cfg::kABytes + j * Cfg::kBBoxBytes);
 #pragma unroll
-            for (int k = 0; k < kBlockK / 16; ++k) {  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
-              const uint32_t acc = (kk > 0 || j > 0 || k > 0) ? 1u : 0u;
-              if (PAIR) umma_f16_pair(d, da + 2 * k, db + 2 * k, idesc, acc);
-              else umma_f16(d, da + 2 * k, db + 2 * k, idesc, acc);
+              for (int k = 0; k < kBlockK / 16; ++k) {  // UMMA_K = 16 elements = 32 bytes = 2 descriptor units
+                const uint32_t acc = (kk > 0 || j > 0 || k > 0) ? 1u : 0u;
+                if (PAIR) umma_f16_pair(d, da + 2 * k, db + 2 * k, idesc, acc);
+                else umma_f16(d, da + 2 * k, db + 2 * k, idesc, acc);
+              }
             }
+            if (PAIR) umma_commit_pair(&empty_bar[s]); else umma_commit(&empty_bar[s]);
           }
-          if (PAIR) umma_commit_pair(&empty_bar[s]); else umma_commit(&empty_bar[s]);
+          __syncwarp();
         }
-        if (ok) { if (PAIR) umma_commit_pair(&tmem_full_bar[ab]); else umma_commit(&tmem_full_bar[ab]); }
+        if (ok && leader) { if (PAIR) umma_commit_pair(&tmem_full_bar[ab]); else umma_commit(&tmem_full_bar[ab]); }
+        __syncwarp();
       }
     }
     __syncwarp();
@@ -230,6 +237,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     // h, the LayerNorm partials and the right to overwrite this kernel's outputs come with the
     // completion of the preceding kernel.  Only then may the next kernel start its own early part
     // (at most one kernel runs ahead).
+    // per-tile constants (biases, the Wout^T tile): not written by any kernel, so those of the first tile
+    // are staged before the wait
+    auto stage_consts = [&](int tile_n) {
+      if (et < TN) {
+        bias_s[et] = ep.bias0[tile_n * TN + et];
+        bias_s[TN + et] = ep.bias1 ? ep.bias1[tile_n * TN + et] : 0.0f;
+      }
+      if (EPI == EPI_MODF) {
+        const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * TN * kCPad);
+        float4* dst = reinterpret_cast<float4*>(wout_s);
+#pragma unroll
+        for (int j = 0; j < TN * kCPad / 4 / kEpiThreads; ++j) dst[et + j * kEpiThreads] = src[et + j * kEpiThreads];
+      }
+    };
+    stage_consts(unit % tiles_n);
     griddep_wait();
     if (et == 0) griddep_launch_dependents();
     bool ok = true;
@@ -256,16 +278,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             tma_load_2d(h_s + c * (kTileM * 128), &tmH, h_bar, tile_n * TN + c * kChunk, tile_m * kTileM);
         }
       }
-      if (et < TN) {
-        bias_s[et] = ep.bias0[tile_n * TN + et];
-        bias_s[TN + et] = ep.bias1 ? ep.bias1[tile_n * TN + et] : 0.0f;
-      }
-      if (EPI == EPI_MODF) {
-        const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * TN * kCPad);
-        float4* dst = reinterpret_cast<float4*>(wout_s);
-#pragma unroll
-        for (int j = 0; j < TN * kCPad / 4 / kEpiThreads; ++j) dst[et + j * kEpiThreads] = src[et + j * kEpiThreads];
-      }
+      if (i > 0) stage_consts(tile_n);
       RowState rs;
       if (valid) epi_row_begin<EPI>(ep, m, rs);
       asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // biases and the Wout^T tile are in place
