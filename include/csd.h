@@ -110,7 +110,8 @@ int64_t csd_launch_count(const csd_ctx *ctx);
  * kernel class, the launches recorded since: their count, device time (ms) and algorithmic FLOPs
  * (2*M*N*K per GEMM).  Classes: 0 condition projection, 1 block MLP first layer (+SiLU),
  * 2 AdaLN modulate (shift|scale), 3 block MLP second layer + gate + residual, 4 final modulate +
- * output projection, 5 per-step boundary kernel. */
+ * output projection, 5 per-step boundary kernel, 6 whole-chain kernel (all layers and steps of one
+ * head in one launch; used when a row block's column slices fit one thread-block cluster). */
 int csd_profile(csd_ctx *ctx, int enable);
 int csd_profile_read(csd_ctx *ctx, int kernel_class, int64_t *launches, double *total_ms,
                      double *total_flops);

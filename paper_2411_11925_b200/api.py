@@ -146,7 +146,7 @@ class Context:
     def launch_count(self) -> int:
         return int(_LIB.csd_launch_count(self._h))
 
-    KERNEL_CLASSES = ("cond_proj", "mlp1_silu", "adaln_modulate", "mlp2_gate_residual", "final_mod_outproj", "step")
+    KERNEL_CLASSES = ("cond_proj", "mlp1_silu", "adaln_modulate", "mlp2_gate_residual", "final_mod_outproj", "step", "chain")
 
     def profile(self, enable: bool):
         self._check(_LIB.csd_profile(self._h, int(enable)))

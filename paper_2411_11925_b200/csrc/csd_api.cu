@@ -15,6 +15,7 @@
 #include <vector>
 
 #include "../../include/csd.h"
+#include "chain.cuh"
 #include "gemm.cuh"
 #include "rowops.cuh"
 
@@ -33,6 +34,8 @@ struct ChainWs {
   // carved per call
   void *zc, *s, *u, *v;
   float *cz, *te, *h, *stats, *epart, *x;
+  // whole-chain kernel only
+  void* s2 = nullptr; float* sched = nullptr; CUtensorMap* amaps = nullptr;
 };
 
 struct ProfRec { cudaEvent_t a, b; int cls; double flops; };
@@ -81,6 +84,10 @@ struct csd_head {
     CUtensorMap Wz{}, Wfss{};
     std::vector<CUtensorMap> Wss, Wg, W1, W2;
   } tm[2];
+  // whole-chain kernel: device copies of the weight tensor maps (per block Wss, Wg, W1, W2; then Wfss) and of
+  // the bias pointers (per block shift, scale, b1, gate, b2; then final shift, scale)
+  CUtensorMap* d_wmaps = nullptr;
+  const float** d_bias = nullptr;
 };
 
 namespace {
@@ -158,7 +165,7 @@ int make_tmap_f32(csd_ctx* ctx, CUtensorMap* m, const void* ptr, uint64_t rows, 
   return CSD_OK;
 }
 
-int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, int T) {
+int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, int T, bool chain_kernel_extras) {
   const size_t asz = d.dtype == CSD_F32 ? 4 : 2;
   const size_t W = d.W;
   size_t off = 0;
@@ -169,6 +176,8 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   const size_t o_st = take(Rh * (W / kStatCols) * 8);
   const size_t o_ep = take(Rh * (W / kStatCols) * kCPad * 4);   // room for 64-wide tiles
   const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
+  size_t o_s2 = 0, o_sched = 0, o_amaps = 0;
+  if (chain_kernel_extras) { o_s2 = take(Rh * W * asz); o_sched = take(static_cast<size_t>(T) * 3 * 4); o_amaps = take(4 * sizeof(CUtensorMap)); }
   if (off > ws.cap) {
     CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamSynchronize(ctx->side[i]));
@@ -186,6 +195,9 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   ws.cz = reinterpret_cast<float*>(b + o_cz); ws.te = reinterpret_cast<float*>(b + o_te);
   ws.h = reinterpret_cast<float*>(b + o_h); ws.stats = reinterpret_cast<float*>(b + o_st);
   ws.epart = reinterpret_cast<float*>(b + o_ep); ws.x = reinterpret_cast<float*>(b + o_x);
+  if (chain_kernel_extras) {
+    ws.s2 = b + o_s2; ws.sched = reinterpret_cast<float*>(b + o_sched); ws.amaps = reinterpret_cast<CUtensorMap*>(b + o_amaps);
+  }
   return CSD_OK;
 }
 
@@ -270,6 +282,32 @@ int check_sched(csd_ctx* ctx, const csd_schedule* s, bool full) {
   return CSD_OK;
 }
 
+// The whole-chain kernel needs the row block's W/128 column slices in one cluster of at most 8 CTAs, each
+// with ~219 KB of shared memory; asked of the driver once per cluster size and operand type.
+bool use_chain_kernel(const csd_head_desc& d) {
+  const int nc = d.W / kTileN;
+  if (d.dtype == CSD_F32 || nc < 1 || nc > kChMaxCluster) return false;
+  static int known[2][kChMaxCluster + 1] = {};   // 0 unknown, 1 usable, -1 not
+  int& k = known[d.dtype == CSD_F16 ? 0 : 1][nc];
+  if (k == 0) {
+    k = -1;
+    const void* fn = d.dtype == CSD_F16 ? reinterpret_cast<const void*>(chain_kernel<__half, 0>)
+                                        : reinterpret_cast<const void*>(chain_kernel<__nv_bfloat16, 1>);
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kChSmemBytes) == cudaSuccess) {
+      cudaLaunchConfig_t lc{};
+      lc.gridDim = dim3(nc); lc.blockDim = dim3(kChThreads); lc.dynamicSmemBytes = kChSmemBytes;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = nc; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.attrs = at; lc.numAttrs = 1;
+      int ncl = 0;
+      if (cudaOccupancyMaxActiveClusters(&ncl, fn, &lc) == cudaSuccess && ncl >= 1) k = 1;
+    }
+    cudaGetLastError();
+  }
+  return k == 1;
+}
+
 // One head's denoising chain for R token rows on stream `st` with workspace slot `slot`:
 // begin() enqueues the per-call work (timestep embedding, condition projection, first boundary
 // kernel), step(t) enqueues the kernels of step t.  Two chains can be interleaved launch by launch.
@@ -277,6 +315,7 @@ struct Chain {
   csd_ctx* ctx; int slot; cudaStream_t st; const csd_head* hd; const csd_schedule* sc;
   int R, cfg; float cfg_scale; const float *z, *x_T, *eps; int sample_last; float *x0, *mu1, *x1;
   int chains = 1;   // chains that run concurrently with this one (itself included)
+  bool allow_chain_kernel = true, whole = false;   // whole: one kernel runs the whole chain
   int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
   bool tc = false, pair = false;
   CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{}, tm_h{};
@@ -311,8 +350,11 @@ struct Chain {
     // used once a kernel has at least two waves of tiles, where L2-to-SM bandwidth is the limit (measured:
     // a few per cent faster at 384 tiles, slower at 64 and 256)
     pair = tc && tn == kTileN && (W / kTileN) * ((Rh + kTileM - 1) / kTileM) >= 2 * ctx->num_sms;
+    // One kernel for the whole chain when a row block's column slices fit one portable cluster.  The choice
+    // depends on the head only, and both paths give the same bits.
+    whole = allow_chain_kernel && tc && use_chain_kernel(d);
     ChainWs& ws = ctx->ws[slot];
-    int rc = ensure_ws(ctx, ws, d, Rh, R, T);
+    int rc = ensure_ws(ctx, ws, d, Rh, R, T, whole);
     if (rc) return rc;
     timestep_embed_kernel<<<T, 256, (d.F + W) * sizeof(float), st>>>(sc->tfeat, hd->Wt1, hd->bt1, hd->Wt2, hd->bt2, W,
                                                                     d.F, ws.te);
@@ -345,10 +387,48 @@ struct Chain {
     sp.stats = ws.stats; sp.s = ws.s;
     sp.te_next = ws.te + static_cast<size_t>(T - 1) * W;
     sp.eps_t = eps;
+    if (whole) return launch_chain_kernel();
     return launch_step(STEP_INIT);
   }
 
+  int launch_chain_kernel() {
+    const csd_head_desc& d = hd->d;
+    ChainWs& ws = ctx->ws[slot];
+    int rc = CSD_OK;
+    CUtensorMap am[4];
+    void* const bufs[4] = {ws.s2, ws.s, ws.u, ws.v};   // s of even t, s of odd t, u, v
+    for (int i = 0; i < 4 && !rc; ++i) rc = make_tmap(ctx, &am[i], d.dtype, bufs[i], Rh, W, W, 64);
+    if (rc) return rc;
+    // small pageable sources: staged by the runtime before the calls return
+    CSD_CUDA(ctx, cudaMemcpyAsync(ws.amaps, am, sizeof(am), cudaMemcpyHostToDevice, st));
+    CSD_CUDA(ctx, cudaMemcpyAsync(ws.sched, sc->a, T * sizeof(float), cudaMemcpyHostToDevice, st));
+    CSD_CUDA(ctx, cudaMemcpyAsync(ws.sched + T, sc->b, T * sizeof(float), cudaMemcpyHostToDevice, st));
+    CSD_CUDA(ctx, cudaMemcpyAsync(ws.sched + 2 * T, sc->sigma, T * sizeof(float), cudaMemcpyHostToDevice, st));
+    ChainParams p{};
+    p.wmaps = hd->d_wmaps; p.amaps = ws.amaps;
+    p.R = R; p.cfg = cfg; p.W = W; p.L = L; p.T = T; p.C = d.C; p.sample_last = sample_last; p.cfg_scale = cfg_scale;
+    p.sched = ws.sched; p.cz = ws.cz; p.te = ws.te; p.bias = hd->d_bias;
+    p.win = hd->win; p.bin = hd->bin; p.wout_t = hd->wout_t; p.bout = hd->bout;
+    p.s[0] = ws.s2; p.s[1] = ws.s; p.u = ws.u; p.v = ws.v; p.stats = ws.stats; p.epart = ws.epart;
+    p.x_T = x_T; p.eps = eps; p.x0 = x0; p.mu1 = mu1; p.x1 = x1; p.err = ctx->d_err;
+    const int nc = W / kTileN, tb_rows = cfg ? kTileM / 2 : kTileM;
+    const int nb = (R + tb_rows - 1) / tb_rows;
+    const double flops_step = 2.0 * Rh * static_cast<double>(W) * W * (5.0 * L + 2.0) + 2.0 * Rh * static_cast<double>(W) * d.C * 2.0;
+    ProfScope ps(ctx, st, 6, flops_step * T);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(nb * nc); lc.blockDim = dim3(kChThreads); lc.dynamicSmemBytes = kChSmemBytes; lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = nc; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, chain_kernel<__half, 0>, p));
+    else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, chain_kernel<__nv_bfloat16, 1>, p));
+    ctx->launches++;
+    return CSD_OK;
+  }
+
   int step(int t) {
+    if (whole) return CSD_OK;   // already enqueued by begin()
     const csd_head_desc& d = hd->d;
     ChainWs& ws = ctx->ws[slot];
     const float* sf = static_cast<const float*>(ws.s);
@@ -400,6 +480,7 @@ int run_chain(csd_ctx* ctx, int slot, cudaStream_t st, const csd_head* hd, const
               float cfg_scale, const float* z, const float* x_T, const float* eps, int sample_last, float* x0,
               float* mu1, float* x1) {
   Chain c{ctx, slot, st, hd, sc, R, cfg, cfg_scale, z, x_T, eps, sample_last, x0, mu1, x1};
+  c.allow_chain_kernel = slot != 2;   // the static-scratch call keeps the layer-by-layer kernels its scratch is sized for
   int rc = c.begin();
   for (int t = sc->T; t >= 1 && !rc; --t) rc = c.step(t);
   return rc;
@@ -547,7 +628,7 @@ int csd_profile(csd_ctx* c, int enable) {
 int csd_profile_read(csd_ctx* c, int kernel_class, int64_t* launches, double* total_ms, double* total_flops) {
   if (!c) return CSD_ERR_INVALID_ARG;
   if (!launches || !total_ms || !total_flops) return fail(c, CSD_ERR_INVALID_ARG, "null output pointer");
-  if (kernel_class < 0 || kernel_class > 5) return fail(c, CSD_ERR_INVALID_ARG, "kernel class %d not in [0, 5]", kernel_class);
+  if (kernel_class < 0 || kernel_class > 6) return fail(c, CSD_ERR_INVALID_ARG, "kernel class %d not in [0, 6]", kernel_class);
   CSD_CUDA(c, cudaStreamSynchronize(c->stream));
   for (int i = 0; i < 2; ++i) CSD_CUDA(c, cudaStreamSynchronize(c->side[i]));
   *launches = 0; *total_ms = 0.0; *total_flops = 0.0;
@@ -669,6 +750,17 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
       if (!rc) rc = make_tmap(ctx, &tm.Wfss, d.dtype, h->Wfss, 2 * W, W, W, 2 * tn);
     }
     if (rc) { csd_head_destroy(h); return rc; }
+    std::vector<CUtensorMap> wm(4 * L + 1);
+    std::vector<const float*> bt(5 * L + 2);
+    for (size_t k = 0; k < L; ++k) {
+      wm[4 * k] = h->tm[1].Wss[k]; wm[4 * k + 1] = h->tm[1].Wg[k]; wm[4 * k + 2] = h->tm[1].W1[k]; wm[4 * k + 3] = h->tm[1].W2[k];
+      bt[5 * k] = h->bsh[k]; bt[5 * k + 1] = h->bsc[k]; bt[5 * k + 2] = h->b1[k]; bt[5 * k + 3] = h->bg[k]; bt[5 * k + 4] = h->b2[k];
+    }
+    wm[4 * L] = h->tm[1].Wfss; bt[5 * L] = h->bfsh; bt[5 * L + 1] = h->bfsc;
+    if (cudaMalloc(&h->d_wmaps, wm.size() * sizeof(CUtensorMap)) != cudaSuccess ||
+        cudaMalloc(&h->d_bias, bt.size() * sizeof(float*)) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the tables"); }
+    if (cudaMemcpy(h->d_wmaps, wm.data(), wm.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(h->d_bias, bt.data(), bt.size() * sizeof(float*), cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "table upload failed");
   }
   *out = h;
   return CSD_OK;
@@ -683,6 +775,8 @@ int csd_head_destroy(csd_head* h) {
   }
   if (h->wblob) cudaFree(h->wblob);
   if (h->fblob) cudaFree(h->fblob);
+  if (h->d_wmaps) cudaFree(h->d_wmaps);
+  if (h->d_bias) cudaFree(h->d_bias);
   cudaGetLastError();
   delete h;
   return CSD_OK;
@@ -814,8 +908,8 @@ int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, cons
     return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
   CSD_CUDA(ctx, cudaSetDevice(ctx->device));
   // workspaces first (growing one synchronises), then fork the two chains
-  if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T))) return rc;
-  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T, use_chain_kernel(head_q->d)))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T, use_chain_kernel(head_p->d)))) return rc;
   CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
   for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
   // the two chains' launches are interleaved step by step so that neither stream starves

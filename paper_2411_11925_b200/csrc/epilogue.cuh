@@ -105,7 +105,7 @@ struct RowState {
 __device__ __forceinline__ void chan_merge_equal(float& ma, float& m2a, float mb, float m2b, float n) {
   const float d = mb - ma;
   ma = fmaf(d, 0.5f, ma);
-  m2a += m2b + d * d * (0.5f * n);
+  m2a = __fadd_rn(m2a, fmaf(__fmul_rn(d, d), 0.5f * n, m2b));
 }
 
 // LayerNorm statistics of row m from its per-64-column (mean, M2) partials.  All partials have the
@@ -113,6 +113,8 @@ __device__ __forceinline__ void chan_merge_equal(float& ma, float& m2a, float mb
 // M2 = sum_g M2_g + n sum_g (mean_g - mean)^2  (Chan et al. for equal counts, all groups at once):
 // no chain of dependent divisions.  Sums run in group order, so the result does not depend on which
 // CTA computes it.  Up to 24 groups (W <= 1536) are loaded once, as one batch of 16-byte loads.
+// CG: read past the L1 cache (the partials were written by other CTAs of the same kernel).
+template <bool CG = false>
 __device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
   const int G = W / kStatCols;   // even: W is a multiple of 128
   const float4* p = reinterpret_cast<const float4*>(stats) + static_cast<size_t>(m) * (G / 2);
@@ -121,7 +123,7 @@ __device__ __forceinline__ void row_stats(const float* stats, int m, int W, floa
   if (G <= 2 * kB) {
     float4 b[kB];
 #pragma unroll
-    for (int j = 0; j < kB; ++j) b[j] = (2 * j < G) ? p[j] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    for (int j = 0; j < kB; ++j) b[j] = (2 * j < G) ? (CG ? __ldcg(p + j) : p[j]) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
 #pragma unroll
     for (int j = 0; j < kB; ++j)
       if (2 * j < G) { sum += b[j].x; sum += b[j].z; m2 += b[j].y; m2 += b[j].w; }
@@ -130,10 +132,10 @@ __device__ __forceinline__ void row_stats(const float* stats, int m, int W, floa
     for (int j = 0; j < kB; ++j)
       if (2 * j < G) { const float d0 = b[j].x - mean, d1 = b[j].z - mean; q = fmaf(d0, d0, q); q = fmaf(d1, d1, q); }
   } else {
-    for (int j = 0; j < G / 2; ++j) { const float4 b = p[j]; sum += b.x; sum += b.z; m2 += b.y; m2 += b.w; }
+    for (int j = 0; j < G / 2; ++j) { const float4 b = CG ? __ldcg(p + j) : p[j]; sum += b.x; sum += b.z; m2 += b.y; m2 += b.w; }
     mean = sum / static_cast<float>(G);
     for (int j = 0; j < G / 2; ++j) {
-      const float4 b = p[j];
+      const float4 b = CG ? __ldcg(p + j) : p[j];
       const float d0 = b.x - mean, d1 = b.z - mean;
       q = fmaf(d0, d0, q); q = fmaf(d1, d1, q);
     }
@@ -144,7 +146,7 @@ __device__ __forceinline__ void row_stats(const float* stats, int m, int W, floa
 
 template <int EPI>
 __device__ __forceinline__ void epi_row_begin(const EpiParams& ep, int m, RowState& rs) {
-  if constexpr (EPI == EPI_MOD || EPI == EPI_MODF) row_stats(ep.stats, m, ep.ldo, rs.mean, rs.rstd);
+  if constexpr (EPI == EPI_MOD || EPI == EPI_MODF) row_stats<false>(ep.stats, m, ep.ldo, rs.mean, rs.rstd);
   if constexpr (EPI == EPI_MODF) {
 #pragma unroll
     for (int c = 0; c < kCPad; ++c) rs.eacc[c] = 0.0f;
@@ -153,6 +155,58 @@ __device__ __forceinline__ void epi_row_begin(const EpiParams& ep, int m, RowSta
 }
 
 template <int EPI> __host__ __device__ constexpr bool epi_reads_h() { return EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES; }
+
+// Residual update of one 32-column chunk, hv += (a1 + b1) (a0 + b0), and its (mean, M2) partial merged
+// into the row state (a thread owns one or two chunks of a 64-column group: the second is merged with
+// equal counts).
+__device__ __forceinline__ void gate_res_chunk(const float* a0, const float* a1, const float* b0, const float* b1,
+                                               float* hv, RowState& rs) {
+  float sum = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kChunk; ++j) {
+    const float y = a0[j] + b0[j];
+    const float g = a1[j] + b1[j];
+    hv[j] = fmaf(g, y, hv[j]);
+    sum += hv[j];
+  }
+  const float mean = sum * (1.0f / kChunk);
+  float m2 = 0.0f;
+#pragma unroll
+  for (int j = 0; j < kChunk; ++j) {
+    const float d = hv[j] - mean;
+    m2 = fmaf(d, d, m2);
+  }
+  if (rs.pn <= 0.0f) { rs.pm = mean; rs.pm2 = m2; }
+  else chan_merge_equal(rs.pm, rs.pm2, mean, m2, static_cast<float>(kChunk));
+  rs.pn += static_cast<float>(kChunk);
+}
+
+// AdaLN modulation of one 32-column chunk: a0 <- LN(h)(1 + a1 + b1) + a0 + b0 (a0 = shift, a1 = scale).
+__device__ __forceinline__ void modulate_chunk(float* a0, const float* a1, const float* b0, const float* b1,
+                                               const float* hv, const RowState& rs) {
+#pragma unroll
+  for (int j = 0; j < kChunk; ++j) {
+    const float shift = a0[j] + b0[j];
+    const float scale = a1[j] + b1[j];
+    a0[j] = fmaf(__fmul_rn(__fsub_rn(hv[j], rs.mean), rs.rstd), __fadd_rn(1.0f, scale), shift);
+  }
+}
+
+// eps_hat partial of one chunk: eacc[c] += sum_j a0[j] Wout^T[j][c]  (wout_c: [32][16]).
+__device__ __forceinline__ void outproj_chunk(const float* a0, const float* wout_c, RowState& rs) {
+#pragma unroll
+  for (int j = 0; j < kChunk; ++j) {
+    const float4* w4 = reinterpret_cast<const float4*>(wout_c + j * kCPad);
+#pragma unroll
+    for (int c4 = 0; c4 < kCPad / 4; ++c4) {
+      const float4 w = w4[c4];
+      rs.eacc[4 * c4 + 0] = fmaf(a0[j], w.x, rs.eacc[4 * c4 + 0]);
+      rs.eacc[4 * c4 + 1] = fmaf(a0[j], w.y, rs.eacc[4 * c4 + 1]);
+      rs.eacc[4 * c4 + 2] = fmaf(a0[j], w.z, rs.eacc[4 * c4 + 2]);
+      rs.eacc[4 * c4 + 3] = fmaf(a0[j], w.w, rs.eacc[4 * c4 + 3]);
+    }
+  }
+}
 
 // a0 / a1: accumulator chunk (32 columns) of the first / second accumulator; n0 = first global
 // output column of the chunk; b0 / b1: the chunk's 32 biases (shared or global memory); hv: the
@@ -172,49 +226,12 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, fl
     for (int j = 0; j < kChunk; ++j) a0[j] = silu_t<FAST>(a0[j] + b0[j]);
     store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
   } else if constexpr (EPI == EPI_MOD || EPI == EPI_MODF) {
-#pragma unroll
-    for (int j = 0; j < kChunk; ++j) {
-      const float shift = a0[j] + b0[j];
-      const float scale = a1[j] + b1[j];
-      a0[j] = (hv[j] - rs.mean) * rs.rstd * (1.0f + scale) + shift;
-    }
-    if constexpr (EPI == EPI_MOD) {
-      store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
-    } else {
-#pragma unroll
-      for (int j = 0; j < kChunk; ++j) {
-        const float4* w4 = reinterpret_cast<const float4*>(wout_c + j * kCPad);
-#pragma unroll
-        for (int c4 = 0; c4 < kCPad / 4; ++c4) {
-          const float4 w = w4[c4];
-          rs.eacc[4 * c4 + 0] = fmaf(a0[j], w.x, rs.eacc[4 * c4 + 0]);
-          rs.eacc[4 * c4 + 1] = fmaf(a0[j], w.y, rs.eacc[4 * c4 + 1]);
-          rs.eacc[4 * c4 + 2] = fmaf(a0[j], w.z, rs.eacc[4 * c4 + 2]);
-          rs.eacc[4 * c4 + 3] = fmaf(a0[j], w.w, rs.eacc[4 * c4 + 3]);
-        }
-      }
-    }
+    modulate_chunk(a0, a1, b0, b1, hv, rs);
+    if constexpr (EPI == EPI_MOD) store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
+    else outproj_chunk(a0, wout_c, rs);
   } else if constexpr (EPI == EPI_GATE_RES) {
-    float sum = 0.0f;
-#pragma unroll
-    for (int j = 0; j < kChunk; ++j) {
-      const float y = a0[j] + b0[j];
-      const float g = a1[j] + b1[j];
-      hv[j] = fmaf(g, y, hv[j]);
-      sum += hv[j];
-    }
+    gate_res_chunk(a0, a1, b0, b1, hv, rs);
     store_chunk<float>(ep.h + off, hv);
-    const float mean = sum * (1.0f / kChunk);
-    float m2 = 0.0f;
-#pragma unroll
-    for (int j = 0; j < kChunk; ++j) {
-      const float d = hv[j] - mean;
-      m2 = fmaf(d, d, m2);
-    }
-    // a thread owns one or two chunks of the tile: the second is merged with equal counts
-    if (rs.pn <= 0.0f) { rs.pm = mean; rs.pm2 = m2; }
-    else chan_merge_equal(rs.pm, rs.pm2, mean, m2, static_cast<float>(kChunk));
-    rs.pn += static_cast<float>(kChunk);
   }
 }
 

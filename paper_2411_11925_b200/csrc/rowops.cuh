@@ -43,6 +43,34 @@ __global__ void convert_act_kernel(const float* __restrict__ src, ACT* __restric
 
 enum StepMode : int { STEP_INIT = 0, STEP_MID = 1, STEP_LAST = 2 };
 
+// Arithmetic of the step boundary, spelled with explicit roundings so that every kernel that
+// finishes a step produces the same bits.
+// guidance: eps_u + s (eps_c - eps_u)
+__device__ __forceinline__ float cfg_combine(float ec, float eu, float scale) { return fmaf(scale, __fsub_rn(ec, eu), eu); }
+// Eq. 3 mean: a x - b eps_hat
+__device__ __forceinline__ float ddpm_mean(float a, float x, float b, float e) { return fmaf(-b, e, __fmul_rn(a, x)); }
+// x_{t-1} = mu + sigma eps
+__device__ __forceinline__ float ddpm_sample(float mu, float sigma, float eps) { return fmaf(sigma, eps, mu); }
+
+// h = Win x + bin for the two columns (64 g + lane, 64 g + 32 + lane) of one row, and the (mean, M2)
+// LayerNorm partial of the row's 64-column group g (warp-wide; every lane returns the same partial).
+// wa / wb: the two columns' rows of Win (16 floats each), ba / bb their biases, xs: the row's x (16).
+__device__ __forceinline__ void input_proj_group(const float* wa, const float* wb, float ba, float bb, const float* xs,
+                                                 float acc[2], float& mean, float& m2) {
+  float a0 = ba, a1 = bb;
+#pragma unroll
+  for (int c = 0; c < kCPad; ++c) { a0 = fmaf(wa[c], xs[c], a0); a1 = fmaf(wb[c], xs[c], a1); }
+  acc[0] = a0; acc[1] = a1;
+  float sum = __fadd_rn(a0, a1);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  mean = sum * (1.0f / kStatCols);
+  const float d0 = a0 - mean, d1 = a1 - mean;
+  m2 = fmaf(d1, d1, __fmul_rn(d0, d0));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
+}
+
 struct StepParams {
   int R, cfg, C, W, NT;          // token rows, guidance flag, token dim, width, number of column tiles
   float cfg_scale, a, b, sigma;  // coefficients of the step being finished (t)
@@ -64,7 +92,7 @@ struct StepParams {
 
 // One block per token row.  Finishes step t (unless STEP_INIT) and prepares the next one:
 //   eps_hat = sum of tile partials + bout; guidance; mu = a x - b eps_hat; x <- mu + sigma eps_t
-//   h = Win x + bin (same for both guidance rows), LayerNorm partials per 32 columns,
+//   h = Win x + bin (same for both guidance rows), LayerNorm partials per 64 columns,
 //   s = SiLU(cz + te_next).
 template <typename ACT>
 __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
@@ -92,10 +120,10 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
       if (tid < p.C) {
         const size_t o = static_cast<size_t>(r) * p.C + tid;
         float e = eh[0][tid];
-        if (p.cfg) e = eh[1][tid] + p.cfg_scale * (eh[0][tid] - eh[1][tid]);
+        if (p.cfg) e = cfg_combine(eh[0][tid], eh[1][tid], p.cfg_scale);
         const float xo = p.x[o];
-        const float mu = p.a * xo - p.b * e;
-        xn = mu + p.sigma * p.eps_t[o];
+        const float mu = ddpm_mean(p.a, xo, p.b, e);
+        xn = ddpm_sample(mu, p.sigma, p.eps_t[o]);
         if (mode == STEP_LAST) {
           p.mu1[o] = mu;
           if (p.x1) p.x1[o] = xo;
@@ -113,30 +141,16 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
   const int lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
   ACT* s = reinterpret_cast<ACT*>(p.s);
   for (int g = warp; g < p.W / kStatCols; g += nwarp) {
-    float acc[2];
-    float sum = 0.0f;
+    float acc[2], mean, m2, wa[kCPad], wb[kCPad];
+    const int na = g * kStatCols + lane, nb = na + 32;
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int n = g * kStatCols + j * 32 + lane;
-      const float4* w4 = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(n) * kCPad);
-      float a = p.bin[n];
-#pragma unroll
-      for (int c4 = 0; c4 < kCPad / 4; ++c4) {
-        const float4 w = w4[c4];
-        a = fmaf(w.x, xs[4 * c4], a); a = fmaf(w.y, xs[4 * c4 + 1], a);
-        a = fmaf(w.z, xs[4 * c4 + 2], a); a = fmaf(w.w, xs[4 * c4 + 3], a);
-      }
-      acc[j] = a;
-      sum += a;
+    for (int c4 = 0; c4 < kCPad / 4; ++c4) {
+      const float4 qa = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(na) * kCPad)[c4];
+      const float4 qb = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(nb) * kCPad)[c4];
+      wa[4 * c4] = qa.x; wa[4 * c4 + 1] = qa.y; wa[4 * c4 + 2] = qa.z; wa[4 * c4 + 3] = qa.w;
+      wb[4 * c4] = qb.x; wb[4 * c4 + 1] = qb.y; wb[4 * c4 + 2] = qb.z; wb[4 * c4 + 3] = qb.w;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    const float mean = sum * (1.0f / kStatCols);
-    float m2 = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 2; ++j) { const float d = acc[j] - mean; m2 = fmaf(d, d, m2); }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m2 += __shfl_xor_sync(0xffffffffu, m2, o);
+    input_proj_group(wa, wb, p.bin[na], p.bin[nb], xs, acc, mean, m2);
     for (int rep = 0; rep < nrep; ++rep) {
       const size_t row = static_cast<size_t>(r) + static_cast<size_t>(rep) * p.R;
       if (lane == 0)
