@@ -23,7 +23,7 @@ CSD_F32, CSD_BF16, CSD_F16 = 0, 1, 2
 DTYPES = {"f32": CSD_F32, "bf16": CSD_BF16, "f16": CSD_F16}
 
 EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launch_count",
-           "csd_profile", "csd_profile_read",
+           "csd_set_chain_mode", "csd_profile", "csd_profile_read",
            "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_draft_denoise_static", "csd_verify",
            "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host")
 
@@ -62,6 +62,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_last_error.argtypes = [vp]; lib.csd_last_error.restype = C.c_char_p
     lib.csd_sync.argtypes = [vp]
     lib.csd_launch_count.argtypes = [vp]; lib.csd_launch_count.restype = C.c_int64
+    lib.csd_set_chain_mode.argtypes = [vp, C.c_int]
     lib.csd_profile.argtypes = [vp, i32]
     lib.csd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_int64), C.POINTER(f64), C.POINTER(f64)]
     lib.csd_head_create.argtypes = [vp, C.POINTER(_HeadDesc), C.POINTER(_HeadWeights), C.POINTER(vp)]
@@ -145,6 +146,10 @@ class Context:
 
     def launch_count(self) -> int:
         return int(_LIB.csd_launch_count(self._h))
+
+    def set_chain_mode(self, cluster: bool):
+        """csd_set_chain_mode: False = one kernel per layer (default), True = one cluster kernel per chain."""
+        self._check(_LIB.csd_set_chain_mode(self._h, 1 if cluster else 0))
 
     KERNEL_CLASSES = ("cond_proj", "mlp1_silu", "adaln_modulate", "mlp2_gate_residual", "final_mod_outproj", "step", "chain")
 

@@ -11,7 +11,10 @@
 // 4-slot TMA ring feeds tcgen05 MMAs into three TMEM accumulators (AdaLN shift|scale 256 columns, gate
 // 128, MLP 128), so the products that depend only on the condition vector s (modulation of the next
 // block, gate of this block) are issued while this block's dependent layers are in their epilogues.
-// Warp 0 requests tiles, warp 1 issues MMAs, 16 epilogue warps (one row x 32 columns per thread).
+// Warp 0 requests activation tiles, the last warp weight tiles (one thread sustains about one TMA request
+// per 300 clk), warp 1 issues MMAs, 16 epilogue warps (one row x 32 columns per thread).  The activations
+// u, v, s are kept in the kernel's own row order (row block after row block), so a tile is one TMA box even
+// with guidance, where a row block holds 64 conditional rows and their 64 unconditional twins.
 //
 // The arithmetic (accumulation order, epilogue formulas, LayerNorm and eps_hat partial layout) is that of
 // the layer-by-layer kernels; the two paths give the same bits.
@@ -25,7 +28,7 @@ constexpr int kChSlots = 4;                     // ring slots: [A tile 16 KB | B
 constexpr int kChSlotBytes = 32768;
 constexpr int kChEpiWarps = 16;
 constexpr int kChEpiThreads = kChEpiWarps * 32;
-constexpr int kChThreads = kChEpiThreads + 64;
+constexpr int kChThreads = kChEpiThreads + 96;   // + TMA (activations), MMA, TMA (weights)
 constexpr int kChHBytes = kTileM * kTileN * 4;  // h slice: 4 chunks of [128 rows][128 B], 128-byte swizzle
 constexpr int kChWoutBytes = kTileN * kCPad * 4;
 constexpr int kChXBytes = kTileM * kCPad * 4;   // x of the row block's tokens
@@ -40,7 +43,7 @@ enum ChainAcc : int { ACC_MOD = 0, ACC_GATE = 1, ACC_MAIN = 2 };
 
 struct ChainParams {
   const CUtensorMap* wmaps;   // device: per block Wss (256-row boxes), Wg, W1, W2 (128-row boxes); then Wfss
-  const CUtensorMap* amaps;   // device: s for even t, s for odd t, u, v (boxes of 64 rows x 64 columns)
+  const CUtensorMap* amaps;   // device: s for even t, s for odd t, u, v (boxes of 128 rows x 64 columns)
   int R, cfg, W, L, T, C, sample_last;
   float cfg_scale;
   const float* sched;         // device [3 T]: a, b, sigma
@@ -48,8 +51,8 @@ struct ChainParams {
   const float* te;            // [T, W]
   const float* const* bias;   // device [5 L + 2]: per block shift, scale, b1, gate, b2 biases; final shift, scale
   const float *win, *bin, *wout_t, *bout;
-  void* s[2];                 // s of even / odd t, [Rh, W]
-  void *u, *v;                // [Rh, W]
+  void* s[2];                 // s of even / odd t, [row blocks * 128, W], the kernel's row order
+  void *u, *v;                // same shape and order
   float* stats;               // [Rh, W/64, 2]
   float* epart;               // [Rh, W/64, 16]
   const float *x_T, *eps;     // [R, C], [T, R, C]
@@ -130,13 +133,12 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
   const int nkb = W / kBlockK;
   const int G = W / kStatCols;
   const int n_base = j * kTileN;
-  // rows of the two 64-row A boxes
-  const int row0 = tb * TB, row1 = p.cfg ? p.R + tb * TB : tb * TB + 64;
+  const int row0 = tb * kTileM;   // first row of the block in u, v, s
   const int syncs_per_step = 3 * L + 2;
 
   const bool run = *reinterpret_cast<const volatile int*>(p.err) == 0;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kChSlots; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < kChSlots; ++s) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
     for (int a = 0; a < 3; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 1); }
     *sync_cnt = 0;
     fence_mbar_init();
@@ -161,32 +163,28 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
       if (ok && c >= kChSlots) { ok = ch_wait<false>(&empty_bar[c % kChSlots], ((c / kChSlots) & 1) ^ 1, p.err); if (!ok && leader) ch_fail(p.err, DEV_ERR_TMA_WAIT, 2, c); }
     };
     // N = 128 segment: one slot per k-block
-    auto seg128 = [&](const CUtensorMap* ta, const CUtensorMap* tw) {
+    auto seg128 = [&](const CUtensorMap* ta) {
       for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
         slot_free(it);
         if (ok && leader) {
           const int s = it % kChSlots;
           uint8_t* dst = ring + s * kChSlotBytes;
-          mbar_arrive_expect_tx(&full_bar[s], kChSlotBytes);
+          mbar_arrive_expect_tx(&full_bar[s], 16384);
           tma_load_2d(dst, ta, &full_bar[s], kb * kBlockK, row0);
-          tma_load_2d(dst + 8192, ta, &full_bar[s], kb * kBlockK, row1);
-          tma_load_2d(dst + 16384, tw, &full_bar[s], kb * kBlockK, n_base);
         }
         __syncwarp();
       }
     };
     // N = 256 segment (packed shift|scale rows): two slots per k-block, the 32 KB weight tile runs from
     // the second half of the first slot through the first half of the second
-    auto seg256 = [&](const CUtensorMap* ta, const CUtensorMap* tw) {
+    auto seg256 = [&](const CUtensorMap* ta) {
       for (int kb = 0; kb < nkb && ok; ++kb, it += 2) {
         slot_free(it); slot_free(it + 1);
         if (ok && leader) {
           const int s = it % kChSlots;
           uint8_t* dst = ring + s * kChSlotBytes;
-          mbar_arrive_expect_tx(&full_bar[s], 16384 + 32768);
+          mbar_arrive_expect_tx(&full_bar[s], 16384);
           tma_load_2d(dst, ta, &full_bar[s], kb * kBlockK, row0);
-          tma_load_2d(dst + 8192, ta, &full_bar[s], kb * kBlockK, row1);
-          tma_load_2d(dst + 16384, tw, &full_bar[s], kb * kBlockK, 2 * n_base);
           mbar_arrive(&full_bar[s + 1]);
         }
         __syncwarp();
@@ -195,20 +193,60 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
     const CUtensorMap* tm_u = p.amaps + 2;
     const CUtensorMap* tm_v = p.amaps + 3;
     sync_until(0);
-    seg256(p.amaps + (T & 1), p.wmaps);                               // modulation of block 0, step T
+    seg256(p.amaps + (T & 1));                                        // modulation of block 0, step T
     for (int si = 0; si < T && ok; ++si) {
       const int t = T - si, base = 1 + si * syncs_per_step;
       const CUtensorMap* tm_s = p.amaps + (t & 1);
       for (int k = 0; k < L && ok; ++k) {
-        const CUtensorMap* wk = p.wmaps + 4 * k;
-        sync_until(base + 3 * k);       seg128(tm_u, wk + 2);          // u W1^T
-        seg128(tm_s, wk + 1);                                         // s Wg^T
-        sync_until(base + 3 * k + 1);   seg128(tm_v, wk + 3);          // v W2^T
-        seg256(tm_s, wk + 4);                                         // modulation of block k + 1 / final
+        sync_until(base + 3 * k);       seg128(tm_u);                  // u W1^T
+        seg128(tm_s);                                                 // s Wg^T
+        sync_until(base + 3 * k + 1);   seg128(tm_v);                  // v W2^T
+        seg256(tm_s);                                                 // modulation of block k + 1 / final
       }
-      if (t > 1) seg256(p.amaps + ((t - 1) & 1), p.wmaps);            // modulation of block 0, next step
+      if (t > 1) seg256(p.amaps + ((t - 1) & 1));                     // modulation of block 0, next step
     }
     if (!ok && leader) ch_fail(p.err, DEV_ERR_TMA_WAIT, 0, 0);
+    __syncwarp();
+  } else if (run && warp == kChEpiWarps + 2) {
+    // ------------------------------------------------------------------ TMA requests, weight tiles
+    // (never wait for the cluster: the ring fills with the weights of layers whose activations are not ready yet)
+    const bool leader = elect_one();
+    bool ok = true;
+    int it = 0;
+    auto slot_free = [&](int c) {
+      if (ok && c >= kChSlots) { ok = ch_wait<false>(&empty_bar[c % kChSlots], ((c / kChSlots) & 1) ^ 1, p.err); if (!ok && leader) ch_fail(p.err, DEV_ERR_TMA_WAIT, 8, c); }
+    };
+    auto seg128 = [&](const CUtensorMap* tw) {
+      for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
+        slot_free(it);
+        if (ok && leader) {
+          const int s = it % kChSlots;
+          mbar_arrive_expect_tx(&full_bar[s], 16384);
+          tma_load_2d(ring + s * kChSlotBytes + 16384, tw, &full_bar[s], kb * kBlockK, n_base);
+        }
+        __syncwarp();
+      }
+    };
+    auto seg256 = [&](const CUtensorMap* tw) {
+      for (int kb = 0; kb < nkb && ok; ++kb, it += 2) {
+        slot_free(it); slot_free(it + 1);
+        if (ok && leader) {
+          const int s = it % kChSlots;
+          mbar_arrive_expect_tx(&full_bar[s], 32768);
+          tma_load_2d(ring + s * kChSlotBytes + 16384, tw, &full_bar[s], kb * kBlockK, 2 * n_base);
+          mbar_arrive(&full_bar[s + 1]);
+        }
+        __syncwarp();
+      }
+    };
+    seg256(p.wmaps);
+    for (int si = 0; si < T && ok; ++si) {
+      for (int k = 0; k < L && ok; ++k) {
+        const CUtensorMap* wk = p.wmaps + 4 * k;
+        seg128(wk + 2); seg128(wk + 1); seg128(wk + 3); seg256(wk + 4);
+      }
+      if (si + 1 < T) seg256(p.wmaps);
+    }
     __syncwarp();
   } else if (run && warp == 1) {
     // ------------------------------------------------------------------ MMA issue
@@ -274,7 +312,7 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
     }
     if (!ok && leader) ch_fail(p.err, DEV_ERR_MMA_WAIT, 0, 0);
     __syncwarp();
-  } else if (run && warp >= 2) {
+  } else if (run && warp >= 2 && warp < kChEpiWarps + 2) {
     // ------------------------------------------------------------------ epilogues
     const int et = static_cast<int>(threadIdx.x) - 64;
     const int ew = warp - 2;
@@ -287,6 +325,7 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
     const int n0 = n_base + cg * kChunk;
     const uint32_t trow = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     uint8_t* h_chunk = h_s + cg * (kTileM * 128);
+    const size_t mi = static_cast<size_t>(row0 + rloc);   // row in u, v, s
     ACT* u_out = reinterpret_cast<ACT*>(p.u);
     ACT* v_out = reinterpret_cast<ACT*>(p.v);
     bool ok = true;
@@ -326,12 +365,13 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
       if (et < 256) bias_s[(bias_buf ^ 1) * 256 + et] = next_bias;
       bias_buf ^= 1;
       tc_fence_before_sync();
-      __threadfence();
       fence_proxy_async_all();
       asm volatile("bar.sync 1, %0;" ::"n"(kChEpiThreads) : "memory");
       if (et == 0 && ok) {
         for (int a = 0; a < 3; ++a)
           if (release_mask & (1 << a)) mbar_arrive(&acc_empty[a]);
+        // one fence for the whole CTA's stores (ordered before it by the barrier), then relaxed signals
+        __threadfence();
         const uint32_t sb = smem_u32(sync_cnt);
         for (int r = 0; r < nc; ++r) red_add_cluster(mapa_shared(sb, static_cast<uint32_t>(r)), 1u);
       }
@@ -378,7 +418,7 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
         load_chunk_f32(p.te + static_cast<size_t>(tp - 1) * W + n_base + cc * kChunk, b);
 #pragma unroll
         for (int i = 0; i < kChunk; ++i) a[i] = silu_f(a[i] + b[i]);
-        store_chunk<ACT>(reinterpret_cast<ACT*>(p.s[tp & 1]) + off, a);
+        store_chunk<ACT>(reinterpret_cast<ACT*>(p.s[tp & 1]) + static_cast<size_t>(row0 + l) * W + n_base + cc * kChunk, a);
       }
     };
 
@@ -416,7 +456,7 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
           const float* b = bias_s + bias_buf * 256 + cg * kChunk;
           modulate_chunk(a0, a1, b, b + 128, hv, rs);
           if (!fin) {
-            if (valid) store_chunk<ACT>(u_out + static_cast<size_t>(m) * W + n0, a0);
+            if (valid) store_chunk<ACT>(u_out + mi * W + n0, a0);
           } else {
 #pragma unroll
             for (int c = 0; c < kCPad; ++c) rs.eacc[c] = 0.0f;
@@ -454,7 +494,7 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
           const float* b = bias_s + bias_buf * 256 + cg * kChunk;
 #pragma unroll
           for (int i = 0; i < kChunk; ++i) a0[i] = silu_t<true>(a0[i] + b[i]);
-          if (valid) store_chunk<ACT>(v_out + static_cast<size_t>(m) * W + n0, a0);
+          if (valid) store_chunk<ACT>(v_out + mi * W + n0, a0);
         }
         phase_end(1 << ACC_MAIN);                                        // sync base + 3 k + 1
 
@@ -497,7 +537,13 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
             for (int rp = 0; rp < nrep; ++rp) {
               const float* src = p.epart + (static_cast<size_t>(tok + rp * p.R) * G) * kCPad + c;
               float acc = 0.0f;
-              for (int nt = 0; nt < G; ++nt) acc += __ldcg(src + nt * kCPad);
+              for (int n8 = 0; n8 < G; n8 += 8) {   // loads in batches, sums in group order
+                float pv[8];
+#pragma unroll
+                for (int i8 = 0; i8 < 8; ++i8) pv[i8] = (n8 + i8 < G) ? __ldcg(src + (n8 + i8) * kCPad) : 0.0f;
+#pragma unroll
+                for (int i8 = 0; i8 < 8; ++i8) if (n8 + i8 < G) acc += pv[i8];
+              }
               e[rp] = acc + p.bout[c];
             }
             const float eh = p.cfg ? cfg_combine(e[0], e[1], p.cfg_scale) : e[0];

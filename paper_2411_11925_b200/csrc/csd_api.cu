@@ -55,6 +55,7 @@ struct csd_ctx {
   cudaEvent_t ev_fork = nullptr, ev_done[2] = {nullptr, nullptr};
   int* d_err = nullptr;
   int64_t launches = 0;
+  int chain_mode = CSD_CHAIN_LAYERS;   // csd_set_chain_mode
   EncodeTiledFn encode = nullptr;
   ChainWs ws[3];   // draft chain, target chain, static-scratch calls
   HostIo io;
@@ -171,13 +172,15 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
   const size_t o_zc = take(static_cast<size_t>(Rh) * d.Dz * asz);
-  const size_t o_s = take(Rh * W * asz), o_u = take(Rh * W * asz), o_v = take(Rh * W * asz);
+  // the whole-chain kernel keeps u, v, s in row blocks of 128 (the last one padded)
+  const size_t Ra = chain_kernel_extras ? static_cast<size_t>(Rh) + 128 : static_cast<size_t>(Rh);
+  const size_t o_s = take(Ra * W * asz), o_u = take(Ra * W * asz), o_v = take(Ra * W * asz);
   const size_t o_cz = take(Rh * W * 4), o_te = take(static_cast<size_t>(T) * W * 4), o_h = take(Rh * W * 4);
   const size_t o_st = take(Rh * (W / kStatCols) * 8);
   const size_t o_ep = take(Rh * (W / kStatCols) * kCPad * 4);   // room for 64-wide tiles
   const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
   size_t o_s2 = 0, o_sched = 0, o_amaps = 0;
-  if (chain_kernel_extras) { o_s2 = take(Rh * W * asz); o_sched = take(static_cast<size_t>(T) * 3 * 4); o_amaps = take(4 * sizeof(CUtensorMap)); }
+  if (chain_kernel_extras) { o_s2 = take(Ra * W * asz); o_sched = take(static_cast<size_t>(T) * 3 * 4); o_amaps = take(4 * sizeof(CUtensorMap)); }
   if (off > ws.cap) {
     CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamSynchronize(ctx->side[i]));
@@ -352,7 +355,7 @@ struct Chain {
     pair = tc && tn == kTileN && (W / kTileN) * ((Rh + kTileM - 1) / kTileM) >= 2 * ctx->num_sms;
     // One kernel for the whole chain when a row block's column slices fit one portable cluster.  The choice
     // depends on the head only, and both paths give the same bits.
-    whole = allow_chain_kernel && tc && use_chain_kernel(d);
+    whole = allow_chain_kernel && tc && ctx->chain_mode == CSD_CHAIN_CLUSTER && use_chain_kernel(d);
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T, whole);
     if (rc) return rc;
@@ -397,7 +400,9 @@ struct Chain {
     int rc = CSD_OK;
     CUtensorMap am[4];
     void* const bufs[4] = {ws.s2, ws.s, ws.u, ws.v};   // s of even t, s of odd t, u, v
-    for (int i = 0; i < 4 && !rc; ++i) rc = make_tmap(ctx, &am[i], d.dtype, bufs[i], Rh, W, W, 64);
+    const int nc = W / kTileN, tb_rows = cfg ? kTileM / 2 : kTileM;
+    const int nb = (R + tb_rows - 1) / tb_rows;
+    for (int i = 0; i < 4 && !rc; ++i) rc = make_tmap(ctx, &am[i], d.dtype, bufs[i], static_cast<uint64_t>(nb) * kTileM, W, W, kTileM);
     if (rc) return rc;
     // small pageable sources: staged by the runtime before the calls return
     CSD_CUDA(ctx, cudaMemcpyAsync(ws.amaps, am, sizeof(am), cudaMemcpyHostToDevice, st));
@@ -411,8 +416,6 @@ struct Chain {
     p.win = hd->win; p.bin = hd->bin; p.wout_t = hd->wout_t; p.bout = hd->bout;
     p.s[0] = ws.s2; p.s[1] = ws.s; p.u = ws.u; p.v = ws.v; p.stats = ws.stats; p.epart = ws.epart;
     p.x_T = x_T; p.eps = eps; p.x0 = x0; p.mu1 = mu1; p.x1 = x1; p.err = ctx->d_err;
-    const int nc = W / kTileN, tb_rows = cfg ? kTileM / 2 : kTileM;
-    const int nb = (R + tb_rows - 1) / tb_rows;
     const double flops_step = 2.0 * Rh * static_cast<double>(W) * W * (5.0 * L + 2.0) + 2.0 * Rh * static_cast<double>(W) * d.C * 2.0;
     ProfScope ps(ctx, st, 6, flops_step * T);
     cudaLaunchConfig_t lc{};
@@ -613,6 +616,13 @@ int csd_sync(csd_ctx* c) {
     return fail(c, CSD_ERR_TIMEOUT, "a device-side bounded wait gave up (code %d: 1 = TMA producer, 2 = MMA issuer, "
                 "3 = epilogue)", e);
   }
+  return CSD_OK;
+}
+
+int csd_set_chain_mode(csd_ctx* c, int mode) {
+  if (!c) return CSD_ERR_INVALID_ARG;
+  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_CLUSTER) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
+  c->chain_mode = mode;
   return CSD_OK;
 }
 
@@ -908,8 +918,8 @@ int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, cons
     return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
   CSD_CUDA(ctx, cudaSetDevice(ctx->device));
   // workspaces first (growing one synchronises), then fork the two chains
-  if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T, use_chain_kernel(head_q->d)))) return rc;
-  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T, use_chain_kernel(head_p->d)))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T, ctx->chain_mode == CSD_CHAIN_CLUSTER && use_chain_kernel(head_q->d)))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T, ctx->chain_mode == CSD_CHAIN_CLUSTER && use_chain_kernel(head_p->d)))) return rc;
   CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
   for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
   // the two chains' launches are interleaved step by step so that neither stream starves

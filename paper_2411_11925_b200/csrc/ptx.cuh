@@ -168,9 +168,10 @@ __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.w
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-// Counter in shared memory that CTAs of the cluster bump remotely: add with release, read with acquire.
+// Counter in shared memory that CTAs of the cluster bump remotely: relaxed add (the caller fences once
+// before a batch of them), read with acquire.
 __device__ __forceinline__ void red_add_cluster(uint32_t cluster_addr, uint32_t v) {
-  asm volatile("red.release.cluster.shared::cluster.add.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+  asm volatile("red.relaxed.cluster.shared::cluster.add.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_acquire_cluster(const uint32_t* smem_word) {
   uint32_t v;

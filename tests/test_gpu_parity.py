@@ -271,3 +271,35 @@ def test_degenerate_sizes_single_row_single_step_widest_scan(op):
     for kw in (dict(B=1, gamma=1, T=1), dict(B=2, gamma=32, T=2), dict(B=1, gamma=3, T=3, cfg=True, cfg_scale=1.5)):
         wl = _wl(bf16=op != "f32", operand=op, draft=gen.HeadSpec(1, 128, 64), target=gen.HeadSpec(1, 128, 128), **kw)
         _check(gen.make_round_inputs(wl), f"degenerate {op} {kw}")
+
+
+@pytest.mark.parametrize("op", ["bf16", "f16"])
+def test_cluster_chain_layout_is_bit_identical_to_layer_kernels(op):
+    # csd_set_chain_mode(CSD_CHAIN_CLUSTER): one cluster kernel per chain.  Same bits as the default layout, with and
+    # without guidance, ragged row blocks (with guidance a block holds 64 tokens, else 128), one to eight CTAs per
+    # cluster, a single step, and a head too wide for a cluster (W = 1152: falls back to the layer kernels).
+    from paper_2411_11925_b200.runner import DeviceRound
+    cases = (dict(B=5, gamma=7, T=6, cfg=True, cfg_scale=3.0),
+             dict(B=23, gamma=7, T=5, cfg=True, cfg_scale=3.0, draft=gen.HeadSpec(1, 256, 128), target=gen.HeadSpec(2, 384, 192)),
+             dict(B=37, gamma=8, T=4, cfg=False, cfg_scale=1.0, draft=gen.HeadSpec(2, 768, 128), target=gen.HeadSpec(1, 1024, 128)),
+             dict(B=1, gamma=1, T=1, draft=gen.HeadSpec(1, 128, 64), target=gen.HeadSpec(1, 128, 128)),
+             dict(B=3, gamma=5, T=3, cfg=True, cfg_scale=2.0, draft=gen.HeadSpec(1, 128, 64), target=gen.HeadSpec(1, 1152, 128)))
+    keys = ("x0", "mu1_q", "mu1_p", "x1_q", "logratio", "n_accept", "accept_mask", "x_new", "n_prop", "flags")
+    for kw in cases:
+        inp = gen.make_round_inputs(_wl(bf16=True, operand=op, **kw))
+        dr = DeviceRound(inp)
+        dr.three_calls()
+        a = dr.results()
+        launches_layers = dr.ctx.launch_count()
+        dr.ctx.set_chain_mode(True)
+        dr.three_calls()
+        b = dr.results()
+        assert dr.ctx.launch_count() - launches_layers < launches_layers   # far fewer launches: the cluster kernels ran
+        for k in keys:
+            np.testing.assert_array_equal(a[k], b[k], err_msg=f"{kw} {k}")
+        dr.fused_round()
+        c = dr.results()
+        for k in keys:
+            if k != "x1_q":
+                np.testing.assert_array_equal(a[k], c[k], err_msg=f"fused {kw} {k}")
+        dr.ctx.close()
