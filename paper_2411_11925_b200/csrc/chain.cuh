@@ -578,3 +578,4 @@ __global__ void __launch_bounds__(kChThreads, 1) chain_kernel(const ChainParams 
 }
 
 }  // namespace csd
+

@@ -114,10 +114,10 @@ __device__ __forceinline__ void chan_merge_equal(float& ma, float& m2a, float mb
 // no chain of dependent divisions.  Sums run in group order, so the result does not depend on which
 // CTA computes it.  Up to 24 groups (W <= 1536) are loaded once, as one batch of 16-byte loads.
 // CG: read past the L1 cache (the partials were written by other CTAs of the same kernel).
+// p: the row's G (mean, M2) pairs, 16-byte aligned.
 template <bool CG = false>
-__device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
+__device__ __forceinline__ void row_stats_at(const float4* p, int W, float& mean, float& rstd) {
   const int G = W / kStatCols;   // even: W is a multiple of 128
-  const float4* p = reinterpret_cast<const float4*>(stats) + static_cast<size_t>(m) * (G / 2);
   constexpr int kB = 12;         // 16-byte loads (two groups each) per batch
   float sum = 0.0f, m2 = 0.0f, q = 0.0f;
   if (G <= 2 * kB) {
@@ -142,6 +142,11 @@ __device__ __forceinline__ void row_stats(const float* stats, int m, int W, floa
   }
   const float m2t = fmaf(static_cast<float>(kStatCols), q, m2);
   rstd = 1.0f / sqrtf(m2t / static_cast<float>(W) + 1e-6f);
+}
+
+template <bool CG = false>
+__device__ __forceinline__ void row_stats(const float* stats, int m, int W, float& mean, float& rstd) {
+  row_stats_at<CG>(reinterpret_cast<const float4*>(stats) + static_cast<size_t>(m) * (W / kStatCols / 2), W, mean, rstd);
 }
 
 template <int EPI>
