@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--workload", default="mar256")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--no-seq", action="store_true", help="skip the sequential-draft variant")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     return ap.parse_args()
 
@@ -228,6 +229,47 @@ def run_ours(args):
     h2d = sum(hosts[0][n].numel() * hosts[0][n].element_size() for n in in_names)
     d2h = sum(hosts[0][n].numel() * hosts[0][n].element_size() for n in out_names)
 
+    # Sequential-draft variant: how an autoregressive loop has to call the draft head, one position at a time
+    # (gamma calls of csd_draft_denoise with B tokens = B (1 + cfg) head rows each).  Few rows per call: the
+    # binding resource is streaming the draft head's weights once per denoising step.
+    seq = None
+    if world == 1 and not args.no_seq:
+        wl1 = gen.Workload(**{**wl.__dict__, "gamma": 1})
+        inp1 = gen.make_round_inputs(wl1, seed_offset=5000, weights=False)
+        inp1.w_q, inp1.w_p = inp0.w_q, inp0.w_p
+        r1 = DeviceRound(inp1, ctx=ctx, device=local, heads=(rounds[0].head_q, rounds[0].head_p))
+        seq_step = lambda i: [r1.draft() for _ in range(wl.gamma)]
+        timed(seq_step, 2)
+        seq_steps = max(2, min(args.steps, 5))
+        seq_secs = timed(seq_step, seq_steps)
+        d = wl.draft
+        wbytes = 2.0 * (d.W * d.Dz + d.L * 5 * d.W * d.W + 2 * d.W * d.W)     # 16-bit GEMM weights of the draft head
+        per_call = seq_secs / (seq_steps * wl.gamma)
+        seq = {"calls_per_round": wl.gamma, "head_rows_per_call": wl.B * (2 if wl.cfg else 1),
+               "ms_per_call": 1e3 * per_call, "value": wl.B * wl.gamma * seq_steps / seq_secs, "unit": UNIT,
+               "bound": "hbm", "weight_bytes_per_step": wbytes,
+               "achieved": wbytes * wl.T / per_call / 1e9, "peak": peaks["hbm_gbs"], "roofline_unit": "GB/s",
+               "frac": wbytes * wl.T / per_call / 1e9 / peaks["hbm_gbs"],
+               "note": "algorithmic bytes = draft weight bytes x T per call; the weights fit L2 (126 MB), so the "
+                       "fraction says how far the call is from streaming them from HBM once per step"}
+
+    # Token pre-filling (Sec. 3.2): the first tokens of an image come from the target head alone, one
+    # csd_draft_denoise call with the target head over B * prefill tokens; timed separately.
+    prefill = None
+    if world == 1 and wl.prefill and wl.prefill == wl.gamma and not args.no_seq:
+        r0 = rounds[0]
+        px0, pmu = torch.zeros_like(r0.x0), torch.zeros_like(r0.x0)
+        pre_step = lambda i: ctx.csd_draft_denoise(r0.head_p, r0.sched_p, wl.R, wl.cfg, wl.cfg_scale, r0.z_p, r0.x_T, r0.eps,
+                                                   px0, pmu, None)
+        timed(pre_step, 1)
+        pre_steps = max(2, min(args.steps, 5))
+        pre_secs = timed(pre_step, pre_steps)
+        t = wl.target
+        fl = (2 if wl.cfg else 1) * wl.R * wl.T * 2.0 * (2 * t.C * t.W + 5 * t.L * t.W * t.W + 2 * t.W * t.W)
+        prefill = {"tokens": wl.R, "ms": 1e3 * pre_secs / pre_steps, "value": wl.R * pre_steps / pre_secs, "unit": "prefilled tokens/s",
+                   "algorithmic_tflops": fl * pre_steps / pre_secs / 1e12,
+                   "frac_of_tensor_peak": fl * pre_steps / pre_secs / 1e12 / peaks["tflops_sustained"]}
+
     # per-kernel-class device time over the same steps (events around every launch: separate pass)
     prof = None
     if not args.no_profile:
@@ -276,6 +318,10 @@ def run_ours(args):
                                                   "share": round(v["ms"] / tot_ms, 4),
                                                   "tflops": (v["flops"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0)}
                                               for k, v in prof.items()}}
+        if seq:
+            line["sequential_draft"] = seq
+        if prefill:
+            line["prefill"] = prefill
         if not args.no_cpu_baseline and world == 1:
             val, threads, desc, _ = time_oracle(args.workload, 15.0)
             line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
