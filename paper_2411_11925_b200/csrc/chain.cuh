@@ -99,7 +99,7 @@ __device__ __forceinline__ bool ch_wait_count(const uint32_t* cnt, uint32_t targ
   }
 }
 
-// 18 warps: the register file is split over four schedulers, so five warps on one of them cap a thread at
+// 19 warps: the register file is split over four schedulers, so five warps on one of them cap a thread at
 // 96 registers.
 // First failing wait of a chain kernel: role (DevErr) | site << 4 | (count & 0xffff) << 8 | (block & 0x7f) << 24.
 __device__ __forceinline__ void ch_fail(int* err, int role, int site, int count) {

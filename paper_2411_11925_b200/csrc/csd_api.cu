@@ -563,8 +563,12 @@ int csd_create(csd_ctx** out, int device, void* cuda_stream) {
   c->num_sms = prop.multiProcessorCount;
   c->stream = static_cast<cudaStream_t>(cuda_stream);
   bool ok = true;
+  // side[1] outranks side[0]: csd_round puts the longer of its two chains there, so that the chain that decides
+  // the round's duration gets free SMs first and the shorter one fills the gaps
+  int prio_lo = 0, prio_hi = 0;
+  cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
   for (int i = 0; i < 2; ++i) {
-    ok = ok && cudaStreamCreateWithFlags(&c->side[i], cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithPriority(&c->side[i], cudaStreamNonBlocking, i == 1 ? prio_hi : prio_lo) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
   }
   ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
@@ -923,8 +927,11 @@ int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, cons
   CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
   for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
   // the two chains' launches are interleaved step by step so that neither stream starves
-  Chain cq{ctx, 0, ctx->side[0], head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr};
-  Chain cp{ctx, 1, ctx->side[1], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr};
+  // the chain with more work per row goes to the higher-priority stream
+  const double wq = static_cast<double>(head_q->d.L) * head_q->d.W * head_q->d.W, wp = static_cast<double>(head_p->d.L) * head_p->d.W * head_p->d.W;
+  const int sq = wq > wp ? 1 : 0;
+  Chain cq{ctx, 0, ctx->side[sq], head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr};
+  Chain cp{ctx, 1, ctx->side[1 - sq], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr};
   cq.chains = cp.chains = 2;
   rc = cp.begin();
   int rc2 = cq.begin();
