@@ -85,6 +85,7 @@ struct csd_head {
     CUtensorMap Wz{}, Wfss{};
     std::vector<CUtensorMap> Wss, Wg, W1, W2;
   } tm[2];
+  std::vector<CUtensorMap> W1_wide;   // first MLP layer with 256-row boxes (W a multiple of 256)
   // whole-chain kernel: device copies of the weight tensor maps (per block Wss, Wg, W1, W2; then Wfss) and of
   // the bias pointers (per block shift, scale, b1, gate, b2; then final shift, scale)
   CUtensorMap* d_wmaps = nullptr;
@@ -320,6 +321,7 @@ struct Chain {
   int chains = 1;   // chains that run concurrently with this one (itself included)
   bool allow_chain_kernel = true, whole = false;   // whole: one kernel runs the whole chain
   int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
+  bool w1_wide = false;   // first MLP layer in 128 x 256 tiles (MMA N = 256)
   bool tc = false, pair = false;
   CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{}, tm_h{};
   EpiParams ep{};
@@ -356,6 +358,14 @@ struct Chain {
     // One kernel for the whole chain when a row block's column slices fit one portable cluster.  The choice
     // depends on the head only, and both paths give the same bits.
     whole = allow_chain_kernel && tc && ctx->chain_mode == CSD_CHAIN_CLUSTER && use_chain_kernel(d);
+    // First MLP layer: 256-wide MMAs keep the tensor pipe busier per issued instruction (measured about 660 clk
+    // per 64-deep k-block and tile against 415 for two 128-wide tiles' worth), but halve the tile count; taken when
+    // that does not cost a wave.
+    {
+      const int row_tiles = (Rh + kTileM - 1) / kTileM, t128 = (W / kTileN) * row_tiles, t256 = (W / 256) * row_tiles;
+      const int waves128 = (t128 + ctx->num_sms - 1) / ctx->num_sms, waves256 = (t256 + ctx->num_sms - 1) / ctx->num_sms;
+      w1_wide = tc && !pair && tn == kTileN && W % 256 == 0 && waves256 * 664 < waves128 * 415;
+    }
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T, whole);
     if (rc) return rc;
@@ -450,7 +460,12 @@ struct Chain {
       if (rc) return rc;
       // v = SiLU(W1 u + b1)
       e.bias0 = hd->b1[k]; e.bias1 = nullptr; e.out_act = ws.v;
-      if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 1>(ctx, d.dtype, tn, pair, st, tm_u, tmw.W1[k], tm_u, tmw.W1[k], tm_h, W, 0, 0, W, e);
+      if (tc && w1_wide) {
+        const CUtensorMap& w1 = hd->W1_wide[k];
+        rc = d.dtype == CSD_F16 ? launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __half, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e)
+                                : launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __nv_bfloat16, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e);
+      }
+      else if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 1>(ctx, d.dtype, tn, pair, st, tm_u, tmw.W1[k], tm_u, tmw.W1[k], tm_h, W, 0, 0, W, e);
       else rc = launch_simt<EPI_SILU_ACT, 1, 128>(ctx, st, uf, W, static_cast<const float*>(hd->W1[k]), W, nullptr, 0,
                                                   nullptr, 0, W, e);
       if (rc) return rc;
@@ -762,6 +777,10 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
         if (!rc) rc = make_tmap(ctx, &tm.W2[k], d.dtype, h->W2[k], W, W, W, tn);
       }
       if (!rc) rc = make_tmap(ctx, &tm.Wfss, d.dtype, h->Wfss, 2 * W, W, W, 2 * tn);
+    }
+    if (!rc && W % 256 == 0) {
+      h->W1_wide.resize(L);
+      for (size_t k = 0; k < L && !rc; ++k) rc = make_tmap(ctx, &h->W1_wide[k], d.dtype, h->W1[k], W, W, W, 256);
     }
     if (rc) { csd_head_destroy(h); return rc; }
     std::vector<CUtensorMap> wm(4 * L + 1);

@@ -21,7 +21,7 @@ constexpr int kBlockK = 64;  // bf16 elements per TMA box row = 128 bytes = one 
 // TN/32 column chunks x 4 TMEM lane quarters; the cheap epilogues of 128-wide tiles run 16 warps
 // (one chunk per thread), everything else 8 warps (two chunks per thread, or one when TN = 64).
 template <int EPI, int TN> struct TcWarps {
-  static constexpr int kEpi = (TN == 128 && (EPI == EPI_SILU_ACT || EPI == EPI_BIAS_F32)) ? 16 : 8;
+  static constexpr int kEpi = (TN >= 128 && (EPI == EPI_SILU_ACT || EPI == EPI_BIAS_F32)) ? 16 : 8;
   static constexpr int kThreads = (kEpi + 3) * 32;
   static constexpr int kChunksPerThread = (TN / kChunk) * 4 / kEpi;
 };
@@ -34,7 +34,7 @@ template <int EPI, int MMA_N, int TN, bool PAIR> struct TcCfg {
   static constexpr bool kStageH = EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES;
   // A stage holds kKps k-blocks of 64 elements (one TMA box per operand and k-block).  The kernels whose
   // MMAs are 128 wide use two: fewer barrier round trips per byte.
-  static constexpr int kKps = (EPI == EPI_SILU_ACT || EPI == EPI_GATE_RES) ? 2 : 1;
+  static constexpr int kKps = ((EPI == EPI_SILU_ACT || EPI == EPI_GATE_RES) && MMA_N <= 128) ? 2 : 1;
   static constexpr int kABoxBytes = kTileM * kBlockK * 2;
   static constexpr int kBRows = PAIR ? MMA_N / 2 : MMA_N;    // rows of the B tile this CTA loads
   static constexpr int kBBoxBytes = kBRows * kBlockK * 2;
