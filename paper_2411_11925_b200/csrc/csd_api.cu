@@ -9,6 +9,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <type_traits>
@@ -321,6 +322,7 @@ struct Chain {
   int chains = 1;   // chains that run concurrently with this one (itself included)
   bool allow_chain_kernel = true, whole = false;   // whole: one kernel runs the whole chain
   int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
+  bool mod64 = false;     // modulate kernels in 64-wide tiles although the others use 128
   bool w1_wide = false;   // first MLP layer in 128 x 256 tiles (MMA N = 256)
   bool tc = false, pair = false;
   CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{}, tm_h{};
@@ -366,6 +368,11 @@ struct Chain {
       const int waves128 = (t128 + ctx->num_sms - 1) / ctx->num_sms, waves256 = (t256 + ctx->num_sms - 1) / ctx->num_sms;
       w1_wide = tc && !pair && tn == kTileN && W % 256 == 0 && waves256 * 664 < waves128 * 415;
     }
+    // The modulate kernels' products never wait for the preceding kernel, only their epilogues do: with 64-wide
+    // tiles the epilogue a thread runs is half as long.  Taken for a chain that has the GPU to itself and whose
+    // 64-wide tiles fit one wave (measured: draft chain of mar256 10.4 -> 9.8 ms, target chain 18.2 -> 17.7 ms;
+    // with two chains side by side the extra CTAs cost more than they save).
+    mod64 = tc && chains == 1 && tn == kTileN && !pair && 2 * (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms;
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T, whole);
     if (rc) return rc;
@@ -454,7 +461,8 @@ struct Chain {
       e.h = ws.h; e.stats = ws.stats;
       // u = LN(h)(1 + scale) + shift
       e.bias0 = hd->bsh[k]; e.bias1 = hd->bsc[k]; e.out_act = ws.u;
-      if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
+      if (tc && mod64) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wss[k], tm_s, hd->tm[0].Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
+      else if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
       else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
                                              nullptr, 0, W, e);
       if (rc) return rc;
@@ -483,7 +491,8 @@ struct Chain {
     }
     EpiParams e = ep;
     e.h = ws.h; e.stats = ws.stats; e.bias0 = hd->bfsh; e.bias1 = hd->bfsc; e.wout_t = hd->wout_t; e.epart = ws.epart;
-    if (tc) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wfss, tm_s, tmw.Wfss, tm_h, W, 0, W, W, e);
+    if (tc && mod64) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wfss, tm_s, hd->tm[0].Wfss, tm_h, W, 0, W, W, e);
+    else if (tc) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wfss, tm_s, tmw.Wfss, tm_h, W, 0, W, W, e);
     else rc = launch_simt<EPI_MODF, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
                                             0, W, e);
     if (rc) return rc;
