@@ -103,17 +103,22 @@ int csd_sync(csd_ctx *ctx);
 /* Number of kernels this context has launched so far (bookkeeping for benchmarks). */
 int64_t csd_launch_count(const csd_ctx *ctx);
 
-/* How a denoising chain (the T steps of Eq. 3 for one head) is laid out on the GPU.  Both layouts compute
- * the same arithmetic in the same order and return the same bits.
+/* How a denoising chain (the T steps of Eq. 3 for one head) is laid out on the GPU.  CSD_CHAIN_LAYERS_PLAIN and
+ * CSD_CHAIN_CLUSTER compute the same arithmetic in the same order and return the same bits.
  *   CSD_CHAIN_LAYERS  (default): one kernel per layer, chained with programmatic dependent launch; a
- *                     layer's independent part overlaps its predecessor on otherwise idle SMs.
+ *                     layer's independent part overlaps its predecessor on otherwise idle SMs.  For 16-bit
+ *                     heads on grids of one wave, blocks 2..L run as two kernels instead of three: LayerNorm
+ *                     is folded into the first layer's epilogue (algebraically the same function, rounded
+ *                     differently: results agree with the other layouts within the parity tolerance, not
+ *                     bit for bit).
+ *   CSD_CHAIN_LAYERS_PLAIN: as above without the folded blocks (three kernels per block everywhere).
  *   CSD_CHAIN_CLUSTER: one kernel per chain; a thread-block cluster of W/128 CTAs owns a block of 128 rows
  *                     for all layers and steps, the residual stream stays in shared memory.  Used for
  *                     16-bit heads with W <= 1024, other heads fall back to CSD_CHAIN_LAYERS.  Measured
  *                     slower than the default at every benchmark size (a row block is confined to W/128
  *                     SMs), kept selectable for small-batch experiments.
  * Takes effect for calls made after it returns. */
-enum { CSD_CHAIN_LAYERS = 0, CSD_CHAIN_CLUSTER = 1 };
+enum { CSD_CHAIN_LAYERS = 0, CSD_CHAIN_CLUSTER = 1, CSD_CHAIN_LAYERS_PLAIN = 2 };
 int csd_set_chain_mode(csd_ctx *ctx, int mode);
 
 /* Optional per-launch timing for benchmarks.  csd_profile(ctx, 1) synchronises, clears the records

@@ -147,9 +147,12 @@ class Context:
     def launch_count(self) -> int:
         return int(_LIB.csd_launch_count(self._h))
 
-    def set_chain_mode(self, cluster: bool):
-        """csd_set_chain_mode: False = one kernel per layer (default), True = one cluster kernel per chain."""
-        self._check(_LIB.csd_set_chain_mode(self._h, 1 if cluster else 0))
+    CHAIN_LAYERS, CHAIN_CLUSTER, CHAIN_LAYERS_PLAIN = 0, 1, 2
+
+    def set_chain_mode(self, mode: int):
+        """csd_set_chain_mode: CHAIN_LAYERS (default: one kernel per layer, folded blocks where they apply),
+        CHAIN_CLUSTER (one cluster kernel per chain) or CHAIN_LAYERS_PLAIN (three kernels per block everywhere)."""
+        self._check(_LIB.csd_set_chain_mode(self._h, int(mode)))
 
     KERNEL_CLASSES = ("cond_proj", "mlp1_silu", "adaln_modulate", "mlp2_gate_residual", "final_mod_outproj", "step", "chain")
 

@@ -17,6 +17,7 @@
 
 #include "../../include/csd.h"
 #include "chain.cuh"
+#include "fold.cuh"
 #include "gemm.cuh"
 #include "rowops.cuh"
 
@@ -37,6 +38,7 @@ struct ChainWs {
   float *cz, *te, *h, *stats, *epart, *x;
   // whole-chain kernel only
   void* s2 = nullptr; float* sched = nullptr; CUtensorMap* amaps = nullptr;
+  void* ap = nullptr;   // a' = h (1 + scale) of the folded blocks
 };
 
 struct ProfRec { cudaEvent_t a, b; int cls; double flops; };
@@ -86,7 +88,12 @@ struct csd_head {
     CUtensorMap Wz{}, Wfss{};
     std::vector<CUtensorMap> Wss, Wg, W1, W2;
   } tm[2];
-  std::vector<CUtensorMap> W1_wide;   // first MLP layer with 256-row boxes (W a multiple of 256)
+  std::vector<CUtensorMap> W1_wide;
+  // folded blocks (fold.cuh): packed [Wg_k | Wscale_{k+1}] (k < L-1) and [W1_k Wscale_k | W1_k Wshift_k] (k >= 1),
+  // 256-row boxes; c1_k = W1_k (1 + bscale_k), c2_k = W1_k bshift_k + b1_k
+  void* xblob = nullptr;
+  std::vector<CUtensorMap> Wgs, Wf;
+  std::vector<float*> c1, c2;   // first MLP layer with 256-row boxes (W a multiple of 256)
   // whole-chain kernel: device copies of the weight tensor maps (per block Wss, Wg, W1, W2; then Wfss) and of
   // the bias pointers (per block shift, scale, b1, gate, b2; then final shift, scale)
   CUtensorMap* d_wmaps = nullptr;
@@ -181,6 +188,7 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   const size_t o_st = take(Rh * (W / kStatCols) * 8);
   const size_t o_ep = take(Rh * (W / kStatCols) * kCPad * 4);   // room for 64-wide tiles
   const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
+  const size_t o_ap = take(d.dtype == CSD_F32 ? 0 : Rh * W * asz);
   size_t o_s2 = 0, o_sched = 0, o_amaps = 0;
   if (chain_kernel_extras) { o_s2 = take(Ra * W * asz); o_sched = take(static_cast<size_t>(T) * 3 * 4); o_amaps = take(4 * sizeof(CUtensorMap)); }
   if (off > ws.cap) {
@@ -200,6 +208,7 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   ws.cz = reinterpret_cast<float*>(b + o_cz); ws.te = reinterpret_cast<float*>(b + o_te);
   ws.h = reinterpret_cast<float*>(b + o_h); ws.stats = reinterpret_cast<float*>(b + o_st);
   ws.epart = reinterpret_cast<float*>(b + o_ep); ws.x = reinterpret_cast<float*>(b + o_x);
+  ws.ap = b + o_ap;
   if (chain_kernel_extras) {
     ws.s2 = b + o_s2; ws.sched = reinterpret_cast<float*>(b + o_sched); ws.amaps = reinterpret_cast<CUtensorMap*>(b + o_amaps);
   }
@@ -287,6 +296,25 @@ int check_sched(csd_ctx* ctx, const csd_schedule* s, bool full) {
   return CSD_OK;
 }
 
+// Shared-memory opt-in of the folded block kernels, once per operand type.
+bool fold_kernels_ready(const csd_head_desc& d) {
+  static int known[2] = {0, 0};
+  int& k = known[d.dtype == CSD_F16 ? 0 : 1];
+  if (k == 0) {
+    bool ok = true;
+    if (d.dtype == CSD_F16) {
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__half, 0, FOLD_W1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_W1>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__half, 0, FOLD_GATE>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_GATE>::kSmemBytes) == cudaSuccess;
+    } else {
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__nv_bfloat16, 1, FOLD_W1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_W1>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__nv_bfloat16, 1, FOLD_GATE>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_GATE>::kSmemBytes) == cudaSuccess;
+    }
+    cudaGetLastError();
+    k = ok ? 1 : -1;
+  }
+  return k == 1;
+}
+
 // The whole-chain kernel needs the row block's W/128 column slices in one cluster of at most 8 CTAs, each
 // with ~219 KB of shared memory; asked of the driver once per cluster size and operand type.
 bool use_chain_kernel(const csd_head_desc& d) {
@@ -322,6 +350,8 @@ struct Chain {
   int chains = 1;   // chains that run concurrently with this one (itself included)
   bool allow_chain_kernel = true, whole = false;   // whole: one kernel runs the whole chain
   int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
+  bool fold = false;      // blocks 1.. run as two kernels (fold.cuh) instead of three
+  CUtensorMap tm_ap{};
   bool mod64 = false;     // modulate kernels in 64-wide tiles although the others use 128
   bool w1_wide = false;   // first MLP layer in 128 x 256 tiles (MMA N = 256)
   bool tc = false, pair = false;
@@ -373,6 +403,9 @@ struct Chain {
     // 64-wide tiles fit one wave (measured: draft chain of mar256 10.4 -> 9.8 ms, target chain 18.2 -> 17.7 ms;
     // with two chains side by side the extra CTAs cost more than they save).
     mod64 = tc && chains == 1 && tn == kTileN && !pair && 2 * (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms;
+    // Folded blocks: one tile per CTA, so only while a layer's 128-wide tiles fit one wave
+    fold = tc && ctx->chain_mode == CSD_CHAIN_LAYERS && !pair && L >= 2 && !hd->Wf.empty() &&
+           (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms && fold_kernels_ready(d);
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T, whole);
     if (rc) return rc;
@@ -392,6 +425,7 @@ struct Chain {
       if ((rc = make_tmap(ctx, &tm_u, d.dtype, ws.u, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_v, d.dtype, ws.v, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap_f32(ctx, &tm_h, ws.h, Rh, W))) return rc;
+      if ((rc = make_tmap(ctx, &tm_ap, d.dtype, ws.ap, Rh, W, W, kTileM))) return rc;
     }
     // cz = z Wz^T + bz
     const csd_head::TmSet& tmw = hd->tm[(tn == 64 || pair) ? 0 : 1];   // pairs load half of each B tile per CTA
@@ -409,6 +443,39 @@ struct Chain {
     sp.eps_t = eps;
     if (whole) return launch_chain_kernel();
     return launch_step(STEP_INIT);
+  }
+
+  int launch_fold(int kind, int k) {
+    const csd_head_desc& d = hd->d;
+    ChainWs& ws = ctx->ws[slot];
+    FoldParams p{};
+    p.M = Rh; p.W = W; p.err = ctx->d_err;
+    const CUtensorMap *tp, *ta, *tw;
+    if (kind == FOLD_W1) {
+      p.c0 = hd->c1[k]; p.c1 = hd->c2[k]; p.c2 = nullptr; p.stats_in = ws.stats; p.out = ws.v;
+      tp = &hd->Wf[k]; ta = &tm_ap; tw = &hd->tm[1].W1[k];
+    } else {
+      p.c0 = hd->bg[k]; p.c1 = hd->b2[k]; p.c2 = hd->bsc[k + 1]; p.stats_out = ws.stats; p.h = ws.h; p.out = ws.ap;
+      tp = &hd->Wgs[k]; ta = &tm_v; tw = &hd->tm[1].W2[k];
+    }
+    const int tiles_n = W / kTileN, row_tiles = (Rh + kTileM - 1) / kTileM;
+    ProfScope ps(ctx, st, kind == FOLD_W1 ? 1 : 3, 2.0 * Rh * static_cast<double>(W) * W * 3.0);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(tiles_n * row_tiles); lc.blockDim = dim3(kFoldThreads); lc.stream = st;
+    lc.dynamicSmemBytes = kind == FOLD_W1 ? FoldCfg<FOLD_W1>::kSmemBytes : FoldCfg<FOLD_GATE>::kSmemBytes;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = ctx->prof_on ? 0 : 1;
+    if (d.dtype == CSD_F16) {
+      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_W1>, tm_s, *tp, *ta, *tw, tiles_n, p));
+      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_GATE>, tm_s, *tp, *ta, *tw, tiles_n, p));
+    } else {
+      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_W1>, tm_s, *tp, *ta, *tw, tiles_n, p));
+      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_GATE>, tm_s, *tp, *ta, *tw, tiles_n, p));
+    }
+    ctx->launches++;
+    return CSD_OK;
   }
 
   int launch_chain_kernel() {
@@ -459,16 +526,26 @@ struct Chain {
     for (int k = 0; k < L; ++k) {
       EpiParams e = ep;
       e.h = ws.h; e.stats = ws.stats;
+      const bool folded_in = fold && k >= 1;        // the block's input is a' = h (1 + scale): no modulate kernel
+      const bool folded_out = fold && k + 1 < L;    // the block's last kernel also forms a' of the next block
+      if (folded_in) {
+        if ((rc = launch_fold(FOLD_W1, k))) return rc;
+        if (folded_out) rc = launch_fold(FOLD_GATE, k);
+        if (rc) return rc;
+        if (folded_out) continue;
+      }
       // u = LN(h)(1 + scale) + shift
       e.bias0 = hd->bsh[k]; e.bias1 = hd->bsc[k]; e.out_act = ws.u;
-      if (tc && mod64) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wss[k], tm_s, hd->tm[0].Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
+      if (folded_in) rc = CSD_OK;
+      else if (tc && mod64) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wss[k], tm_s, hd->tm[0].Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
       else if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
       else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
                                              nullptr, 0, W, e);
       if (rc) return rc;
       // v = SiLU(W1 u + b1)
       e.bias0 = hd->b1[k]; e.bias1 = nullptr; e.out_act = ws.v;
-      if (tc && w1_wide) {
+      if (folded_in) rc = CSD_OK;
+      else if (tc && w1_wide) {
         const CUtensorMap& w1 = hd->W1_wide[k];
         rc = d.dtype == CSD_F16 ? launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __half, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e)
                                 : launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __nv_bfloat16, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e);
@@ -480,7 +557,8 @@ struct Chain {
       // h += gate * (W2 v + b2).  On the tensor-core path the gate product s Wg^T comes first: it does
       // not depend on the preceding kernel (which writes v) and overlaps with it.
       e.bias0 = hd->b2[k]; e.bias1 = hd->bg[k]; e.out_act = nullptr;
-      if (tc) {
+      if (folded_out) rc = launch_fold(FOLD_GATE, k);
+      else if (tc) {
         EpiParams g = e;
         g.bias0 = hd->bg[k]; g.bias1 = hd->b2[k];
         rc = launch_tc<EPI_GATE_RES, 2, 1>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wg[k], tm_v, tmw.W2[k], tm_h, W, W, W, W, g);
@@ -649,7 +727,7 @@ int csd_sync(csd_ctx* c) {
 
 int csd_set_chain_mode(csd_ctx* c, int mode) {
   if (!c) return CSD_ERR_INVALID_ARG;
-  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_CLUSTER) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
+  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_CLUSTER && mode != CSD_CHAIN_LAYERS_PLAIN) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
   c->chain_mode = mode;
   return CSD_OK;
 }
@@ -763,12 +841,31 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
     f_b1[k] = put(w->b1 + k * W, W); f_b2[k] = put(w->b2 + k * W, W);
   }
   const size_t f_bfsh = put(w->bfada, W), f_bfsc = put(w->bfada + W, W);
+  // folded blocks: c1_k = W1_k (1 + bscale_k), c2_k = W1_k bshift_k + b1_k  (double accumulation, rounded once)
+  const bool folded = d.dtype != CSD_F32 && L >= 2;
+  std::vector<size_t> f_c1(L, 0), f_c2(L, 0);
+  if (folded) {
+    std::vector<float> v1(W), v2(W);
+    for (size_t k = 1; k < L; ++k) {
+      const float* W1k = w->W1 + k * W * W;
+      const float* bsh = w->bada + k * 3 * W;
+      const float* bsc = bsh + W;
+      for (size_t n = 0; n < W; ++n) {
+        double a1 = 0.0, a2 = 0.0;
+        for (size_t j = 0; j < W; ++j) { a1 += static_cast<double>(W1k[n * W + j]) * (1.0 + bsc[j]); a2 += static_cast<double>(W1k[n * W + j]) * bsh[j]; }
+        v1[n] = static_cast<float>(a1); v2[n] = static_cast<float>(a2 + w->b1[k * W + n]);
+      }
+      f_c1[k] = put(v1.data(), W); f_c2[k] = put(v2.data(), W);
+    }
+  }
   if (cudaMalloc(&h->fblob, fs.size() * 4) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the parameters"); }
   if (cudaMemcpy(h->fblob, fs.data(), fs.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "parameter upload failed");
   float* fb = h->fblob;
   h->bz = fb + f_bz; h->Wt1 = fb + f_wt1; h->bt1 = fb + f_bt1; h->Wt2 = fb + f_wt2; h->bt2 = fb + f_bt2;
   h->win = fb + f_win; h->bin = fb + f_bin; h->wout_t = fb + f_wout; h->bout = fb + f_bout;
   h->bfsh = fb + f_bfsh; h->bfsc = fb + f_bfsc;
+  h->c1.assign(L, nullptr); h->c2.assign(L, nullptr);
+  if (folded) for (size_t k = 1; k < L; ++k) { h->c1[k] = fb + f_c1[k]; h->c2[k] = fb + f_c2[k]; }
   h->bsh.resize(L); h->bsc.resize(L); h->bg.resize(L); h->b1.resize(L); h->b2.resize(L);
   for (size_t k = 0; k < L; ++k) { h->bsh[k] = fb + f_bsh[k]; h->bsc[k] = fb + f_bsc[k]; h->bg[k] = fb + f_bg[k]; h->b1[k] = fb + f_b1[k]; h->b2[k] = fb + f_b2[k]; }
 
@@ -786,6 +883,43 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
         if (!rc) rc = make_tmap(ctx, &tm.W2[k], d.dtype, h->W2[k], W, W, W, tn);
       }
       if (!rc) rc = make_tmap(ctx, &tm.Wfss, d.dtype, h->Wfss, 2 * W, W, W, 2 * tn);
+    }
+    if (!rc && folded) {
+      // xblob: Wgs_0 .. Wgs_{L-2} | Wf_1 .. Wf_{L-1}, each [2 W, W] in operand format
+      const size_t per = 2 * W * W, nx = 2 * (L - 1) * per;
+      std::vector<float> xs;
+      try { xs.resize(nx); } catch (...) { return bail(CSD_ERR_WORKSPACE, "out of host memory"); }
+      float *dA = nullptr, *dB = nullptr, *dC = nullptr;
+      std::vector<float> f1(W * W), f2(W * W);
+      bool okx = cudaMalloc(&dA, W * W * 4) == cudaSuccess && cudaMalloc(&dB, W * W * 4) == cudaSuccess && cudaMalloc(&dC, W * W * 4) == cudaSuccess;
+      for (size_t k = 0; k + 1 < L && okx; ++k)     // gate of block k | scale of block k + 1
+        interleave(w->Wada + k * 3 * W * W + 2 * W * W, w->Wada + (k + 1) * 3 * W * W + W * W, &xs[k * per]);
+      for (size_t k = 1; k < L && okx; ++k) {       // W1_k Wscale_k | W1_k Wshift_k
+        const float* ada = w->Wada + k * 3 * W * W;
+        const dim3 grid(static_cast<unsigned>(W / 32), static_cast<unsigned>(W / 32));
+        okx = okx && cudaMemcpy(dA, w->W1 + k * W * W, W * W * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+        okx = okx && cudaMemcpy(dB, ada + W * W, W * W * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+        if (okx) square_matmul_kernel<<<grid, 256>>>(dA, dB, dC, static_cast<int>(W));
+        okx = okx && cudaMemcpy(f1.data(), dC, W * W * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+        okx = okx && cudaMemcpy(dB, ada, W * W * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+        if (okx) square_matmul_kernel<<<grid, 256>>>(dA, dB, dC, static_cast<int>(W));
+        okx = okx && cudaMemcpy(f2.data(), dC, W * W * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+        if (okx) interleave(f1.data(), f2.data(), &xs[(L - 1 + k - 1) * per]);
+      }
+      if (dA) cudaFree(dA);
+      if (dB) cudaFree(dB);
+      if (dC) cudaFree(dC);
+      if (!okx) { cudaGetLastError(); return bail(CSD_ERR_CUDA, "fused weight products failed"); }
+      std::vector<uint16_t> xb;
+      try { xb.resize(nx); } catch (...) { return bail(CSD_ERR_WORKSPACE, "out of host memory"); }
+      if (d.dtype == CSD_BF16) { for (size_t i = 0; i < nx; ++i) xb[i] = f32_to_bf16_bits(xs[i]); }
+      else { for (size_t i = 0; i < nx; ++i) { const __half hv = __float2half_rn(xs[i]); memcpy(&xb[i], &hv, 2); } }
+      if (cudaMalloc(&h->xblob, nx * 2) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the fused weights"); }
+      if (cudaMemcpy(h->xblob, xb.data(), nx * 2, cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "fused weight upload failed");
+      h->Wgs.resize(L); h->Wf.resize(L);
+      char* xbase = static_cast<char*>(h->xblob);
+      for (size_t k = 0; k + 1 < L && !rc; ++k) rc = make_tmap(ctx, &h->Wgs[k], d.dtype, xbase + k * per * 2, 2 * W, W, W, 256);
+      for (size_t k = 1; k < L && !rc; ++k) rc = make_tmap(ctx, &h->Wf[k], d.dtype, xbase + (L - 1 + k - 1) * per * 2, 2 * W, W, W, 256);
     }
     if (!rc && W % 256 == 0) {
       h->W1_wide.resize(L);
@@ -819,6 +953,7 @@ int csd_head_destroy(csd_head* h) {
   if (h->fblob) cudaFree(h->fblob);
   if (h->d_wmaps) cudaFree(h->d_wmaps);
   if (h->d_bias) cudaFree(h->d_bias);
+  if (h->xblob) cudaFree(h->xblob);
   cudaGetLastError();
   delete h;
   return CSD_OK;
@@ -860,6 +995,7 @@ int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_sched
   take(Rh * d.Dz * asz); take(Rh * W * asz); take(Rh * W * asz); take(Rh * W * asz);
   take(Rh * W * 4); take(static_cast<size_t>(sched->T) * W * 4); take(Rh * W * 4);
   take(Rh * (W / kStatCols) * 8); take(Rh * (W / kStatCols) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
+  take(d.dtype == CSD_F32 ? 0 : Rh * W * asz);
   if (need > kStaticScratchBytes)
     return fail(ctx, CSD_ERR_WORKSPACE,
                 "csd_draft_denoise_static: this call needs %zu bytes of scratch but the built-in array holds %zu "
