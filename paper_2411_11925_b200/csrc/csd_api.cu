@@ -403,9 +403,15 @@ struct Chain {
     // 64-wide tiles fit one wave (measured: draft chain of mar256 10.4 -> 9.8 ms, target chain 18.2 -> 17.7 ms;
     // with two chains side by side the extra CTAs cost more than they save).
     mod64 = tc && chains == 1 && tn == kTileN && !pair && 2 * (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms;
-    // Folded blocks: one tile per CTA, so only while a layer's 128-wide tiles fit one wave
-    fold = tc && ctx->chain_mode == CSD_CHAIN_LAYERS && !pair && L >= 2 && !hd->Wf.empty() &&
-           (W / kTileN) * ((Rh + kTileM - 1) / kTileM) <= ctx->num_sms && fold_kernels_ready(d);
+    // Folded blocks: one 128-wide tile per CTA, and their early products want idle SMs to overlap the preceding
+    // kernel: taken when the layer's tiles fill between an eighth and half of the SMs (measured slower on tiny grids,
+    // which run 64-wide tiles, and on a full wave)
+    // (the rule looks at this chain alone, so that csd_round and the three separate calls take the same path).
+    {
+      const int t128 = (W / kTileN) * ((Rh + kTileM - 1) / kTileM);
+      fold = tc && ctx->chain_mode == CSD_CHAIN_LAYERS && !pair && L >= 2 && !hd->Wf.empty() &&
+             8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && fold_kernels_ready(d);
+    }
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T, whole);
     if (rc) return rc;
