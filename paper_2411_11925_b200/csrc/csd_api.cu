@@ -39,6 +39,7 @@ struct ChainWs {
   // whole-chain kernel only
   void* s2 = nullptr; float* sched = nullptr; CUtensorMap* amaps = nullptr;
   void* ap = nullptr;   // a' = h (1 + scale) of the folded blocks
+  float* hid = nullptr; // hidden layer of the timestep embedding [T, W]
 };
 
 struct ProfRec { cudaEvent_t a, b; int cls; double flops; };
@@ -189,6 +190,7 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   const size_t o_ep = take(Rh * (W / kStatCols) * kCPad * 4);   // room for 64-wide tiles
   const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
   const size_t o_ap = take(d.dtype == CSD_F32 ? 0 : Rh * W * asz);
+  const size_t o_hid = take(static_cast<size_t>(T) * W * 4);
   size_t o_s2 = 0, o_sched = 0, o_amaps = 0;
   if (chain_kernel_extras) { o_s2 = take(Ra * W * asz); o_sched = take(static_cast<size_t>(T) * 3 * 4); o_amaps = take(4 * sizeof(CUtensorMap)); }
   if (off > ws.cap) {
@@ -208,7 +210,7 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   ws.cz = reinterpret_cast<float*>(b + o_cz); ws.te = reinterpret_cast<float*>(b + o_te);
   ws.h = reinterpret_cast<float*>(b + o_h); ws.stats = reinterpret_cast<float*>(b + o_st);
   ws.epart = reinterpret_cast<float*>(b + o_ep); ws.x = reinterpret_cast<float*>(b + o_x);
-  ws.ap = b + o_ap;
+  ws.ap = b + o_ap; ws.hid = reinterpret_cast<float*>(b + o_hid);
   if (chain_kernel_extras) {
     ws.s2 = b + o_s2; ws.sched = reinterpret_cast<float*>(b + o_sched); ws.amaps = reinterpret_cast<CUtensorMap*>(b + o_amaps);
   }
@@ -415,8 +417,12 @@ struct Chain {
     ChainWs& ws = ctx->ws[slot];
     int rc = ensure_ws(ctx, ws, d, Rh, R, T, whole);
     if (rc) return rc;
-    timestep_embed_kernel<<<T, 256, (d.F + W) * sizeof(float), st>>>(sc->tfeat, hd->Wt1, hd->bt1, hd->Wt2, hd->bt2, W,
-                                                                    d.F, ws.te);
+    {
+      const dim3 grid((W + 31) / 32, (T + 31) / 32);
+      small_gemm_nt_kernel<true><<<grid, 256, 0, st>>>(sc->tfeat, hd->Wt1, hd->bt1, ws.hid, T, W, d.F);
+      small_gemm_nt_kernel<false><<<grid, 256, 0, st>>>(ws.hid, hd->Wt2, hd->bt2, ws.te, T, W, W);
+      ctx->launches++;
+    }
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
     ep.M = Rh; ep.ldo = W;
@@ -775,8 +781,6 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
   if (d.W % kTileN != 0) return fail(ctx, CSD_ERR_UNSUPPORTED, "width W = %d must be a multiple of 128", d.W);
   const int kmul = d.dtype != CSD_F32 ? kBlockK : kSimtBK;
   if (d.Dz % kmul != 0) return fail(ctx, CSD_ERR_UNSUPPORTED, "Dz = %d must be a multiple of %d", d.Dz, kmul);
-  if (static_cast<size_t>(d.F + d.W) * 4 > 40 * 1024)
-    return fail(ctx, CSD_ERR_UNSUPPORTED, "F + W = %d too large for the timestep-embedding kernel", d.F + d.W);
   const float* const* ptrs = reinterpret_cast<const float* const*>(w);
   for (size_t i = 0; i < sizeof(csd_head_weights) / sizeof(float*); ++i)
     if (!ptrs[i]) return fail(ctx, CSD_ERR_INVALID_ARG, "weight pointer #%zu is null", i);
@@ -1002,6 +1006,7 @@ int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_sched
   take(Rh * W * 4); take(static_cast<size_t>(sched->T) * W * 4); take(Rh * W * 4);
   take(Rh * (W / kStatCols) * 8); take(Rh * (W / kStatCols) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
   take(d.dtype == CSD_F32 ? 0 : Rh * W * asz);
+  take(static_cast<size_t>(sched->T) * W * 4);
   if (need > kStaticScratchBytes)
     return fail(ctx, CSD_ERR_WORKSPACE,
                 "csd_draft_denoise_static: this call needs %zu bytes of scratch but the built-in array holds %zu "

@@ -7,31 +7,40 @@
 
 namespace csd {
 
-// te[t, n] = Wt2[n, :] . SiLU(Wt1 tfeat_t + bt1) + bt2[n]   (one block per timestep)
+// Timestep embedding te[t, :] = Wt2 SiLU(Wt1 tfeat_t + bt1) + bt2 for all T steps: two small fp32 products
+// C[m, n] = act(sum_k A[m, k] B[n, k] + bias[n]) in 32 x 32 tiles (each weight row is read once per 32 steps,
+// not once per step).
+template <bool SILU>
 __global__ void __launch_bounds__(256)
-timestep_embed_kernel(const float* __restrict__ tfeat, const float* __restrict__ Wt1,
-                      const float* __restrict__ bt1, const float* __restrict__ Wt2,
-                      const float* __restrict__ bt2, int W, int F, float* __restrict__ te) {
-  extern __shared__ float sm[];  // tf[F] | hid[W]
-  float* tf = sm;
-  float* hid = sm + F;
-  const int t = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  for (int i = threadIdx.x; i < F; i += blockDim.x) tf[i] = tfeat[static_cast<size_t>(t) * F + i];
-  __syncthreads();
-  for (int n = warp; n < W; n += nwarp) {
-    float acc = 0.0f;
-    for (int k = lane; k < F; k += 32) acc = fmaf(Wt1[static_cast<size_t>(n) * F + k], tf[k], acc);
+small_gemm_nt_kernel(const float* __restrict__ A, const float* __restrict__ B, const float* __restrict__ bias,
+                     float* __restrict__ C, int M, int N, int K) {
+  __shared__ float As[32][33], Bs[32][33];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;      // 32 x 8 threads, 4 rows of the tile each
+  const int m0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+  for (int k0 = 0; k0 < K; k0 += 32) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) hid[n] = silu_f(acc + bt1[n]);
+    for (int r = 0; r < 4; ++r) {
+      const int row = ty * 4 + r, k = k0 + tx;
+      As[row][tx] = (m0 + row < M && k < K) ? A[static_cast<size_t>(m0 + row) * K + k] : 0.0f;
+      Bs[row][tx] = (n0 + row < N && k < K) ? B[static_cast<size_t>(n0 + row) * K + k] : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+      const float b = Bs[tx][k];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) acc[r] = fmaf(As[ty * 4 + r][k], b, acc[r]);
+    }
+    __syncthreads();
   }
-  __syncthreads();
-  for (int n = warp; n < W; n += nwarp) {
-    float acc = 0.0f;
-    for (int k = lane; k < W; k += 32) acc = fmaf(Wt2[static_cast<size_t>(n) * W + k], hid[k], acc);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) te[static_cast<size_t>(t) * W + n] = acc + bt2[n];
+  for (int r = 0; r < 4; ++r) {
+    const int m = m0 + ty * 4 + r, n = n0 + tx;
+    if (m < M && n < N) {
+      const float v = acc[r] + bias[n];
+      C[static_cast<size_t>(m) * N + n] = SILU ? silu_f(v) : v;
+    }
   }
 }
 
