@@ -462,13 +462,13 @@ struct Chain {
     ChainWs& ws = ctx->ws[slot];
     FoldParams p{};
     p.M = Rh; p.W = W; p.err = ctx->d_err;
-    const CUtensorMap *tp, *ta, *tw;
+    const CUtensorMap *tp, *ta, *tw, *tout;
     if (kind == FOLD_W1) {
       p.c0 = hd->c1[k]; p.c1 = hd->c2[k]; p.c2 = nullptr; p.stats_in = ws.stats; p.out = ws.v;
-      tp = &hd->Wf[k]; ta = &tm_ap; tw = &hd->tm[1].W1[k];
+      tp = &hd->Wf[k]; ta = &tm_ap; tw = &hd->tm[1].W1[k]; tout = &tm_v;
     } else {
       p.c0 = hd->bg[k]; p.c1 = hd->b2[k]; p.c2 = hd->bsc[k + 1]; p.stats_out = ws.stats; p.h = ws.h; p.out = ws.ap;
-      tp = &hd->Wgs[k]; ta = &tm_v; tw = &hd->tm[1].W2[k];
+      tp = &hd->Wgs[k]; ta = &tm_v; tw = &hd->tm[1].W2[k]; tout = &tm_ap;
     }
     const int tiles_n = W / kTileN, row_tiles = (Rh + kTileM - 1) / kTileM;
     ProfScope ps(ctx, st, kind == FOLD_W1 ? 1 : 3, 2.0 * Rh * static_cast<double>(W) * W * 3.0);
@@ -480,11 +480,11 @@ struct Chain {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = at; lc.numAttrs = ctx->prof_on ? 0 : 1;
     if (d.dtype == CSD_F16) {
-      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_W1>, tm_s, *tp, *ta, *tw, tiles_n, p));
-      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_GATE>, tm_s, *tp, *ta, *tw, tiles_n, p));
+      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_W1>, tm_s, *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
+      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_GATE>, tm_s, *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
     } else {
-      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_W1>, tm_s, *tp, *ta, *tw, tiles_n, p));
-      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_GATE>, tm_s, *tp, *ta, *tw, tiles_n, p));
+      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_W1>, tm_s, *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
+      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_GATE>, tm_s, *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
     }
     ctx->launches++;
     return CSD_OK;

@@ -48,7 +48,8 @@ template <typename ACT, int AB_FMT, int KIND>
 __global__ void __launch_bounds__(kFoldThreads, 1)
 fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmWp,
             const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
-            int tiles_n, const FoldParams p) {
+            const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmHst, int tiles_n,
+            const FoldParams p) {
   using Cfg = FoldCfg<KIND>;
   constexpr int S = Cfg::kSlots, SP = S / 2, kPairBytes = 2 * kChSlotBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -68,6 +69,8 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
   const bool run = *reinterpret_cast<const volatile int*>(p.err) == 0;
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmS); tma_prefetch_desc(&tmWp); tma_prefetch_desc(&tmA); tma_prefetch_desc(&tmW);
+    tma_prefetch_desc(&tmOut);
+    if (KIND == FOLD_GATE) tma_prefetch_desc(&tmHst);
     for (int s = 0; s < SP; ++s) { mbar_init(&full_bar[s], 3); mbar_init(&empty_bar[s], 1); }
     mbar_init(&acc_full[0], 1); mbar_init(&acc_full[1], 1);
     fence_mbar_init();
@@ -203,6 +206,18 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
         }
       }
     }
+    // The outputs leave through shared memory and TMA stores: a thread owns a row, so direct stores would touch 32
+    // rows per instruction, 16 bytes each (measured: they, not the arithmetic, set the epilogue's length).  The ring
+    // is free once the last MMA has completed: 16-bit tile in two boxes of 64 columns at its start, fp32 h behind.
+    auto stage_act = [&](int c, const float* v) {
+      uint8_t* row = ring + (c >> 1) * (kTileM * 128) + rloc * 128;
+      ACT o[kChunk];
+#pragma unroll
+      for (int j = 0; j < kChunk; ++j) o[j] = to_act<ACT>(v[j]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<uint4*>(row + ((((c & 1) * 4 + i) ^ (rloc & 7)) << 4)) = reinterpret_cast<const uint4*>(o)[i];
+    };
     RowState rs;
     rs.mean = 0.0f; rs.rstd = 0.0f; rs.pm = 0.0f; rs.pm2 = 0.0f; rs.pn = 0.0f;
     if (KIND == FOLD_W1 && valid) row_stats<true>(p.stats_in, m, W, rs.mean, rs.rstd);
@@ -229,19 +244,31 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
             const float t1 = __fsub_rn(am[j], __fmul_rn(rs.mean, __fadd_rn(a0[j], k1[j])));
             am[j] = silu_t<true>(fmaf(rs.rstd, t1, __fadd_rn(a1[j], k2[j])));
           }
-          if (valid) store_chunk<ACT>(reinterpret_cast<ACT*>(p.out) + static_cast<size_t>(m) * W + n0, am);
+          stage_act(c, am);
         } else {
           float* hv = hv2[ci];
           gate_res_chunk(a0, am, bias_s + c * kChunk, bias_s + 128 + c * kChunk, hv, rs);
-          if (valid) store_chunk<float>(p.h + static_cast<size_t>(m) * W + n0, hv);
+          store_swizzled_row32(ring + 32768 + c * (kTileM * 128), rloc, hv);   // new h, one fp32 box per chunk
           const float* ks = bias_s + 256 + c * kChunk;
 #pragma unroll
           for (int j = 0; j < kChunk; ++j) hv[j] = __fmul_rn(hv[j], __fadd_rn(1.0f, __fadd_rn(a1[j], ks[j])));
-          if (valid) store_chunk<ACT>(reinterpret_cast<ACT*>(p.out) + static_cast<size_t>(m) * W + n0, hv);
+          stage_act(c, hv);
         }
       }
       if (KIND == FOLD_GATE && valid)
         reinterpret_cast<float2*>(p.stats_out)[static_cast<size_t>(m) * (W / kStatCols) + tile_n * 2 + half] = make_float2(rs.pm, rs.pm2);
+    }
+    fence_proxy_async_smem();
+    asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+    if (et == 0 && ok) {
+      tma_store_2d(&tmOut, ring, n_base, row0);
+      tma_store_2d(&tmOut, ring + kTileM * 128, n_base + 64, row0);
+      if (KIND == FOLD_GATE) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tma_store_2d(&tmHst, ring + 32768 + c * (kTileM * 128), n_base + c * kChunk, row0);
+      }
+      tma_store_commit();
+      tma_store_wait_all();
     }
   }
   tc_fence_before_sync();
