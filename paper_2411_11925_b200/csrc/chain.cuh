@@ -60,13 +60,6 @@ struct ChainParams {
   int* err;
 };
 
-__device__ __forceinline__ void store_swizzled_row32(uint8_t* tile, int r, const float* v) {
-  uint8_t* row = tile + r * 128;
-#pragma unroll
-  for (int j = 0; j < 8; ++j)
-    *reinterpret_cast<float4*>(row + ((j ^ (r & 7)) << 4)) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-}
-
 // Bounded wait that also gives up once any kernel of the context has raised the error flag.
 template <bool CLUSTER>
 __device__ __forceinline__ bool ch_wait(uint64_t* bar, uint32_t parity, const int* err) {

@@ -62,6 +62,14 @@ __device__ __forceinline__ void load_swizzled_row32(const uint8_t* tile, int r, 
   }
 }
 
+// The inverse: writes 32 floats of row r in the layout a TMA store with the 128-byte swizzle expects.
+__device__ __forceinline__ void store_swizzled_row32(uint8_t* tile, int r, const float* v) {
+  uint8_t* row = tile + r * 128;
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    *reinterpret_cast<float4*>(row + ((j ^ (r & 7)) << 4)) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+}
+
 // Persistent over tiles: CTA b handles output tiles b, b + gridDim.x, ... (column tile fastest).  The
 // shared-memory ring runs on across tiles; the accumulators are double-buffered in TMEM, so the
 // epilogue of one tile overlaps the MMAs of the next.
@@ -269,6 +277,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           if (PAIR) mbar_arrive_cluster(mapa_shared(smem_u32(&tmem_empty_bar[ab ^ 1]), 0));
           else mbar_arrive(&tmem_empty_bar[ab ^ 1]);
         }
+        if (EPI == EPI_GATE_RES && i >= 1) {
+          // the previous tile's new h sits in the h tile (the threads that own its rows wrote it in place): TMA
+          // stores instead of row-per-thread stores, which touch 32 rows per instruction
+          const int tp = unit + (i - 1) * nunits;
+          const int pn = tp % tiles_n, pm = PAIR ? 2 * (tp / tiles_n) + rank : tp / tiles_n;
+#pragma unroll
+          for (int c = 0; c < NC; ++c) tma_store_2d(&tmH, h_s + c * (kTileM * 128), pn * TN + c * kChunk, pm * kTileM);
+          tma_store_commit();
+          tma_store_wait_read();   // before the next h tile lands on it
+        }
         if (Cfg::kStageH) {
           // requested before this thread block's further pipeline traffic queues up behind it: ordinary
           // loads issued while the pipeline saturates the SM's shared-memory port take thousands of cycles
@@ -303,7 +321,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
             for (int e = 0; e < kCPad; ++e) { efirst[e] = rs.eacc[e]; rs.eacc[e] = 0.0f; }
           }
-          if (valid)
+          if (EPI == EPI_GATE_RES) {
+            gate_res_chunk(a0, a1, bias_s + c * kChunk, bias_s + TN + c * kChunk, hv, rs);
+            store_swizzled_row32(h_s + c * (kTileM * 128), rloc, hv);   // in place; leaves by TMA store
+          } else if (valid)
             epi_chunk<EPI, ACT, true>(ep, m, tile_n * TN + c * kChunk, a0, a1, bias_s + c * kChunk,
                                       bias_s + TN + c * kChunk, hv, rs, wout_s + c * kChunk * kCPad);
           if (EPI == EPI_MODF && ci == 1) {
@@ -311,6 +332,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             for (int e = 0; e < kCPad; ++e) rs.eacc[e] = efirst[e] + rs.eacc[e];
           }
         }
+        if (EPI == EPI_GATE_RES) fence_proxy_async_smem();
         tc_fence_before_sync();   // orders the TMEM reads before the barrier that releases the buffer
       }
       if (EPI == EPI_GATE_RES) {
@@ -346,6 +368,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           }
         }
       }
+    }
+    if (EPI == EPI_GATE_RES) {
+      // the last tile's new h
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+      if (et == 0 && ok) {
+        const int tp = unit + (my_tiles - 1) * nunits;
+        const int pn = tp % tiles_n, pm = PAIR ? 2 * (tp / tiles_n) + rank : tp / tiles_n;
+#pragma unroll
+        for (int c = 0; c < NC; ++c) tma_store_2d(&tmH, h_s + c * (kTileM * 128), pn * TN + c * kChunk, pm * kTileM);
+        tma_store_commit();
+      }
+      if (et == 0) tma_store_wait_all();
     }
   }
   tc_fence_before_sync();
