@@ -191,8 +191,9 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
   const size_t o_ap = take(d.dtype == CSD_F32 ? 0 : Rh * W * asz);
   const size_t o_hid = take(static_cast<size_t>(T) * W * 4);
-  size_t o_s2 = 0, o_sched = 0, o_amaps = 0;
-  if (chain_kernel_extras) { o_s2 = take(Ra * W * asz); o_sched = take(static_cast<size_t>(T) * 3 * 4); o_amaps = take(4 * sizeof(CUtensorMap)); }
+  const size_t o_s2 = take(Ra * W * asz);   // s of even steps (s of odd steps: o_s)
+  size_t o_sched = 0, o_amaps = 0;
+  if (chain_kernel_extras) { o_sched = take(static_cast<size_t>(T) * 3 * 4); o_amaps = take(4 * sizeof(CUtensorMap)); }
   if (off > ws.cap) {
     CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamSynchronize(ctx->side[i]));
@@ -211,8 +212,9 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
   ws.h = reinterpret_cast<float*>(b + o_h); ws.stats = reinterpret_cast<float*>(b + o_st);
   ws.epart = reinterpret_cast<float*>(b + o_ep); ws.x = reinterpret_cast<float*>(b + o_x);
   ws.ap = b + o_ap; ws.hid = reinterpret_cast<float*>(b + o_hid);
+  ws.s2 = b + o_s2;
   if (chain_kernel_extras) {
-    ws.s2 = b + o_s2; ws.sched = reinterpret_cast<float*>(b + o_sched); ws.amaps = reinterpret_cast<CUtensorMap*>(b + o_amaps);
+    ws.sched = reinterpret_cast<float*>(b + o_sched); ws.amaps = reinterpret_cast<CUtensorMap*>(b + o_amaps);
   }
   return CSD_OK;
 }
@@ -357,7 +359,11 @@ struct Chain {
   bool mod64 = false;     // modulate kernels in 64-wide tiles although the others use 128
   bool w1_wide = false;   // first MLP layer in 128 x 256 tiles (MMA N = 256)
   bool tc = false, pair = false;
-  CUtensorMap tm_z{}, tm_s{}, tm_u{}, tm_v{}, tm_h{};
+  // s is double-buffered by step parity (index t & 1): the boundary kernel that ends step t writes s of step t - 2,
+  // so no product of s ever waits for the kernel right before it
+  CUtensorMap tm_z{}, tm_sb[2]{}, tm_u{}, tm_v{}, tm_h{};
+  void* sbuf[2] = {nullptr, nullptr};
+  int cur_t = 0;
   EpiParams ep{};
   StepParams sp{};
 
@@ -433,7 +439,8 @@ struct Chain {
       else convert_act_kernel<__nv_bfloat16><<<nblk, 256, 0, st>>>(z, static_cast<__nv_bfloat16*>(ws.zc), nz);
       ctx->launches++;
       if ((rc = make_tmap(ctx, &tm_z, d.dtype, ws.zc, Rh, d.Dz, d.Dz, kTileM))) return rc;
-      if ((rc = make_tmap(ctx, &tm_s, d.dtype, ws.s, Rh, W, W, kTileM))) return rc;
+      if ((rc = make_tmap(ctx, &tm_sb[1], d.dtype, ws.s, Rh, W, W, kTileM))) return rc;
+      if ((rc = make_tmap(ctx, &tm_sb[0], d.dtype, ws.s2, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_u, d.dtype, ws.u, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_v, d.dtype, ws.v, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap_f32(ctx, &tm_h, ws.h, Rh, W))) return rc;
@@ -450,8 +457,11 @@ struct Chain {
     sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = tc ? W / kStatCols : W / kTileN; sp.cfg_scale = cfg_scale;
     sp.sample_last = sample_last; sp.epart = ws.epart; sp.bout = hd->bout; sp.x_src = x_T; sp.x = ws.x;
     sp.x0 = x0; sp.mu1 = mu1; sp.x1 = x1; sp.win = hd->win; sp.bin = hd->bin; sp.cz = ws.cz; sp.h = ws.h;
-    sp.stats = ws.stats; sp.s = ws.s;
+    sbuf[0] = ws.s2; sbuf[1] = ws.s;
+    sp.stats = ws.stats; sp.s = sbuf[T & 1];
     sp.te_next = ws.te + static_cast<size_t>(T - 1) * W;
+    sp.s_b = T >= 2 ? sbuf[(T - 1) & 1] : nullptr;   // the first boundary also prepares s of step T - 1
+    sp.te_b = T >= 2 ? ws.te + static_cast<size_t>(T - 2) * W : nullptr;
     sp.eps_t = eps;
     if (whole) return launch_chain_kernel();
     return launch_step(STEP_INIT);
@@ -480,11 +490,11 @@ struct Chain {
     at[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = at; lc.numAttrs = ctx->prof_on ? 0 : 1;
     if (d.dtype == CSD_F16) {
-      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_W1>, tm_s, *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
-      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_GATE>, tm_s, *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
+      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_W1>, tm_sb[cur_t & 1], *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
+      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_GATE>, tm_sb[cur_t & 1], *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
     } else {
-      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_W1>, tm_s, *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
-      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_GATE>, tm_s, *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
+      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_W1>, tm_sb[cur_t & 1], *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
+      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_GATE>, tm_sb[cur_t & 1], *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
     }
     ctx->launches++;
     return CSD_OK;
@@ -530,7 +540,9 @@ struct Chain {
     if (whole) return CSD_OK;   // already enqueued by begin()
     const csd_head_desc& d = hd->d;
     ChainWs& ws = ctx->ws[slot];
-    const float* sf = static_cast<const float*>(ws.s);
+    cur_t = t;
+    const CUtensorMap& tm_s = tm_sb[t & 1];
+    const float* sf = static_cast<const float*>(sbuf[t & 1]);
     const float* uf = static_cast<const float*>(ws.u);
     const float* vf = static_cast<const float*>(ws.v);
     const csd_head::TmSet& tmw = hd->tm[(tn == 64 || pair) ? 0 : 1];   // pairs load half of each B tile per CTA
@@ -548,9 +560,11 @@ struct Chain {
       }
       // u = LN(h)(1 + scale) + shift
       e.bias0 = hd->bsh[k]; e.bias1 = hd->bsc[k]; e.out_act = ws.u;
+      // s of the first step is written by the kernel right before the first modulate kernel; every later s is older
+      const int dep_mod = (k == 0 && t == T) ? 0 : W;
       if (folded_in) rc = CSD_OK;
-      else if (tc && mod64) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wss[k], tm_s, hd->tm[0].Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
-      else if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, k == 0 ? 0 : W, W, e);
+      else if (tc && mod64) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wss[k], tm_s, hd->tm[0].Wss[k], tm_h, W, 0, dep_mod, W, e);
+      else if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, dep_mod, W, e);
       else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
                                              nullptr, 0, W, e);
       if (rc) return rc;
@@ -588,7 +602,10 @@ struct Chain {
     if (rc) return rc;
     sp.a = sc->a[t - 1]; sp.b = sc->b[t - 1]; sp.sigma = sc->sigma[t - 1];
     sp.eps_t = eps + static_cast<size_t>(t - 1) * R * d.C;
-    if (t > 1) sp.te_next = ws.te + static_cast<size_t>(t - 2) * W;
+    // this boundary prepares h of step t - 1 and s of step t - 2
+    sp.s = t >= 3 ? sbuf[(t - 2) & 1] : nullptr;
+    if (t >= 3) sp.te_next = ws.te + static_cast<size_t>(t - 3) * W;
+    sp.s_b = nullptr; sp.te_b = nullptr;
     return launch_step(t > 1 ? STEP_MID : STEP_LAST);
   }
 };
@@ -1007,6 +1024,7 @@ int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_sched
   take(Rh * (W / kStatCols) * 8); take(Rh * (W / kStatCols) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
   take(d.dtype == CSD_F32 ? 0 : Rh * W * asz);
   take(static_cast<size_t>(sched->T) * W * 4);
+  take(Rh * W * asz);
   if (need > kStaticScratchBytes)
     return fail(ctx, CSD_ERR_WORKSPACE,
                 "csd_draft_denoise_static: this call needs %zu bytes of scratch but the built-in array holds %zu "

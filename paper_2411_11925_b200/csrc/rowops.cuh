@@ -96,13 +96,15 @@ struct StepParams {
   const float* te_next;          // [W] embedding of the step being prepared
   float* h;                      // [Rh, W]
   float* stats;                  // [Rh, W/64, 2]
-  void* s;                       // [Rh, W] activations
+  void* s;                       // [Rh, W] activations: s of the step te_next belongs to (null: none)
+  void* s_b;                     // a second s to prepare (first boundary only), with its embedding te_b
+  const float* te_b;
 };
 
 // One block per token row.  Finishes step t (unless STEP_INIT) and prepares the next one:
 //   eps_hat = sum of tile partials + bout; guidance; mu = a x - b eps_hat; x <- mu + sigma eps_t
 //   h = Win x + bin (same for both guidance rows), LayerNorm partials per 64 columns,
-//   s = SiLU(cz + te_next).
+//   s = SiLU(cz + te_next) of the step after that (s is double-buffered, see the host code).
 template <typename ACT>
 __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
   __shared__ float xs[kCPad];
@@ -168,7 +170,8 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
       for (int j = 0; j < 2; ++j) {
         const int n = g * kStatCols + j * 32 + lane;
         p.h[row * p.W + n] = acc[j];
-        s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + p.te_next[n]));
+        if (s) s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + p.te_next[n]));
+        if (p.s_b) reinterpret_cast<ACT*>(p.s_b)[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + p.te_b[n]));
       }
     }
   }
