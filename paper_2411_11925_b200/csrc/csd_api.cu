@@ -481,7 +481,9 @@ struct Chain {
       tp = &hd->Wgs[k]; ta = &tm_v; tw = &hd->tm[1].W2[k]; tout = &tm_ap;
     }
     const int tiles_n = W / kTileN, row_tiles = (Rh + kTileM - 1) / kTileM;
-    ProfScope ps(ctx, st, kind == FOLD_W1 ? 1 : 3, 2.0 * Rh * static_cast<double>(W) * W * 3.0);
+    // algorithmic FLOPs: the block's five W x W products are split 2 (first layer and the modulation folded into
+    // it; the kernel executes three products) + 3 (gate, next scale, second layer)
+    ProfScope ps(ctx, st, kind == FOLD_W1 ? 1 : 3, 2.0 * Rh * static_cast<double>(W) * W * (kind == FOLD_W1 ? 2.0 : 3.0));
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(tiles_n * row_tiles); lc.blockDim = dim3(kFoldThreads); lc.stream = st;
     lc.dynamicSmemBytes = kind == FOLD_W1 ? FoldCfg<FOLD_W1>::kSmemBytes : FoldCfg<FOLD_GATE>::kSmemBytes;
