@@ -371,14 +371,16 @@ struct Chain {
     const csd_head_desc& d = hd->d;
     ProfScope ps(ctx, st, 5, 2.0 * Rh * static_cast<double>(W) * d.C);
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(R); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    // four token rows per block once that still leaves every SM several blocks (the choice does not change a bit)
+    const bool rb4 = R >= 8 * ctx->num_sms;
+    cfg.gridDim = dim3(rb4 ? (R + 3) / 4 : R); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at; cfg.numAttrs = (ctx->prof_on || !tc) ? 0 : 1;
-    if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, step_kernel<__half>, sp, mode));
-    else if (d.dtype == CSD_BF16) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, step_kernel<__nv_bfloat16>, sp, mode));
-    else CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, step_kernel<float>, sp, mode));
+    if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<__half, 4> : step_kernel<__half, 1>, sp, mode));
+    else if (d.dtype == CSD_BF16) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<__nv_bfloat16, 4> : step_kernel<__nv_bfloat16, 1>, sp, mode));
+    else CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<float, 4> : step_kernel<float, 1>, sp, mode));
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
     return CSD_OK;

@@ -101,37 +101,50 @@ struct StepParams {
   const float* te_b;
 };
 
-// One block per token row.  Finishes step t (unless STEP_INIT) and prepares the next one:
+// RB token rows per block.  Finishes step t (unless STEP_INIT) and prepares the next one:
 //   eps_hat = sum of tile partials + bout; guidance; mu = a x - b eps_hat; x <- mu + sigma eps_t
 //   h = Win x + bin (same for both guidance rows), LayerNorm partials per 64 columns,
 //   s = SiLU(cz + te_next) of the step after that (s is double-buffered, see the host code).
-template <typename ACT>
+// With one row per block the kernel is bound by re-reading Win (64 B per column and row) through L1; RB = 4 reads a
+// group's columns once for four rows.  The arithmetic of a row does not depend on RB.
+template <typename ACT, int RB>
 __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
-  __shared__ float xs[kCPad];
-  __shared__ float eh[2][kCPad];
-  const int r = blockIdx.x, tid = threadIdx.x;
+  __shared__ float xs[RB][kCPad];
+  __shared__ float eh[RB][2][kCPad];
+  const int r0 = blockIdx.x * RB, tid = threadIdx.x;
   const int nrep = p.cfg ? 2 : 1;
+  const int nrow = min(RB, p.R - r0);
   griddep_wait();
   if (tid == 0) griddep_launch_dependents();
   if (mode == STEP_INIT) {
-    if (tid < kCPad) xs[tid] = (tid < p.C) ? p.x_src[static_cast<size_t>(r) * p.C + tid] : 0.0f;
-    if (tid < p.C) p.x[static_cast<size_t>(r) * p.C + tid] = p.x_src[static_cast<size_t>(r) * p.C + tid];
-    __syncthreads();
-  } else {
-    if (tid < nrep * kCPad) {
-      const int rep = tid / kCPad, c = tid % kCPad;
-      const float* e = p.epart + (static_cast<size_t>(r + rep * p.R) * p.NT) * kCPad + c;
-      float acc = 0.0f;
-      for (int nt = 0; nt < p.NT; ++nt) acc += e[nt * kCPad];
-      eh[rep][c] = acc + p.bout[c];
+    if (tid < RB * kCPad) {
+      const int rr = tid / kCPad, c = tid % kCPad;
+      float v = 0.0f;
+      if (rr < nrow && c < p.C) {
+        v = p.x_src[static_cast<size_t>(r0 + rr) * p.C + c];
+        p.x[static_cast<size_t>(r0 + rr) * p.C + c] = v;
+      }
+      xs[rr][c] = v;
     }
     __syncthreads();
-    if (tid < kCPad) {
+  } else {
+    if (tid < RB * 2 * kCPad) {
+      const int c = tid % kCPad, rep = (tid / kCPad) & 1, rr = tid / (2 * kCPad);
+      if (rr < nrow && rep < nrep) {
+        const float* e = p.epart + (static_cast<size_t>(r0 + rr + rep * p.R) * p.NT) * kCPad + c;
+        float acc = 0.0f;
+        for (int nt = 0; nt < p.NT; ++nt) acc += e[nt * kCPad];
+        eh[rr][rep][c] = acc + p.bout[c];
+      }
+    }
+    __syncthreads();
+    if (tid < RB * kCPad) {
+      const int rr = tid / kCPad, c = tid % kCPad;
       float xn = 0.0f;
-      if (tid < p.C) {
-        const size_t o = static_cast<size_t>(r) * p.C + tid;
-        float e = eh[0][tid];
-        if (p.cfg) e = cfg_combine(eh[0][tid], eh[1][tid], p.cfg_scale);
+      if (rr < nrow && c < p.C) {
+        const size_t o = static_cast<size_t>(r0 + rr) * p.C + c;
+        float e = eh[rr][0][c];
+        if (p.cfg) e = cfg_combine(eh[rr][0][c], eh[rr][1][c], p.cfg_scale);
         const float xo = p.x[o];
         const float mu = ddpm_mean(p.a, xo, p.b, e);
         xn = ddpm_sample(mu, p.sigma, p.eps_t[o]);
@@ -143,7 +156,7 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
           p.x[o] = xn;
         }
       }
-      xs[tid] = xn;
+      xs[rr][c] = xn;
     }
     if (mode == STEP_LAST) return;
     __syncthreads();
@@ -151,8 +164,9 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
   // prepare: each warp handles 64 consecutive columns at a time (lane, lane + 32): one LayerNorm partial
   const int lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
   ACT* s = reinterpret_cast<ACT*>(p.s);
+  ACT* s_b = reinterpret_cast<ACT*>(p.s_b);
   for (int g = warp; g < p.W / kStatCols; g += nwarp) {
-    float acc[2], mean, m2, wa[kCPad], wb[kCPad];
+    float wa[kCPad], wb[kCPad];
     const int na = g * kStatCols + lane, nb = na + 32;
 #pragma unroll
     for (int c4 = 0; c4 < kCPad / 4; ++c4) {
@@ -161,17 +175,26 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
       wa[4 * c4] = qa.x; wa[4 * c4 + 1] = qa.y; wa[4 * c4 + 2] = qa.z; wa[4 * c4 + 3] = qa.w;
       wb[4 * c4] = qb.x; wb[4 * c4 + 1] = qb.y; wb[4 * c4 + 2] = qb.z; wb[4 * c4 + 3] = qb.w;
     }
-    input_proj_group(wa, wb, p.bin[na], p.bin[nb], xs, acc, mean, m2);
-    for (int rep = 0; rep < nrep; ++rep) {
-      const size_t row = static_cast<size_t>(r) + static_cast<size_t>(rep) * p.R;
-      if (lane == 0)
-        reinterpret_cast<float2*>(p.stats)[row * (p.W / kStatCols) + g] = make_float2(mean, m2);
+    const float ba = p.bin[na], bb = p.bin[nb];
+    float te[2] = {0.0f, 0.0f}, teb[2] = {0.0f, 0.0f};
+    if (s) { te[0] = p.te_next[na]; te[1] = p.te_next[nb]; }
+    if (s_b) { teb[0] = p.te_b[na]; teb[1] = p.te_b[nb]; }
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const int n = g * kStatCols + j * 32 + lane;
-        p.h[row * p.W + n] = acc[j];
-        if (s) s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + p.te_next[n]));
-        if (p.s_b) reinterpret_cast<ACT*>(p.s_b)[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + p.te_b[n]));
+    for (int rr = 0; rr < RB; ++rr) {
+      if (rr >= nrow) break;
+      float acc[2], mean, m2;
+      input_proj_group(wa, wb, ba, bb, xs[rr], acc, mean, m2);
+      for (int rep = 0; rep < nrep; ++rep) {
+        const size_t row = static_cast<size_t>(r0 + rr) + static_cast<size_t>(rep) * p.R;
+        if (lane == 0)
+          reinterpret_cast<float2*>(p.stats)[row * (p.W / kStatCols) + g] = make_float2(mean, m2);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int n = g * kStatCols + j * 32 + lane;
+          p.h[row * p.W + n] = acc[j];
+          if (s) s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + te[j]));
+          if (s_b) s_b[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + teb[j]));
+        }
       }
     }
   }
