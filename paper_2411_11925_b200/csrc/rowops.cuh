@@ -179,12 +179,26 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
     float te[2] = {0.0f, 0.0f}, teb[2] = {0.0f, 0.0f};
     if (s) { te[0] = p.te_next[na]; te[1] = p.te_next[nb]; }
     if (s_b) { teb[0] = p.te_b[na]; teb[1] = p.te_b[nb]; }
+    // every cz value of the group first: the loads are independent, but behind the stores below the compiler must
+    // assume they are not, and each row would wait for its own trip to memory
+    float czv[RB][2][2];
+#pragma unroll
+    for (int rr = 0; rr < RB; ++rr)
+#pragma unroll
+      for (int rep = 0; rep < 2; ++rep)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const size_t row = static_cast<size_t>(r0 + rr) + static_cast<size_t>(rep) * p.R;
+          czv[rr][rep][j] = (rr < nrow && rep < nrep && (s || s_b)) ? __ldg(p.cz + row * p.W + g * kStatCols + j * 32 + lane) : 0.0f;
+        }
 #pragma unroll
     for (int rr = 0; rr < RB; ++rr) {
       if (rr >= nrow) break;
       float acc[2], mean, m2;
       input_proj_group(wa, wb, ba, bb, xs[rr], acc, mean, m2);
-      for (int rep = 0; rep < nrep; ++rep) {
+#pragma unroll
+      for (int rep = 0; rep < 2; ++rep) {
+        if (rep >= nrep) break;
         const size_t row = static_cast<size_t>(r0 + rr) + static_cast<size_t>(rep) * p.R;
         if (lane == 0)
           reinterpret_cast<float2*>(p.stats)[row * (p.W / kStatCols) + g] = make_float2(mean, m2);
@@ -192,8 +206,8 @@ __global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
         for (int j = 0; j < 2; ++j) {
           const int n = g * kStatCols + j * 32 + lane;
           p.h[row * p.W + n] = acc[j];
-          if (s) s[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + te[j]));
-          if (s_b) s_b[row * p.W + n] = to_act<ACT>(silu_f(p.cz[row * p.W + n] + teb[j]));
+          if (s) s[row * p.W + n] = to_act<ACT>(silu_f(czv[rr][rep][j] + te[j]));
+          if (s_b) s_b[row * p.W + n] = to_act<ACT>(silu_f(czv[rr][rep][j] + teb[j]));
         }
       }
     }
