@@ -108,7 +108,7 @@ struct StepParams {
 // With one row per block the kernel is bound by re-reading Win (64 B per column and row) through L1; RB = 4 reads a
 // group's columns once for four rows.  The arithmetic of a row does not depend on RB.
 template <typename ACT, int RB>
-__global__ void __launch_bounds__(256) step_kernel(StepParams p, int mode) {
+__global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p, int mode) {
   __shared__ float xs[RB][kCPad];
   __shared__ float eh[RB][2][kCPad];
   const int r0 = blockIdx.x * RB, tid = threadIdx.x;
