@@ -15,6 +15,10 @@ What pins each function (see tests/test_oracle_pins.py):
   log_sigma_term, log_ratio_*   long form (Eq. 4) == closed form (Eq. 7, 8);
                            identical heads give exactly 0; 1-D Gaussian toy
                            head matches an independently composed affine map
+  log_ratio_single_path    T = 1 reduces to Eq. 8; identical heads give exactly 0;
+                           1-D Gaussian toy heads: equals the difference of two
+                           multivariate-normal log-densities of the whole path
+                           (library routine); E_q[p(Y)/q(Y)] = 1 by Monte Carlo
   accept_prefix            brute force over all accept masks (Alg. 1)
   resample                 KS test against the numerically integrated
                            max(0, Sigma*p - q) (Eq. 5, Eq. 11, Cor. 1); textbook
@@ -212,6 +216,23 @@ def log_ratio_long(dq: dict, dp: dict, sched_q, sched_p) -> np.ndarray:
     return total
 
 
+def log_ratio_single_path(eps_p: Callable[[np.ndarray, int], np.ndarray], sched_q, sched_p,
+                          dq: dict) -> np.ndarray:
+    """log p(Y_q)/q(Y_q) of Eq. 2: the exact criterion, in which BOTH models score the
+    draft's own trajectory Y_q = (x_T, x^q_{T-1}, ..., x^q_0).  Step t contributes
+    log N(x^q_{t-1}; mu^p_t(x^q_t), sigma_p,t^2) - log N(x^q_{t-1}; mu^q_t(x^q_t), sigma_q,t^2);
+    p(x_T) = q(x_T) cancels.  dq is a keep=True draft run: xs[j] = x^q_{T-j}, mus[j] = mu^q_{T-j}."""
+    T = len(sched_q["a"])
+    total = 0.0
+    for j in range(T):
+        t = T - j
+        x_t, x_next = dq["xs"][j], dq["xs"][j + 1]
+        mu_p = sched_p["a"][t - 1] * x_t - sched_p["b"][t - 1] * eps_p(x_t, t)
+        total = total + gaussian_logpdf_iso(x_next, mu_p, sched_p["sigma"][t - 1]) \
+                      - gaussian_logpdf_iso(x_next, dq["mus"][j], sched_q["sigma"][t - 1])
+    return total
+
+
 # --------------------------------------------------------------------------
 # Verification (Alg. 1: draw r_i, accept while r_i <= ratio, n = first reject)
 # --------------------------------------------------------------------------
@@ -286,6 +307,20 @@ def csd_round(eps_q, eps_p, sched_q, sched_p, x_T, noise, u, xi, v, B, gamma, ca
     if keep:
         out["dq"], out["dp"] = dq, dp
     return out
+
+
+def single_path_from_inputs(inp) -> Dict[str, np.ndarray]:
+    """Draft trajectories of a RoundInputs bundle and the exact ratio of Eq. 2 on them,
+    with the accept scan of Alg. 1 applied to that ratio."""
+    wl = inp.wl
+    sched = ddpm_schedule(inp.beta, wl.tau)
+    eq = make_mlp_head(inp.w_q, inp.z_q, inp.tfeat, wl.cfg, wl.cfg_scale)
+    ep = make_mlp_head(inp.w_p, inp.z_p, inp.tfeat, wl.cfg, wl.cfg_scale)
+    dq = denoise(eq, sched, inp.x_T, inp.eps, sample_last=True, keep=True)
+    logr = log_ratio_single_path(ep, sched, sched, dq).reshape(wl.B, wl.gamma)
+    n, acc = accept_prefix(logr, inp.u)
+    return {"traj_x": np.stack(dq["xs"]), "traj_mu": np.stack(dq["mus"]), "logratio": logr,
+            "n_accept": n, "accept": acc}
 
 
 def round_from_inputs(inp, keep: bool = False) -> Dict[str, np.ndarray]:

@@ -310,6 +310,87 @@ def test_toy_gaussian_logratio_matches_independent_affine_composition():
         assert abs(got[r] - want) < 1e-8 * max(1.0, abs(want))
 
 
+# ------------------------------------------------- single-path exact ratio (Eq. 2)
+def test_single_path_ratio_with_one_step_is_the_final_step_ratio():
+    # T = 1: both trajectories consist of x_T = x_1 only, so Eq. 2 and Eq. 8 coincide (Sigma = 1).
+    beta = gen.beta_linear(1, 0.02, 0.02)
+    sq, sp = orc.ddpm_schedule(beta, 1.0), orc.ddpm_schedule(beta, 0.8)
+    eq = orc.make_gaussian_toy_head(0.3, 0.8, sq["alphabar"])
+    ep = orc.make_gaussian_toy_head(-0.1, 1.1, sp["alphabar"])
+    rng = np.random.default_rng(40)
+    x_T, noise = rng.standard_normal((5, 3)), rng.standard_normal((1, 5, 3))
+    dq, dp = orc.run_pair(eq, ep, sq, sp, x_T, noise, keep=True)
+    closed = orc.log_ratio_closed(dq["x0"], dq["mu1"], dp["mu1"], sq["sigma"][0], sp["sigma"][0], 0.0)
+    np.testing.assert_allclose(orc.log_ratio_single_path(ep, sq, sp, dq), closed, atol=1e-12)
+
+
+def test_single_path_ratio_of_identical_heads_is_exactly_zero():
+    wl = gen.WORKLOADS["tiny_fp32"]
+    inp = gen.make_round_inputs(wl)
+    inp.w_q, inp.z_q = inp.w_p, inp.z_p
+    out = orc.single_path_from_inputs(inp)
+    assert np.all(out["logratio"] == 0.0) and np.all(out["n_accept"] == wl.gamma)
+    assert out["traj_x"].shape == (wl.T + 1, wl.R, 16) and out["traj_mu"].shape == (wl.T, wl.R, 16)
+
+
+def _toy_path_gaussian(m, s, tau, beta, xT):
+    # 1-D Gaussian toy head: x_{t-1} = A_t x_t + D_t + sigma_t eps_t.  The path y = (x_{T-1}, ..., x_0) given
+    # x_T solves M y = d + S eps, hence y ~ N(M^-1 d, M^-1 S S^T M^-T).
+    T = len(beta)
+    ab = np.cumprod(1 - beta)
+    M, d, S = np.eye(T), np.zeros(T), np.zeros((T, T))
+    for i, t in enumerate(range(T, 0, -1)):
+        k = math.sqrt(1 - ab[t - 1]) / (ab[t - 1] * s * s + 1 - ab[t - 1])
+        bt = beta[t - 1] / (math.sqrt(1 - beta[t - 1]) * math.sqrt(1 - ab[t - 1]))
+        A, D = 1 / math.sqrt(1 - beta[t - 1]) - bt * k, bt * k * math.sqrt(ab[t - 1]) * m
+        d[i] = D + (A * xT if i == 0 else 0.0)
+        if i > 0:
+            M[i, i - 1] = -A
+        S[i, i] = tau * math.sqrt(beta[t - 1])
+    Minv = np.linalg.inv(M)
+    return Minv @ d, Minv @ S @ S.T @ Minv.T
+
+
+def test_single_path_ratio_matches_multivariate_normal_path_densities():
+    # With toy heads the whole path given x_T is jointly Gaussian under either model, so Eq. 2 is the difference
+    # of two multivariate-normal log-densities (scipy), evaluated at the draft's path: no stepping, no per-step terms.
+    T = 8
+    beta = gen.beta_linear(T, 0.01, 0.2)
+    tau_q, tau_p = 1.0, 0.9
+    sq, sp = orc.ddpm_schedule(beta, tau_q), orc.ddpm_schedule(beta, tau_p)
+    eq = orc.make_gaussian_toy_head(0.4, 0.6, sq["alphabar"])
+    ep = orc.make_gaussian_toy_head(-0.2, 0.9, sp["alphabar"])
+    rng = np.random.default_rng(41)
+    N = 5
+    x_T, noise = rng.standard_normal((N, 1)), rng.standard_normal((T, N, 1))
+    dq = orc.denoise(eq, sq, x_T, noise, sample_last=True, keep=True)
+    got = orc.log_ratio_single_path(ep, sq, sp, dq)
+    for r in range(N):
+        y = np.array([dq["xs"][j + 1][r, 0] for j in range(T)])
+        mq, cq = _toy_path_gaussian(0.4, 0.6, tau_q, beta, x_T[r, 0])
+        mp, cp = _toy_path_gaussian(-0.2, 0.9, tau_p, beta, x_T[r, 0])
+        want = st.multivariate_normal(mp, cp).logpdf(y) - st.multivariate_normal(mq, cq).logpdf(y)
+        assert abs(got[r] - want) < 1e-8 * max(1.0, abs(want))
+
+
+def test_single_path_ratio_has_unit_expectation_under_the_draft():
+    # E_{Y ~ q}[p(Y)/q(Y)] = 1 (importance-weight identity stated with the bias analysis of the surrogate ratio);
+    # a dropped step, a wrong sign or a wrong variance in Eq. 2 breaks it.
+    T, N = 3, 400_000
+    beta = gen.beta_linear(T, 0.05, 0.2)
+    sq, sp = orc.ddpm_schedule(beta, 1.0), orc.ddpm_schedule(beta, 0.95)
+    eq = orc.make_gaussian_toy_head(0.1, 0.9, sq["alphabar"])
+    ep = orc.make_gaussian_toy_head(0.0, 1.0, sp["alphabar"])
+    rng = np.random.default_rng(42)
+    x_T = np.tile(rng.standard_normal((1, 1)), (N, 1))
+    noise = rng.standard_normal((T, N, 1))
+    dq = orc.denoise(eq, sq, x_T, noise, sample_last=True, keep=True)
+    w = np.exp(orc.log_ratio_single_path(ep, sq, sp, dq))
+    se = w.std() / math.sqrt(N)
+    assert abs(w.mean() - 1.0) < 5 * se + 1e-3, (w.mean(), se)
+    assert w.std() > 0.05          # not vacuous: the two models differ
+
+
 # --------------------------------------------------------------- accept scan
 @pytest.mark.parametrize("gamma", [1, 3, 8])
 def test_accept_prefix_brute_force_all_masks(gamma):
