@@ -200,6 +200,43 @@ int csd_accept_scan(csd_ctx *ctx, int B, int gamma, int C, double log_sigma_term
                     float sigma1_q, const float *x0_q, const float *mu1_q, const float *mu1_p,
                     const float *u, float *logratio, int32_t *n_accept, uint32_t *accept_mask);
 
+/* ---- Exact single-path criterion (Eq. 2; Table 1 "p(Y_q)/q(Y_q)") ------------------------------
+ * Eq. 2 scores the DRAFT's own trajectory Y_q = (x_T, x^q_{T-1}, ..., x^q_0) under both models:
+ *   log p(Y_q)/q(Y_q) = sum_{t=1..T} [ log N(x^q_{t-1}; mu^p_t(x^q_t), sigma_p,t^2 I)
+ *                                    - log N(x^q_{t-1}; mu^q_t(x^q_t), sigma_q,t^2 I) ].
+ * The paper shows this exact ratio accepts almost nothing and replaces it by Eq. 4; it is provided as the
+ * diagnostic the approximated criterion of csd_verify is measured against.
+ *
+ * csd_draft_denoise_traj: csd_draft_denoise that records the whole trajectory.
+ *   traj_x  device [T+1, R, C] out: slot j = x_{T-j} (slot 0 = x_T, slot T = x_0)
+ *   traj_mu device [T,   R, C] out: slot j = mu_{T-j} (the mean from which slot j+1 of traj_x was drawn)
+ *   other arguments as in csd_draft_denoise; x_0 and mu_1 are the last slots. */
+int csd_draft_denoise_traj(csd_ctx *ctx, const csd_head *head, const csd_schedule *sched, int R, int cfg,
+                           float cfg_scale, const float *z, const float *x_T, const float *eps,
+                           float *traj_x, float *traj_mu);
+
+/* csd_verify_single_path: evaluates the target head at every state of the draft's trajectory and
+ * returns the log of Eq. 2 per token, then the accept test and prefix count of Alg. 1 on it
+ * (accept iff log u <= logratio).  Given the trajectory, the T target evaluations do not depend on
+ * one another: they run as ceil(T / steps_per_pass) passes of the layers over steps_per_pass * R
+ * token rows each instead of T dependent steps.  Per step the two quadratic forms are rounded
+ * separately, so a target that reproduces the draft's means bit for bit gives exactly 0.
+ *   sched_p: full schedule of the target; sched_q: only T and sigma are read (same T).
+ *   z_p device [B*gamma*(1+cfg), Dz_p]; traj_x, traj_mu_q device, as written by
+ *   csd_draft_denoise_traj for R = B*gamma; u device [B, gamma] in (0,1];
+ *   steps_per_pass: 0 = chosen by the library (about 32768 head rows per pass).  The steps are
+ *   summed in trajectory order whatever the split; with CSD_CHAIN_LAYERS_PLAIN the result does not
+ *   depend on it by a bit, in the default mode the block layout follows a pass's row count and
+ *   results of different splits agree within the parity tolerance;
+ *   logratio device [B, gamma] out; n_accept device int32 [B] out; accept_mask device uint32 [B]
+ *   out or NULL.
+ * The library keeps a side buffer of steps_per_pass * R * C floats besides the chain workspace. */
+int csd_verify_single_path(csd_ctx *ctx, const csd_head *head_p, const csd_schedule *sched_p,
+                           const csd_schedule *sched_q, int B, int gamma, int cfg, float cfg_scale,
+                           const float *z_p, const float *traj_x, const float *traj_mu_q,
+                           const float *u, int steps_per_pass, float *logratio, int32_t *n_accept,
+                           uint32_t *accept_mask);
+
 /* Resampling from the modified distribution max(0, p - q)/Z (Eq. 5) by acceptance-rejection with
  * the bound M = 1/Z (Eq. 9-11) in the inference-free form of Corollary 1.  For each sequence with
  * n_accept[b] < gamma, row j = b*gamma + n_accept[b]: for k = 0..cap-1

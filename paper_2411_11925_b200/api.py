@@ -25,7 +25,8 @@ DTYPES = {"f32": CSD_F32, "bf16": CSD_BF16, "f16": CSD_F16}
 EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launch_count",
            "csd_set_chain_mode", "csd_profile", "csd_profile_read",
            "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_draft_denoise_static", "csd_verify",
-           "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host")
+           "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host", "csd_draft_denoise_traj",
+           "csd_verify_single_path")
 
 WEIGHT_FIELDS = ("Wz", "bz", "Wt1", "bt1", "Wt2", "bt2", "Win", "bin", "Wada", "bada",
                  "W1", "b1", "W2", "b2", "Wfada", "bfada", "Wout", "bout")
@@ -70,6 +71,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_draft_denoise.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, f32] + [vp] * 6
     lib.csd_draft_denoise_static.argtypes = lib.csd_draft_denoise.argtypes
     lib.csd_verify.argtypes = [vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32] + [vp] * 10
+    lib.csd_draft_denoise_traj.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, f32] + [vp] * 5
+    lib.csd_verify_single_path.argtypes = ([vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32]
+                                           + [vp] * 4 + [i32] + [vp] * 3)
     lib.csd_accept_scan.argtypes = [vp, i32, i32, i32, f64, f32, f32] + [vp] * 7
     lib.csd_resample.argtypes = [vp, i32, i32, i32, i32, f64, f32, f32] + [vp] * 9
     round_args = [vp, vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32, i32] + [vp] * 17
@@ -195,6 +199,17 @@ class Context:
         self._check(_LIB.csd_verify(self._h, head_p._h, C.byref(sched_p.c), C.byref(sched_q.c), B, gamma, int(cfg),
                                     cfg_scale, _ptr(z_p), _ptr(x_T), _ptr(eps), _ptr(x0_q), _ptr(mu1_q), _ptr(u),
                                     _ptr(logratio), _ptr(n_accept), _ptr(accept_mask), _ptr(mu1_p)))
+
+    def csd_draft_denoise_traj(self, head: "Head", sched: Schedule, R, cfg, cfg_scale, z, x_T, eps, traj_x, traj_mu):
+        self._check(_LIB.csd_draft_denoise_traj(self._h, head._h, C.byref(sched.c), R, int(cfg), cfg_scale,
+                                                _ptr(z), _ptr(x_T), _ptr(eps), _ptr(traj_x), _ptr(traj_mu)))
+
+    def csd_verify_single_path(self, head_p: "Head", sched_p: Schedule, sched_q: Schedule, B, gamma, cfg, cfg_scale,
+                               z_p, traj_x, traj_mu_q, u, steps_per_pass, logratio, n_accept, accept_mask=None):
+        self._check(_LIB.csd_verify_single_path(self._h, head_p._h, C.byref(sched_p.c), C.byref(sched_q.c), B, gamma,
+                                                int(cfg), cfg_scale, _ptr(z_p), _ptr(traj_x), _ptr(traj_mu_q),
+                                                _ptr(u), int(steps_per_pass), _ptr(logratio), _ptr(n_accept),
+                                                _ptr(accept_mask)))
 
     def csd_accept_scan(self, B, gamma, Cdim, log_sigma, sigma1_p, sigma1_q, x0_q, mu1_q, mu1_p, u, logratio,
                         n_accept, accept_mask=None):

@@ -63,6 +63,7 @@ struct csd_ctx {
   EncodeTiledFn encode = nullptr;
   ChainWs ws[3];   // draft chain, target chain, static-scratch calls
   HostIo io;
+  HostIo sp;       // csd_verify_single_path: schedule constants, mu^p of one pass, running log-ratio
   char err[512] = {0};
   // optional per-launch timing (csd_profile)
   bool prof_on = false;
@@ -366,6 +367,45 @@ struct Chain {
   int cur_t = 0;
   EpiParams ep{};
   StepParams sp{};
+  // trajectory recording (csd_draft_denoise_traj): [T + 1, R, C] states and [T, R, C] means, or null
+  float *traj_x = nullptr, *traj_mu = nullptr;
+  // batched evaluation on a given trajectory (csd_verify_single_path): R = batch_steps * batch_Rin token rows,
+  // one pass of the layers; slot batch_j0 of batch_traj is the first step of the pass
+  int batch_Rin = 0, batch_j0 = 0, Ts = 0;
+  const float *batch_traj = nullptr, *batch_sched = nullptr;
+  float* batch_mu = nullptr;
+
+  template <typename ACT>
+  int launch_step_t(cudaLaunchConfig_t& cfg, bool rb4, int mode) {
+    if (traj_x) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<ACT, 4, true> : step_kernel<ACT, 1, true>, sp, mode));
+    else CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<ACT, 4> : step_kernel<ACT, 1>, sp, mode));
+    return CSD_OK;
+  }
+
+  // kind 0: prepare the pass (h, LayerNorm partials, s); kind 1: finish it (eps_hat, guidance, mu^p)
+  int launch_batch(int kind) {
+    const csd_head_desc& d = hd->d;
+    ChainWs& ws = ctx->ws[slot];
+    BatchParams b{};
+    b.Rin = batch_Rin; b.Rtok = R; b.cfg = cfg; b.C = d.C; b.W = W; b.NT = tc ? W / kStatCols : W / kTileN;
+    b.T = Ts; b.j0 = batch_j0; b.cfg_scale = cfg_scale; b.sched = batch_sched; b.traj_x = batch_traj;
+    b.win = hd->win; b.bin = hd->bin; b.cz = ws.cz; b.te = ws.te; b.h = ws.h; b.stats = ws.stats; b.s = ws.s;
+    b.epart = ws.epart; b.bout = hd->bout; b.mu_p = batch_mu;
+    ProfScope ps(ctx, st, 5, 2.0 * Rh * static_cast<double>(W) * d.C);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(kind == 0 ? (R + 3) / 4 : (R + 15) / 16); lc.blockDim = dim3(256); lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at; lc.numAttrs = (ctx->prof_on || !tc) ? 0 : 1;
+    if (kind == 1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, batch_finish_kernel, b));
+    else if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, batch_prepare_kernel<__half>, b));
+    else if (d.dtype == CSD_BF16) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, batch_prepare_kernel<__nv_bfloat16>, b));
+    else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, batch_prepare_kernel<float>, b));
+    ctx->launches++;
+    CSD_CUDA(ctx, cudaGetLastError());
+    return CSD_OK;
+  }
 
   int launch_step(int mode) {
     const csd_head_desc& d = hd->d;
@@ -378,9 +418,11 @@ struct Chain {
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at; cfg.numAttrs = (ctx->prof_on || !tc) ? 0 : 1;
-    if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<__half, 4> : step_kernel<__half, 1>, sp, mode));
-    else if (d.dtype == CSD_BF16) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<__nv_bfloat16, 4> : step_kernel<__nv_bfloat16, 1>, sp, mode));
-    else CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<float, 4> : step_kernel<float, 1>, sp, mode));
+    int rc;
+    if (d.dtype == CSD_F16) rc = launch_step_t<__half>(cfg, rb4, mode);
+    else if (d.dtype == CSD_BF16) rc = launch_step_t<__nv_bfloat16>(cfg, rb4, mode);
+    else rc = launch_step_t<float>(cfg, rb4, mode);
+    if (rc) return rc;
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
     return CSD_OK;
@@ -388,7 +430,8 @@ struct Chain {
 
   int begin() {
     const csd_head_desc& d = hd->d;
-    Rh = R * (cfg ? 2 : 1); W = d.W; L = d.L; T = sc->T;
+    Rh = R * (cfg ? 2 : 1); W = d.W; L = d.L; Ts = sc->T;
+    T = batch_Rin ? 1 : Ts;   // a batched pass runs the layers once
     tc = d.dtype != CSD_F32;
     // 64-wide output tiles when 128-wide ones (of all chains running side by side) would occupy at most a
     // quarter of the SMs: a kernel and the early part of its successor should both find free SMs
@@ -423,24 +466,26 @@ struct Chain {
              8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && fold_kernels_ready(d);
     }
     ChainWs& ws = ctx->ws[slot];
-    int rc = ensure_ws(ctx, ws, d, Rh, R, T, whole);
+    int rc = ensure_ws(ctx, ws, d, Rh, R, Ts, whole);
     if (rc) return rc;
     {
-      const dim3 grid((W + 31) / 32, (T + 31) / 32);
-      small_gemm_nt_kernel<true><<<grid, 256, 0, st>>>(sc->tfeat, hd->Wt1, hd->bt1, ws.hid, T, W, d.F);
-      small_gemm_nt_kernel<false><<<grid, 256, 0, st>>>(ws.hid, hd->Wt2, hd->bt2, ws.te, T, W, W);
+      const dim3 grid((W + 31) / 32, (Ts + 31) / 32);
+      small_gemm_nt_kernel<true><<<grid, 256, 0, st>>>(sc->tfeat, hd->Wt1, hd->bt1, ws.hid, Ts, W, d.F);
+      small_gemm_nt_kernel<false><<<grid, 256, 0, st>>>(ws.hid, hd->Wt2, hd->bt2, ws.te, Ts, W, W);
       ctx->launches++;
     }
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
     ep.M = Rh; ep.ldo = W;
+    // rows of z: one per head row, or one per row of a step when the steps of a trajectory are batched
+    const int Rz = batch_Rin ? batch_Rin * (cfg ? 2 : 1) : Rh;
     if (tc) {
-      const size_t nz = static_cast<size_t>(Rh) * d.Dz;
+      const size_t nz = static_cast<size_t>(Rz) * d.Dz;
       const unsigned nblk = static_cast<unsigned>((nz + 255) / 256);
       if (d.dtype == CSD_F16) convert_act_kernel<__half><<<nblk, 256, 0, st>>>(z, static_cast<__half*>(ws.zc), nz);
       else convert_act_kernel<__nv_bfloat16><<<nblk, 256, 0, st>>>(z, static_cast<__nv_bfloat16*>(ws.zc), nz);
       ctx->launches++;
-      if ((rc = make_tmap(ctx, &tm_z, d.dtype, ws.zc, Rh, d.Dz, d.Dz, kTileM))) return rc;
+      if ((rc = make_tmap(ctx, &tm_z, d.dtype, ws.zc, Rz, d.Dz, d.Dz, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_sb[1], d.dtype, ws.s, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_sb[0], d.dtype, ws.s2, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_u, d.dtype, ws.u, Rh, W, W, kTileM))) return rc;
@@ -451,15 +496,18 @@ struct Chain {
     // cz = z Wz^T + bz
     const csd_head::TmSet& tmw = hd->tm[(tn == 64 || pair) ? 0 : 1];   // pairs load half of each B tile per CTA
     EpiParams e = ep;
+    e.M = Rz;
     e.bias0 = hd->bz; e.out_f32 = ws.cz;
     if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 1>(ctx, d.dtype, tn, pair, st, tm_z, tmw.Wz, tm_z, tmw.Wz, tm_h, d.Dz, 0, 0, W, e);
     else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
                                                 nullptr, 0, W, e);
     if (rc) return rc;
+    sbuf[0] = ws.s2; sbuf[1] = ws.s;
+    if (batch_Rin) return launch_batch(0);   // a pass has one step (t = 1): its s is sbuf[1]
+    sp.traj_x = traj_x; sp.traj_mu = nullptr;
     sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = tc ? W / kStatCols : W / kTileN; sp.cfg_scale = cfg_scale;
     sp.sample_last = sample_last; sp.epart = ws.epart; sp.bout = hd->bout; sp.x_src = x_T; sp.x = ws.x;
     sp.x0 = x0; sp.mu1 = mu1; sp.x1 = x1; sp.win = hd->win; sp.bin = hd->bin; sp.cz = ws.cz; sp.h = ws.h;
-    sbuf[0] = ws.s2; sbuf[1] = ws.s;
     sp.stats = ws.stats; sp.s = sbuf[T & 1];
     sp.te_next = ws.te + static_cast<size_t>(T - 1) * W;
     sp.s_b = T >= 2 ? sbuf[(T - 1) & 1] : nullptr;   // the first boundary also prepares s of step T - 1
@@ -604,6 +652,11 @@ struct Chain {
     else rc = launch_simt<EPI_MODF, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
                                             0, W, e);
     if (rc) return rc;
+    if (batch_Rin) return launch_batch(1);
+    if (traj_x) {   // slot j holds x_{T-j} and mu_{T-j}: this boundary produces x_{t-1} and mu_t
+      sp.traj_x = traj_x + static_cast<size_t>(T - t + 1) * R * d.C;
+      sp.traj_mu = traj_mu + static_cast<size_t>(T - t) * R * d.C;
+    }
     sp.a = sc->a[t - 1]; sp.b = sc->b[t - 1]; sp.sigma = sc->sigma[t - 1];
     sp.eps_t = eps + static_cast<size_t>(t - 1) * R * d.C;
     // this boundary prepares h of step t - 1 and s of step t - 2
@@ -735,6 +788,7 @@ int csd_destroy(csd_ctx* c) {
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->io.base) cudaFree(c->io.base);
+  if (c->sp.base) cudaFree(c->sp.base);
   if (c->d_err) cudaFree(c->d_err);
   cudaGetLastError();
   delete c;
@@ -1082,6 +1136,99 @@ int csd_verify(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p
   const int C = head_p->d.C;
   return accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term(sched_q, sched_p, C), sched_p->sigma[0],
                      sched_q->sigma[0], x0_q, mu1_q, mu1_p, u, logratio, n_accept, accept_mask);
+}
+
+int csd_draft_denoise_traj(csd_ctx* ctx, const csd_head* head, const csd_schedule* sched, int R, int cfg,
+                           float cfg_scale, const float* z, const float* x_T, const float* eps, float* traj_x,
+                           float* traj_mu) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_chain_args(ctx, head, sched, R, cfg, z, x_T, eps);
+  if (rc) return rc;
+  if (!traj_x || !traj_mu) return fail(ctx, CSD_ERR_INVALID_ARG, "traj_x / traj_mu is null");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  const size_t slot = static_cast<size_t>(R) * head->d.C;
+  const int T = sched->T;
+  // the last boundary writes x_0 and mu_1 through the chain's ordinary outputs, which are the last slots
+  Chain c{ctx, 0, ctx->stream, head, sched, R, cfg, cfg_scale, z, x_T, eps, 1, traj_x + T * slot,
+          traj_mu + (T - 1) * slot, nullptr};
+  c.allow_chain_kernel = false;   // the whole-chain kernel keeps its states on chip
+  c.traj_x = traj_x; c.traj_mu = traj_mu;
+  rc = c.begin();
+  for (int t = T; t >= 1 && !rc; --t) rc = c.step(t);
+  return rc;
+}
+
+int csd_verify_single_path(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p,
+                           const csd_schedule* sched_q, int B, int gamma, int cfg, float cfg_scale, const float* z_p,
+                           const float* traj_x, const float* traj_mu_q, const float* u, int steps_per_pass,
+                           float* logratio, int32_t* n_accept, uint32_t* accept_mask) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
+  if (static_cast<int64_t>(B) * gamma > (1 << 24)) return fail(ctx, CSD_ERR_UNSUPPORTED, "B * gamma exceeds 2^24 rows");
+  const int R = B * gamma;
+  int rc = check_chain_args(ctx, head_p, sched_p, R, cfg, z_p, traj_x, traj_mu_q);
+  if (rc) return rc;
+  if ((rc = check_sched(ctx, sched_q, false))) return rc;
+  if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
+  if ((rc = check_verify_dims(ctx, B, gamma, head_p->d.C))) return rc;
+  if (!u || !logratio || !n_accept) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  if (steps_per_pass < 0) return fail(ctx, CSD_ERR_INVALID_ARG, "steps_per_pass = %d must be >= 0", steps_per_pass);
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  const int T = sched_p->T, C = head_p->d.C, Rh1 = R * (cfg ? 2 : 1);
+  // steps per pass: enough head rows to fill the GPU several times over, few enough to keep the workspace
+  // (about 16 W bytes per head row) modest
+  constexpr int kRowsPerPass = 32768;
+  int tb = steps_per_pass ? steps_per_pass : (kRowsPerPass + Rh1 - 1) / Rh1;
+  if (tb > T) tb = T;
+  if (static_cast<int64_t>(tb) * Rh1 > (int64_t(1) << 26)) return fail(ctx, CSD_ERR_UNSUPPORTED, "pass of %d steps has too many rows", tb);
+  // device side buffer: [5, T] constants | mu^p of a pass [tb R, C] | running sum [R] (double)
+  const size_t o_mu = align_up(static_cast<size_t>(5) * T * 4, 256);
+  const size_t o_acc = align_up(o_mu + static_cast<size_t>(tb) * R * C * 4, 256);
+  const size_t need = o_acc + static_cast<size_t>(R) * 8;
+  cudaStream_t st = ctx->stream;
+  if (need > ctx->sp.cap) {
+    CSD_CUDA(ctx, cudaStreamSynchronize(st));
+    if (ctx->sp.base) CSD_CUDA(ctx, cudaFree(ctx->sp.base));
+    ctx->sp.base = nullptr; ctx->sp.cap = 0;
+    if (cudaMalloc(&ctx->sp.base, need) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes for the single-path buffers", need);
+    }
+    ctx->sp.cap = need;
+  }
+  char* base = static_cast<char*>(ctx->sp.base);
+  float* d_sched = reinterpret_cast<float*>(base);
+  float* d_mu = reinterpret_cast<float*>(base + o_mu);
+  double* d_acc = reinterpret_cast<double*>(base + o_acc);
+  {
+    // per step: a_t, b_t of the target, C (log sigma_q,t - log sigma_p,t), 1 / (2 sigma_p,t^2), 1 / (2 sigma_q,t^2)
+    std::vector<float> hs(static_cast<size_t>(5) * T);
+    for (int t = 0; t < T; ++t) {
+      const double sp = sched_p->sigma[t], sq = sched_q->sigma[t];
+      hs[t] = sched_p->a[t]; hs[T + t] = sched_p->b[t];
+      hs[2 * T + t] = static_cast<float>(C * (std::log(sq) - std::log(sp)));
+      hs[3 * T + t] = static_cast<float>(0.5 / (sp * sp));
+      hs[4 * T + t] = static_cast<float>(0.5 / (sq * sq));
+    }
+    // pageable source: the runtime stages it before the call returns
+    CSD_CUDA(ctx, cudaMemcpyAsync(d_sched, hs.data(), hs.size() * 4, cudaMemcpyHostToDevice, st));
+  }
+  for (int j0 = 0; j0 < T; j0 += tb) {
+    const int n = T - j0 < tb ? T - j0 : tb;
+    Chain c{ctx, 1, st, head_p, sched_p, n * R, cfg, cfg_scale, z_p, nullptr, nullptr, 0, nullptr, nullptr, nullptr};
+    c.allow_chain_kernel = false;
+    c.batch_Rin = R; c.batch_j0 = j0; c.batch_traj = traj_x; c.batch_sched = d_sched; c.batch_mu = d_mu;
+    if ((rc = c.begin())) return rc;
+    if ((rc = c.step(1))) return rc;
+    single_path_accum_kernel<<<(R + 127) / 128, 128, 0, st>>>(R, C, T, j0, n, d_sched, traj_x, traj_mu_q, d_mu, d_acc,
+                                                              j0 == 0 ? 1 : 0);
+    ctx->launches++;
+    CSD_CUDA(ctx, cudaGetLastError());
+  }
+  accept_from_logratio_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, gamma, d_acc, u, logratio, n_accept, accept_mask);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
 }
 
 int csd_resample(csd_ctx* ctx, int B, int gamma, int C, int cap, double log_sigma_term_, float sigma1_p, float sigma1_q,

@@ -99,6 +99,8 @@ struct StepParams {
   void* s;                       // [Rh, W] activations: s of the step te_next belongs to (null: none)
   void* s_b;                     // a second s to prepare (first boundary only), with its embedding te_b
   const float* te_b;
+  float* traj_x;                 // TRAJ kernels: where the state this boundary produces is recorded ([R, C])
+  float* traj_mu;                // TRAJ kernels: where the mean of the step being finished is recorded ([R, C])
 };
 
 // RB token rows per block.  Finishes step t (unless STEP_INIT) and prepares the next one:
@@ -107,7 +109,8 @@ struct StepParams {
 //   s = SiLU(cz + te_next) of the step after that (s is double-buffered, see the host code).
 // With one row per block the kernel is bound by re-reading Win (64 B per column and row) through L1; RB = 4 reads a
 // group's columns once for four rows.  The arithmetic of a row does not depend on RB.
-template <typename ACT, int RB>
+// TRAJ: also record the whole trajectory (every state and every mean), for the single-path ratio of Eq. 2.
+template <typename ACT, int RB, bool TRAJ = false>
 __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p, int mode) {
   __shared__ float xs[RB][kCPad];
   __shared__ float eh[RB][2][kCPad];
@@ -123,6 +126,7 @@ __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p
       if (rr < nrow && c < p.C) {
         v = p.x_src[static_cast<size_t>(r0 + rr) * p.C + c];
         p.x[static_cast<size_t>(r0 + rr) * p.C + c] = v;
+        if (TRAJ) p.traj_x[static_cast<size_t>(r0 + rr) * p.C + c] = v;
       }
       xs[rr][c] = v;
     }
@@ -154,6 +158,7 @@ __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p
           if (p.sample_last && p.x0) p.x0[o] = xn;
         } else {
           p.x[o] = xn;
+          if (TRAJ) { p.traj_x[o] = xn; p.traj_mu[o] = mu; }
         }
       }
       xs[rr][c] = xn;
@@ -211,6 +216,155 @@ __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p
         }
       }
     }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Single-path ratio (Eq. 2): the target head scores the DRAFT's trajectory, so its T evaluations do not depend
+// on one another and several steps are evaluated as one batch of rows.  Token row r' = j * Rin + r of a pass is
+// row r of trajectory slot j0 + j (timestep t = T - j0 - j); with guidance its head rows are r' and Rtok + r'.
+struct BatchParams {
+  int Rin, Rtok, cfg, C, W, NT, T, j0;   // rows per step, token rows of the pass, ..., first trajectory slot
+  float cfg_scale;
+  const float* sched;    // device [5, T] of the target / draft pair: a, b, log-constant, 1/(2 sigma_p^2), 1/(2 sigma_q^2)
+  const float* traj_x;   // [T + 1, Rin, C]: slot j holds x_{T-j}
+  const float* win;      // [W, 16] (zero padded), bin [W]
+  const float* bin;
+  const float* cz;       // [Rin (1 + cfg), W]: one condition projection per row, shared by all steps
+  const float* te;       // [T, W]
+  float* h;              // [Rh, W]
+  float* stats;          // [Rh, W/64, 2]
+  void* s;               // [Rh, W] activations
+  const float* epart;    // [Rh, NT, 16] eps_hat partial sums
+  const float* bout;     // [16]
+  float* mu_p;           // [Rtok, C] out: mean of the target's transition at the draft's state
+};
+
+// Prepares a pass: h = Win x + bin, its LayerNorm partials and s = SiLU(cz + te_t), four token rows per block,
+// with the arithmetic of step_kernel (the same device functions), so a row gets the bits it gets there.
+template <typename ACT>
+__global__ void __launch_bounds__(256) batch_prepare_kernel(BatchParams p) {
+  constexpr int RB = 4;
+  __shared__ float xs[RB][kCPad];
+  const int r0 = blockIdx.x * RB, tid = threadIdx.x;
+  const int nrep = p.cfg ? 2 : 1;
+  const int nrow = min(RB, p.Rtok - r0);
+  griddep_wait();
+  if (tid == 0) griddep_launch_dependents();
+  if (tid < RB * kCPad) {
+    const int rr = tid / kCPad, c = tid % kCPad;
+    float v = 0.0f;
+    if (rr < nrow && c < p.C) v = p.traj_x[(static_cast<size_t>(p.j0) * p.Rin + r0 + rr) * p.C + c];
+    xs[rr][c] = v;
+  }
+  __syncthreads();
+  const int lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
+  ACT* s = reinterpret_cast<ACT*>(p.s);
+  for (int g = warp; g < p.W / kStatCols; g += nwarp) {
+    float wa[kCPad], wb[kCPad];
+    const int na = g * kStatCols + lane, nb = na + 32;
+#pragma unroll
+    for (int c4 = 0; c4 < kCPad / 4; ++c4) {
+      const float4 qa = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(na) * kCPad)[c4];
+      const float4 qb = reinterpret_cast<const float4*>(p.win + static_cast<size_t>(nb) * kCPad)[c4];
+      wa[4 * c4] = qa.x; wa[4 * c4 + 1] = qa.y; wa[4 * c4 + 2] = qa.z; wa[4 * c4 + 3] = qa.w;
+      wb[4 * c4] = qb.x; wb[4 * c4 + 1] = qb.y; wb[4 * c4 + 2] = qb.z; wb[4 * c4 + 3] = qb.w;
+    }
+    const float ba = p.bin[na], bb = p.bin[nb];
+#pragma unroll
+    for (int rr = 0; rr < RB; ++rr) {
+      if (rr >= nrow) break;
+      const int rt = r0 + rr, j = rt / p.Rin, ri = rt - j * p.Rin;
+      const float* te = p.te + static_cast<size_t>(p.T - 1 - p.j0 - j) * p.W;
+      const float te0 = te[na], te1 = te[nb];
+      float acc[2], mean, m2;
+      input_proj_group(wa, wb, ba, bb, xs[rr], acc, mean, m2);
+#pragma unroll
+      for (int rep = 0; rep < 2; ++rep) {
+        if (rep >= nrep) break;
+        const size_t row = static_cast<size_t>(rt) + static_cast<size_t>(rep) * p.Rtok;
+        const size_t zrow = static_cast<size_t>(ri) + static_cast<size_t>(rep) * p.Rin;
+        if (lane == 0)
+          reinterpret_cast<float2*>(p.stats)[row * (p.W / kStatCols) + g] = make_float2(mean, m2);
+        p.h[row * p.W + na] = acc[0];
+        p.h[row * p.W + nb] = acc[1];
+        s[row * p.W + na] = to_act<ACT>(silu_f(__ldg(p.cz + zrow * p.W + na) + te0));
+        s[row * p.W + nb] = to_act<ACT>(silu_f(__ldg(p.cz + zrow * p.W + nb) + te1));
+      }
+    }
+  }
+}
+
+// Finishes a pass: eps_hat = sum of tile partials + bout, guidance, mu^p_t = a_t x_t - b_t eps_hat (Eq. 3 mean),
+// 16 token rows per block of 256 threads (thread = row, coordinate).
+__global__ void __launch_bounds__(256) batch_finish_kernel(BatchParams p) {
+  const int rt = blockIdx.x * 16 + (threadIdx.x >> 4), c = threadIdx.x & 15;
+  griddep_wait();
+  if (rt >= p.Rtok || c >= p.C) return;
+  float e[2] = {0.0f, 0.0f};
+  for (int rep = 0; rep < (p.cfg ? 2 : 1); ++rep) {
+    const float* ep = p.epart + (static_cast<size_t>(rt) + static_cast<size_t>(rep) * p.Rtok) * p.NT * kCPad + c;
+    float acc = 0.0f;
+    for (int nt = 0; nt < p.NT; ++nt) acc += ep[nt * kCPad];
+    e[rep] = acc + p.bout[c];
+  }
+  const float eh = p.cfg ? cfg_combine(e[0], e[1], p.cfg_scale) : e[0];
+  const int ti = p.T - 1 - p.j0 - rt / p.Rin;   // t - 1
+  const float x = p.traj_x[(static_cast<size_t>(p.j0) * p.Rin + rt) * p.C + c];
+  p.mu_p[static_cast<size_t>(rt) * p.C + c] = ddpm_mean(p.sched[ti], x, p.sched[p.T + ti], eh);
+}
+
+// Adds the steps of one pass to the running log-ratio of Eq. 2, one thread per token row, steps in trajectory
+// order (so the sum does not depend on how the steps were split into passes):
+//   term_t = C (log sigma_q,t - log sigma_p,t) - |x_{t-1} - mu^p_t|^2 / (2 sigma_p,t^2) + |x_{t-1} - mu^q_t|^2 / (2 sigma_q,t^2).
+// The two quadratic forms are rounded separately, so identical means give a term of exactly zero.
+__global__ void __launch_bounds__(128)
+single_path_accum_kernel(int Rin, int C, int T, int j0, int nsteps, const float* __restrict__ sched,
+                         const float* __restrict__ traj_x, const float* __restrict__ traj_mu,
+                         const float* __restrict__ mu_p, double* __restrict__ acc, int first) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= Rin) return;
+  double total = first ? 0.0 : acc[r];
+  for (int j = 0; j < nsteps; ++j) {
+    const int ti = T - 1 - j0 - j;
+    const float* xn = traj_x + (static_cast<size_t>(j0 + j + 1) * Rin + r) * C;
+    const float* mq = traj_mu + (static_cast<size_t>(j0 + j) * Rin + r) * C;
+    const float* mp = mu_p + (static_cast<size_t>(j) * Rin + r) * C;
+    float dp = 0.0f, dq = 0.0f;
+    for (int c = 0; c < C; ++c) {
+      const float x = xn[c];
+      const float ep = x - mp[c], eq = x - mq[c];
+      dp = fmaf(ep, ep, dp);
+      dq = fmaf(eq, eq, dq);
+    }
+    const float term = sched[2 * T + ti] + __fsub_rn(__fmul_rn(dq, sched[4 * T + ti]), __fmul_rn(dp, sched[3 * T + ti]));
+    total += static_cast<double>(term);
+  }
+  acc[r] = total;
+}
+
+// Accept test and prefix scan of Alg. 1 on a log-ratio that is already there: one warp per sequence.
+__global__ void __launch_bounds__(128)
+accept_from_logratio_kernel(int B, int gamma, const double* __restrict__ acc, const float* __restrict__ u,
+                            float* __restrict__ logratio, int32_t* __restrict__ n_accept,
+                            uint32_t* __restrict__ accept_mask) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  bool ok = true;
+  if (lane < gamma) {
+    const size_t row = static_cast<size_t>(b) * gamma + lane;
+    const float lr = static_cast<float>(acc[row]);
+    logratio[row] = lr;
+    ok = logf(u[row]) <= lr;
+  }
+  const uint32_t ballot = __ballot_sync(0xffffffffu, ok);
+  if (lane == 0) {
+    const uint32_t rej = ~ballot;
+    int n = rej ? (__ffs(rej) - 1) : gamma;
+    if (n > gamma) n = gamma;
+    n_accept[b] = n;
+    if (accept_mask) accept_mask[b] = (gamma >= 32) ? ballot : (ballot & ((1u << gamma) - 1u));
   }
 }
 

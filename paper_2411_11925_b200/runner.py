@@ -69,6 +69,23 @@ class DeviceRound:
                               float(self.sched_q.sigma[0]), self.n_accept, self.mu1_p, self.mu1_q, self.xi,
                               self.v, self.x_new, self.n_prop, self.flags, self.cap_hits)
 
+    def draft_traj(self):
+        """Draft trajectories with every state and mean recorded (input of the single-path ratio, Eq. 2)."""
+        wl = self.wl
+        if not hasattr(self, "traj_x"):
+            T = len(self.sched_q.sigma)
+            self.traj_x = torch.zeros(T + 1, wl.R, self.C, dtype=torch.float32, device=self.dev)
+            self.traj_mu = torch.zeros(T, wl.R, self.C, dtype=torch.float32, device=self.dev)
+        self.ctx.csd_draft_denoise_traj(self.head_q, self.sched_q, wl.R, wl.cfg, wl.cfg_scale, self.z_q, self.x_T,
+                                        self.eps, self.traj_x, self.traj_mu)
+
+    def verify_single_path(self, steps_per_pass: int = 0, traj_x=None, traj_mu=None):
+        wl = self.wl
+        self.ctx.csd_verify_single_path(self.head_p, self.sched_p, self.sched_q, wl.B, wl.gamma, wl.cfg, wl.cfg_scale,
+                                        self.z_p, self.traj_x if traj_x is None else traj_x,
+                                        self.traj_mu if traj_mu is None else traj_mu, self.u, steps_per_pass,
+                                        self.logratio, self.n_accept, self.accept_mask)
+
     def three_calls(self):
         self.draft(); self.verify(); self.resample()
 

@@ -1,0 +1,242 @@
+"""GPU parity of the exact single-path criterion (Eq. 2): the recorded draft trajectory and the log-ratio that the
+batched target evaluation returns, against the float64 checker on the same seeded inputs."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import csd_oracle as orc
+from paper_2411_11925_b200 import inputs as gen
+
+from _parity import TOL_LOGR, TOL_MU, TOL_X
+
+pytestmark = pytest.mark.gpu
+
+
+def _wl(base="tiny_fp32", **kw):
+    return gen.Workload(**{**gen.WORKLOADS[base].__dict__, **kw})
+
+
+def _device_round(inp, **kw):
+    from paper_2411_11925_b200.runner import DeviceRound
+    return DeviceRound(inp, **kw)
+
+
+def _np(t):
+    return t.cpu().numpy().copy()
+
+
+def _oracle_parts(inp, tau_q=None, tau_p=None):
+    wl = inp.wl
+    sq = orc.ddpm_schedule(inp.beta, wl.tau if tau_q is None else tau_q)
+    sp = orc.ddpm_schedule(inp.beta, wl.tau if tau_p is None else tau_p)
+    eq = orc.make_mlp_head(inp.w_q, inp.z_q, inp.tfeat, wl.cfg, wl.cfg_scale)
+    ep = orc.make_mlp_head(inp.w_p, inp.z_p, inp.tfeat, wl.cfg, wl.cfg_scale)
+    dq = orc.denoise(eq, sq, inp.x_T, inp.eps, sample_last=True, keep=True)
+    return sq, sp, ep, dq
+
+
+def _logr_tolerance(ep, sq, sp, dq, delta_mu):
+    # Each step's term is as ill-conditioned in its mean as Eq. 8 is: d term / d mu = (x_{t-1} - mu) / sigma_t^2.
+    # A per-coordinate error delta_mu in every mean moves the sum by at most
+    # sum_t (sqrt(2 Qp_t) / sigma_p,t + sqrt(2 Qq_t) / sigma_q,t) sqrt(C) delta_mu, Q = |x_{t-1} - mu|^2 / (2 sigma^2).
+    T = len(sq["a"])
+    C = dq["xs"][0].shape[1]
+    cond = 0.0
+    for j in range(T):
+        t = T - j
+        mu_p = sp["a"][t - 1] * dq["xs"][j] - sp["b"][t - 1] * ep(dq["xs"][j], t)
+        rp = np.sqrt(np.sum((dq["xs"][j + 1] - mu_p) ** 2, axis=1)) / sp["sigma"][t - 1] ** 2
+        rq = np.sqrt(np.sum((dq["xs"][j + 1] - dq["mus"][j]) ** 2, axis=1)) / sq["sigma"][t - 1] ** 2
+        cond = cond + (rp + rq) * math.sqrt(C)
+    return TOL_LOGR + cond * delta_mu
+
+
+def _check_scan(dr, wl, u):
+    lr = _np(dr.logratio)
+    mask = _np(dr.accept_mask).astype(np.int64) & 0xFFFFFFFF
+    acc = ((mask[:, None] >> np.arange(wl.gamma)[None, :]) & 1).astype(bool)
+    logu32 = np.log(u.astype(np.float32)).astype(np.float32)
+    knife = np.abs(logu32.astype(np.float64) - lr) < 1e-5
+    assert np.array_equal(acc | knife, (logu32 <= lr) | knife)
+    own = np.array([(list(r) + [False]).index(False) for r in acc])
+    np.testing.assert_array_equal(_np(dr.n_accept), own)
+    return lr, acc
+
+
+CASES = [("f32", dict(B=3, gamma=4, T=10)),
+         ("f32", dict(B=5, gamma=7, T=6, cfg=True, cfg_scale=2.0)),
+         ("f16", dict(B=9, gamma=8, T=8, bf16=True, cfg=True, cfg_scale=3.0)),
+         ("bf16", dict(B=9, gamma=8, T=8, bf16=True, operand="bf16", cfg=True, cfg_scale=3.0)),
+         # 37 * 8 * 2 = 592 head rows per step: several 128-row tiles and a ragged tail in every pass
+         ("f16", dict(B=37, gamma=8, T=5, bf16=True, cfg=True, cfg_scale=3.0, draft=gen.HeadSpec(1, 256, 128),
+                      target=gen.HeadSpec(2, 256, 256)))]
+
+
+@pytest.mark.parametrize("op,kw", CASES)
+def test_recorded_trajectory_matches_checker_and_the_plain_draft_call(op, kw):
+    inp = gen.make_round_inputs(_wl(**kw))
+    wl = inp.wl
+    dr = _device_round(inp)
+    dr.draft()
+    dr.draft_traj()
+    dr.ctx.sync()
+    tx, tm = _np(dr.traj_x), _np(dr.traj_mu)
+    np.testing.assert_array_equal(tx[0], inp.x_T.astype(np.float32))
+    np.testing.assert_array_equal(tx[-1], _np(dr.x0))
+    np.testing.assert_array_equal(tm[-1], _np(dr.mu1_q))
+    np.testing.assert_array_equal(tx[-2], _np(dr.x1_q))
+    _, _, _, dq = _oracle_parts(inp)
+    assert np.max(np.abs(tx - np.stack(dq["xs"]))) <= TOL_X[op]
+    assert np.max(np.abs(tm - np.stack(dq["mus"]))) <= TOL_X[op]
+    dr.ctx.close()
+
+
+@pytest.mark.parametrize("op,kw", CASES)
+def test_single_path_logratio_on_the_checkers_trajectory(op, kw):
+    # The trajectory is an input of the call: give it the checker's (rounded to fp32), so that the comparison
+    # isolates the batched target evaluation and the sum of Eq. 2.
+    inp = gen.make_round_inputs(_wl(**kw))
+    wl = inp.wl
+    sq, sp, ep, dq = _oracle_parts(inp, tau_p=0.9 * wl.tau)
+    dq32 = {"xs": [x.astype(np.float32).astype(np.float64) for x in dq["xs"]],
+            "mus": [m.astype(np.float32).astype(np.float64) for m in dq["mus"]]}
+    want = orc.log_ratio_single_path(ep, sq, sp, dq32).reshape(wl.B, wl.gamma)
+    tol = _logr_tolerance(ep, sq, sp, dq32, TOL_MU[op]).reshape(wl.B, wl.gamma)
+    dr = _device_round(inp, tau_p=0.9 * wl.tau)
+    tx = torch.from_numpy(np.stack(dq32["xs"]).astype(np.float32)).to(dr.dev)
+    tm = torch.from_numpy(np.stack(dq32["mus"]).astype(np.float32)).to(dr.dev)
+    from paper_2411_11925_b200 import api
+    for mode in (api.Context.CHAIN_LAYERS, api.Context.CHAIN_LAYERS_PLAIN):
+        dr.ctx.set_chain_mode(mode)
+        first = None
+        for spp in (0, 1, 3, wl.T):
+            dr.verify_single_path(spp, tx, tm)
+            dr.ctx.sync()
+            lr, acc = _check_scan(dr, wl, inp.u)
+            err = np.abs(lr - want)
+            assert np.all(err <= tol), (op, mode, spp, float(err.max()), float((err / tol).max()))
+            if op == "f32":
+                assert err.max() <= TOL_LOGR   # the fp32 path meets the flat stated tolerance
+            if first is None:
+                first = lr
+                print(op, kw, "mode", mode, "single-path logR err", float(err.max()), "of tol", float((err / tol).max()),
+                      "median |logR|", float(np.median(np.abs(want))))
+            elif mode == api.Context.CHAIN_LAYERS_PLAIN:
+                # with the three-kernel blocks a row's bits do not depend on the row count of a pass, and the steps
+                # are summed in trajectory order: the split into passes does not change a bit
+                np.testing.assert_array_equal(lr, first)
+            n_ref, acc_ref = orc.accept_prefix(want, inp.u)
+            in_band = np.abs(want - np.log(inp.u.astype(np.float64))) <= tol
+            assert not np.any((acc != acc_ref) & ~in_band)
+    dr.ctx.close()
+
+
+@pytest.mark.parametrize("op,kw", CASES[:4])
+def test_single_path_end_to_end_matches_checker(op, kw):
+    inp = gen.make_round_inputs(_wl(**kw))
+    wl = inp.wl
+    sq, sp, ep, dq = _oracle_parts(inp)
+    want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(wl.B, wl.gamma)
+    # here the target also sees the accumulated error of the draft's trajectory: delta = the trajectory tolerance
+    tol = _logr_tolerance(ep, sq, sp, dq, TOL_X[op] + TOL_MU[op]).reshape(wl.B, wl.gamma)
+    dr = _device_round(inp)
+    dr.draft_traj()
+    dr.verify_single_path()
+    dr.ctx.sync()
+    lr, acc = _check_scan(dr, wl, inp.u)
+    err = np.abs(lr - want)
+    print(op, kw, "end-to-end single-path logR err", float(err.max()), "of tol", float((err / tol).max()))
+    assert np.all(err <= tol)
+    if op == "f32":
+        assert err.max() <= TOL_LOGR
+    dr.ctx.close()
+
+
+@pytest.mark.parametrize("op", ["f32", "bf16", "f16"])
+def test_identical_heads_give_exactly_zero_single_path_ratio(op):
+    # Eq. 2 with p = q is 1.  The three-kernel block layout returns the same bits whatever the row count, so the
+    # batched target evaluation reproduces the draft's means exactly and every step's term is exactly 0.
+    from paper_2411_11925_b200 import api
+    wl = _wl(B=6, gamma=5, T=8, bf16=op != "f32", operand=op, cfg=True, cfg_scale=3.0, draft=gen.HeadSpec(2, 256, 256))
+    inp = gen.make_round_inputs(wl)
+    inp.w_q, inp.z_q = inp.w_p, inp.z_p
+    dr = _device_round(inp)
+    dr.ctx.set_chain_mode(api.Context.CHAIN_LAYERS_PLAIN)
+    dr.draft_traj()
+    dr.verify_single_path(3)
+    dr.ctx.sync()
+    assert np.all(_np(dr.logratio) == 0.0)
+    assert np.all(_np(dr.n_accept) == wl.gamma)
+    dr.ctx.close()
+
+
+def test_close_heads_fp32_single_path_ratio_is_tight():
+    # Target = draft + small perturbation: log-ratios of order 1..100, where the flat tolerance is meaningful.
+    wl = _wl(B=8, gamma=4, T=10)
+    inp = gen.make_round_inputs(wl)
+    rng = np.random.default_rng(7)
+    inp.w_q = gen.perturb_head_weights(inp.w_p, rng, 0.002)
+    inp.z_q = inp.z_p
+    sq, sp, ep, dq = _oracle_parts(inp)
+    want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(wl.B, wl.gamma)
+    dr = _device_round(inp)
+    dr.draft_traj()
+    dr.verify_single_path()
+    dr.ctx.sync()
+    lr = _np(dr.logratio)
+    err = np.abs(lr - want)
+    print("close heads fp32: median |logR|", float(np.median(np.abs(want))), "max err", float(err.max()))
+    assert np.all(err <= TOL_LOGR + 1e-3 * np.abs(want))
+    dr.ctx.close()
+
+
+def test_single_path_argument_checks():
+    from paper_2411_11925_b200 import api
+    inp = gen.make_round_inputs(_wl(B=2, gamma=3, T=4))
+    dr = _device_round(inp)
+    dr.draft_traj()
+    with pytest.raises(api.CsdError) as e:
+        dr.ctx.csd_verify_single_path(dr.head_p, dr.sched_p, dr.sched_q, 2, 3, 0, 1.0, dr.z_p, None, dr.traj_mu, dr.u,
+                                      0, dr.logratio, dr.n_accept)
+    assert e.value.code == -1
+    with pytest.raises(api.CsdError) as e:
+        dr.verify_single_path(-1)
+    assert e.value.code == -1
+    with pytest.raises(api.CsdError) as e:
+        dr.ctx.csd_verify_single_path(dr.head_p, dr.sched_p, dr.sched_q, 2, 33, 0, 1.0, dr.z_p, dr.traj_x, dr.traj_mu,
+                                      dr.u, 0, dr.logratio, dr.n_accept)
+    assert e.value.code == -3
+    dr.ctx.sync()
+    dr.ctx.close()
+
+
+def test_mar256_full_size_single_path_sampled_sequences():
+    # The benchmark's configuration (B=64, gamma=8, T=100, guidance, 32 steps = 32768 head rows per pass); the
+    # checker evaluates two sequences end to end.
+    wl = gen.WORKLOADS["mar256"]
+    inp = gen.make_round_inputs(wl)
+    dr = _device_round(inp)
+    dr.draft_traj()
+    dr.verify_single_path()
+    dr.ctx.sync()
+    lr, acc = _check_scan(dr, wl, inp.u)
+    assert np.all(np.isfinite(lr))
+    seqs = [0, 63]
+    sub = gen.select_sequences(inp, seqs)
+    sq, sp, ep, dq = _oracle_parts(sub)
+    want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(len(seqs), wl.gamma)
+    op = wl.operand_format
+    tol = _logr_tolerance(ep, sq, sp, dq, TOL_X[op] + TOL_MU[op]).reshape(len(seqs), wl.gamma)
+    rows = sub.extras["rows"]
+    assert np.max(np.abs(_np(dr.traj_x)[:, rows] - np.stack(dq["xs"]))) <= TOL_X[op]
+    err = np.abs(lr[seqs] - want)
+    print("mar256 single-path: max err", float(err.max()), "of tol", float((err / tol).max()),
+          "median |logR|", float(np.median(np.abs(want))))
+    assert np.all(err <= tol)
+    # a second call repeats bit for bit
+    dr.verify_single_path()
+    dr.ctx.sync()
+    np.testing.assert_array_equal(_np(dr.logratio), lr)
+    dr.ctx.close()
