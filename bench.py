@@ -270,6 +270,25 @@ def run_ours(args):
                    "algorithmic_tflops": fl * pre_steps / pre_secs / 1e12,
                    "frac_of_tensor_peak": fl * pre_steps / pre_secs / 1e12 / peaks["tflops_sustained"]}
 
+    # Exact single-path criterion (Eq. 2): the target scores the draft's recorded trajectory.  Its T evaluations are
+    # independent rows, so the call is throughput-bound: reported against the tensor roofline with algorithmic
+    # FLOPs = (1 + cfg) R T F_target.
+    single = None
+    if world == 1 and not args.no_seq:
+        r0 = rounds[0]
+        r0.draft_traj()
+        sp_step = lambda i: r0.verify_single_path()
+        timed(sp_step, 2)
+        l1 = ctx.launch_count()
+        sp_steps = max(2, min(args.steps, 5))
+        sp_secs = timed(sp_step, sp_steps)
+        t = wl.target
+        fl = (2 if wl.cfg else 1) * wl.R * wl.T * 2.0 * (2 * t.C * t.W + 5 * t.L * t.W * t.W + 2 * t.W * t.W)
+        single = {"call": "csd_verify_single_path", "ms": 1e3 * sp_secs / sp_steps, "value": wl.R * sp_steps / sp_secs,
+                  "unit": "verified tokens/s", "launches_per_call": int((ctx.launch_count() - l1) // sp_steps),
+                  "bound": "tensor", "achieved": fl * sp_steps / sp_secs / 1e12, "peak": peaks["tflops_sustained"],
+                  "roofline_unit": "TFLOP/s", "frac": fl * sp_steps / sp_secs / 1e12 / peaks["tflops_sustained"]}
+
     # per-kernel-class device time over the same steps (events around every launch: separate pass)
     prof = None
     if not args.no_profile:
@@ -324,6 +343,8 @@ def run_ours(args):
             line["sequential_draft"] = seq
         if prefill:
             line["prefill"] = prefill
+        if single:
+            line["single_path"] = single
         if not args.no_cpu_baseline and world == 1:
             val, threads, desc, _ = time_oracle(args.workload, 15.0)
             line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
