@@ -372,6 +372,8 @@ struct Chain {
   // batched evaluation on a given trajectory (csd_verify_single_path): R = batch_steps * batch_Rin token rows,
   // one pass of the layers; slot batch_j0 of batch_traj is the first step of the pass
   int batch_Rin = 0, batch_j0 = 0, Ts = 0;
+  int ws_steps = 0;          // steps the workspace is carved for (the same for every pass of a call, so that the
+  bool batch_reuse = false;  // timestep embedding and the condition projection of the first pass stay where they are)
   const float *batch_traj = nullptr, *batch_sched = nullptr;
   float* batch_mu = nullptr;
 
@@ -466,25 +468,27 @@ struct Chain {
              8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && fold_kernels_ready(d);
     }
     ChainWs& ws = ctx->ws[slot];
-    int rc = ensure_ws(ctx, ws, d, Rh, R, Ts, whole);
+    int rc = batch_Rin ? ensure_ws(ctx, ws, d, ws_steps * batch_Rin * (cfg ? 2 : 1), ws_steps * batch_Rin, Ts, false)
+                       : ensure_ws(ctx, ws, d, Rh, R, Ts, whole);
     if (rc) return rc;
-    {
+    if (!batch_reuse) {
       const dim3 grid((W + 31) / 32, (Ts + 31) / 32);
       small_gemm_nt_kernel<true><<<grid, 256, 0, st>>>(sc->tfeat, hd->Wt1, hd->bt1, ws.hid, Ts, W, d.F);
       small_gemm_nt_kernel<false><<<grid, 256, 0, st>>>(ws.hid, hd->Wt2, hd->bt2, ws.te, Ts, W, W);
-      ctx->launches++;
+      ctx->launches += 2;
     }
-    ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
     ep.M = Rh; ep.ldo = W;
     // rows of z: one per head row, or one per row of a step when the steps of a trajectory are batched
     const int Rz = batch_Rin ? batch_Rin * (cfg ? 2 : 1) : Rh;
     if (tc) {
-      const size_t nz = static_cast<size_t>(Rz) * d.Dz;
-      const unsigned nblk = static_cast<unsigned>((nz + 255) / 256);
-      if (d.dtype == CSD_F16) convert_act_kernel<__half><<<nblk, 256, 0, st>>>(z, static_cast<__half*>(ws.zc), nz);
-      else convert_act_kernel<__nv_bfloat16><<<nblk, 256, 0, st>>>(z, static_cast<__nv_bfloat16*>(ws.zc), nz);
-      ctx->launches++;
+      if (!batch_reuse) {
+        const size_t nz = static_cast<size_t>(Rz) * d.Dz;
+        const unsigned nblk = static_cast<unsigned>((nz + 255) / 256);
+        if (d.dtype == CSD_F16) convert_act_kernel<__half><<<nblk, 256, 0, st>>>(z, static_cast<__half*>(ws.zc), nz);
+        else convert_act_kernel<__nv_bfloat16><<<nblk, 256, 0, st>>>(z, static_cast<__nv_bfloat16*>(ws.zc), nz);
+        ctx->launches++;
+      }
       if ((rc = make_tmap(ctx, &tm_z, d.dtype, ws.zc, Rz, d.Dz, d.Dz, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_sb[1], d.dtype, ws.s, Rh, W, W, kTileM))) return rc;
       if ((rc = make_tmap(ctx, &tm_sb[0], d.dtype, ws.s2, Rh, W, W, kTileM))) return rc;
@@ -498,7 +502,8 @@ struct Chain {
     EpiParams e = ep;
     e.M = Rz;
     e.bias0 = hd->bz; e.out_f32 = ws.cz;
-    if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 1>(ctx, d.dtype, tn, pair, st, tm_z, tmw.Wz, tm_z, tmw.Wz, tm_h, d.Dz, 0, 0, W, e);
+    if (batch_reuse) rc = CSD_OK;
+    else if (tc) rc = launch_tc<EPI_BIAS_F32, 1, 1>(ctx, d.dtype, tn, pair, st, tm_z, tmw.Wz, tm_z, tmw.Wz, tm_h, d.Dz, 0, 0, W, e);
     else rc = launch_simt<EPI_BIAS_F32, 1, 128>(ctx, st, z, d.Dz, static_cast<const float*>(hd->Wz), d.Dz, nullptr, 0,
                                                 nullptr, 0, W, e);
     if (rc) return rc;
@@ -1181,10 +1186,10 @@ int csd_verify_single_path(csd_ctx* ctx, const csd_head* head_p, const csd_sched
   int tb = steps_per_pass ? steps_per_pass : (kRowsPerPass + Rh1 - 1) / Rh1;
   if (tb > T) tb = T;
   if (static_cast<int64_t>(tb) * Rh1 > (int64_t(1) << 26)) return fail(ctx, CSD_ERR_UNSUPPORTED, "pass of %d steps has too many rows", tb);
-  // device side buffer: [5, T] constants | mu^p of a pass [tb R, C] | running sum [R] (double)
+  // device side buffer: [5, T] constants | mu^p of a pass [tb R, C] | per-step terms [T, R]
   const size_t o_mu = align_up(static_cast<size_t>(5) * T * 4, 256);
   const size_t o_acc = align_up(o_mu + static_cast<size_t>(tb) * R * C * 4, 256);
-  const size_t need = o_acc + static_cast<size_t>(R) * 8;
+  const size_t need = o_acc + static_cast<size_t>(T) * R * 4;
   cudaStream_t st = ctx->stream;
   if (need > ctx->sp.cap) {
     CSD_CUDA(ctx, cudaStreamSynchronize(st));
@@ -1199,7 +1204,7 @@ int csd_verify_single_path(csd_ctx* ctx, const csd_head* head_p, const csd_sched
   char* base = static_cast<char*>(ctx->sp.base);
   float* d_sched = reinterpret_cast<float*>(base);
   float* d_mu = reinterpret_cast<float*>(base + o_mu);
-  double* d_acc = reinterpret_cast<double*>(base + o_acc);
+  float* d_terms = reinterpret_cast<float*>(base + o_acc);
   {
     // per step: a_t, b_t of the target, C (log sigma_q,t - log sigma_p,t), 1 / (2 sigma_p,t^2), 1 / (2 sigma_q,t^2)
     std::vector<float> hs(static_cast<size_t>(5) * T);
@@ -1218,14 +1223,14 @@ int csd_verify_single_path(csd_ctx* ctx, const csd_head* head_p, const csd_sched
     Chain c{ctx, 1, st, head_p, sched_p, n * R, cfg, cfg_scale, z_p, nullptr, nullptr, 0, nullptr, nullptr, nullptr};
     c.allow_chain_kernel = false;
     c.batch_Rin = R; c.batch_j0 = j0; c.batch_traj = traj_x; c.batch_sched = d_sched; c.batch_mu = d_mu;
+    c.ws_steps = tb; c.batch_reuse = j0 > 0;
     if ((rc = c.begin())) return rc;
     if ((rc = c.step(1))) return rc;
-    single_path_accum_kernel<<<(R + 127) / 128, 128, 0, st>>>(R, C, T, j0, n, d_sched, traj_x, traj_mu_q, d_mu, d_acc,
-                                                              j0 == 0 ? 1 : 0);
+    single_path_terms_kernel<<<(n * R + 127) / 128, 128, 0, st>>>(R, C, T, j0, n, d_sched, traj_x, traj_mu_q, d_mu, d_terms);
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
   }
-  accept_from_logratio_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, gamma, d_acc, u, logratio, n_accept, accept_mask);
+  single_path_accept_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, gamma, T, d_terms, u, logratio, n_accept, accept_mask);
   ctx->launches++;
   CSD_CUDA(ctx, cudaGetLastError());
   return CSD_OK;

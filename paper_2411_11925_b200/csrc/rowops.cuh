@@ -271,25 +271,37 @@ __global__ void __launch_bounds__(256) batch_prepare_kernel(BatchParams p) {
       wb[4 * c4] = qb.x; wb[4 * c4 + 1] = qb.y; wb[4 * c4 + 2] = qb.z; wb[4 * c4 + 3] = qb.w;
     }
     const float ba = p.bin[na], bb = p.bin[nb];
+    // every cz and te value of the group first: independent loads in flight together (one trip to memory per
+    // group instead of one per row)
+    float czv[RB][2][2], tev[RB][2];
+#pragma unroll
+    for (int rr = 0; rr < RB; ++rr) {
+      const int rt = min(r0 + rr, p.Rtok - 1), j = rt / p.Rin, ri = rt - j * p.Rin;
+      const float* te = p.te + static_cast<size_t>(p.T - 1 - p.j0 - j) * p.W;
+      tev[rr][0] = te[na]; tev[rr][1] = te[nb];
+#pragma unroll
+      for (int rep = 0; rep < 2; ++rep) {
+        const size_t zrow = static_cast<size_t>(ri) + static_cast<size_t>(rep < nrep ? rep : 0) * p.Rin;
+        czv[rr][rep][0] = __ldg(p.cz + zrow * p.W + na);
+        czv[rr][rep][1] = __ldg(p.cz + zrow * p.W + nb);
+      }
+    }
 #pragma unroll
     for (int rr = 0; rr < RB; ++rr) {
       if (rr >= nrow) break;
-      const int rt = r0 + rr, j = rt / p.Rin, ri = rt - j * p.Rin;
-      const float* te = p.te + static_cast<size_t>(p.T - 1 - p.j0 - j) * p.W;
-      const float te0 = te[na], te1 = te[nb];
+      const int rt = r0 + rr;
       float acc[2], mean, m2;
       input_proj_group(wa, wb, ba, bb, xs[rr], acc, mean, m2);
 #pragma unroll
       for (int rep = 0; rep < 2; ++rep) {
         if (rep >= nrep) break;
         const size_t row = static_cast<size_t>(rt) + static_cast<size_t>(rep) * p.Rtok;
-        const size_t zrow = static_cast<size_t>(ri) + static_cast<size_t>(rep) * p.Rin;
         if (lane == 0)
           reinterpret_cast<float2*>(p.stats)[row * (p.W / kStatCols) + g] = make_float2(mean, m2);
         p.h[row * p.W + na] = acc[0];
         p.h[row * p.W + nb] = acc[1];
-        s[row * p.W + na] = to_act<ACT>(silu_f(__ldg(p.cz + zrow * p.W + na) + te0));
-        s[row * p.W + nb] = to_act<ACT>(silu_f(__ldg(p.cz + zrow * p.W + nb) + te1));
+        s[row * p.W + na] = to_act<ACT>(silu_f(czv[rr][rep][0] + tev[rr][0]));
+        s[row * p.W + nb] = to_act<ACT>(silu_f(czv[rr][rep][1] + tev[rr][1]));
       }
     }
   }
@@ -314,47 +326,47 @@ __global__ void __launch_bounds__(256) batch_finish_kernel(BatchParams p) {
   p.mu_p[static_cast<size_t>(rt) * p.C + c] = ddpm_mean(p.sched[ti], x, p.sched[p.T + ti], eh);
 }
 
-// Adds the steps of one pass to the running log-ratio of Eq. 2, one thread per token row, steps in trajectory
-// order (so the sum does not depend on how the steps were split into passes):
+// Per-step terms of the log-ratio of Eq. 2 for the steps of one pass, one thread per (step, token row):
 //   term_t = C (log sigma_q,t - log sigma_p,t) - |x_{t-1} - mu^p_t|^2 / (2 sigma_p,t^2) + |x_{t-1} - mu^q_t|^2 / (2 sigma_q,t^2).
 // The two quadratic forms are rounded separately, so identical means give a term of exactly zero.
 __global__ void __launch_bounds__(128)
-single_path_accum_kernel(int Rin, int C, int T, int j0, int nsteps, const float* __restrict__ sched,
+single_path_terms_kernel(int Rin, int C, int T, int j0, int nsteps, const float* __restrict__ sched,
                          const float* __restrict__ traj_x, const float* __restrict__ traj_mu,
-                         const float* __restrict__ mu_p, double* __restrict__ acc, int first) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= Rin) return;
-  double total = first ? 0.0 : acc[r];
-  for (int j = 0; j < nsteps; ++j) {
-    const int ti = T - 1 - j0 - j;
-    const float* xn = traj_x + (static_cast<size_t>(j0 + j + 1) * Rin + r) * C;
-    const float* mq = traj_mu + (static_cast<size_t>(j0 + j) * Rin + r) * C;
-    const float* mp = mu_p + (static_cast<size_t>(j) * Rin + r) * C;
-    float dp = 0.0f, dq = 0.0f;
-    for (int c = 0; c < C; ++c) {
-      const float x = xn[c];
-      const float ep = x - mp[c], eq = x - mq[c];
-      dp = fmaf(ep, ep, dp);
-      dq = fmaf(eq, eq, dq);
-    }
-    const float term = sched[2 * T + ti] + __fsub_rn(__fmul_rn(dq, sched[4 * T + ti]), __fmul_rn(dp, sched[3 * T + ti]));
-    total += static_cast<double>(term);
+                         const float* __restrict__ mu_p, float* __restrict__ terms) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= nsteps * Rin) return;
+  const int j = i / Rin, r = i - j * Rin;
+  const int ti = T - 1 - j0 - j;
+  const float* xn = traj_x + (static_cast<size_t>(j0 + j + 1) * Rin + r) * C;
+  const float* mq = traj_mu + (static_cast<size_t>(j0 + j) * Rin + r) * C;
+  const float* mp = mu_p + static_cast<size_t>(i) * C;
+  float dp = 0.0f, dq = 0.0f;
+  for (int c = 0; c < C; ++c) {
+    const float x = xn[c];
+    const float ep = x - mp[c], eq = x - mq[c];
+    dp = fmaf(ep, ep, dp);
+    dq = fmaf(eq, eq, dq);
   }
-  acc[r] = total;
+  terms[static_cast<size_t>(j0 + j) * Rin + r] =
+      sched[2 * T + ti] + __fsub_rn(__fmul_rn(dq, sched[4 * T + ti]), __fmul_rn(dp, sched[3 * T + ti]));
 }
 
-// Accept test and prefix scan of Alg. 1 on a log-ratio that is already there: one warp per sequence.
+// Sum of the T terms in trajectory order (in double, so the order of magnitude of the early terms does not cost the
+// late ones their digits), then the accept test and prefix scan of Alg. 1: one warp per sequence.
 __global__ void __launch_bounds__(128)
-accept_from_logratio_kernel(int B, int gamma, const double* __restrict__ acc, const float* __restrict__ u,
-                            float* __restrict__ logratio, int32_t* __restrict__ n_accept,
-                            uint32_t* __restrict__ accept_mask) {
+single_path_accept_kernel(int B, int gamma, int T, const float* __restrict__ terms, const float* __restrict__ u,
+                          float* __restrict__ logratio, int32_t* __restrict__ n_accept,
+                          uint32_t* __restrict__ accept_mask) {
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (b >= B) return;
   bool ok = true;
   if (lane < gamma) {
     const size_t row = static_cast<size_t>(b) * gamma + lane;
-    const float lr = static_cast<float>(acc[row]);
+    const size_t R = static_cast<size_t>(B) * gamma;
+    double total = 0.0;
+    for (int j = 0; j < T; ++j) total += static_cast<double>(terms[j * R + row]);
+    const float lr = static_cast<float>(total);
     logratio[row] = lr;
     ok = logf(u[row]) <= lr;
   }
