@@ -373,6 +373,31 @@ def test_single_path_ratio_matches_multivariate_normal_path_densities():
         assert abs(got[r] - want) < 1e-8 * max(1.0, abs(want))
 
 
+def test_unaligned_long_product_matches_multivariate_normal_path_densities():
+    # Ablation without trajectory alignment (the target draws its own noise): p(Y_p)/q(Y_q) of Eq. 4 is the joint
+    # density of the target's path (ending in the draft's x_0) under p over that of the draft's path under q; with toy
+    # heads both joints are multivariate normal (scipy), no per-step terms involved.
+    T = 7
+    beta = gen.beta_linear(T, 0.01, 0.2)
+    tau_q, tau_p = 1.0, 0.9
+    sq, sp = orc.ddpm_schedule(beta, tau_q), orc.ddpm_schedule(beta, tau_p)
+    eq = orc.make_gaussian_toy_head(0.4, 0.6, sq["alphabar"])
+    ep = orc.make_gaussian_toy_head(-0.2, 0.9, sp["alphabar"])
+    rng = np.random.default_rng(43)
+    N = 5
+    x_T = rng.standard_normal((N, 1))
+    noise, noise_p = rng.standard_normal((T, N, 1)), rng.standard_normal((T, N, 1))
+    dq, dp = orc.run_pair(eq, ep, sq, sp, x_T, noise, noise_p=noise_p, keep=True)
+    got = orc.log_ratio_long(dq, dp, sq, sp)
+    for r in range(N):
+        yq = np.array([dq["xs"][j + 1][r, 0] for j in range(T)])
+        yp = np.array([dp["xs"][j + 1][r, 0] for j in range(T - 1)] + [dq["x0"][r, 0]])
+        mq, cq = _toy_path_gaussian(0.4, 0.6, tau_q, beta, x_T[r, 0])
+        mp, cp = _toy_path_gaussian(-0.2, 0.9, tau_p, beta, x_T[r, 0])
+        want = st.multivariate_normal(mp, cp).logpdf(yp) - st.multivariate_normal(mq, cq).logpdf(yq)
+        assert abs(got[r] - want) < 1e-8 * max(1.0, abs(want))
+
+
 def test_single_path_ratio_has_unit_expectation_under_the_draft():
     # E_{Y ~ q}[p(Y)/q(Y)] = 1 (importance-weight identity stated with the bias analysis of the surrogate ratio);
     # a dropped step, a wrong sign or a wrong variance in Eq. 2 breaks it.
