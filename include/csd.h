@@ -200,6 +200,20 @@ int csd_accept_scan(csd_ctx *ctx, int B, int gamma, int C, double log_sigma_term
                     float sigma1_q, const float *x0_q, const float *mu1_q, const float *mu1_p,
                     const float *u, float *logratio, int32_t *n_accept, uint32_t *accept_mask);
 
+/* Verification WITHOUT denoising trajectory alignment (the ablation of the paper's alignment study:
+ * the target draws its own noise).  As csd_verify, but the target's chain uses eps_p while the
+ * draft's used eps_q, so the per-step exponentials of Eq. 4 no longer cancel into Eq. 7/8: with
+ * x^m_{t-1} - mu^m_t = sigma_m,t eps^m_t,
+ *   logratio = [Eq. 8 evaluated with this target's mu1_p]
+ *              + sum_{t=2..T} (|eps^q_t|^2 - |eps^p_t|^2) / 2.
+ * With eps_p == eps_q the extra sum is exactly 0 and the call returns csd_verify's bits.
+ *   eps_p, eps_q device [T, B*gamma, C]; everything else as in csd_verify. */
+int csd_verify_unaligned(csd_ctx *ctx, const csd_head *head_p, const csd_schedule *sched_p,
+                         const csd_schedule *sched_q, int B, int gamma, int cfg, float cfg_scale,
+                         const float *z_p, const float *x_T, const float *eps_p, const float *eps_q,
+                         const float *x0_q, const float *mu1_q, const float *u, float *logratio,
+                         int32_t *n_accept, uint32_t *accept_mask, float *mu1_p);
+
 /* ---- Exact single-path criterion (Eq. 2; Table 1 "p(Y_q)/q(Y_q)") ------------------------------
  * Eq. 2 scores the DRAFT's own trajectory Y_q = (x_T, x^q_{T-1}, ..., x^q_0) under both models:
  *   log p(Y_q)/q(Y_q) = sum_{t=1..T} [ log N(x^q_{t-1}; mu^p_t(x^q_t), sigma_p,t^2 I)

@@ -26,7 +26,7 @@ EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launc
            "csd_set_chain_mode", "csd_profile", "csd_profile_read",
            "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_draft_denoise_static", "csd_verify",
            "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host", "csd_draft_denoise_traj",
-           "csd_verify_single_path")
+           "csd_verify_single_path", "csd_verify_unaligned")
 
 WEIGHT_FIELDS = ("Wz", "bz", "Wt1", "bt1", "Wt2", "bt2", "Win", "bin", "Wada", "bada",
                  "W1", "b1", "W2", "b2", "Wfada", "bfada", "Wout", "bout")
@@ -74,6 +74,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_draft_denoise_traj.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, f32] + [vp] * 5
     lib.csd_verify_single_path.argtypes = ([vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32]
                                            + [vp] * 4 + [i32] + [vp] * 3)
+    lib.csd_verify_unaligned.argtypes = ([vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32]
+                                         + [vp] * 11)
     lib.csd_accept_scan.argtypes = [vp, i32, i32, i32, f64, f32, f32] + [vp] * 7
     lib.csd_resample.argtypes = [vp, i32, i32, i32, i32, f64, f32, f32] + [vp] * 9
     round_args = [vp, vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32, i32] + [vp] * 17
@@ -210,6 +212,13 @@ class Context:
                                                 int(cfg), cfg_scale, _ptr(z_p), _ptr(traj_x), _ptr(traj_mu_q),
                                                 _ptr(u), int(steps_per_pass), _ptr(logratio), _ptr(n_accept),
                                                 _ptr(accept_mask)))
+
+    def csd_verify_unaligned(self, head_p: "Head", sched_p: Schedule, sched_q: Schedule, B, gamma, cfg, cfg_scale,
+                             z_p, x_T, eps_p, eps_q, x0_q, mu1_q, u, logratio, n_accept, accept_mask, mu1_p):
+        self._check(_LIB.csd_verify_unaligned(self._h, head_p._h, C.byref(sched_p.c), C.byref(sched_q.c), B, gamma,
+                                              int(cfg), cfg_scale, _ptr(z_p), _ptr(x_T), _ptr(eps_p), _ptr(eps_q),
+                                              _ptr(x0_q), _ptr(mu1_q), _ptr(u), _ptr(logratio), _ptr(n_accept),
+                                              _ptr(accept_mask), _ptr(mu1_p)))
 
     def csd_accept_scan(self, B, gamma, Cdim, log_sigma, sigma1_p, sigma1_q, x0_q, mu1_q, mu1_p, u, logratio,
                         n_accept, accept_mask=None):

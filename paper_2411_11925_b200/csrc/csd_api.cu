@@ -63,6 +63,7 @@ struct csd_ctx {
   EncodeTiledFn encode = nullptr;
   ChainWs ws[3];   // draft chain, target chain, static-scratch calls
   HostIo io;
+  HostIo un;       // csd_verify_unaligned: per-row noise terms
   HostIo sp;       // csd_verify_single_path: schedule constants, mu^p of one pass, running log-ratio
   char err[512] = {0};
   // optional per-launch timing (csd_profile)
@@ -702,12 +703,12 @@ double log_sigma_term(const csd_schedule* q, const csd_schedule* p, int C) {
 
 int accept_scan(csd_ctx* ctx, cudaStream_t st, int B, int gamma, int C, double log_sigma, float sp1, float sq1,
                 const float* x0, const float* mu_q, const float* mu_p, const float* u, float* logratio,
-                int32_t* n_accept, uint32_t* mask) {
+                int32_t* n_accept, uint32_t* mask, const float* offset = nullptr) {
   const double lc = log_sigma + C * (std::log(static_cast<double>(sq1)) - std::log(static_cast<double>(sp1)));
   const float inv2vp = static_cast<float>(0.5 / (static_cast<double>(sp1) * sp1));
   const float inv2vq = static_cast<float>(0.5 / (static_cast<double>(sq1) * sq1));
   accept_scan_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, gamma, C, static_cast<float>(lc), inv2vp, inv2vq, x0, mu_q, mu_p, u,
-                                                  logratio, n_accept, mask);
+                                                  logratio, n_accept, mask, offset);
   ctx->launches++;
   CSD_CUDA(ctx, cudaGetLastError());
   return CSD_OK;
@@ -794,6 +795,7 @@ int csd_destroy(csd_ctx* c) {
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->io.base) cudaFree(c->io.base);
   if (c->sp.base) cudaFree(c->sp.base);
+  if (c->un.base) cudaFree(c->un.base);
   if (c->d_err) cudaFree(c->d_err);
   cudaGetLastError();
   delete c;
@@ -1141,6 +1143,41 @@ int csd_verify(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p
   const int C = head_p->d.C;
   return accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term(sched_q, sched_p, C), sched_p->sigma[0],
                      sched_q->sigma[0], x0_q, mu1_q, mu1_p, u, logratio, n_accept, accept_mask);
+}
+
+int csd_verify_unaligned(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p, const csd_schedule* sched_q,
+                         int B, int gamma, int cfg, float cfg_scale, const float* z_p, const float* x_T,
+                         const float* eps_p, const float* eps_q, const float* x0_q, const float* mu1_q, const float* u,
+                         float* logratio, int32_t* n_accept, uint32_t* accept_mask, float* mu1_p) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
+  int rc = check_chain_args(ctx, head_p, sched_p, B * gamma, cfg, z_p, x_T, eps_p);
+  if (rc) return rc;
+  if ((rc = check_sched(ctx, sched_q, false))) return rc;
+  if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
+  if ((rc = check_verify_dims(ctx, B, gamma, head_p->d.C))) return rc;
+  if (!eps_q || !x0_q || !mu1_q || !u || !logratio || !n_accept || !mu1_p) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  const int R = B * gamma, C = head_p->d.C, T = sched_p->T;
+  const size_t need = static_cast<size_t>(R) * 4;
+  if (need > ctx->un.cap) {
+    CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (ctx->un.base) CSD_CUDA(ctx, cudaFree(ctx->un.base));
+    ctx->un.base = nullptr; ctx->un.cap = 0;
+    if (cudaMalloc(&ctx->un.base, need) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes for the noise terms", need);
+    }
+    ctx->un.cap = need;
+  }
+  float* d_off = static_cast<float*>(ctx->un.base);
+  rc = run_chain(ctx, 1, ctx->stream, head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps_p, 0, nullptr, mu1_p, nullptr);
+  if (rc) return rc;
+  noise_norm_term_kernel<<<(R + 127) / 128, 128, 0, ctx->stream>>>(R, C, T, eps_q, eps_p, d_off);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term(sched_q, sched_p, C), sched_p->sigma[0],
+                     sched_q->sigma[0], x0_q, mu1_q, mu1_p, u, logratio, n_accept, accept_mask, d_off);
 }
 
 int csd_draft_denoise_traj(csd_ctx* ctx, const csd_head* head, const csd_schedule* sched, int R, int cfg,

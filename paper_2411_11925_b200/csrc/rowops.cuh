@@ -389,7 +389,7 @@ accept_scan_kernel(int B, int gamma, int C, float log_const, float inv2vp, float
                    const float* __restrict__ x0, const float* __restrict__ mu_q,
                    const float* __restrict__ mu_p, const float* __restrict__ u,
                    float* __restrict__ logratio, int32_t* __restrict__ n_accept,
-                   uint32_t* __restrict__ accept_mask) {
+                   uint32_t* __restrict__ accept_mask, const float* __restrict__ offset = nullptr) {
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (b >= B) return;
@@ -406,7 +406,8 @@ accept_scan_kernel(int B, int gamma, int C, float log_const, float inv2vp, float
     }
     // Both products are rounded separately (no FMA contraction), so that identical draft and target
     // means give a difference of exactly zero.
-    const float lr = log_const + __fsub_rn(__fmul_rn(dq, inv2vq), __fmul_rn(dp, inv2vp));
+    float lr = log_const + __fsub_rn(__fmul_rn(dq, inv2vq), __fmul_rn(dp, inv2vp));
+    if (offset) lr = __fadd_rn(lr, offset[row]);   // terms of the steps t >= 2 when the noise is not shared
     logratio[row] = lr;
     acc = logf(u[row]) <= lr;
   }
@@ -418,6 +419,25 @@ accept_scan_kernel(int B, int gamma, int C, float log_const, float inv2vp, float
     n_accept[b] = n;
     if (accept_mask) accept_mask[b] = (gamma >= 32) ? ballot : (ballot & ((1u << gamma) - 1u));
   }
+}
+
+// Without trajectory alignment the exponentials of the steps t >= 2 of Eq. 4 do not cancel: x^m_{t-1} - mu^m_t =
+// sigma_m,t eps^m_t, so step t contributes (|eps^q_t|^2 - |eps^p_t|^2) / 2 beyond the Sigma term.  One thread per
+// token row, steps in order, double accumulation; identical noise gives exactly 0.
+__global__ void __launch_bounds__(128)
+noise_norm_term_kernel(int R, int C, int T, const float* __restrict__ eps_q, const float* __restrict__ eps_p,
+                       float* __restrict__ offset) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= R) return;
+  double total = 0.0;
+  for (int t = 1; t < T; ++t) {   // slices 1..T-1 = steps 2..T
+    const float* a = eps_q + (static_cast<size_t>(t) * R + r) * C;
+    const float* b = eps_p + (static_cast<size_t>(t) * R + r) * C;
+    float nq = 0.0f, np = 0.0f;
+    for (int c = 0; c < C; ++c) { nq = fmaf(a[c], a[c], nq); np = fmaf(b[c], b[c], np); }
+    total += 0.5 * (static_cast<double>(nq) - static_cast<double>(np));
+  }
+  offset[r] = static_cast<float>(total);
 }
 
 // Resampling: one warp per sequence, lane c < C = coordinate.  Proposals are consumed in order.

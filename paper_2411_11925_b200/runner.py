@@ -86,6 +86,13 @@ class DeviceRound:
                                         self.traj_mu if traj_mu is None else traj_mu, self.u, steps_per_pass,
                                         self.logratio, self.n_accept, self.accept_mask)
 
+    def verify_unaligned(self, eps_p):
+        """csd_verify with the target's own noise eps_p (no trajectory alignment)."""
+        wl = self.wl
+        self.ctx.csd_verify_unaligned(self.head_p, self.sched_p, self.sched_q, wl.B, wl.gamma, wl.cfg, wl.cfg_scale,
+                                      self.z_p, self.x_T, eps_p, self.eps, self.x0, self.mu1_q, self.u, self.logratio,
+                                      self.n_accept, self.accept_mask, self.mu1_p)
+
     def three_calls(self):
         self.draft(); self.verify(); self.resample()
 

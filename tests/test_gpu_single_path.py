@@ -192,6 +192,48 @@ def test_close_heads_fp32_single_path_ratio_is_tight():
     dr.ctx.close()
 
 
+@pytest.mark.parametrize("op,kw", CASES[:4])
+def test_unaligned_verify_matches_checker_and_reduces_to_verify(op, kw):
+    # Ablation without trajectory alignment: the target runs on its own noise; the checker's value is the long
+    # product of Eq. 4 over both recorded paths.
+    inp = gen.make_round_inputs(_wl(**kw))
+    wl = inp.wl
+    rng = np.random.default_rng(99)
+    eps_p = rng.standard_normal(inp.eps.shape).astype(np.float32)
+    sq = orc.ddpm_schedule(inp.beta, wl.tau)
+    sp = orc.ddpm_schedule(inp.beta, 0.9 * wl.tau)
+    eq = orc.make_mlp_head(inp.w_q, inp.z_q, inp.tfeat, wl.cfg, wl.cfg_scale)
+    ep = orc.make_mlp_head(inp.w_p, inp.z_p, inp.tfeat, wl.cfg, wl.cfg_scale)
+    dq, dp = orc.run_pair(eq, ep, sq, sp, inp.x_T, inp.eps, noise_p=eps_p, keep=True)
+    want = orc.log_ratio_long(dq, dp, sq, sp).reshape(wl.B, wl.gamma)
+    dr = _device_round(inp, tau_p=0.9 * wl.tau)
+    dr.draft()
+    # aligned noise: the extra sum is exactly zero, the call is csd_verify bit for bit
+    dr.verify()
+    dr.ctx.sync()
+    lr_v, mu_v = _np(dr.logratio), _np(dr.mu1_p)
+    dr.verify_unaligned(dr.eps)
+    dr.ctx.sync()
+    np.testing.assert_array_equal(_np(dr.logratio), lr_v)
+    np.testing.assert_array_equal(_np(dr.mu1_p), mu_v)
+    # own noise
+    dr.verify_unaligned(torch.from_numpy(eps_p).to(dr.dev))
+    dr.ctx.sync()
+    lr, acc = _check_scan(dr, wl, inp.u)
+    assert np.max(np.abs(_np(dr.mu1_p) - dp["mu1"])) <= TOL_MU[op]
+    s1q, s1p = sq["sigma"][0], sp["sigma"][0]
+    Qp = np.sum((dq["x0"] - dp["mu1"]) ** 2, axis=1) / (2 * s1p ** 2)
+    Qq = np.sum((dq["x0"] - dq["mu1"]) ** 2, axis=1) / (2 * s1q ** 2)
+    tol = (TOL_LOGR + (np.sqrt(2 * Qp) / s1p + np.sqrt(2 * Qq) / s1q) * 4.0 * TOL_MU[op]).reshape(wl.B, wl.gamma)
+    # fp32 result of magnitude |want|: half an ulp of the sum on top
+    tol = tol + 1e-6 * np.abs(want)
+    err = np.abs(lr - want)
+    print(op, kw, "unaligned logR err", float(err.max()), "of tol", float((err / tol).max()), "median |logR|",
+          float(np.median(np.abs(want))))
+    assert np.all(err <= tol)
+    dr.ctx.close()
+
+
 def test_single_path_argument_checks():
     from paper_2411_11925_b200 import api
     inp = gen.make_round_inputs(_wl(B=2, gamma=3, T=4))
