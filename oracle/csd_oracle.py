@@ -10,6 +10,9 @@ otherwise in the paper's order: no blocking, fusion or reordering.
 
 What pins each function (see tests/test_oracle_pins.py):
 
+  ddim_schedule            marginal preservation on Gaussian data for every eta (the sampler's
+                           defining property), eta = 1 on the full ladder is the DDPM posterior,
+                           last-step mean is x0_hat
   ddpm_schedule            textbook special case (N(0,1) data: mu_t = sqrt(alpha_t) x_t)
   denoise / run_pair       Theorem 1 pathwise identity and its Monte-Carlo form
   log_sigma_term, log_ratio_*   long form (Eq. 4) == closed form (Eq. 7, 8);
@@ -52,6 +55,29 @@ def ddpm_schedule(beta: np.ndarray, tau: float = 1.0) -> Dict[str, np.ndarray]:
     b = beta / (np.sqrt(alpha) * np.sqrt(1.0 - alphabar))
     sigma = tau * np.sqrt(beta)
     return {"a": a, "b": b, "sigma": sigma, "alphabar": alphabar, "beta": beta}
+
+
+def ddim_schedule(beta_full: np.ndarray, steps: np.ndarray, eta: float) -> Dict[str, np.ndarray]:
+    """DDIM sampler (Appendix "More Variants of Diffusion Model") derived from a DDPM trained with beta_full,
+    run on the ascending sub-sequence `steps` (1-based timesteps) with stochasticity eta in (0, 1].  The
+    transition is the Gaussian q_sigma(x_prev | x_t, x0_hat) of the DDIM paper:
+      x0_hat = (x_t - sqrt(1-ab_t) eps_hat) / sqrt(ab_t)
+      x_prev = sqrt(ab_prev) x0_hat + sqrt(1 - ab_prev - sigma^2) eps_hat + sigma eps,
+      sigma  = eta sqrt((1-ab_prev)/(1-ab_t)) sqrt(1 - ab_t/ab_prev),
+    i.e. mean a x_t - b eps_hat, so it enters the method exactly like Eq. 3.  At the last step ab_prev = 1 makes
+    sigma = 0, a point mass that has no density ratio: there sigma = eta sqrt(1 - ab_t) (the variance of the
+    respaced chain's forward step), mean x0_hat.  Index k-1 of the result is the k-th step counted from x_0."""
+    ab_full = np.cumprod(1.0 - np.asarray(beta_full, dtype=f64))
+    steps = np.asarray(steps, dtype=np.int64)
+    ab = ab_full[steps - 1]
+    ab_prev = np.concatenate([[1.0], ab[:-1]])
+    sigma = eta * np.sqrt((1.0 - ab_prev) / (1.0 - ab)) * np.sqrt(1.0 - ab / ab_prev)
+    sigma[0] = eta * np.sqrt(1.0 - ab[0])
+    direction = np.sqrt(np.maximum(0.0, 1.0 - ab_prev - sigma ** 2))
+    direction[0] = 0.0
+    a = np.sqrt(ab_prev / ab)
+    b = a * np.sqrt(1.0 - ab) - direction
+    return {"a": a, "b": b, "sigma": sigma, "alphabar": ab, "beta": 1.0 - ab / ab_prev}
 
 
 # --------------------------------------------------------------------------

@@ -49,6 +49,45 @@ def test_schedule_point_mass_data_gives_ddpm_posterior_mean():
         np.testing.assert_allclose(mu, want, rtol=0, atol=1e-13)
 
 
+@pytest.mark.parametrize("eta", [0.3, 1.0])
+def test_ddim_schedule_preserves_gaussian_marginals(eta):
+    # Defining property of DDIM: given the true x_0, for every sigma the reverse step maps the marginal of x_t
+    # onto that of x_prev.  Point-mass data x_0 = m (the predictor then returns the true noise):
+    # x_t ~ N(sqrt(ab) m, 1 - ab), the step is affine x_prev = A x_t + D + sigma eps, so mean and variance can
+    # be pushed through by hand.
+    N, m, s_ = 200, 0.7, 0.0
+    beta = gen.beta_linear(N)
+    steps = np.arange(10, N + 1, 10)
+    sch = orc.ddim_schedule(beta, steps, eta)
+    eps_fn = orc.make_gaussian_toy_head(m, s_, sch["alphabar"])
+    ab = sch["alphabar"]
+    for k in range(len(steps), 1, -1):           # steps with a proper predecessor marginal (ab_prev < 1)
+        x = np.array([[0.0], [1.0]])
+        mu = sch["a"][k - 1] * x - sch["b"][k - 1] * eps_fn(x, k)
+        A, D = mu[1, 0] - mu[0, 0], mu[0, 0]
+        mean_t, var_t = math.sqrt(ab[k - 1]) * m, ab[k - 1] * s_ ** 2 + 1 - ab[k - 1]
+        mean_p, var_p = math.sqrt(ab[k - 2]) * m, ab[k - 2] * s_ ** 2 + 1 - ab[k - 2]
+        assert abs(A * mean_t + D - mean_p) < 1e-12
+        assert abs(A * A * var_t + sch["sigma"][k - 1] ** 2 - var_p) < 1e-12
+
+
+def test_ddim_with_eta_one_on_the_full_ladder_is_the_ddpm_posterior():
+    # Song et al.: eta = 1 recovers DDPM: same mean coefficients as the eps-parameterised DDPM mean and the posterior
+    # variance beta~_t = (1 - ab_{t-1}) / (1 - ab_t) beta_t (Ho et al., Eq. 7).
+    T = 30
+    beta = gen.beta_linear(T)
+    dd, dp = orc.ddim_schedule(beta, np.arange(1, T + 1), 1.0), orc.ddpm_schedule(beta)
+    ab = np.cumprod(1 - beta)
+    np.testing.assert_allclose(dd["a"], dp["a"], rtol=1e-12)
+    np.testing.assert_allclose(dd["b"][1:], dp["b"][1:], rtol=1e-10)
+    np.testing.assert_allclose(dd["sigma"][1:] ** 2, (1 - ab[:-1]) / (1 - ab[1:]) * beta[1:], rtol=1e-12)
+    # last step: the mean is the predicted x_0 (for point-mass data it is the data point itself)
+    eps_fn = orc.make_gaussian_toy_head(0.4, 0.0, dd["alphabar"])
+    x = np.array([[-1.0], [2.5]])
+    np.testing.assert_allclose(dd["a"][0] * x - dd["b"][0] * eps_fn(x, 1), 0.4, atol=1e-12)
+    assert abs(dd["sigma"][0] - math.sqrt(1 - ab[0])) < 1e-15
+
+
 def test_temperature_scales_sigma_only():
     beta = gen.beta_linear(10)
     s1, s2 = orc.ddpm_schedule(beta, 1.0), orc.ddpm_schedule(beta, 0.8)
