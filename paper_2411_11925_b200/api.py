@@ -101,6 +101,31 @@ def ddpm_coefficients(beta: np.ndarray, tau: float = 1.0) -> Dict[str, np.ndarra
             "sigma": (tau * np.sqrt(beta)).astype(np.float32)}
 
 
+def ddim_coefficients(beta_full: np.ndarray, steps, eta: float) -> Dict[str, np.ndarray]:
+    """Host helper: a DDIM sampler with stochasticity eta in (0, 1] on the ascending sub-sequence `steps` (1-based)
+    of a DDPM's timesteps, written as the coefficients csd_schedule takes (mu = a x_t - b eps_hat, then
+    + sigma eps): the library needs nothing else to run DDIM (Appendix "More Variants of Diffusion Model").
+    Entry k-1 is the k-th step counted from x_0; pass the feature-table rows of the same timesteps as tfeat.
+    The last step (to x_0) would have sigma = 0, which has no density to take ratios of: it gets
+    sigma = eta sqrt(1 - alphabar) around the predicted x_0."""
+    if not 0.0 < eta <= 1.0:
+        raise ValueError("eta must be in (0, 1]")
+    abar_all = np.cumprod(1.0 - np.asarray(beta_full, dtype=np.float64))
+    idx = np.asarray(list(steps), dtype=np.int64) - 1
+    if idx.size == 0 or np.any(np.diff(idx) <= 0) or idx[0] < 0 or idx[-1] >= abar_all.size:
+        raise ValueError("steps must be ascending timesteps within 1..len(beta_full)")
+    cur = abar_all[idx]
+    prv = np.ones_like(cur)
+    prv[1:] = cur[:-1]
+    sig = eta * np.sqrt((1.0 - prv) * (1.0 - cur / prv) / (1.0 - cur))
+    sig[0] = eta * np.sqrt(1.0 - cur[0])
+    keep = np.sqrt(np.clip(1.0 - prv - sig * sig, 0.0, None))     # weight of eps_hat in the direction to x_t
+    keep[0] = 0.0
+    scale = np.sqrt(prv / cur)
+    return {"a": scale.astype(np.float32), "b": (scale * np.sqrt(1.0 - cur) - keep).astype(np.float32),
+            "sigma": sig.astype(np.float32)}
+
+
 def _ptr(t) -> Optional[int]:
     if t is None:
         return None

@@ -15,7 +15,10 @@ class DeviceRound:
     """Device-resident heads, schedules, inputs and outputs of one speculative round."""
 
     def __init__(self, inp: RoundInputs, ctx: Optional[api.Context] = None, device: int = 0,
-                 heads: Optional[tuple] = None, tau_q: Optional[float] = None, tau_p: Optional[float] = None):
+                 heads: Optional[tuple] = None, tau_q: Optional[float] = None, tau_p: Optional[float] = None,
+                 coeffs_q: Optional[dict] = None, coeffs_p: Optional[dict] = None):
+        """coeffs_q / coeffs_p: transition coefficients {"a", "b", "sigma"} to use instead of the DDPM ones of
+        inp.beta (for instance api.ddim_coefficients); inp.tfeat must then hold the rows of the same timesteps."""
         wl = inp.wl
         self.inp, self.wl = inp, wl
         self.dev = torch.device("cuda", device)
@@ -26,8 +29,8 @@ class DeviceRound:
         else:
             self.head_q, self.head_p = heads
         self.tfeat = torch.from_numpy(inp.tfeat).to(self.dev)
-        cq = api.ddpm_coefficients(inp.beta, wl.tau if tau_q is None else tau_q)
-        cp = api.ddpm_coefficients(inp.beta, wl.tau if tau_p is None else tau_p)
+        cq = coeffs_q or api.ddpm_coefficients(inp.beta, wl.tau if tau_q is None else tau_q)
+        cp = coeffs_p or api.ddpm_coefficients(inp.beta, wl.tau if tau_p is None else tau_p)
         self.sched_q = api.Schedule(cq["a"], cq["b"], cq["sigma"], self.tfeat)
         self.sched_p = api.Schedule(cp["a"], cp["b"], cp["sigma"], self.tfeat)
         self.C = wl.draft.C

@@ -101,3 +101,23 @@ def test_select_sequences_slices_rows_consistently():
     full, part = orc.round_from_inputs(inp), orc.round_from_inputs(sub)
     np.testing.assert_allclose(part["logratio"], full["logratio"][[2, 0]], rtol=1e-9)
     np.testing.assert_allclose(part["x0"][:g], full["x0"][2 * g:3 * g], atol=1e-12)
+
+
+def test_ddim_coefficients_agree_with_the_checker_and_reject_bad_arguments():
+    import numpy as np
+    import pytest
+    from oracle import csd_oracle as orc
+    from paper_2411_11925_b200 import api, inputs as gen
+    beta = gen.beta_linear(1000)
+    steps = np.linspace(10, 1000, 100).astype(np.int64)
+    for eta in (0.2, 1.0):
+        got, want = api.ddim_coefficients(beta, steps, eta), orc.ddim_schedule(beta, steps, eta)
+        for k in ("a", "b", "sigma"):
+            np.testing.assert_allclose(got[k], want[k], rtol=2e-7, atol=1e-9)
+        assert np.all(got["sigma"] > 0)
+    with pytest.raises(ValueError):
+        api.ddim_coefficients(beta, steps, 0.0)
+    with pytest.raises(ValueError):
+        api.ddim_coefficients(beta, [5, 3], 1.0)
+    with pytest.raises(ValueError):
+        api.ddim_coefficients(beta, [1, 1001], 1.0)
