@@ -335,6 +335,16 @@ def csd_round(eps_q, eps_p, sched_q, sched_p, x_T, noise, u, xi, v, B, gamma, ca
     return out
 
 
+def bonus_token(eps_p_next, sched_p, x_T_next, noise_next, n_accept, gamma) -> Dict[str, np.ndarray]:
+    """Alg. 1, all-accepted branch: a sequence whose gamma drafts were all accepted also gets the token of
+    position gamma+1, an ordinary sample x_0 of the target head's reverse process at that position (noise at every
+    step, as for the draft).  Rows of other sequences are left at zero with taken = False."""
+    d = denoise(eps_p_next, sched_p, x_T_next, noise_next, sample_last=True)
+    taken = np.asarray(n_accept) >= gamma
+    x = np.where(taken[:, None], d["x0"], 0.0)
+    return {"x_bonus": x, "taken": taken, "x0_all": d["x0"]}
+
+
 def single_path_from_inputs(inp) -> Dict[str, np.ndarray]:
     """Draft trajectories of a RoundInputs bundle and the exact ratio of Eq. 2 on them,
     with the accept scan of Alg. 1 applied to that ratio."""

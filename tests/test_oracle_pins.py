@@ -455,6 +455,25 @@ def test_single_path_ratio_has_unit_expectation_under_the_draft():
     assert w.std() > 0.05          # not vacuous: the two models differ
 
 
+def test_bonus_token_is_a_target_sample_exactly_where_everything_was_accepted():
+    # The all-accepted branch of Alg. 1: on Gaussian data with point mass m the target's samples end within a few
+    # sigma_1 of m (its reverse process contracts onto the data), and only sequences with n = gamma receive one.
+    T, B, gamma = 40, 6, 4
+    sp = orc.ddpm_schedule(gen.beta_linear(T))
+    ep = orc.make_gaussian_toy_head(0.25, 0.0, sp["alphabar"])
+    rng = np.random.default_rng(50)
+    x_T, noise = rng.standard_normal((B, 2)), rng.standard_normal((T, B, 2))
+    n = np.array([4, 0, 3, 4, 2, 4])
+    out = orc.bonus_token(ep, sp, x_T, noise, n, gamma)
+    np.testing.assert_array_equal(out["taken"], [True, False, False, True, False, True])
+    assert np.all(out["x_bonus"][~out["taken"]] == 0.0)
+    assert np.all(np.abs(out["x_bonus"][out["taken"]] - 0.25) < 6 * sp["sigma"][0])
+    # and it is the last state of the plain reverse process with noise at every step
+    d = orc.denoise(ep, sp, x_T, noise, sample_last=True)
+    np.testing.assert_array_equal(out["x_bonus"][out["taken"]], d["x0"][out["taken"]])
+    np.testing.assert_allclose(d["x0"], d["mu1"] + sp["sigma"][0] * noise[0], atol=1e-15)
+
+
 # --------------------------------------------------------------- accept scan
 @pytest.mark.parametrize("gamma", [1, 3, 8])
 def test_accept_prefix_brute_force_all_masks(gamma):
