@@ -214,6 +214,18 @@ int csd_verify_unaligned(csd_ctx *ctx, const csd_head *head_p, const csd_schedul
                          const float *x0_q, const float *mu1_q, const float *u, float *logratio,
                          int32_t *n_accept, uint32_t *accept_mask, float *mu1_p);
 
+/* Bonus token (Alg. 1, the branch in which all gamma drafts were accepted: "sample x from p_{gamma+1}").
+ * Runs the target head's reverse process (t = T..1, noise at every step, as csd_draft_denoise does) for
+ * position gamma+1 of every sequence and keeps the sample where n_accept[b] == gamma.  All B rows are
+ * evaluated because n_accept lives on the device; the selection costs no host synchronisation.
+ *   z_next device [B*(1+cfg), Dz_p] (the target backbone's output at position gamma+1);
+ *   x_T_next device [B, C]; eps_next device [T, B, C]; n_accept device int32 [B] (from csd_verify);
+ *   x_bonus device [B, C] out, untouched where n_accept[b] < gamma;
+ *   taken device uint32 [B] out or NULL: 1 where a bonus token was written. */
+int csd_bonus_token(csd_ctx *ctx, const csd_head *head_p, const csd_schedule *sched_p, int B, int gamma,
+                    int cfg, float cfg_scale, const float *z_next, const float *x_T_next,
+                    const float *eps_next, const int32_t *n_accept, float *x_bonus, uint32_t *taken);
+
 /* ---- Exact single-path criterion (Eq. 2; Table 1 "p(Y_q)/q(Y_q)") ------------------------------
  * Eq. 2 scores the DRAFT's own trajectory Y_q = (x_T, x^q_{T-1}, ..., x^q_0) under both models:
  *   log p(Y_q)/q(Y_q) = sum_{t=1..T} [ log N(x^q_{t-1}; mu^p_t(x^q_t), sigma_p,t^2 I)

@@ -26,7 +26,7 @@ EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launc
            "csd_set_chain_mode", "csd_profile", "csd_profile_read",
            "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_draft_denoise_static", "csd_verify",
            "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host", "csd_draft_denoise_traj",
-           "csd_verify_single_path", "csd_verify_unaligned")
+           "csd_verify_single_path", "csd_verify_unaligned", "csd_bonus_token")
 
 WEIGHT_FIELDS = ("Wz", "bz", "Wt1", "bt1", "Wt2", "bt2", "Win", "bin", "Wada", "bada",
                  "W1", "b1", "W2", "b2", "Wfada", "bfada", "Wout", "bout")
@@ -76,6 +76,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
                                            + [vp] * 4 + [i32] + [vp] * 3)
     lib.csd_verify_unaligned.argtypes = ([vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32]
                                          + [vp] * 11)
+    lib.csd_bonus_token.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, i32, f32] + [vp] * 6
     lib.csd_accept_scan.argtypes = [vp, i32, i32, i32, f64, f32, f32] + [vp] * 7
     lib.csd_resample.argtypes = [vp, i32, i32, i32, i32, f64, f32, f32] + [vp] * 9
     round_args = [vp, vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32, i32] + [vp] * 17
@@ -244,6 +245,12 @@ class Context:
                                               int(cfg), cfg_scale, _ptr(z_p), _ptr(x_T), _ptr(eps_p), _ptr(eps_q),
                                               _ptr(x0_q), _ptr(mu1_q), _ptr(u), _ptr(logratio), _ptr(n_accept),
                                               _ptr(accept_mask), _ptr(mu1_p)))
+
+    def csd_bonus_token(self, head_p: "Head", sched_p: Schedule, B, gamma, cfg, cfg_scale, z_next, x_T_next, eps_next,
+                        n_accept, x_bonus, taken=None):
+        self._check(_LIB.csd_bonus_token(self._h, head_p._h, C.byref(sched_p.c), B, gamma, int(cfg), cfg_scale,
+                                         _ptr(z_next), _ptr(x_T_next), _ptr(eps_next), _ptr(n_accept), _ptr(x_bonus),
+                                         _ptr(taken)))
 
     def csd_accept_scan(self, B, gamma, Cdim, log_sigma, sigma1_p, sigma1_q, x0_q, mu1_q, mu1_p, u, logratio,
                         n_accept, accept_mask=None):

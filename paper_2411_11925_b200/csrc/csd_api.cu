@@ -64,6 +64,7 @@ struct csd_ctx {
   ChainWs ws[3];   // draft chain, target chain, static-scratch calls
   HostIo io;
   HostIo un;       // csd_verify_unaligned: per-row noise terms
+  HostIo bn;       // csd_bonus_token: samples of every sequence before the selection
   HostIo sp;       // csd_verify_single_path: schedule constants, mu^p of one pass, running log-ratio
   char err[512] = {0};
   // optional per-launch timing (csd_profile)
@@ -796,6 +797,7 @@ int csd_destroy(csd_ctx* c) {
   if (c->io.base) cudaFree(c->io.base);
   if (c->sp.base) cudaFree(c->sp.base);
   if (c->un.base) cudaFree(c->un.base);
+  if (c->bn.base) cudaFree(c->bn.base);
   if (c->d_err) cudaFree(c->d_err);
   cudaGetLastError();
   delete c;
@@ -1178,6 +1180,38 @@ int csd_verify_unaligned(csd_ctx* ctx, const csd_head* head_p, const csd_schedul
   CSD_CUDA(ctx, cudaGetLastError());
   return accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term(sched_q, sched_p, C), sched_p->sigma[0],
                      sched_q->sigma[0], x0_q, mu1_q, mu1_p, u, logratio, n_accept, accept_mask, d_off);
+}
+
+int csd_bonus_token(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p, int B, int gamma, int cfg,
+                    float cfg_scale, const float* z_next, const float* x_T_next, const float* eps_next,
+                    const int32_t* n_accept, float* x_bonus, uint32_t* taken) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "gamma = %d must be >= 1", gamma);
+  int rc = check_chain_args(ctx, head_p, sched_p, B, cfg, z_next, x_T_next, eps_next);
+  if (rc) return rc;
+  if (!n_accept || !x_bonus) return fail(ctx, CSD_ERR_INVALID_ARG, "n_accept / x_bonus is null");
+  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  const int C = head_p->d.C;
+  const size_t need = static_cast<size_t>(2) * B * C * 4;
+  if (need > ctx->bn.cap) {
+    CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (ctx->bn.base) CSD_CUDA(ctx, cudaFree(ctx->bn.base));
+    ctx->bn.base = nullptr; ctx->bn.cap = 0;
+    if (cudaMalloc(&ctx->bn.base, need) != cudaSuccess) {
+      cudaGetLastError();
+      return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes for the bonus samples", need);
+    }
+    ctx->bn.cap = need;
+  }
+  float* d_x0 = static_cast<float*>(ctx->bn.base);
+  float* d_mu = d_x0 + static_cast<size_t>(B) * C;
+  // the masks live on the device, so every sequence is sampled and the selection is a kernel: no host round trip
+  rc = run_chain(ctx, 1, ctx->stream, head_p, sched_p, B, cfg, cfg_scale, z_next, x_T_next, eps_next, 1, d_x0, d_mu, nullptr);
+  if (rc) return rc;
+  bonus_select_kernel<<<(B * C + 255) / 256, 256, 0, ctx->stream>>>(B, C, gamma, n_accept, d_x0, x_bonus, taken);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
 }
 
 int csd_draft_denoise_traj(csd_ctx* ctx, const csd_head* head, const csd_schedule* sched, int R, int cfg,

@@ -440,6 +440,18 @@ noise_norm_term_kernel(int R, int C, int T, const float* __restrict__ eps_q, con
   offset[r] = static_cast<float>(total);
 }
 
+// All-accepted branch of Alg. 1: sequence b keeps its sample of position gamma + 1 only if n_accept[b] == gamma.
+__global__ void __launch_bounds__(256)
+bonus_select_kernel(int B, int C, int gamma, const int32_t* __restrict__ n_accept, const float* __restrict__ x0,
+                    float* __restrict__ x_bonus, uint32_t* __restrict__ taken) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * C) return;
+  const int b = i / C;
+  const bool all = n_accept[b] >= gamma;
+  if (all) x_bonus[i] = x0[i];
+  if (taken && i == b * C) taken[b] = all ? 1u : 0u;
+}
+
 // Resampling: one warp per sequence, lane c < C = coordinate.  Proposals are consumed in order.
 __global__ void __launch_bounds__(128)
 resample_kernel(int B, int gamma, int C, int cap, float log_sigma, float sp1, float sq1,
