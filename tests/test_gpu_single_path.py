@@ -282,3 +282,29 @@ def test_mar256_full_size_single_path_sampled_sequences():
     dr.ctx.sync()
     np.testing.assert_array_equal(_np(dr.logratio), lr)
     dr.ctx.close()
+
+
+def test_ar_stress_full_size_single_path_sampled_sequences():
+    # Perturbed-draft workload at full size (B=256, gamma=16, T=50, no guidance: 4096 rows per step, 8 steps per
+    # pass), with the draft's condition vectors given to the target so that the heads are close and the log-ratios
+    # moderate; the checker evaluates the first and the last sequence.
+    wl = gen.WORKLOADS["ar_stress"]
+    inp = gen.make_round_inputs(wl)
+    inp.z_p = inp.z_q
+    dr = _device_round(inp)
+    dr.draft_traj()
+    dr.verify_single_path()
+    dr.ctx.sync()
+    lr, acc = _check_scan(dr, wl, inp.u)
+    assert np.all(np.isfinite(lr))
+    seqs = [0, wl.B - 1]
+    sub = gen.select_sequences(inp, seqs)
+    sq, sp, ep, dq = _oracle_parts(sub)
+    want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(len(seqs), wl.gamma)
+    op = wl.operand_format
+    tol = _logr_tolerance(ep, sq, sp, dq, TOL_X[op] + TOL_MU[op]).reshape(len(seqs), wl.gamma)
+    err = np.abs(lr[seqs] - want)
+    print("ar_stress single-path: max err", float(err.max()), "of tol", float((err / tol).max()),
+          "median |logR|", float(np.median(np.abs(want))), "accepted", float(acc.mean()))
+    assert np.all(err <= tol)
+    dr.ctx.close()
