@@ -1242,6 +1242,7 @@ int csd_verify_single_path(csd_ctx* ctx, const csd_head* head_p, const csd_sched
   if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
   if (static_cast<int64_t>(B) * gamma > (1 << 24)) return fail(ctx, CSD_ERR_UNSUPPORTED, "B * gamma exceeds 2^24 rows");
   const int R = B * gamma;
+  if (!traj_x || !traj_mu_q) return fail(ctx, CSD_ERR_INVALID_ARG, "traj_x / traj_mu_q is null");
   int rc = check_chain_args(ctx, head_p, sched_p, R, cfg, z_p, traj_x, traj_mu_q);
   if (rc) return rc;
   if ((rc = check_sched(ctx, sched_q, false))) return rc;

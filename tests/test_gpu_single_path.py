@@ -308,3 +308,26 @@ def test_ar_stress_full_size_single_path_sampled_sequences():
           "median |logR|", float(np.median(np.abs(want))), "accepted", float(acc.mean()))
     assert np.all(err <= tol)
     dr.ctx.close()
+
+
+@pytest.mark.parametrize("kw", [dict(B=1, gamma=1, T=1), dict(B=1, gamma=32, T=2), dict(B=2, gamma=1, T=3, cfg=True, cfg_scale=1.5)])
+def test_single_path_and_unaligned_degenerate_sizes(kw):
+    # one row, one step (Eq. 2 is then Eq. 8 with Sigma = 1), the widest prefix scan, one position per sequence
+    inp = gen.make_round_inputs(_wl(**kw))
+    wl = inp.wl
+    sq, sp, ep, dq = _oracle_parts(inp)
+    want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(wl.B, wl.gamma)
+    dr = _device_round(inp)
+    dr.draft_traj()
+    dr.verify_single_path(7)          # more steps per pass than there are steps
+    dr.ctx.sync()
+    lr, acc = _check_scan(dr, wl, inp.u)
+    tol = _logr_tolerance(ep, sq, sp, dq, TOL_X["f32"] + TOL_MU["f32"]).reshape(wl.B, wl.gamma)
+    assert np.all(np.abs(lr - want) <= tol)
+    if wl.T == 1:
+        # same number as the aligned criterion, which for T = 1 has no step before the last
+        dr.draft(); dr.verify(); dr.ctx.sync()
+        np.testing.assert_allclose(_np(dr.logratio), lr, rtol=1e-5, atol=1e-3)
+        dr.verify_unaligned(dr.eps); dr.ctx.sync()
+        np.testing.assert_allclose(_np(dr.logratio), lr, rtol=1e-5, atol=1e-3)
+    dr.ctx.close()
