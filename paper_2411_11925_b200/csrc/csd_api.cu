@@ -630,6 +630,13 @@ struct Chain {
       // v = SiLU(W1 u + b1)
       e.bias0 = hd->b1[k]; e.bias1 = nullptr; e.out_act = ws.v;
       if (folded_in) rc = CSD_OK;
+      else if (tc && pair && W % 256 == 0) {
+        // CTA pairs over 256 x 256 tiles: per MMA byte the pair loads half as many operand bytes as with 256 x 128
+        // tiles, and the first layer (one accumulator, K = W) is the kernel bound by that feed
+        const CUtensorMap& w1 = hd->tm[1].W1[k];   // 128-row boxes: each CTA of the pair loads half of the 256 rows
+        rc = d.dtype == CSD_F16 ? launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __half, true>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e)
+                                : launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __nv_bfloat16, true>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e);
+      }
       else if (tc && w1_wide) {
         const CUtensorMap& w1 = hd->W1_wide[k];
         rc = d.dtype == CSD_F16 ? launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __half, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e)
