@@ -27,13 +27,14 @@ def _worker(rank, world, port, B, q):
     inp = gen.make_round_inputs(wl)                       # same seed on every rank: replicated heads + inputs
     mine = gen.shard_sequences(B, world, rank)
     out = orc.round_from_inputs(gen.select_sequences(inp, mine))
+    sp_local = orc.single_path_from_inputs(gen.select_sequences(inp, mine))["logratio"]   # Eq. 2 shards the same way
     n_local = torch.full((B,), -1, dtype=torch.int32)
     n_local[mine.start:mine.stop] = torch.from_numpy(out["n_accept"])
     dist.all_reduce(n_local, op=dist.ReduceOp.MAX)        # gather for a host-side AR scheduler
     t = torch.tensor([0.010 * (rank + 1)], dtype=torch.float64)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)              # benchmark timing: max over ranks
     if rank == 0:
-        q.put((n_local.numpy(), float(t), out["logratio"]))
+        q.put((n_local.numpy(), float(t), out["logratio"], sp_local))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -48,7 +49,7 @@ def test_two_ranks_shard_sequences_without_exchange():
     procs = [ctx.Process(target=_worker, args=(r, world, port, B, q)) for r in range(world)]
     for p in procs:
         p.start()
-    n_all, tmax, lr0 = q.get(timeout=240)
+    n_all, tmax, lr0, sp0 = q.get(timeout=240)
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
@@ -56,4 +57,5 @@ def test_two_ranks_shard_sequences_without_exchange():
     full = orc.round_from_inputs(gen.make_round_inputs(wl))
     np.testing.assert_array_equal(n_all, full["n_accept"])          # sharded == unsharded
     np.testing.assert_allclose(lr0, full["logratio"][:3], rtol=1e-9)
+    np.testing.assert_allclose(sp0, orc.single_path_from_inputs(gen.make_round_inputs(wl))["logratio"][:3], rtol=1e-9)
     assert abs(tmax - 0.020) < 1e-12
