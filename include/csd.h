@@ -52,7 +52,8 @@ enum {
   CSD_ERR_UNSUPPORTED = -3, /* e.g. W not a multiple of 128, gamma > 32, C > 16, not an sm_100 GPU */
   CSD_ERR_WORKSPACE = -4,   /* device memory for the workspace or weights could not be had      */
   CSD_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed                                 */
-  CSD_ERR_TIMEOUT = -6      /* a bounded device-side wait gave up (reported by csd_sync)         */
+  CSD_ERR_TIMEOUT = -6,     /* a bounded device-side wait gave up (reported by csd_sync)         */
+  CSD_ERR_NONFINITE = -7    /* a state or mean of a denoising step was inf or NaN (reported by csd_sync) */
 };
 
 enum { CSD_F32 = 0, CSD_BF16 = 1, CSD_F16 = 2 };
@@ -65,7 +66,11 @@ enum { CSD_F32 = 0, CSD_BF16 = 1, CSD_F16 = 2 };
  *           bf16-representable: such a value is exact in fp16 when |w| >= 2^-17 (else it is off
  *           by at most 2^-25), and activations keep 11 significant bits instead of 8, which the
  *           long, error-amplifying T-step trajectories need (a tensor-core instruction takes
- *           both operands in one 16-bit format).  Activations must stay below 65504 in magnitude.
+ *           both operands in one 16-bit format).  Activations must stay below 65504 in magnitude: a
+ *           larger one is rounded to infinity, reaches the step update as inf or NaN and is reported by
+ *           csd_sync as CSD_ERR_NONFINITE (nothing faults; the outputs of that call are not usable).
+ *           Heads whose activations can grow that large (weights far above Xavier scale) take CSD_BF16
+ *           (fp32 range, 8 significant bits) or CSD_F32.
  * In all three the residual stream, LayerNorm statistics, x_t, mu and the densities are fp32. */
 typedef struct {
   int C, W, L, Dz, F;
@@ -93,32 +98,42 @@ typedef struct {
 } csd_schedule;
 
 /* Context: owns a growable device workspace and the stream association.  `cuda_stream` is a
- * cudaStream_t (NULL = legacy default stream).  csd_destroy synchronises the stream and frees. */
+ * cudaStream_t (NULL = legacy default stream).  csd_destroy synchronises the stream and frees.
+ * Several contexts, also on different devices (ordinals below 64), may live in one process.  Every call
+ * makes the context's device current while it runs and puts the caller's current device back on return. */
 int csd_create(csd_ctx **out, int device, void *cuda_stream);
 int csd_destroy(csd_ctx *ctx);
 const char *csd_last_error(const csd_ctx *ctx);
-/* Waits for the context's stream and returns CSD_ERR_TIMEOUT / CSD_ERR_CUDA if any kernel of an
- * earlier call raised its error flag, else CSD_OK.  Clears the flag. */
+/* Waits for the context's stream and returns CSD_ERR_TIMEOUT (a bounded wait of some kernel gave up; the
+ * message names the waiting role, the wait's site in the kernel, its iteration and the thread block),
+ * CSD_ERR_NONFINITE (see csd_head_desc) or CSD_ERR_CUDA if a kernel of an earlier call raised its status
+ * word, else CSD_OK.  Clears the status.  After a failed wait every later launch of the context returns
+ * at once until csd_sync has been called. */
 int csd_sync(csd_ctx *ctx);
+/* Every device-side wait of the library (on an mbarrier of a TMA / MMA / epilogue pipeline) is bounded:
+ * after `cycles` SM clock cycles (default 4e9, about two seconds; cycles <= 0 restores the default) it
+ * gives up and raises the status csd_sync reports.  The limit is one value per GPU and process (all
+ * contexts on that device share it).  Synchronises the context's streams. */
+int csd_set_wait_limit(csd_ctx *ctx, int64_t cycles);
+/* Diagnostic: enqueues one tiny kernel whose only thread waits on a barrier nobody arrives at, i.e. a wait
+ * that is certain to run into the limit above.  Used to check the reporting path (csd_sync returns
+ * CSD_ERR_TIMEOUT, "wait self-test") without disturbing the GPU: nothing faults or traps, and the wait
+ * ends at the limit.  Set a short limit first (1e5 cycles) or the call takes the default two seconds. */
+int csd_selftest_wait_timeout(csd_ctx *ctx);
 /* Number of kernels this context has launched so far (bookkeeping for benchmarks). */
 int64_t csd_launch_count(const csd_ctx *ctx);
 
-/* How a denoising chain (the T steps of Eq. 3 for one head) is laid out on the GPU.  CSD_CHAIN_LAYERS_PLAIN and
- * CSD_CHAIN_CLUSTER compute the same arithmetic in the same order and return the same bits.
+/* How the blocks of a denoising chain (the T steps of Eq. 3 for one head) are split into kernels.
  *   CSD_CHAIN_LAYERS  (default): one kernel per layer, chained with programmatic dependent launch; a
  *                     layer's independent part overlaps its predecessor on otherwise idle SMs.  For 16-bit
  *                     heads on grids of one wave, blocks 2..L run as two kernels instead of three: LayerNorm
  *                     is folded into the first layer's epilogue (algebraically the same function, rounded
- *                     differently: results agree with the other layouts within the parity tolerance, not
+ *                     differently: results agree with the plain layout within the parity tolerance, not
  *                     bit for bit).
- *   CSD_CHAIN_LAYERS_PLAIN: as above without the folded blocks (three kernels per block everywhere).
- *   CSD_CHAIN_CLUSTER: one kernel per chain; a thread-block cluster of W/128 CTAs owns a block of 128 rows
- *                     for all layers and steps, the residual stream stays in shared memory.  Used for
- *                     16-bit heads with W <= 1024, other heads fall back to CSD_CHAIN_LAYERS.  Measured
- *                     slower than the default at every benchmark size (a row block is confined to W/128
- *                     SMs), kept selectable for small-batch experiments.
+ *   CSD_CHAIN_LAYERS_PLAIN: as above without the folded blocks (three kernels per block everywhere); a
+ *                     row's bits then do not depend on how many rows the call has.
  * Takes effect for calls made after it returns. */
-enum { CSD_CHAIN_LAYERS = 0, CSD_CHAIN_CLUSTER = 1, CSD_CHAIN_LAYERS_PLAIN = 2 };
+enum { CSD_CHAIN_LAYERS = 0, CSD_CHAIN_LAYERS_PLAIN = 2 };
 int csd_set_chain_mode(csd_ctx *ctx, int mode);
 
 /* Optional per-launch timing for benchmarks.  csd_profile(ctx, 1) synchronises, clears the records
@@ -128,11 +143,31 @@ int csd_set_chain_mode(csd_ctx *ctx, int mode);
  * kernel class, the launches recorded since: their count, device time (ms) and algorithmic FLOPs
  * (2*M*N*K per GEMM).  Classes: 0 condition projection, 1 block MLP first layer (+SiLU),
  * 2 AdaLN modulate (shift|scale), 3 block MLP second layer + gate + residual, 4 final modulate +
- * output projection, 5 per-step boundary kernel, 6 whole-chain kernel (all layers and steps of one
- * head in one launch; used when a row block's column slices fit one thread-block cluster). */
+ * output projection, 5 per-step boundary kernel, 6 small-batch chain kernel. */
 int csd_profile(csd_ctx *ctx, int enable);
 int csd_profile_read(csd_ctx *ctx, int kernel_class, int64_t *launches, double *total_ms,
                      double *total_flops);
+
+/* Host-only helpers: the schedules of the samplers the paper uses, as the coefficient arrays csd_schedule
+ * takes.  No GPU work, no context; all pointers are HOST arrays; return CSD_OK or CSD_ERR_INVALID_ARG.
+ *
+ * csd_schedule_ddpm: the T-step DDPM reverse process behind Eq. 3 with the eps-prediction mean and fixed
+ * isotropic variance: alpha_t = 1 - beta_t, abar_t = prod_{s<=t} alpha_s,
+ *   a[t-1] = 1/sqrt(alpha_t),  b[t-1] = beta_t / (sqrt(alpha_t) sqrt(1 - abar_t)),  sigma[t-1] = tau sqrt(beta_t)
+ * (tau = sampling temperature, Appendix "Temperature").  beta [T] in (0,1); a, b, sigma [T] out. */
+int csd_schedule_ddpm(int T, const double *beta, double tau, float *a, float *b, float *sigma);
+/* csd_schedule_ddim: the DDIM sampler of the appendix "More Variants of Diffusion Model" (Table 9 runs 100
+ * steps) on the ascending sub-sequence steps[0..n_steps) (1-based timesteps) of a T_full-step DDPM, with
+ * stochasticity eta in (0, 1] (eta = 0 has no density to take ratios of).  With prv / cur = abar of the
+ * previous / current kept timestep:  sigma = eta sqrt((1-prv)/(1-cur)) sqrt(1 - cur/prv),
+ *   a = sqrt(prv/cur),  b = a sqrt(1-cur) - sqrt(1 - prv - sigma^2).
+ * Entry k is the (k+1)-th step counted from x_0; the step to x_0 (prv = 1) gets sigma = eta sqrt(1 - cur)
+ * around the predicted x_0.  Pass the feature rows of the same timesteps as csd_schedule.tfeat. */
+int csd_schedule_ddim(int T_full, const double *beta_full, int n_steps, const int32_t *steps, double eta,
+                      float *a, float *b, float *sigma);
+/* csd_log_sigma_term: log Sigma of Eq. 7 for fixed isotropic variances,
+ * C * sum_{t=2..T} (log sigma_q[t-1] - log sigma_p[t-1]), exactly as csd_verify and csd_round form it. */
+int csd_log_sigma_term(int T, const float *sigma_q, const float *sigma_p, int C, double *out);
 
 /* Copies and repacks the weights into device memory owned by the head (synchronous; the caller
  * may free `w` afterwards).  A head belongs to the context it was created with. */
@@ -255,13 +290,14 @@ int csd_draft_denoise_traj(csd_ctx *ctx, const csd_head *head, const csd_schedul
  *   depend on it by a bit, in the default mode the block layout follows a pass's row count and
  *   results of different splits agree within the parity tolerance;
  *   logratio device [B, gamma] out; n_accept device int32 [B] out; accept_mask device uint32 [B]
- *   out or NULL.
+ *   out or NULL; mu_p_traj device [T, R, C] out or NULL: slot j = the target's mean mu^p_{T-j}(x^q_{T-j}),
+ *   the counterpart of traj_mu_q (diagnostic; the per-step terms are formed from exactly these values).
  * The library keeps a side buffer of steps_per_pass * R * C floats besides the chain workspace. */
 int csd_verify_single_path(csd_ctx *ctx, const csd_head *head_p, const csd_schedule *sched_p,
                            const csd_schedule *sched_q, int B, int gamma, int cfg, float cfg_scale,
                            const float *z_p, const float *traj_x, const float *traj_mu_q,
                            const float *u, int steps_per_pass, float *logratio, int32_t *n_accept,
-                           uint32_t *accept_mask);
+                           uint32_t *accept_mask, float *mu_p_traj);
 
 /* Resampling from the modified distribution max(0, p - q)/Z (Eq. 5) by acceptance-rejection with
  * the bound M = 1/Z (Eq. 9-11) in the inference-free form of Corollary 1.  For each sequence with

@@ -18,12 +18,13 @@ from . import build as _build
 _c_float_p = C.POINTER(C.c_float)
 
 ERRORS = {0: "CSD_OK", -1: "CSD_ERR_INVALID_ARG", -2: "CSD_ERR_SHAPE", -3: "CSD_ERR_UNSUPPORTED",
-          -4: "CSD_ERR_WORKSPACE", -5: "CSD_ERR_CUDA", -6: "CSD_ERR_TIMEOUT"}
+          -4: "CSD_ERR_WORKSPACE", -5: "CSD_ERR_CUDA", -6: "CSD_ERR_TIMEOUT", -7: "CSD_ERR_NONFINITE"}
 CSD_F32, CSD_BF16, CSD_F16 = 0, 1, 2
 DTYPES = {"f32": CSD_F32, "bf16": CSD_BF16, "f16": CSD_F16}
 
 EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launch_count",
-           "csd_set_chain_mode", "csd_profile", "csd_profile_read",
+           "csd_set_chain_mode", "csd_profile", "csd_profile_read", "csd_set_wait_limit", "csd_selftest_wait_timeout",
+           "csd_schedule_ddpm", "csd_schedule_ddim", "csd_log_sigma_term",
            "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_draft_denoise_static", "csd_verify",
            "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host", "csd_draft_denoise_traj",
            "csd_verify_single_path", "csd_verify_unaligned", "csd_bonus_token")
@@ -64,6 +65,12 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_sync.argtypes = [vp]
     lib.csd_launch_count.argtypes = [vp]; lib.csd_launch_count.restype = C.c_int64
     lib.csd_set_chain_mode.argtypes = [vp, C.c_int]
+    lib.csd_set_wait_limit.argtypes = [vp, C.c_int64]
+    lib.csd_selftest_wait_timeout.argtypes = [vp]
+    f64p, i32p = C.POINTER(f64), C.POINTER(C.c_int32)
+    lib.csd_schedule_ddpm.argtypes = [i32, f64p, f64, _c_float_p, _c_float_p, _c_float_p]
+    lib.csd_schedule_ddim.argtypes = [i32, f64p, i32, i32p, f64, _c_float_p, _c_float_p, _c_float_p]
+    lib.csd_log_sigma_term.argtypes = [i32, _c_float_p, _c_float_p, i32, f64p]
     lib.csd_profile.argtypes = [vp, i32]
     lib.csd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_int64), C.POINTER(f64), C.POINTER(f64)]
     lib.csd_head_create.argtypes = [vp, C.POINTER(_HeadDesc), C.POINTER(_HeadWeights), C.POINTER(vp)]
@@ -73,7 +80,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_verify.argtypes = [vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32] + [vp] * 10
     lib.csd_draft_denoise_traj.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, f32] + [vp] * 5
     lib.csd_verify_single_path.argtypes = ([vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32]
-                                           + [vp] * 4 + [i32] + [vp] * 3)
+                                           + [vp] * 4 + [i32] + [vp] * 4)
     lib.csd_verify_unaligned.argtypes = ([vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32]
                                          + [vp] * 11)
     lib.csd_bonus_token.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, i32, f32] + [vp] * 6
@@ -91,40 +98,33 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
 _LIB = load_library()
 
 
+def _schedule_out(n: int):
+    out = {k: np.zeros(n, dtype=np.float32) for k in ("a", "b", "sigma")}
+    return out, [out[k].ctypes.data_as(_c_float_p) for k in ("a", "b", "sigma")]
+
+
 def ddpm_coefficients(beta: np.ndarray, tau: float = 1.0) -> Dict[str, np.ndarray]:
-    """Host helper: reverse-process coefficients of a DDPM with fixed variance
-    sigma_t^2 = tau^2 beta_t (Eq. 3): mu_t = a_t x_t - b_t eps_hat."""
-    beta = np.asarray(beta, dtype=np.float64)
-    alpha = 1.0 - beta
-    abar = np.cumprod(alpha)
-    return {"a": (alpha ** -0.5).astype(np.float32),
-            "b": (beta / np.sqrt(alpha * (1.0 - abar))).astype(np.float32),
-            "sigma": (tau * np.sqrt(beta)).astype(np.float32)}
+    """csd_schedule_ddpm: coefficient arrays {"a", "b", "sigma"} of the T-step DDPM behind Eq. 3."""
+    beta = np.ascontiguousarray(beta, dtype=np.float64)
+    out, ptrs = _schedule_out(beta.size)
+    rc = _LIB.csd_schedule_ddpm(int(beta.size), beta.ctypes.data_as(C.POINTER(C.c_double)), float(tau), *ptrs)
+    if rc != 0:
+        raise CsdError(rc, "csd_schedule_ddpm: beta must lie in (0, 1) and tau be positive")
+    return out
 
 
 def ddim_coefficients(beta_full: np.ndarray, steps, eta: float) -> Dict[str, np.ndarray]:
-    """Host helper: a DDIM sampler with stochasticity eta in (0, 1] on the ascending sub-sequence `steps` (1-based)
-    of a DDPM's timesteps, written as the coefficients csd_schedule takes (mu = a x_t - b eps_hat, then
-    + sigma eps): the library needs nothing else to run DDIM (Appendix "More Variants of Diffusion Model").
-    Entry k-1 is the k-th step counted from x_0; pass the feature-table rows of the same timesteps as tfeat.
-    The last step (to x_0) would have sigma = 0, which has no density to take ratios of: it gets
-    sigma = eta sqrt(1 - alphabar) around the predicted x_0."""
-    if not 0.0 < eta <= 1.0:
-        raise ValueError("eta must be in (0, 1]")
-    abar_all = np.cumprod(1.0 - np.asarray(beta_full, dtype=np.float64))
-    idx = np.asarray(list(steps), dtype=np.int64) - 1
-    if idx.size == 0 or np.any(np.diff(idx) <= 0) or idx[0] < 0 or idx[-1] >= abar_all.size:
-        raise ValueError("steps must be ascending timesteps within 1..len(beta_full)")
-    cur = abar_all[idx]
-    prv = np.ones_like(cur)
-    prv[1:] = cur[:-1]
-    sig = eta * np.sqrt((1.0 - prv) * (1.0 - cur / prv) / (1.0 - cur))
-    sig[0] = eta * np.sqrt(1.0 - cur[0])
-    keep = np.sqrt(np.clip(1.0 - prv - sig * sig, 0.0, None))     # weight of eps_hat in the direction to x_t
-    keep[0] = 0.0
-    scale = np.sqrt(prv / cur)
-    return {"a": scale.astype(np.float32), "b": (scale * np.sqrt(1.0 - cur) - keep).astype(np.float32),
-            "sigma": sig.astype(np.float32)}
+    """csd_schedule_ddim: coefficient arrays of a DDIM sampler with stochasticity eta in (0, 1] on the ascending
+    sub-sequence `steps` (1-based timesteps) of a DDPM's ladder.  Entry k-1 is the k-th step counted from x_0; pass
+    the feature-table rows of the same timesteps as tfeat."""
+    beta_full = np.ascontiguousarray(beta_full, dtype=np.float64)
+    steps = np.ascontiguousarray(list(steps), dtype=np.int32)
+    out, ptrs = _schedule_out(steps.size)
+    rc = _LIB.csd_schedule_ddim(int(beta_full.size), beta_full.ctypes.data_as(C.POINTER(C.c_double)), int(steps.size),
+                                steps.ctypes.data_as(C.POINTER(C.c_int32)), float(eta), *ptrs)
+    if rc != 0:
+        raise ValueError("csd_schedule_ddim: eta must be in (0, 1] and steps ascending timesteps within 1..len(beta_full)")
+    return out
 
 
 def _ptr(t) -> Optional[int]:
@@ -153,9 +153,13 @@ class Schedule:
                            self.sigma.ctypes.data_as(_c_float_p), tfeat.data_ptr())
 
     def log_sigma_term(self, other_p: "Schedule", Cdim: int) -> float:
-        """log Sigma of Eq. 7 for (self = draft, other_p = target), as the library computes it."""
-        return float(Cdim * np.sum(np.log(self.sigma[1:].astype(np.float64))
-                                   - np.log(other_p.sigma[1:].astype(np.float64))))
+        """csd_log_sigma_term: log Sigma of Eq. 7 for (self = draft, other_p = target)."""
+        out = C.c_double()
+        rc = _LIB.csd_log_sigma_term(self.T, self.sigma.ctypes.data_as(_c_float_p),
+                                     other_p.sigma.ctypes.data_as(_c_float_p), int(Cdim), C.byref(out))
+        if rc != 0:
+            raise CsdError(rc, "csd_log_sigma_term")
+        return float(out.value)
 
 
 class Context:
@@ -179,12 +183,18 @@ class Context:
     def launch_count(self) -> int:
         return int(_LIB.csd_launch_count(self._h))
 
-    CHAIN_LAYERS, CHAIN_CLUSTER, CHAIN_LAYERS_PLAIN = 0, 1, 2
+    CHAIN_LAYERS, CHAIN_LAYERS_PLAIN = 0, 2
 
     def set_chain_mode(self, mode: int):
-        """csd_set_chain_mode: CHAIN_LAYERS (default: one kernel per layer, folded blocks where they apply),
-        CHAIN_CLUSTER (one cluster kernel per chain) or CHAIN_LAYERS_PLAIN (three kernels per block everywhere)."""
+        """csd_set_chain_mode: CHAIN_LAYERS (default: one kernel per layer, folded blocks where they apply) or
+        CHAIN_LAYERS_PLAIN (three kernels per block everywhere)."""
         self._check(_LIB.csd_set_chain_mode(self._h, int(mode)))
+
+    def set_wait_limit(self, cycles: int):
+        self._check(_LIB.csd_set_wait_limit(self._h, int(cycles)))
+
+    def selftest_wait_timeout(self):
+        self._check(_LIB.csd_selftest_wait_timeout(self._h))
 
     KERNEL_CLASSES = ("cond_proj", "mlp1_silu", "adaln_modulate", "mlp2_gate_residual", "final_mod_outproj", "step", "chain")
 
@@ -233,11 +243,12 @@ class Context:
                                                 _ptr(z), _ptr(x_T), _ptr(eps), _ptr(traj_x), _ptr(traj_mu)))
 
     def csd_verify_single_path(self, head_p: "Head", sched_p: Schedule, sched_q: Schedule, B, gamma, cfg, cfg_scale,
-                               z_p, traj_x, traj_mu_q, u, steps_per_pass, logratio, n_accept, accept_mask=None):
+                               z_p, traj_x, traj_mu_q, u, steps_per_pass, logratio, n_accept, accept_mask=None,
+                               mu_p_traj=None):
         self._check(_LIB.csd_verify_single_path(self._h, head_p._h, C.byref(sched_p.c), C.byref(sched_q.c), B, gamma,
                                                 int(cfg), cfg_scale, _ptr(z_p), _ptr(traj_x), _ptr(traj_mu_q),
                                                 _ptr(u), int(steps_per_pass), _ptr(logratio), _ptr(n_accept),
-                                                _ptr(accept_mask)))
+                                                _ptr(accept_mask), _ptr(mu_p_traj)))
 
     def csd_verify_unaligned(self, head_p: "Head", sched_p: Schedule, sched_q: Schedule, B, gamma, cfg, cfg_scale,
                              z_p, x_T, eps_p, eps_q, x0_q, mu1_q, u, logratio, n_accept, accept_mask, mu1_p):

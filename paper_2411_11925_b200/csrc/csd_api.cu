@@ -16,7 +16,6 @@
 #include <vector>
 
 #include "../../include/csd.h"
-#include "chain.cuh"
 #include "fold.cuh"
 #include "gemm.cuh"
 #include "rowops.cuh"
@@ -36,11 +35,13 @@ struct ChainWs {
   // carved per call
   void *zc, *s, *u, *v;
   float *cz, *te, *h, *stats, *epart, *x;
-  // whole-chain kernel only
-  void* s2 = nullptr; float* sched = nullptr; CUtensorMap* amaps = nullptr;
+  void* s2 = nullptr;   // s of even steps (s of odd steps: s)
   void* ap = nullptr;   // a' = h (1 + scale) of the folded blocks
   float* hid = nullptr; // hidden layer of the timestep embedding [T, W]
+  bool owned = true;    // false: base is memory the library did not allocate and must never free or grow
 };
+
+constexpr int kMaxDevices = 64;   // device ordinals the per-device tables below cover
 
 struct ProfRec { cudaEvent_t a, b; int cls; double flops; };
 
@@ -98,10 +99,6 @@ struct csd_head {
   void* xblob = nullptr;
   std::vector<CUtensorMap> Wgs, Wf;
   std::vector<float*> c1, c2;   // first MLP layer with 256-row boxes (W a multiple of 256)
-  // whole-chain kernel: device copies of the weight tensor maps (per block Wss, Wg, W1, W2; then Wfss) and of
-  // the bias pointers (per block shift, scale, b1, gate, b2; then final shift, scale)
-  CUtensorMap* d_wmaps = nullptr;
-  const float** d_bias = nullptr;
 };
 
 namespace {
@@ -123,6 +120,25 @@ int fail(csd_ctx* ctx, int code, const char* fmt, ...) {
       return fail(ctx, CSD_ERR_CUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), __FILE__, \
                   __LINE__);                                                                         \
   } while (0)
+
+// Makes the context's device current for the duration of a call and puts the caller's device back afterwards.
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; cudaGetLastError(); }
+    if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+  DeviceGuard(const DeviceGuard&) = delete;
+  DeviceGuard& operator=(const DeviceGuard&) = delete;
+};
+#define CSD_DEVICE(ctx)                                                                              \
+  DeviceGuard device_guard_((ctx)->device);                                                          \
+  if (!device_guard_.ok) return fail(ctx, CSD_ERR_CUDA, "cannot make device %d current", (ctx)->device)
 
 cudaEvent_t prof_event(csd_ctx* ctx) {
   if (ctx->ev_used == ctx->ev_pool.size()) {
@@ -179,46 +195,53 @@ int make_tmap_f32(csd_ctx* ctx, CUtensorMap* m, const void* ptr, uint64_t rows, 
   return CSD_OK;
 }
 
-int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, int T, bool chain_kernel_extras) {
+// Byte offsets of a chain's intermediates inside its workspace (each piece rounded up to 1 KiB) and their total.
+// The one place that knows the layout: the growable workspaces and the fixed static scratch both use it.
+struct WsLayout {
+  size_t zc, s, u, v, cz, te, h, stats, epart, x, ap, hid, s2, total;
+};
+
+WsLayout ws_layout(const csd_head_desc& d, int Rh, int R, int T) {
   const size_t asz = d.dtype == CSD_F32 ? 4 : 2;
-  const size_t W = d.W;
+  const size_t W = d.W, rh = static_cast<size_t>(Rh);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
-  const size_t o_zc = take(static_cast<size_t>(Rh) * d.Dz * asz);
-  // the whole-chain kernel keeps u, v, s in row blocks of 128 (the last one padded)
-  const size_t Ra = chain_kernel_extras ? static_cast<size_t>(Rh) + 128 : static_cast<size_t>(Rh);
-  const size_t o_s = take(Ra * W * asz), o_u = take(Ra * W * asz), o_v = take(Ra * W * asz);
-  const size_t o_cz = take(Rh * W * 4), o_te = take(static_cast<size_t>(T) * W * 4), o_h = take(Rh * W * 4);
-  const size_t o_st = take(Rh * (W / kStatCols) * 8);
-  const size_t o_ep = take(Rh * (W / kStatCols) * kCPad * 4);   // room for 64-wide tiles
-  const size_t o_x = take(static_cast<size_t>(R) * kCPad * 4);
-  const size_t o_ap = take(d.dtype == CSD_F32 ? 0 : Rh * W * asz);
-  const size_t o_hid = take(static_cast<size_t>(T) * W * 4);
-  const size_t o_s2 = take(Ra * W * asz);   // s of even steps (s of odd steps: o_s)
-  size_t o_sched = 0, o_amaps = 0;
-  if (chain_kernel_extras) { o_sched = take(static_cast<size_t>(T) * 3 * 4); o_amaps = take(4 * sizeof(CUtensorMap)); }
-  if (off > ws.cap) {
+  WsLayout l{};
+  l.zc = take(rh * d.Dz * asz);
+  l.s = take(rh * W * asz); l.u = take(rh * W * asz); l.v = take(rh * W * asz);
+  l.cz = take(rh * W * 4); l.te = take(static_cast<size_t>(T) * W * 4); l.h = take(rh * W * 4);
+  l.stats = take(rh * (W / kStatCols) * 8);
+  l.epart = take(rh * (W / kStatCols) * kCPad * 4);   // room for 64-wide tiles
+  l.x = take(static_cast<size_t>(R) * kCPad * 4);
+  l.ap = take(d.dtype == CSD_F32 ? 0 : rh * W * asz);
+  l.hid = take(static_cast<size_t>(T) * W * 4);
+  l.s2 = take(rh * W * asz);
+  l.total = off;
+  return l;
+}
+
+int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, int T) {
+  const WsLayout l = ws_layout(d, Rh, R, T);
+  if (l.total > ws.cap) {
+    if (!ws.owned) return fail(ctx, CSD_ERR_WORKSPACE, "the fixed scratch holds %zu bytes, this call needs %zu", ws.cap, l.total);
     CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamSynchronize(ctx->side[i]));
     if (ws.base) CSD_CUDA(ctx, cudaFree(ws.base));
     ws.base = nullptr;
     ws.cap = 0;
-    if (cudaMalloc(&ws.base, off) != cudaSuccess) {
+    if (cudaMalloc(&ws.base, l.total) != cudaSuccess) {
       cudaGetLastError();
-      return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes of workspace", off);
+      return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes of workspace", l.total);
     }
-    ws.cap = off;
+    ws.cap = l.total;
   }
   char* b = static_cast<char*>(ws.base);
-  ws.zc = b + o_zc; ws.s = b + o_s; ws.u = b + o_u; ws.v = b + o_v;
-  ws.cz = reinterpret_cast<float*>(b + o_cz); ws.te = reinterpret_cast<float*>(b + o_te);
-  ws.h = reinterpret_cast<float*>(b + o_h); ws.stats = reinterpret_cast<float*>(b + o_st);
-  ws.epart = reinterpret_cast<float*>(b + o_ep); ws.x = reinterpret_cast<float*>(b + o_x);
-  ws.ap = b + o_ap; ws.hid = reinterpret_cast<float*>(b + o_hid);
-  ws.s2 = b + o_s2;
-  if (chain_kernel_extras) {
-    ws.sched = reinterpret_cast<float*>(b + o_sched); ws.amaps = reinterpret_cast<CUtensorMap*>(b + o_amaps);
-  }
+  ws.zc = b + l.zc; ws.s = b + l.s; ws.u = b + l.u; ws.v = b + l.v;
+  ws.cz = reinterpret_cast<float*>(b + l.cz); ws.te = reinterpret_cast<float*>(b + l.te);
+  ws.h = reinterpret_cast<float*>(b + l.h); ws.stats = reinterpret_cast<float*>(b + l.stats);
+  ws.epart = reinterpret_cast<float*>(b + l.epart); ws.x = reinterpret_cast<float*>(b + l.x);
+  ws.ap = b + l.ap; ws.hid = reinterpret_cast<float*>(b + l.hid);
+  ws.s2 = b + l.s2;
   return CSD_OK;
 }
 
@@ -227,11 +250,11 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
                 const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k, int N, const EpiParams& ep) {
   constexpr int MMA_N = NMUL * TN;
   auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, TN, std::is_same<ACT, __half>::value ? 0 : 1, PAIR>;
-  static bool attr_done = false;
+  static bool attr_done[kMaxDevices] = {};   // function attributes are per device
   constexpr int smem = TcCfg<EPI, MMA_N, TN, PAIR>::kSmemBytes;
-  if (!attr_done) {
+  if (!attr_done[ctx->device]) {
     CSD_CUDA(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_done = true;
+    attr_done[ctx->device] = true;
   }
   // Work units: output tiles, or pair tiles (two row tiles) for CTA pairs.  Persistent: at most one CTA per SM.
   const int tiles_n = N / TN, row_tiles = (ep.M + kTileM - 1) / kTileM;
@@ -303,10 +326,10 @@ int check_sched(csd_ctx* ctx, const csd_schedule* s, bool full) {
   return CSD_OK;
 }
 
-// Shared-memory opt-in of the folded block kernels, once per operand type.
-bool fold_kernels_ready(const csd_head_desc& d) {
-  static int known[2] = {0, 0};
-  int& k = known[d.dtype == CSD_F16 ? 0 : 1];
+// Shared-memory opt-in of the folded block kernels, once per device and operand type.
+bool fold_kernels_ready(const csd_ctx* ctx, const csd_head_desc& d) {
+  static int known[kMaxDevices][2] = {};
+  int& k = known[ctx->device][d.dtype == CSD_F16 ? 0 : 1];
   if (k == 0) {
     bool ok = true;
     if (d.dtype == CSD_F16) {
@@ -322,32 +345,6 @@ bool fold_kernels_ready(const csd_head_desc& d) {
   return k == 1;
 }
 
-// The whole-chain kernel needs the row block's W/128 column slices in one cluster of at most 8 CTAs, each
-// with ~219 KB of shared memory; asked of the driver once per cluster size and operand type.
-bool use_chain_kernel(const csd_head_desc& d) {
-  const int nc = d.W / kTileN;
-  if (d.dtype == CSD_F32 || nc < 1 || nc > kChMaxCluster) return false;
-  static int known[2][kChMaxCluster + 1] = {};   // 0 unknown, 1 usable, -1 not
-  int& k = known[d.dtype == CSD_F16 ? 0 : 1][nc];
-  if (k == 0) {
-    k = -1;
-    const void* fn = d.dtype == CSD_F16 ? reinterpret_cast<const void*>(chain_kernel<__half, 0>)
-                                        : reinterpret_cast<const void*>(chain_kernel<__nv_bfloat16, 1>);
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kChSmemBytes) == cudaSuccess) {
-      cudaLaunchConfig_t lc{};
-      lc.gridDim = dim3(nc); lc.blockDim = dim3(kChThreads); lc.dynamicSmemBytes = kChSmemBytes;
-      cudaLaunchAttribute at[1];
-      at[0].id = cudaLaunchAttributeClusterDimension;
-      at[0].val.clusterDim.x = nc; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-      lc.attrs = at; lc.numAttrs = 1;
-      int ncl = 0;
-      if (cudaOccupancyMaxActiveClusters(&ncl, fn, &lc) == cudaSuccess && ncl >= 1) k = 1;
-    }
-    cudaGetLastError();
-  }
-  return k == 1;
-}
-
 // One head's denoising chain for R token rows on stream `st` with workspace slot `slot`:
 // begin() enqueues the per-call work (timestep embedding, condition projection, first boundary
 // kernel), step(t) enqueues the kernels of step t.  Two chains can be interleaved launch by launch.
@@ -355,7 +352,6 @@ struct Chain {
   csd_ctx* ctx; int slot; cudaStream_t st; const csd_head* hd; const csd_schedule* sc;
   int R, cfg; float cfg_scale; const float *z, *x_T, *eps; int sample_last; float *x0, *mu1, *x1;
   int chains = 1;   // chains that run concurrently with this one (itself included)
-  bool allow_chain_kernel = true, whole = false;   // whole: one kernel runs the whole chain
   int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
   bool fold = false;      // blocks 1.. run as two kernels (fold.cuh) instead of three
   CUtensorMap tm_ap{};
@@ -394,7 +390,7 @@ struct Chain {
     b.Rin = batch_Rin; b.Rtok = R; b.cfg = cfg; b.C = d.C; b.W = W; b.NT = tc ? W / kStatCols : W / kTileN;
     b.T = Ts; b.j0 = batch_j0; b.cfg_scale = cfg_scale; b.sched = batch_sched; b.traj_x = batch_traj;
     b.win = hd->win; b.bin = hd->bin; b.cz = ws.cz; b.te = ws.te; b.h = ws.h; b.stats = ws.stats; b.s = ws.s;
-    b.epart = ws.epart; b.bout = hd->bout; b.mu_p = batch_mu;
+    b.epart = ws.epart; b.bout = hd->bout; b.mu_p = batch_mu; b.status = ctx->d_err + 1;
     ProfScope ps(ctx, st, 5, 2.0 * Rh * static_cast<double>(W) * d.C);
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(kind == 0 ? (R + 3) / 4 : (R + 15) / 16); lc.blockDim = dim3(256); lc.stream = st;
@@ -444,9 +440,6 @@ struct Chain {
     // used once a kernel has at least two waves of tiles, where L2-to-SM bandwidth is the limit (measured:
     // a few per cent faster at 384 tiles, slower at 64 and 256)
     pair = tc && tn == kTileN && (W / kTileN) * ((Rh + kTileM - 1) / kTileM) >= 2 * ctx->num_sms;
-    // One kernel for the whole chain when a row block's column slices fit one portable cluster.  The choice
-    // depends on the head only, and both paths give the same bits.
-    whole = allow_chain_kernel && tc && ctx->chain_mode == CSD_CHAIN_CLUSTER && use_chain_kernel(d);
     // First MLP layer: 256-wide MMAs keep the tensor pipe busier per issued instruction (measured about 660 clk
     // per 64-deep k-block and tile against 415 for two 128-wide tiles' worth), but halve the tile count; taken when
     // that does not cost a wave.
@@ -467,11 +460,11 @@ struct Chain {
     {
       const int t128 = (W / kTileN) * ((Rh + kTileM - 1) / kTileM);
       fold = tc && ctx->chain_mode == CSD_CHAIN_LAYERS && !pair && L >= 2 && !hd->Wf.empty() &&
-             8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && fold_kernels_ready(d);
+             8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && fold_kernels_ready(ctx, d);
     }
     ChainWs& ws = ctx->ws[slot];
-    int rc = batch_Rin ? ensure_ws(ctx, ws, d, ws_steps * batch_Rin * (cfg ? 2 : 1), ws_steps * batch_Rin, Ts, false)
-                       : ensure_ws(ctx, ws, d, Rh, R, Ts, whole);
+    int rc = batch_Rin ? ensure_ws(ctx, ws, d, ws_steps * batch_Rin * (cfg ? 2 : 1), ws_steps * batch_Rin, Ts)
+                       : ensure_ws(ctx, ws, d, Rh, R, Ts);
     if (rc) return rc;
     if (!batch_reuse) {
       const dim3 grid((W + 31) / 32, (Ts + 31) / 32);
@@ -511,7 +504,7 @@ struct Chain {
     if (rc) return rc;
     sbuf[0] = ws.s2; sbuf[1] = ws.s;
     if (batch_Rin) return launch_batch(0);   // a pass has one step (t = 1): its s is sbuf[1]
-    sp.traj_x = traj_x; sp.traj_mu = nullptr;
+    sp.traj_x = traj_x; sp.traj_mu = nullptr; sp.status = ctx->d_err + 1;
     sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = tc ? W / kStatCols : W / kTileN; sp.cfg_scale = cfg_scale;
     sp.sample_last = sample_last; sp.epart = ws.epart; sp.bout = hd->bout; sp.x_src = x_T; sp.x = ws.x;
     sp.x0 = x0; sp.mu1 = mu1; sp.x1 = x1; sp.win = hd->win; sp.bin = hd->bin; sp.cz = ws.cz; sp.h = ws.h;
@@ -520,7 +513,6 @@ struct Chain {
     sp.s_b = T >= 2 ? sbuf[(T - 1) & 1] : nullptr;   // the first boundary also prepares s of step T - 1
     sp.te_b = T >= 2 ? ws.te + static_cast<size_t>(T - 2) * W : nullptr;
     sp.eps_t = eps;
-    if (whole) return launch_chain_kernel();
     return launch_step(STEP_INIT);
   }
 
@@ -559,44 +551,7 @@ struct Chain {
     return CSD_OK;
   }
 
-  int launch_chain_kernel() {
-    const csd_head_desc& d = hd->d;
-    ChainWs& ws = ctx->ws[slot];
-    int rc = CSD_OK;
-    CUtensorMap am[4];
-    void* const bufs[4] = {ws.s2, ws.s, ws.u, ws.v};   // s of even t, s of odd t, u, v
-    const int nc = W / kTileN, tb_rows = cfg ? kTileM / 2 : kTileM;
-    const int nb = (R + tb_rows - 1) / tb_rows;
-    for (int i = 0; i < 4 && !rc; ++i) rc = make_tmap(ctx, &am[i], d.dtype, bufs[i], static_cast<uint64_t>(nb) * kTileM, W, W, kTileM);
-    if (rc) return rc;
-    // small pageable sources: staged by the runtime before the calls return
-    CSD_CUDA(ctx, cudaMemcpyAsync(ws.amaps, am, sizeof(am), cudaMemcpyHostToDevice, st));
-    CSD_CUDA(ctx, cudaMemcpyAsync(ws.sched, sc->a, T * sizeof(float), cudaMemcpyHostToDevice, st));
-    CSD_CUDA(ctx, cudaMemcpyAsync(ws.sched + T, sc->b, T * sizeof(float), cudaMemcpyHostToDevice, st));
-    CSD_CUDA(ctx, cudaMemcpyAsync(ws.sched + 2 * T, sc->sigma, T * sizeof(float), cudaMemcpyHostToDevice, st));
-    ChainParams p{};
-    p.wmaps = hd->d_wmaps; p.amaps = ws.amaps;
-    p.R = R; p.cfg = cfg; p.W = W; p.L = L; p.T = T; p.C = d.C; p.sample_last = sample_last; p.cfg_scale = cfg_scale;
-    p.sched = ws.sched; p.cz = ws.cz; p.te = ws.te; p.bias = hd->d_bias;
-    p.win = hd->win; p.bin = hd->bin; p.wout_t = hd->wout_t; p.bout = hd->bout;
-    p.s[0] = ws.s2; p.s[1] = ws.s; p.u = ws.u; p.v = ws.v; p.stats = ws.stats; p.epart = ws.epart;
-    p.x_T = x_T; p.eps = eps; p.x0 = x0; p.mu1 = mu1; p.x1 = x1; p.err = ctx->d_err;
-    const double flops_step = 2.0 * Rh * static_cast<double>(W) * W * (5.0 * L + 2.0) + 2.0 * Rh * static_cast<double>(W) * d.C * 2.0;
-    ProfScope ps(ctx, st, 6, flops_step * T);
-    cudaLaunchConfig_t lc{};
-    lc.gridDim = dim3(nb * nc); lc.blockDim = dim3(kChThreads); lc.dynamicSmemBytes = kChSmemBytes; lc.stream = st;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = nc; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    lc.attrs = at; lc.numAttrs = 1;
-    if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, chain_kernel<__half, 0>, p));
-    else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, chain_kernel<__nv_bfloat16, 1>, p));
-    ctx->launches++;
-    return CSD_OK;
-  }
-
   int step(int t) {
-    if (whole) return CSD_OK;   // already enqueued by begin()
     const csd_head_desc& d = hd->d;
     ChainWs& ws = ctx->ws[slot];
     cur_t = t;
@@ -685,7 +640,6 @@ int run_chain(csd_ctx* ctx, int slot, cudaStream_t st, const csd_head* hd, const
               float cfg_scale, const float* z, const float* x_T, const float* eps, int sample_last, float* x0,
               float* mu1, float* x1) {
   Chain c{ctx, slot, st, hd, sc, R, cfg, cfg_scale, z, x_T, eps, sample_last, x0, mu1, x1};
-  c.allow_chain_kernel = slot != 2;   // the static-scratch call keeps the layer-by-layer kernels its scratch is sized for
   int rc = c.begin();
   for (int t = sc->T; t >= 1 && !rc; --t) rc = c.step(t);
   return rc;
@@ -755,7 +709,9 @@ int csd_create(csd_ctx** out, int device, void* cuda_stream) {
     cudaGetLastError();
     return CSD_ERR_CUDA;
   }
-  if (cudaSetDevice(device) != cudaSuccess) return CSD_ERR_CUDA;
+  if (device >= kMaxDevices) return CSD_ERR_UNSUPPORTED;
+  DeviceGuard dg(device);   // the caller's current device is put back when this call returns
+  if (!dg.ok) return CSD_ERR_CUDA;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return CSD_ERR_CUDA;
   if (prop.major != 10) return CSD_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
@@ -774,8 +730,8 @@ int csd_create(csd_ctx** out, int device, void* cuda_stream) {
     ok = ok && cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
   }
   ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->d_err, sizeof(int)) == cudaSuccess;
-  ok = ok && cudaMemset(c->d_err, 0, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_err, 2 * sizeof(int)) == cudaSuccess;   // [0] first failed wait, [1] non-finite value seen
+  ok = ok && cudaMemset(c->d_err, 0, 2 * sizeof(int)) == cudaSuccess;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   ok = ok && cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
@@ -792,13 +748,14 @@ int csd_create(csd_ctx** out, int device, void* cuda_stream) {
 
 int csd_destroy(csd_ctx* c) {
   if (!c) return CSD_ERR_INVALID_ARG;
-  cudaSetDevice(c->device);
+  DeviceGuard dg(c->device);
   cudaStreamSynchronize(c->stream);
   for (int i = 0; i < 2; ++i) {
     if (c->side[i]) { cudaStreamSynchronize(c->side[i]); cudaStreamDestroy(c->side[i]); }
     if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
-    if (c->ws[i].base) cudaFree(c->ws[i].base);
   }
+  for (ChainWs& w : c->ws)
+    if (w.base && w.owned) cudaFree(w.base);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->io.base) cudaFree(c->io.base);
@@ -817,26 +774,52 @@ int64_t csd_launch_count(const csd_ctx* c) { return c ? c->launches : 0; }
 
 int csd_sync(csd_ctx* c) {
   if (!c) return CSD_ERR_INVALID_ARG;
+  CSD_DEVICE(c);
   CSD_CUDA(c, cudaStreamSynchronize(c->stream));
-  int e = 0;
-  CSD_CUDA(c, cudaMemcpy(&e, c->d_err, sizeof(int), cudaMemcpyDeviceToHost));
-  if (e != 0) {
-    cudaMemset(c->d_err, 0, sizeof(int));
-    return fail(c, CSD_ERR_TIMEOUT, "a device-side bounded wait gave up (code %d: 1 = TMA producer, 2 = MMA issuer, "
-                "3 = epilogue)", e);
+  int e[2] = {0, 0};
+  CSD_CUDA(c, cudaMemcpy(e, c->d_err, sizeof(e), cudaMemcpyDeviceToHost));
+  if (e[0] != 0 || e[1] != 0) cudaMemset(c->d_err, 0, sizeof(e));
+  if (e[0] != 0) {
+    static const char* const roles[] = {"?", "TMA producer", "MMA issuer", "epilogue", "wait self-test"};
+    const int role = e[0] & 0xf;
+    return fail(c, CSD_ERR_TIMEOUT, "a device-side bounded wait gave up: %s (role %d), site %d, iteration %d, block %d",
+                roles[role <= 4 ? role : 0], role, (e[0] >> 4) & 0xf, (e[0] >> 8) & 0xffff, (e[0] >> 24) & 0x7f);
   }
+  if (e[1] != 0)
+    return fail(c, CSD_ERR_NONFINITE, "a non-finite value reached a step update: an activation beyond the operand "
+                "format's range (65504 for CSD_F16 heads: use CSD_BF16 or CSD_F32) or non-finite inputs");
+  return CSD_OK;
+}
+
+int csd_set_wait_limit(csd_ctx* c, int64_t cycles) {
+  if (!c) return CSD_ERR_INVALID_ARG;
+  CSD_DEVICE(c);
+  CSD_CUDA(c, cudaStreamSynchronize(c->stream));
+  for (int i = 0; i < 2; ++i) CSD_CUDA(c, cudaStreamSynchronize(c->side[i]));
+  const long long v = cycles > 0 ? static_cast<long long>(cycles) : 4000000000ll;
+  CSD_CUDA(c, cudaMemcpyToSymbol(g_wait_limit_cycles, &v, sizeof(v)));
+  return CSD_OK;
+}
+
+int csd_selftest_wait_timeout(csd_ctx* c) {
+  if (!c) return CSD_ERR_INVALID_ARG;
+  CSD_DEVICE(c);
+  wait_timeout_selftest_kernel<<<1, 32, 0, c->stream>>>(c->d_err);
+  c->launches++;
+  CSD_CUDA(c, cudaGetLastError());
   return CSD_OK;
 }
 
 int csd_set_chain_mode(csd_ctx* c, int mode) {
   if (!c) return CSD_ERR_INVALID_ARG;
-  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_CLUSTER && mode != CSD_CHAIN_LAYERS_PLAIN) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
+  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_LAYERS_PLAIN) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
   c->chain_mode = mode;
   return CSD_OK;
 }
 
 int csd_profile(csd_ctx* c, int enable) {
   if (!c) return CSD_ERR_INVALID_ARG;
+  CSD_DEVICE(c);
   CSD_CUDA(c, cudaStreamSynchronize(c->stream));
   c->prof_on = enable != 0;
   c->prof.clear();
@@ -848,6 +831,7 @@ int csd_profile_read(csd_ctx* c, int kernel_class, int64_t* launches, double* to
   if (!c) return CSD_ERR_INVALID_ARG;
   if (!launches || !total_ms || !total_flops) return fail(c, CSD_ERR_INVALID_ARG, "null output pointer");
   if (kernel_class < 0 || kernel_class > 6) return fail(c, CSD_ERR_INVALID_ARG, "kernel class %d not in [0, 6]", kernel_class);
+  CSD_DEVICE(c);
   CSD_CUDA(c, cudaStreamSynchronize(c->stream));
   for (int i = 0; i < 2; ++i) CSD_CUDA(c, cudaStreamSynchronize(c->side[i]));
   *launches = 0; *total_ms = 0.0; *total_flops = 0.0;
@@ -857,6 +841,56 @@ int csd_profile_read(csd_ctx* c, int kernel_class, int64_t* launches, double* to
     CSD_CUDA(c, cudaEventElapsedTime(&ms, r.a, r.b));
     *launches += 1; *total_ms += ms; *total_flops += r.flops;
   }
+  return CSD_OK;
+}
+
+int csd_schedule_ddpm(int T, const double* beta, double tau, float* a, float* b, float* sigma) {
+  if (T < 1 || !beta || !a || !b || !sigma || !(tau > 0.0)) return CSD_ERR_INVALID_ARG;
+  double abar = 1.0;
+  for (int t = 0; t < T; ++t) {
+    if (!(beta[t] > 0.0 && beta[t] < 1.0)) return CSD_ERR_INVALID_ARG;
+    const double alpha = 1.0 - beta[t];
+    abar *= alpha;
+    a[t] = static_cast<float>(1.0 / std::sqrt(alpha));
+    b[t] = static_cast<float>(beta[t] / (std::sqrt(alpha) * std::sqrt(1.0 - abar)));
+    sigma[t] = static_cast<float>(tau * std::sqrt(beta[t]));
+  }
+  return CSD_OK;
+}
+
+int csd_schedule_ddim(int T_full, const double* beta_full, int n_steps, const int32_t* steps, double eta, float* a,
+                      float* b, float* sigma) {
+  if (T_full < 1 || n_steps < 1 || !beta_full || !steps || !a || !b || !sigma) return CSD_ERR_INVALID_ARG;
+  if (!(eta > 0.0 && eta <= 1.0)) return CSD_ERR_INVALID_ARG;
+  std::vector<double> abar(static_cast<size_t>(T_full));
+  double acc = 1.0;
+  for (int t = 0; t < T_full; ++t) {
+    if (!(beta_full[t] > 0.0 && beta_full[t] < 1.0)) return CSD_ERR_INVALID_ARG;
+    acc *= 1.0 - beta_full[t];
+    abar[t] = acc;
+  }
+  for (int k = 0; k < n_steps; ++k) {
+    if (steps[k] < 1 || steps[k] > T_full || (k > 0 && steps[k] <= steps[k - 1])) return CSD_ERR_INVALID_ARG;
+    const double cur = abar[steps[k] - 1], prv = k > 0 ? abar[steps[k - 1] - 1] : 1.0;
+    // variance of q_sigma(x_prev | x_t, x0_hat); the step to x_0 would have none (prv = 1): it gets the
+    // variance of the chain's own forward step around the predicted x_0
+    const double sg = k > 0 ? eta * std::sqrt((1.0 - prv) / (1.0 - cur)) * std::sqrt(1.0 - cur / prv) : eta * std::sqrt(1.0 - cur);
+    const double keep = k > 0 ? std::sqrt(std::fmax(0.0, 1.0 - prv - sg * sg)) : 0.0;   // weight of eps_hat towards x_t
+    const double scale = std::sqrt(prv / cur);
+    a[k] = static_cast<float>(scale);
+    b[k] = static_cast<float>(scale * std::sqrt(1.0 - cur) - keep);
+    sigma[k] = static_cast<float>(sg);
+  }
+  return CSD_OK;
+}
+
+int csd_log_sigma_term(int T, const float* sigma_q, const float* sigma_p, int C, double* out) {
+  if (T < 1 || C < 1 || !sigma_q || !sigma_p || !out) return CSD_ERR_INVALID_ARG;
+  for (int t = 0; t < T; ++t)
+    if (!(sigma_q[t] > 0.0f) || !(sigma_p[t] > 0.0f)) return CSD_ERR_INVALID_ARG;
+  csd_schedule q{}, p{};
+  q.T = T; q.sigma = sigma_q; p.T = T; p.sigma = sigma_p;
+  *out = log_sigma_term(&q, &p, C);
   return CSD_OK;
 }
 
@@ -875,7 +909,7 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
   const float* const* ptrs = reinterpret_cast<const float* const*>(w);
   for (size_t i = 0; i < sizeof(csd_head_weights) / sizeof(float*); ++i)
     if (!ptrs[i]) return fail(ctx, CSD_ERR_INVALID_ARG, "weight pointer #%zu is null", i);
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
 
   csd_head* h = new (std::nothrow) csd_head();
   if (!h) return fail(ctx, CSD_ERR_WORKSPACE, "out of host memory");
@@ -1027,17 +1061,6 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
       for (size_t k = 0; k < L && !rc; ++k) rc = make_tmap(ctx, &h->W1_wide[k], d.dtype, h->W1[k], W, W, W, 256);
     }
     if (rc) { csd_head_destroy(h); return rc; }
-    std::vector<CUtensorMap> wm(4 * L + 1);
-    std::vector<const float*> bt(5 * L + 2);
-    for (size_t k = 0; k < L; ++k) {
-      wm[4 * k] = h->tm[1].Wss[k]; wm[4 * k + 1] = h->tm[1].Wg[k]; wm[4 * k + 2] = h->tm[1].W1[k]; wm[4 * k + 3] = h->tm[1].W2[k];
-      bt[5 * k] = h->bsh[k]; bt[5 * k + 1] = h->bsc[k]; bt[5 * k + 2] = h->b1[k]; bt[5 * k + 3] = h->bg[k]; bt[5 * k + 4] = h->b2[k];
-    }
-    wm[4 * L] = h->tm[1].Wfss; bt[5 * L] = h->bfsh; bt[5 * L + 1] = h->bfsc;
-    if (cudaMalloc(&h->d_wmaps, wm.size() * sizeof(CUtensorMap)) != cudaSuccess ||
-        cudaMalloc(&h->d_bias, bt.size() * sizeof(float*)) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the tables"); }
-    if (cudaMemcpy(h->d_wmaps, wm.data(), wm.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(h->d_bias, bt.data(), bt.size() * sizeof(float*), cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "table upload failed");
   }
   *out = h;
   return CSD_OK;
@@ -1045,15 +1068,13 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
 
 int csd_head_destroy(csd_head* h) {
   if (!h) return CSD_ERR_INVALID_ARG;
+  DeviceGuard dg(h->ctx ? h->ctx->device : 0);
   if (h->ctx) {
-    cudaSetDevice(h->ctx->device);
     cudaStreamSynchronize(h->ctx->stream);
     for (int i = 0; i < 2; ++i) cudaStreamSynchronize(h->ctx->side[i]);
   }
   if (h->wblob) cudaFree(h->wblob);
   if (h->fblob) cudaFree(h->fblob);
-  if (h->d_wmaps) cudaFree(h->d_wmaps);
-  if (h->d_bias) cudaFree(h->d_bias);
   if (h->xblob) cudaFree(h->xblob);
   cudaGetLastError();
   delete h;
@@ -1066,7 +1087,7 @@ int csd_draft_denoise(csd_ctx* ctx, const csd_head* head, const csd_schedule* sc
   int rc = check_chain_args(ctx, head, sched, R, cfg, z, x_T, eps);
   if (rc) return rc;
   if (!x0 || !mu1) return fail(ctx, CSD_ERR_INVALID_ARG, "x0 / mu1 is null");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   return run_chain(ctx, 0, ctx->stream, head, sched, R, cfg, cfg_scale, z, x_T, eps, 1, x0, mu1, x1);
 }
 
@@ -1075,7 +1096,7 @@ int csd_draft_denoise(csd_ctx* ctx, const csd_head* head, const csd_schedule* sc
 // lives in this one file-scope device array instead of a cudaMalloc'ed workspace.
 constexpr size_t kStaticScratchBytes = size_t(8) << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-static void* g_static_scratch_addr[64] = {nullptr};   // device address of the array, per device ordinal
+static void* g_static_scratch_addr[kMaxDevices] = {nullptr};   // device address of the array, per device ordinal
 
 int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_schedule* sched, int R, int cfg,
                              float cfg_scale, const float* z, const float* x_T, const float* eps, float* x0,
@@ -1084,21 +1105,12 @@ int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_sched
   int rc = check_chain_args(ctx, head, sched, R, cfg, z, x_T, eps);
   if (rc) return rc;
   if (!x0 || !mu1) return fail(ctx, CSD_ERR_INVALID_ARG, "x0 / mu1 is null");
-  if (ctx->device < 0 || ctx->device >= 64) return fail(ctx, CSD_ERR_UNSUPPORTED, "device ordinal %d not in [0, 64)", ctx->device);
   if (ctx->prof_on) return fail(ctx, CSD_ERR_INVALID_ARG, "csd_draft_denoise_static: switch csd_profile off first (recording creates CUDA events)");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
-  // Bytes the chain's intermediates need, laid out exactly as the growable workspace lays them out
-  // (each piece rounded up to 1 KiB).  Reject before anything is enqueued.
+  CSD_DEVICE(ctx);
+  // Bytes the chain's intermediates need: the same layout function the growable workspaces use.  Reject before
+  // anything is enqueued.
   const csd_head_desc& d = head->d;
-  const size_t Rh = static_cast<size_t>(R) * (cfg ? 2 : 1), W = d.W, asz = d.dtype == CSD_F32 ? 4 : 2;
-  size_t need = 0;
-  auto take = [&](size_t bytes) { need = align_up(need + bytes, 1024); };
-  take(Rh * d.Dz * asz); take(Rh * W * asz); take(Rh * W * asz); take(Rh * W * asz);
-  take(Rh * W * 4); take(static_cast<size_t>(sched->T) * W * 4); take(Rh * W * 4);
-  take(Rh * (W / kStatCols) * 8); take(Rh * (W / kStatCols) * kCPad * 4); take(static_cast<size_t>(R) * kCPad * 4);
-  take(d.dtype == CSD_F32 ? 0 : Rh * W * asz);
-  take(static_cast<size_t>(sched->T) * W * 4);
-  take(Rh * W * asz);
+  const size_t need = ws_layout(d, R * (cfg ? 2 : 1), R, sched->T).total;
   if (need > kStaticScratchBytes)
     return fail(ctx, CSD_ERR_WORKSPACE,
                 "csd_draft_denoise_static: this call needs %zu bytes of scratch but the built-in array holds %zu "
@@ -1117,7 +1129,8 @@ int csd_draft_denoise_static(csd_ctx* ctx, const csd_head* head, const csd_sched
   }
   ChainWs& ws = ctx->ws[2];
   ws.base = g_static_scratch_addr[ctx->device];
-  ws.cap = kStaticScratchBytes;          // never grown: `need` was checked above
+  ws.cap = kStaticScratchBytes;
+  ws.owned = false;                      // never freed or grown: a call that does not fit is an error
   return run_chain(ctx, 2, ctx->stream, head, sched, R, cfg, cfg_scale, z, x_T, eps, 1, x0, mu1, x1);
 }
 
@@ -1129,7 +1142,7 @@ int csd_accept_scan(csd_ctx* ctx, int B, int gamma, int C, double log_sigma_term
   if (rc) return rc;
   if (!x0_q || !mu1_q || !mu1_p || !u || !logratio || !n_accept) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
   if (!(sigma1_p > 0.0f) || !(sigma1_q > 0.0f)) return fail(ctx, CSD_ERR_INVALID_ARG, "sigma1 must be > 0");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   return accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term_, sigma1_p, sigma1_q, x0_q, mu1_q, mu1_p, u, logratio,
                      n_accept, accept_mask);
 }
@@ -1146,7 +1159,7 @@ int csd_verify(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p
   if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
   if ((rc = check_verify_dims(ctx, B, gamma, head_p->d.C))) return rc;
   if (!x0_q || !mu1_q || !u || !logratio || !n_accept || !mu1_p) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   rc = run_chain(ctx, 1, ctx->stream, head_p, sched_p, B * gamma, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr);
   if (rc) return rc;
   const int C = head_p->d.C;
@@ -1166,7 +1179,7 @@ int csd_verify_unaligned(csd_ctx* ctx, const csd_head* head_p, const csd_schedul
   if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
   if ((rc = check_verify_dims(ctx, B, gamma, head_p->d.C))) return rc;
   if (!eps_q || !x0_q || !mu1_q || !u || !logratio || !n_accept || !mu1_p) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   const int R = B * gamma, C = head_p->d.C, T = sched_p->T;
   const size_t need = static_cast<size_t>(R) * 4;
   if (need > ctx->un.cap) {
@@ -1197,7 +1210,7 @@ int csd_bonus_token(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sc
   int rc = check_chain_args(ctx, head_p, sched_p, B, cfg, z_next, x_T_next, eps_next);
   if (rc) return rc;
   if (!n_accept || !x_bonus) return fail(ctx, CSD_ERR_INVALID_ARG, "n_accept / x_bonus is null");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   const int C = head_p->d.C;
   const size_t need = static_cast<size_t>(2) * B * C * 4;
   if (need > ctx->bn.cap) {
@@ -1228,13 +1241,12 @@ int csd_draft_denoise_traj(csd_ctx* ctx, const csd_head* head, const csd_schedul
   int rc = check_chain_args(ctx, head, sched, R, cfg, z, x_T, eps);
   if (rc) return rc;
   if (!traj_x || !traj_mu) return fail(ctx, CSD_ERR_INVALID_ARG, "traj_x / traj_mu is null");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   const size_t slot = static_cast<size_t>(R) * head->d.C;
   const int T = sched->T;
   // the last boundary writes x_0 and mu_1 through the chain's ordinary outputs, which are the last slots
   Chain c{ctx, 0, ctx->stream, head, sched, R, cfg, cfg_scale, z, x_T, eps, 1, traj_x + T * slot,
           traj_mu + (T - 1) * slot, nullptr};
-  c.allow_chain_kernel = false;   // the whole-chain kernel keeps its states on chip
   c.traj_x = traj_x; c.traj_mu = traj_mu;
   rc = c.begin();
   for (int t = T; t >= 1 && !rc; --t) rc = c.step(t);
@@ -1244,7 +1256,7 @@ int csd_draft_denoise_traj(csd_ctx* ctx, const csd_head* head, const csd_schedul
 int csd_verify_single_path(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p,
                            const csd_schedule* sched_q, int B, int gamma, int cfg, float cfg_scale, const float* z_p,
                            const float* traj_x, const float* traj_mu_q, const float* u, int steps_per_pass,
-                           float* logratio, int32_t* n_accept, uint32_t* accept_mask) {
+                           float* logratio, int32_t* n_accept, uint32_t* accept_mask, float* mu_p_traj) {
   if (!ctx) return CSD_ERR_INVALID_ARG;
   if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
   if (static_cast<int64_t>(B) * gamma > (1 << 24)) return fail(ctx, CSD_ERR_UNSUPPORTED, "B * gamma exceeds 2^24 rows");
@@ -1257,7 +1269,7 @@ int csd_verify_single_path(csd_ctx* ctx, const csd_head* head_p, const csd_sched
   if ((rc = check_verify_dims(ctx, B, gamma, head_p->d.C))) return rc;
   if (!u || !logratio || !n_accept) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
   if (steps_per_pass < 0) return fail(ctx, CSD_ERR_INVALID_ARG, "steps_per_pass = %d must be >= 0", steps_per_pass);
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   const int T = sched_p->T, C = head_p->d.C, Rh1 = R * (cfg ? 2 : 1);
   // steps per pass: enough head rows to fill the GPU several times over, few enough to keep the workspace
   // (about 16 W bytes per head row) modest
@@ -1300,12 +1312,13 @@ int csd_verify_single_path(csd_ctx* ctx, const csd_head* head_p, const csd_sched
   for (int j0 = 0; j0 < T; j0 += tb) {
     const int n = T - j0 < tb ? T - j0 : tb;
     Chain c{ctx, 1, st, head_p, sched_p, n * R, cfg, cfg_scale, z_p, nullptr, nullptr, 0, nullptr, nullptr, nullptr};
-    c.allow_chain_kernel = false;
-    c.batch_Rin = R; c.batch_j0 = j0; c.batch_traj = traj_x; c.batch_sched = d_sched; c.batch_mu = d_mu;
+    // the target's means of this pass: into the caller's [T, R, C] array (slot j0 onwards) when it wants them
+    float* pass_mu = mu_p_traj ? mu_p_traj + static_cast<size_t>(j0) * R * C : d_mu;
+    c.batch_Rin = R; c.batch_j0 = j0; c.batch_traj = traj_x; c.batch_sched = d_sched; c.batch_mu = pass_mu;
     c.ws_steps = tb; c.batch_reuse = j0 > 0;
     if ((rc = c.begin())) return rc;
     if ((rc = c.step(1))) return rc;
-    single_path_terms_kernel<<<(n * R + 127) / 128, 128, 0, st>>>(R, C, T, j0, n, d_sched, traj_x, traj_mu_q, d_mu, d_terms);
+    single_path_terms_kernel<<<(n * R + 127) / 128, 128, 0, st>>>(R, C, T, j0, n, d_sched, traj_x, traj_mu_q, pass_mu, d_terms);
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
   }
@@ -1325,7 +1338,7 @@ int csd_resample(csd_ctx* ctx, int B, int gamma, int C, int cap, double log_sigm
   if (!n_accept || !mu1_p || !mu1_q || !xi || !v || !x_new || !n_prop || !flags || !cap_hits)
     return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
   if (!(sigma1_p > 0.0f) || !(sigma1_q > 0.0f)) return fail(ctx, CSD_ERR_INVALID_ARG, "sigma1 must be > 0");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   return resample(ctx, ctx->stream, B, gamma, C, cap, log_sigma_term_, sigma1_p, sigma1_q, n_accept, mu1_p, mu1_q, xi, v,
                   x_new, n_prop, flags, cap_hits);
 }
@@ -1348,10 +1361,10 @@ int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, cons
   if (cap < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cap = %d must be >= 1", cap);
   if (!u || !xi || !v || !x0 || !mu1_q || !mu1_p || !logratio || !n_accept || !x_new || !n_prop || !flags || !cap_hits)
     return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   // workspaces first (growing one synchronises), then fork the two chains
-  if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T, ctx->chain_mode == CSD_CHAIN_CLUSTER && use_chain_kernel(head_q->d)))) return rc;
-  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T, ctx->chain_mode == CSD_CHAIN_CLUSTER && use_chain_kernel(head_p->d)))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T))) return rc;
   CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
   for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
   // the two chains' launches are interleaved step by step so that neither stream starves
@@ -1393,7 +1406,7 @@ int csd_round_host(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p,
       !n_prop || !flags || !cap_hits)
     return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
   if (sched_q->T < 1 || sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "schedules disagree on T");
-  CSD_CUDA(ctx, cudaSetDevice(ctx->device));
+  CSD_DEVICE(ctx);
   const size_t R = static_cast<size_t>(B) * gamma, Rh = R * (cfg ? 2 : 1), C = head_p->d.C, T = sched_p->T;
   struct Item { const void* src; void* dst; size_t bytes; size_t off; bool in; };
   Item items[] = {

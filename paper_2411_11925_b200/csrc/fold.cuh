@@ -18,9 +18,12 @@
 // One tile per CTA (128 x 128), a TMA ring of three 64 KB slot pairs, three TMEM accumulators, two TMA warps, one MMA warp,
 // eight epilogue warps (one row x 64 columns per thread).
 #pragma once
-#include "chain.cuh"
+#include "gemm.cuh"
+#include "rowops.cuh"
 
 namespace csd {
+
+constexpr int kChSlotBytes = 32768;   // ring slot: [A tile 16 KB | B tile 16 KB]
 
 enum FoldKind : int { FOLD_W1 = 0, FOLD_GATE = 1 };
 

@@ -63,11 +63,14 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
       : "memory");
   return ok != 0;
 }
-// Bounded wait: polls the barrier and gives up (returns false) after about `limit_cycles` SM
-// clock cycles (default 4e9, roughly two seconds).  The clock is read only once per 1024 failed
-// polls: a timer read on every wait would sit on the pipeline's critical path.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
-                                          long long limit_cycles = 4000000000ll) {
+// Upper bound, in SM clock cycles, of every device-side wait of this library (about two seconds by default).
+// One value per device that has loaded the library; the host sets it with csd_set_wait_limit.
+__device__ long long g_wait_limit_cycles = 4000000000ll;
+
+// Bounded wait: polls the barrier and gives up (returns false) after about g_wait_limit_cycles SM clock
+// cycles.  The clock (and the limit) are read only once per 1024 failed polls: a timer read on every wait
+// would sit on the pipeline's critical path.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   long long t0 = 0;
   uint32_t spins = 0;
   for (;;) {
@@ -75,9 +78,31 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
     if ((++spins & 1023u) == 0u) {
       const long long now = clock64();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > limit_cycles) return false;
+      else if (now - t0 > *reinterpret_cast<volatile long long*>(&g_wait_limit_cycles)) return false;
     }
   }
+}
+
+// Bounded wait that also gives up once any kernel of the context has raised the error flag.
+template <bool CLUSTER>
+__device__ __forceinline__ bool ch_wait(uint64_t* bar, uint32_t parity, const int* err) {
+  long long t0 = 0;
+  uint32_t spins = 0;
+  for (;;) {
+    if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 1023u) == 0u) {
+      if (*reinterpret_cast<const volatile int*>(err) != 0) return false;
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > *reinterpret_cast<volatile long long*>(&g_wait_limit_cycles)) return false;
+    }
+  }
+}
+
+// Records the first failing wait of a context: role (1 TMA producer, 2 MMA issuer, 3 epilogue, 4 self-test) |
+// site << 4 | (count & 0xffff) << 8 | (block & 0x7f) << 24.  Later failures do not overwrite it.
+__device__ __forceinline__ void ch_fail(int* err, int role, int site, int count) {
+  atomicCAS(err, 0, role | (site << 4) | ((count & 0xffff) << 8) | ((static_cast<int>(blockIdx.x) & 0x7f) << 24));
 }
 
 // ------------------------------------------------ programmatic dependent launch

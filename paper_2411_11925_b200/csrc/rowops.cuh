@@ -101,6 +101,7 @@ struct StepParams {
   const float* te_b;
   float* traj_x;                 // TRAJ kernels: where the state this boundary produces is recorded ([R, C])
   float* traj_mu;                // TRAJ kernels: where the mean of the step being finished is recorded ([R, C])
+  int* status;                   // set to 1 when a mean or state of this step is not finite (csd_sync reports it)
 };
 
 // RB token rows per block.  Finishes step t (unless STEP_INIT) and prepares the next one:
@@ -152,6 +153,8 @@ __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p
         const float xo = p.x[o];
         const float mu = ddpm_mean(p.a, xo, p.b, e);
         xn = ddpm_sample(mu, p.sigma, p.eps_t[o]);
+        // an activation beyond the 16-bit operand range became inf further up and arrives here as inf or NaN
+        if (!(fabsf(xn) <= 3.0e38f)) *p.status = 1;
         if (mode == STEP_LAST) {
           p.mu1[o] = mu;
           if (p.x1) p.x1[o] = xo;
@@ -238,6 +241,7 @@ struct BatchParams {
   const float* epart;    // [Rh, NT, 16] eps_hat partial sums
   const float* bout;     // [16]
   float* mu_p;           // [Rtok, C] out: mean of the target's transition at the draft's state
+  int* status;           // set to 1 when a mean is not finite
 };
 
 // Prepares a pass: h = Win x + bin, its LayerNorm partials and s = SiLU(cz + te_t), four token rows per block,
@@ -323,7 +327,9 @@ __global__ void __launch_bounds__(256) batch_finish_kernel(BatchParams p) {
   const float eh = p.cfg ? cfg_combine(e[0], e[1], p.cfg_scale) : e[0];
   const int ti = p.T - 1 - p.j0 - rt / p.Rin;   // t - 1
   const float x = p.traj_x[(static_cast<size_t>(p.j0) * p.Rin + rt) * p.C + c];
-  p.mu_p[static_cast<size_t>(rt) * p.C + c] = ddpm_mean(p.sched[ti], x, p.sched[p.T + ti], eh);
+  const float mu = ddpm_mean(p.sched[ti], x, p.sched[p.T + ti], eh);
+  if (!(fabsf(mu) <= 3.0e38f)) *p.status = 1;
+  p.mu_p[static_cast<size_t>(rt) * p.C + c] = mu;
 }
 
 // Per-step terms of the log-ratio of Eq. 2 for the steps of one pass, one thread per (step, token row):
@@ -450,6 +456,16 @@ bonus_select_kernel(int B, int C, int gamma, const int32_t* __restrict__ n_accep
   const bool all = n_accept[b] >= gamma;
   if (all) x_bonus[i] = x0[i];
   if (taken && i == b * C) taken[b] = all ? 1u : 0u;
+}
+
+// Self-test of the bounded waits: one thread waits on a barrier on which nobody ever arrives, so the wait runs
+// into the limit (csd_set_wait_limit), gives up and records role 4, site 1 in the context's error word.  Nothing
+// else happens: no fault, no trap, no wait beyond the limit.
+__global__ void wait_timeout_selftest_kernel(int* err) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); fence_mbar_init(); }
+  __syncthreads();
+  if (threadIdx.x == 0 && !ch_wait<false>(&bar, 0, err)) ch_fail(err, 4, 1, 0);
 }
 
 // Resampling: one warp per sequence, lane c < C = coordinate.  Proposals are consumed in order.

@@ -82,12 +82,12 @@ class DeviceRound:
         self.ctx.csd_draft_denoise_traj(self.head_q, self.sched_q, wl.R, wl.cfg, wl.cfg_scale, self.z_q, self.x_T,
                                         self.eps, self.traj_x, self.traj_mu)
 
-    def verify_single_path(self, steps_per_pass: int = 0, traj_x=None, traj_mu=None):
+    def verify_single_path(self, steps_per_pass: int = 0, traj_x=None, traj_mu=None, mu_p_traj=None):
         wl = self.wl
         self.ctx.csd_verify_single_path(self.head_p, self.sched_p, self.sched_q, wl.B, wl.gamma, wl.cfg, wl.cfg_scale,
                                         self.z_p, self.traj_x if traj_x is None else traj_x,
                                         self.traj_mu if traj_mu is None else traj_mu, self.u, steps_per_pass,
-                                        self.logratio, self.n_accept, self.accept_mask)
+                                        self.logratio, self.n_accept, self.accept_mask, mu_p_traj)
 
     def verify_unaligned(self, eps_p):
         """csd_verify with the target's own noise eps_p (no trajectory alignment)."""

@@ -9,7 +9,7 @@ import torch
 from oracle import csd_oracle as orc
 from paper_2411_11925_b200 import inputs as gen
 
-from _parity import TOL_LOGR, TOL_MU, TOL_X
+from _parity import F32_EPS, K_MEASURED, TOL_LOGR, TOL_MU, TOL_X
 
 pytestmark = pytest.mark.gpu
 
@@ -37,20 +37,37 @@ def _oracle_parts(inp, tau_q=None, tau_p=None):
     return sq, sp, ep, dq
 
 
-def _logr_tolerance(ep, sq, sp, dq, delta_mu):
-    # Each step's term is as ill-conditioned in its mean as Eq. 8 is: d term / d mu = (x_{t-1} - mu) / sigma_t^2.
-    # A per-coordinate error delta_mu in every mean moves the sum by at most
-    # sum_t (sqrt(2 Qp_t) / sigma_p,t + sqrt(2 Qq_t) / sigma_q,t) sqrt(C) delta_mu, Q = |x_{t-1} - mu|^2 / (2 sigma^2).
+# Flat ceilings on the single-path log-ratio error of 16-bit operand heads at the sizes tested here (sum of T terms,
+# each as ill-conditioned in its mean as Eq. 8: |logR| is 1e2..1e3 with unrelated random heads); fp32 meets 5e-2.
+CEIL_SP = {"f32": TOL_LOGR, "f16": 0.15, "bf16": 1.0}
+
+
+def _logr_tolerance(ep, sq, sp, dq, g_mu_p, g_traj_x=None, g_traj_mu=None):
+    """5e-2 + K times the exact first- plus second-order effect, on the sum of Eq. 2, of the errors MEASURED in this
+    run: the target's per-step means (mu_p_traj output of the call) and, when the GPU's own recorded trajectory was
+    scored, its states and draft means.  d term_t / d mu = (x_{t-1} - mu) / sigma_t^2, so each step amplifies its
+    mean error by up to 1e4; with K = 1 the bound is the Taylor expansion itself, K = 2 leaves room for the fp32
+    evaluation.  Also returns the checker's per-step target means."""
     T = len(sq["a"])
-    C = dq["xs"][0].shape[1]
-    cond = 0.0
+    bound, qsum = 0.0, 0.0
     for j in range(T):
         t = T - j
-        mu_p = sp["a"][t - 1] * dq["xs"][j] - sp["b"][t - 1] * ep(dq["xs"][j], t)
-        rp = np.sqrt(np.sum((dq["xs"][j + 1] - mu_p) ** 2, axis=1)) / sp["sigma"][t - 1] ** 2
-        rq = np.sqrt(np.sum((dq["xs"][j + 1] - dq["mus"][j]) ** 2, axis=1)) / sq["sigma"][t - 1] ** 2
-        cond = cond + (rp + rq) * math.sqrt(C)
-    return TOL_LOGR + cond * delta_mu
+        x_t, x_n = dq["xs"][j], dq["xs"][j + 1]
+        mu_p = sp["a"][t - 1] * x_t - sp["b"][t - 1] * ep(x_t, t)
+        vp, vq = sp["sigma"][t - 1] ** 2, sq["sigma"][t - 1] ** 2
+        d_xn = 0.0 if g_traj_x is None else g_traj_x[j + 1].astype(np.float64) - x_n
+        d_mq = 0.0 if g_traj_mu is None else g_traj_mu[j].astype(np.float64) - dq["mus"][j]
+        d_p = g_mu_p[j].astype(np.float64) - mu_p - d_xn          # change of (mu_p - x_{t-1})
+        d_q = d_mq - d_xn
+        bound = bound + np.sum(np.abs(x_n - mu_p) / vp * np.abs(d_p) + np.abs(x_n - dq["mus"][j]) / vq * np.abs(d_q), axis=1) \
+            + np.sum(d_p * d_p, axis=1) / (2 * vp) + np.sum(d_q * d_q, axis=1) / (2 * vq)
+        qsum = qsum + np.sum((x_n - mu_p) ** 2, axis=1) / (2 * vp) + np.sum((x_n - dq["mus"][j]) ** 2, axis=1) / (2 * vq)
+    return TOL_LOGR + K_MEASURED * bound + 8.0 * F32_EPS * qsum
+
+
+def _mu_buffer(dr, wl):
+    T = len(dr.sched_q.sigma)
+    return torch.zeros(T, wl.R, dr.C, dtype=torch.float32, device=dr.dev)
 
 
 def _check_scan(dr, wl, u):
@@ -103,8 +120,8 @@ def test_single_path_logratio_on_the_checkers_trajectory(op, kw):
     dq32 = {"xs": [x.astype(np.float32).astype(np.float64) for x in dq["xs"]],
             "mus": [m.astype(np.float32).astype(np.float64) for m in dq["mus"]]}
     want = orc.log_ratio_single_path(ep, sq, sp, dq32).reshape(wl.B, wl.gamma)
-    tol = _logr_tolerance(ep, sq, sp, dq32, TOL_MU[op]).reshape(wl.B, wl.gamma)
     dr = _device_round(inp, tau_p=0.9 * wl.tau)
+    mu_buf = _mu_buffer(dr, wl)
     tx = torch.from_numpy(np.stack(dq32["xs"]).astype(np.float32)).to(dr.dev)
     tm = torch.from_numpy(np.stack(dq32["mus"]).astype(np.float32)).to(dr.dev)
     from paper_2411_11925_b200 import api
@@ -112,13 +129,13 @@ def test_single_path_logratio_on_the_checkers_trajectory(op, kw):
         dr.ctx.set_chain_mode(mode)
         first = None
         for spp in (0, 1, 3, wl.T):
-            dr.verify_single_path(spp, tx, tm)
+            dr.verify_single_path(spp, tx, tm, mu_p_traj=mu_buf)
             dr.ctx.sync()
             lr, acc = _check_scan(dr, wl, inp.u)
+            tol = _logr_tolerance(ep, sq, sp, dq32, _np(mu_buf)).reshape(wl.B, wl.gamma)
             err = np.abs(lr - want)
             assert np.all(err <= tol), (op, mode, spp, float(err.max()), float((err / tol).max()))
-            if op == "f32":
-                assert err.max() <= TOL_LOGR   # the fp32 path meets the flat stated tolerance
+            assert err.max() <= CEIL_SP[op], (op, mode, spp, float(err.max()))   # fp32: the flat stated 5e-2
             if first is None:
                 first = lr
                 print(op, kw, "mode", mode, "single-path logR err", float(err.max()), "of tol", float((err / tol).max()),
@@ -139,18 +156,18 @@ def test_single_path_end_to_end_matches_checker(op, kw):
     wl = inp.wl
     sq, sp, ep, dq = _oracle_parts(inp)
     want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(wl.B, wl.gamma)
-    # here the target also sees the accumulated error of the draft's trajectory: delta = the trajectory tolerance
-    tol = _logr_tolerance(ep, sq, sp, dq, TOL_X[op] + TOL_MU[op]).reshape(wl.B, wl.gamma)
     dr = _device_round(inp)
+    mu_buf = _mu_buffer(dr, wl)
     dr.draft_traj()
-    dr.verify_single_path()
+    dr.verify_single_path(mu_p_traj=mu_buf)
     dr.ctx.sync()
     lr, acc = _check_scan(dr, wl, inp.u)
+    # here the target also sees the accumulated error of the draft's trajectory: all three measured errors enter
+    tol = _logr_tolerance(ep, sq, sp, dq, _np(mu_buf), _np(dr.traj_x), _np(dr.traj_mu)).reshape(wl.B, wl.gamma)
     err = np.abs(lr - want)
     print(op, kw, "end-to-end single-path logR err", float(err.max()), "of tol", float((err / tol).max()))
     assert np.all(err <= tol)
-    if op == "f32":
-        assert err.max() <= TOL_LOGR
+    assert err.max() <= CEIL_SP[op], (op, float(err.max()))
     dr.ctx.close()
 
 
@@ -222,10 +239,13 @@ def test_unaligned_verify_matches_checker_and_reduces_to_verify(op, kw):
     lr, acc = _check_scan(dr, wl, inp.u)
     assert np.max(np.abs(_np(dr.mu1_p) - dp["mu1"])) <= TOL_MU[op]
     s1q, s1p = sq["sigma"][0], sp["sigma"][0]
-    Qp = np.sum((dq["x0"] - dp["mu1"]) ** 2, axis=1) / (2 * s1p ** 2)
-    Qq = np.sum((dq["x0"] - dq["mu1"]) ** 2, axis=1) / (2 * s1q ** 2)
-    tol = (TOL_LOGR + (np.sqrt(2 * Qp) / s1p + np.sqrt(2 * Qq) / s1q) * 4.0 * TOL_MU[op]).reshape(wl.B, wl.gamma)
-    # fp32 result of magnitude |want|: half an ulp of the sum on top
+    # the steps t >= 2 contribute exact functions of the input noise; the final step is Eq. 8 with this target's
+    # mean: the band comes from the measured errors of x0, mu1_q, mu1_p as in the aligned comparison
+    from _parity import measured_effect
+    effect = measured_effect({"x0": dq["x0"], "mu1_q": dq["mu1"], "mu1_p": dp["mu1"]},
+                             {"x0": _np(dr.x0), "mu1_q": _np(dr.mu1_q), "mu1_p": _np(dr.mu1_p)}, s1q, s1p)
+    tol = (TOL_LOGR + K_MEASURED * effect).reshape(wl.B, wl.gamma)
+    # fp32 result of magnitude |want|: a few ulp of the sum on top
     tol = tol + 1e-6 * np.abs(want)
     err = np.abs(lr - want)
     print(op, kw, "unaligned logR err", float(err.max()), "of tol", float((err / tol).max()), "median |logR|",
@@ -260,23 +280,26 @@ def test_mar256_full_size_single_path_sampled_sequences():
     wl = gen.WORKLOADS["mar256"]
     inp = gen.make_round_inputs(wl)
     dr = _device_round(inp)
+    mu_buf = _mu_buffer(dr, wl)
     dr.draft_traj()
-    dr.verify_single_path()
+    dr.verify_single_path(mu_p_traj=mu_buf)
     dr.ctx.sync()
     lr, acc = _check_scan(dr, wl, inp.u)
     assert np.all(np.isfinite(lr))
-    seqs = [0, 63]
+    seqs = [0, 15, 16, 63]       # first, last, both sides of a 128-row tile boundary
     sub = gen.select_sequences(inp, seqs)
     sq, sp, ep, dq = _oracle_parts(sub)
     want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(len(seqs), wl.gamma)
     op = wl.operand_format
-    tol = _logr_tolerance(ep, sq, sp, dq, TOL_X[op] + TOL_MU[op]).reshape(len(seqs), wl.gamma)
     rows = sub.extras["rows"]
+    tol = _logr_tolerance(ep, sq, sp, dq, _np(mu_buf)[:, rows], _np(dr.traj_x)[:, rows],
+                          _np(dr.traj_mu)[:, rows]).reshape(len(seqs), wl.gamma)
     assert np.max(np.abs(_np(dr.traj_x)[:, rows] - np.stack(dq["xs"]))) <= TOL_X[op]
     err = np.abs(lr[seqs] - want)
     print("mar256 single-path: max err", float(err.max()), "of tol", float((err / tol).max()),
           "median |logR|", float(np.median(np.abs(want))))
     assert np.all(err <= tol)
+    assert err.max() <= 0.25, float(err.max())    # measured 0.10 on |logR| of about 1200
     # a second call repeats bit for bit
     dr.verify_single_path()
     dr.ctx.sync()
@@ -292,17 +315,20 @@ def test_ar_stress_full_size_single_path_sampled_sequences():
     inp = gen.make_round_inputs(wl)
     inp.z_p = inp.z_q
     dr = _device_round(inp)
+    mu_buf = _mu_buffer(dr, wl)
     dr.draft_traj()
-    dr.verify_single_path()
+    dr.verify_single_path(mu_p_traj=mu_buf)
     dr.ctx.sync()
     lr, acc = _check_scan(dr, wl, inp.u)
     assert np.all(np.isfinite(lr))
-    seqs = [0, wl.B - 1]
+    seqs = [0, 7, 8, wl.B - 1]
     sub = gen.select_sequences(inp, seqs)
     sq, sp, ep, dq = _oracle_parts(sub)
     want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(len(seqs), wl.gamma)
     op = wl.operand_format
-    tol = _logr_tolerance(ep, sq, sp, dq, TOL_X[op] + TOL_MU[op]).reshape(len(seqs), wl.gamma)
+    rows = sub.extras["rows"]
+    tol = _logr_tolerance(ep, sq, sp, dq, _np(mu_buf)[:, rows], _np(dr.traj_x)[:, rows],
+                          _np(dr.traj_mu)[:, rows]).reshape(len(seqs), wl.gamma)
     err = np.abs(lr[seqs] - want)
     print("ar_stress single-path: max err", float(err.max()), "of tol", float((err / tol).max()),
           "median |logR|", float(np.median(np.abs(want))), "accepted", float(acc.mean()))
@@ -318,12 +344,14 @@ def test_single_path_and_unaligned_degenerate_sizes(kw):
     sq, sp, ep, dq = _oracle_parts(inp)
     want = orc.log_ratio_single_path(ep, sq, sp, dq).reshape(wl.B, wl.gamma)
     dr = _device_round(inp)
+    mu_buf = _mu_buffer(dr, wl)
     dr.draft_traj()
-    dr.verify_single_path(7)          # more steps per pass than there are steps
+    dr.verify_single_path(7, mu_p_traj=mu_buf)          # more steps per pass than there are steps
     dr.ctx.sync()
     lr, acc = _check_scan(dr, wl, inp.u)
-    tol = _logr_tolerance(ep, sq, sp, dq, TOL_X["f32"] + TOL_MU["f32"]).reshape(wl.B, wl.gamma)
+    tol = _logr_tolerance(ep, sq, sp, dq, _np(mu_buf), _np(dr.traj_x), _np(dr.traj_mu)).reshape(wl.B, wl.gamma)
     assert np.all(np.abs(lr - want) <= tol)
+    assert np.max(np.abs(lr - want)) <= TOL_LOGR
     if wl.T == 1:
         # same number as the aligned criterion, which for T = 1 has no step before the last
         dr.draft(); dr.verify(); dr.ctx.sync()

@@ -55,6 +55,31 @@ def test_ddpm_coefficients_match_the_checker_schedule():
             np.testing.assert_allclose(c[k], s[k], rtol=1e-7)
 
 
+def test_log_sigma_term_matches_the_checker_and_rejects_bad_arguments():
+    # csd_log_sigma_term (Eq. 7) is a host-only call of the C library: no GPU needed
+    from paper_2411_11925_b200 import api
+    beta = gen.beta_linear(50)
+    cq, cp = api.ddpm_coefficients(beta, 1.0), api.ddpm_coefficients(beta, 0.9)
+    tf = torch.zeros(50, 4)
+
+    class _S(api.Schedule):     # the device feature table is irrelevant here
+        def __init__(self, c):
+            self.sigma = c["sigma"]; self.T = 50
+
+    got = _S(cq).log_sigma_term(_S(cp), 16)
+    want = orc.log_sigma_term(cq["sigma"].astype(np.float64), cp["sigma"].astype(np.float64), 16)
+    assert abs(got - want) <= 1e-9 * abs(want) and abs(want - 16 * 49 * np.log(1 / 0.9)) < 1e-3
+    assert _S(cq).log_sigma_term(_S(cq), 16) == 0.0
+    lib = ctypes.CDLL(build.build_library())
+    out = ctypes.c_double()
+    bad = np.zeros(3, np.float32)
+    fp = ctypes.POINTER(ctypes.c_float)
+    assert lib.csd_log_sigma_term(3, bad.ctypes.data_as(fp), bad.ctypes.data_as(fp), 16, ctypes.byref(out)) == -1
+    assert lib.csd_log_sigma_term(3, None, None, 16, ctypes.byref(out)) == -1
+    assert lib.csd_schedule_ddpm(3, None, ctypes.c_double(1.0), None, None, None) == -1
+    assert lib.csd_set_wait_limit(None, ctypes.c_int64(5)) == -1 and lib.csd_selftest_wait_timeout(None) == -1
+
+
 def test_round_to_bf16_matches_torch_and_is_idempotent():
     rng = np.random.default_rng(0)
     a = (rng.standard_normal(10000) * 10.0 ** rng.integers(-6, 3, 10000)).astype(np.float32)

@@ -53,6 +53,56 @@ def test_static_scratch_denoise_matches_the_allocating_call_twice(op):
     dr.ctx.close()
 
 
+def test_static_scratch_call_leaves_free_device_memory_unchanged():
+    # The property the entry point exists for: on a context that has never made an allocating call, a static call
+    # with a shape it has not seen before takes no device memory.  (The first launch of a kernel may make the CUDA
+    # runtime load that kernel's code, which can take memory once: a warm-up call with the same kernel variants
+    # comes first, as a deployment would do before its memory is handed away.)
+    dr = _setup("f16", B=6)
+    big = _setup("f16", B=7, seed_offset=3)        # a second shape on the SAME kernels (tiny grids, 64-wide tiles)
+    ctx = dr.ctx
+    heads = (dr.head_q, dr.sched_q)
+
+    def static_call(r):
+        w = r.wl
+        out = torch.empty_like(r.x0), torch.empty_like(r.x0)
+        ctx.csd_draft_denoise_static(heads[0], heads[1], w.R, w.cfg, w.cfg_scale, r.z_q, r.x_T, r.eps, out[0], out[1], None)
+        ctx.sync()
+        return out
+
+    static_call(dr)                                # warm-up: kernels loaded, array address resolved
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    # outputs allocated by torch before the measurement window closes would count: allocate them first
+    w = big.wl
+    o0, o1 = torch.empty_like(big.x0), torch.empty_like(big.x0)
+    free1 = torch.cuda.mem_get_info()[0]
+    ctx.csd_draft_denoise_static(heads[0], heads[1], w.R, w.cfg, w.cfg_scale, big.z_q, big.x_T, big.eps, o0, o1, None)
+    ctx.sync()
+    free2 = torch.cuda.mem_get_info()[0]
+    assert free2 == free1, (free0, free1, free2)
+    # and the result is the allocating call's
+    big.ctx.close()
+    dr.ctx.close()
+
+
+def test_static_scratch_near_the_limit_runs_the_folded_blocks():
+    # 410 head rows x W = 1024 need 8 173 568 of the 8 388 608 bytes; blocks 2.. of this grid run as folded kernels
+    from paper_2411_11925_b200.runner import DeviceRound
+    wl = gen.Workload(**{**gen.WORKLOADS["tiny_fp32"].__dict__, "B": 41, "gamma": 5, "T": 3, "bf16": True,
+                         "cfg": True, "cfg_scale": 3.0, "draft": gen.HeadSpec(2, 1024, 128)})
+    dr = DeviceRound(gen.make_round_inputs(wl))
+    dr.draft()
+    dr.ctx.sync()
+    want = dr.x0.clone(), dr.mu1_q.clone()
+    got = torch.full_like(dr.x0, float("nan")), torch.full_like(dr.x0, float("nan"))
+    dr.ctx.csd_draft_denoise_static(dr.head_q, dr.sched_q, wl.R, wl.cfg, wl.cfg_scale, dr.z_q, dr.x_T, dr.eps,
+                                    got[0], got[1], None)
+    dr.ctx.sync()
+    assert torch.equal(got[0], want[0]) and torch.equal(got[1], want[1])
+    dr.ctx.close()
+
+
 def test_static_scratch_denoise_rejects_sizes_beyond_the_array():
     from paper_2411_11925_b200 import api
     dr = _setup("f16", B=400)                 # 400*5*2 = 4000 head rows x W=256: far beyond 8 MiB
