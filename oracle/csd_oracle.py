@@ -22,6 +22,12 @@ What pins each function (see tests/test_oracle_pins.py):
                            1-D Gaussian toy heads: equals the difference of two
                            multivariate-normal log-densities of the whole path
                            (library routine); E_q[p(Y)/q(Y)] = 1 by Monte Carlo
+  lv_schedule, denoise_lv, log_ratio_*_lv, resample_lv, csd_round_lv (learned diagonal variances)
+                           a head whose variance output is the constant +1 reproduces the fixed-variance
+                           round exactly; long form (Eq. 4) == closed form (Eq. 7, 8) per token; 1-D toy
+                           heads against scipy's normal densities over the whole pair of paths; posterior
+                           variance against the textbook closed form; KS of the resampler with different
+                           per-dimension variances against the numerically integrated max(0, Sigma p - q)
   accept_prefix            brute force over all accept masks (Alg. 1)
   resample                 KS test against the numerically integrated
                            max(0, Sigma*p - q) (Eq. 5, Eq. 11, Cor. 1); textbook
@@ -367,3 +373,146 @@ def round_from_inputs(inp, keep: bool = False) -> Dict[str, np.ndarray]:
     ep = make_mlp_head(inp.w_p, inp.z_p, inp.tfeat, wl.cfg, wl.cfg_scale)
     return csd_round(eq, ep, sched, sched, inp.x_T, inp.eps, inp.u, inp.xi, inp.v,
                      wl.B, wl.gamma, wl.cap, keep=keep)
+
+
+# --------------------------------------------------------------------------
+# Learned per-dimension variances: the general transition of Eq. 3,
+# N(x_{t-1}; mu_theta(x_t, t), Sigma_theta(x_t, t)) with a diagonal Sigma_theta that the head predicts
+# next to eps_hat (the paper cites the improved-DDPM work for this network).  The head then has 2C
+# outputs [eps_hat | w]; the log-variance of coordinate d interpolates, with f = (w_d + 1) / 2, between
+# two per-step bounds:   log var_{t,d} = lv_min[t] + f * (lv_max[t] - lv_min[t]).
+# lv_schedule gives the bounds of that work for a DDPM: lv_max = log beta_t, lv_min = log of the
+# posterior variance beta~_t = beta_t (1 - abar_{t-1}) / (1 - abar_t), with beta~_1 (= 0) replaced by
+# beta~_2; a temperature tau scales both standard deviations (adds 2 log tau).
+# --------------------------------------------------------------------------
+def lv_schedule(beta: np.ndarray, tau: float = 1.0) -> Dict[str, np.ndarray]:
+    s = ddpm_schedule(beta, 1.0)
+    abar = s["alphabar"]
+    abar_prev = np.concatenate([[1.0], abar[:-1]])
+    post = s["beta"] * (1.0 - abar_prev) / (1.0 - abar)
+    if len(post) > 1:
+        post[0] = post[1]
+    else:
+        post[0] = s["beta"][0]
+    return {"a": s["a"], "b": s["b"], "lv_min": np.log(post) + 2.0 * np.log(tau),
+            "lv_max": np.log(s["beta"]) + 2.0 * np.log(tau), "alphabar": abar, "beta": s["beta"]}
+
+
+def make_mlp_head_lv(w: Dict[str, np.ndarray], z: np.ndarray, tfeat: np.ndarray, cfg: bool, cfg_scale: float):
+    """Head with 2C outputs: returns fn(x_t [R,C], t) -> (eps_hat [R,C], w [R,C]).  With classifier-free
+    guidance eps_hat is guided as in make_mlp_head; the variance output is the conditional row's own
+    (guidance acts on the predicted noise only)."""
+    w = {k: np.asarray(v, dtype=f64) for k, v in w.items()}
+
+    def fn(x_t: np.ndarray, t: int):
+        R, C = x_t.shape
+        if cfg:
+            o = head_eps(w, np.concatenate([x_t, x_t], axis=0), tfeat[t - 1], z)
+            e_c, e_u = o[:R, :C], o[R:, :C]
+            return e_u + cfg_scale * (e_c - e_u), o[:R, C:]
+        o = head_eps(w, x_t, tfeat[t - 1], z)
+        return o[:, :C], o[:, C:]
+    return fn
+
+
+def denoise_lv(fn, sched: Dict[str, np.ndarray], x_T: np.ndarray, noise: np.ndarray, sample_last: bool = True,
+               keep: bool = False) -> Dict[str, np.ndarray]:
+    """As denoise(), with the transition's diagonal variance predicted at every step:
+    x_{t-1} = mu_t + exp(lv_t / 2) * noise_t.  Returns also lv1 (log-variance of the last step, [R,C]) and
+    half_logdet = (1/2) sum_{t>=2} sum_d lv_{t,d}, i.e. log prod_{t>=2} sqrt|Sigma_t| of this trajectory."""
+    T = len(sched["a"])
+    x = x_T.astype(f64)
+    xs = [x.copy()] if keep else None
+    mus, lvs = ([] if keep else None), ([] if keep else None)
+    half_logdet = np.zeros(x.shape[0], dtype=f64)
+    x1 = mu1 = x0 = lv1 = None
+    for t in range(T, 0, -1):
+        e_hat, wv = fn(x, t)
+        lv = sched["lv_min"][t - 1] + 0.5 * (wv + 1.0) * (sched["lv_max"][t - 1] - sched["lv_min"][t - 1])
+        mu = sched["a"][t - 1] * x - sched["b"][t - 1] * e_hat
+        if t == 1:
+            x1, mu1, lv1 = x, mu, lv
+        else:
+            half_logdet = half_logdet + 0.5 * np.sum(lv, axis=-1)
+        if t > 1 or sample_last:
+            x = mu + np.exp(0.5 * lv) * noise[t - 1].astype(f64)
+            if t == 1:
+                x0 = x
+        if keep:
+            mus.append(mu.copy()); lvs.append(lv.copy())
+            if t > 1 or sample_last:
+                xs.append(x.copy())
+    out = {"x1": x1, "mu1": mu1, "x0": x0, "lv1": lv1, "half_logdet": half_logdet}
+    if keep:
+        out["xs"], out["mus"], out["lvs"] = xs, mus, lvs
+    return out
+
+
+def gaussian_logpdf_diag(x: np.ndarray, mu: np.ndarray, lv: np.ndarray) -> np.ndarray:
+    """log N(x; mu, diag(exp(lv))) over the last axis."""
+    C = x.shape[-1]
+    d = x - mu
+    return -0.5 * C * np.log(2.0 * np.pi) - 0.5 * np.sum(lv, axis=-1) - 0.5 * np.sum(d * d * np.exp(-lv), axis=-1)
+
+
+def log_ratio_closed_lv(x0, mu1_q, lv1_q, mu1_p, lv1_p, log_sigma_rows) -> np.ndarray:
+    """Eq. 8 with Sigma of Eq. 7 per token: log Sigma[r] = half_logdet_q[r] - half_logdet_p[r]."""
+    return log_sigma_rows + gaussian_logpdf_diag(x0, mu1_p, lv1_p) - gaussian_logpdf_diag(x0, mu1_q, lv1_q)
+
+
+def log_ratio_long_lv(dq: dict, dp: dict) -> np.ndarray:
+    """The full product of Eq. 4 over t = 1..T with x_0^p := x_0^q (keep=True runs of denoise_lv)."""
+    T = len(dq["mus"])
+    total = 0.0
+    for j in range(T):
+        t = T - j
+        xp_next = dp["xs"][j + 1] if t > 1 else dq["xs"][j + 1]
+        total = total + gaussian_logpdf_diag(xp_next, dp["mus"][j], dp["lvs"][j]) \
+                      - gaussian_logpdf_diag(dq["xs"][j + 1], dq["mus"][j], dq["lvs"][j])
+    return total
+
+
+def resample_lv(n_accept, mu1_p, lv1_p, mu1_q, lv1_q, log_sigma_rows, xi, v, gamma, cap):
+    """Corollary 1 with diagonal final-step covariances: propose x' = mu_p + exp(lv_p / 2) xi, accept with
+    alpha_s = max(0, 1 - q(x') / (Sigma p(x'))), Sigma the rejected token's own (Eq. 7)."""
+    B = len(n_accept)
+    C = mu1_p.shape[-1]
+    x_new = np.zeros((B, C), dtype=f64)
+    n_prop = np.zeros(B, dtype=np.int32)
+    flags = np.zeros(B, dtype=np.uint32)
+    for b in range(B):
+        n = int(n_accept[b])
+        if n >= gamma:
+            continue
+        j = b * gamma + n
+        flags[b] |= 1
+        done = False
+        for k in range(cap):
+            xp = mu1_p[j] + np.exp(0.5 * lv1_p[j]) * xi[b, k].astype(f64)
+            lp = gaussian_logpdf_diag(xp, mu1_p[j], lv1_p[j])
+            lq = gaussian_logpdf_diag(xp, mu1_q[j], lv1_q[j])
+            alpha_s = max(0.0, -np.expm1(min(0.0, lq - log_sigma_rows[j] - lp)))
+            x_new[b] = xp
+            n_prop[b] = k + 1
+            if float(v[b, k]) <= alpha_s:
+                done = True
+                break
+        if not done:
+            flags[b] |= 2
+    return {"x_new": x_new, "n_prop": n_prop, "flags": flags, "cap_hits": int(np.sum((flags & 2) != 0))}
+
+
+def csd_round_lv(fn_q, fn_p, sched_q, sched_p, x_T, noise, u, xi, v, B, gamma, cap, keep=False):
+    """One round of Alg. 1 with heads that predict their variances."""
+    dq = denoise_lv(fn_q, sched_q, x_T, noise, sample_last=True, keep=keep)
+    dp = denoise_lv(fn_p, sched_p, x_T, noise, sample_last=False, keep=keep)
+    ls = dq["half_logdet"] - dp["half_logdet"]
+    logr = log_ratio_closed_lv(dq["x0"], dq["mu1"], dq["lv1"], dp["mu1"], dp["lv1"], ls)
+    n, acc = accept_prefix(logr.reshape(B, gamma), u)
+    rs = resample_lv(n, dp["mu1"], dp["lv1"], dq["mu1"], dq["lv1"], ls, xi, v, gamma, cap)
+    out = {"x0": dq["x0"], "mu1_q": dq["mu1"], "lv1_q": dq["lv1"], "x1_q": dq["x1"], "mu1_p": dp["mu1"],
+           "lv1_p": dp["lv1"], "half_logdet_q": dq["half_logdet"], "half_logdet_p": dp["half_logdet"],
+           "log_sigma_rows": ls, "logratio": logr.reshape(B, gamma), "n_accept": n, "accept": acc, **rs}
+    if keep:
+        out["dq"], out["dp"] = dq, dp
+    return out

@@ -55,8 +55,8 @@ def _logr_tolerance(ep, sq, sp, dq, g_mu_p, g_traj_x=None, g_traj_mu=None):
         x_t, x_n = dq["xs"][j], dq["xs"][j + 1]
         mu_p = sp["a"][t - 1] * x_t - sp["b"][t - 1] * ep(x_t, t)
         vp, vq = sp["sigma"][t - 1] ** 2, sq["sigma"][t - 1] ** 2
-        d_xn = 0.0 if g_traj_x is None else g_traj_x[j + 1].astype(np.float64) - x_n
-        d_mq = 0.0 if g_traj_mu is None else g_traj_mu[j].astype(np.float64) - dq["mus"][j]
+        d_xn = np.zeros_like(x_n) if g_traj_x is None else g_traj_x[j + 1].astype(np.float64) - x_n
+        d_mq = np.zeros_like(x_n) if g_traj_mu is None else g_traj_mu[j].astype(np.float64) - dq["mus"][j]
         d_p = g_mu_p[j].astype(np.float64) - mu_p - d_xn          # change of (mu_p - x_{t-1})
         d_q = d_mq - d_xn
         bound = bound + np.sum(np.abs(x_n - mu_p) / vp * np.abs(d_p) + np.abs(x_n - dq["mus"][j]) / vq * np.abs(d_q), axis=1) \

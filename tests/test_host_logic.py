@@ -146,3 +146,30 @@ def test_ddim_coefficients_agree_with_the_checker_and_reject_bad_arguments():
         api.ddim_coefficients(beta, [5, 3], 1.0)
     with pytest.raises(ValueError):
         api.ddim_coefficients(beta, [1, 1001], 1.0)
+
+
+def test_bench_launches_its_own_ranks_and_counts_decisions(monkeypatch):
+    import argparse
+    import bench
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    a = argparse.Namespace(gpus=2, master_port=29999)
+    cmd = bench.reexec_argv(a, ["--gpus", "2", "--steps", "4"])
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-4:] == ["--gpus", "2", "--steps", "4"]
+    assert cmd[-5].endswith("bench.py")
+    assert bench.reexec_argv(argparse.Namespace(gpus=1, master_port=1), []) is None
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    assert bench.reexec_argv(a, []) is None          # already a rank: no second launch
+    # decision counters, on a round of the checker standing in for the library's outputs
+    wl = gen.Workload(**{**gen.WORKLOADS["tiny_fp32"].__dict__, "B": 6, "T": 3, "perturb_std": 1e-4})
+    inp = gen.make_round_inputs(wl)
+    inp.z_q = inp.z_p
+    ref = orc.round_from_inputs(inp)
+    res = {k: np.asarray(ref[k]) for k in ("logratio", "n_accept", "n_prop", "flags", "x0")}
+    res["cap_hits"] = np.array([ref["cap_hits"]])
+    res["accept_mask"] = (ref["accept"].astype(np.int64) << np.arange(wl.gamma)[None, :]).sum(axis=1)
+    d = bench.decision_counts(res, inp.u, wl.gamma)
+    assert d["decisions"] == 24 and d["resampled"] == int((ref["n_accept"] < wl.gamma).sum())
+    assert abs(d["accept_rate"] - ref["accept"].mean()) < 1e-12
+    c = bench.checker_counts(res, ref, inp.u, wl, wl.B)
+    assert c["accept_mismatch"] == 0 and c["n_prop_mismatch"] == 0 and c["x0_err"] == 0.0
