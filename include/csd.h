@@ -74,12 +74,16 @@ enum { CSD_F32 = 0, CSD_BF16 = 1, CSD_F16 = 2 };
  * In all three the residual stream, LayerNorm statistics, x_t, mu and the densities are fp32. */
 typedef struct {
   int C, W, L, Dz, F;
-  int dtype; /* CSD_F32 | CSD_BF16 | CSD_F16 */
+  int dtype;   /* CSD_F32 | CSD_BF16 | CSD_F16 */
+  int var_out; /* 0: the head predicts eps_hat (C outputs) and the transition's variance is the schedule's fixed
+                  sigma_t^2; 1: the head also predicts the diagonal of Sigma_theta(x_t, t) of Eq. 3 (2C outputs,
+                  Wout [2C, W], bout [2C]: rows C..2C are the variance parameter w) - such a head is used with the
+                  _lv calls below */
 } csd_head_desc;
 
 /* HOST pointers to fp32 parameters, each matrix row-major [out, in]:
  * Wz[W,Dz] bz[W] Wt1[W,F] bt1[W] Wt2[W,W] bt2[W] Win[W,C] bin[W] Wada[L,3W,W] bada[L,3W]
- * W1[L,W,W] b1[L,W] W2[L,W,W] b2[L,W] Wfada[2W,W] bfada[2W] Wout[C,W] bout[C].
+ * W1[L,W,W] b1[L,W] W2[L,W,W] b2[L,W] Wfada[2W,W] bfada[2W] Wout[C,W] bout[C]  (Wout[2C,W] bout[2C] if var_out).
  * For CSD_BF16 / CSD_F16 heads the matrices are converted to that format (round to nearest
  * even); callers that want bit-defined results pass values that are already representable. */
 typedef struct {
@@ -261,6 +265,21 @@ int csd_bonus_token(csd_ctx *ctx, const csd_head *head_p, const csd_schedule *sc
                     int cfg, float cfg_scale, const float *z_next, const float *x_T_next,
                     const float *eps_next, const int32_t *n_accept, float *x_bonus, uint32_t *taken);
 
+/* csd_verify with the bonus token folded in.  Alg. 1 obtains p_{gamma+1} from the same parallel target pass that
+ * yields p_1..p_gamma, so here the B rows of position gamma+1 ride along as rows R..R+B of the verifying chain
+ * (one chain of R + B token rows instead of a second, latency-bound chain of B rows): those rows sample x_0 at
+ * the last step, and x_bonus[b] is written where n_accept[b] == gamma.  logratio, n_accept, accept_mask, mu1_p as
+ * csd_verify; z_next, x_T_next, eps_next, x_bonus, taken as csd_bonus_token.  The inputs are gathered into a
+ * side buffer the library keeps ((R + B) rows of z, x_T, eps).  Results equal csd_verify followed by
+ * csd_bonus_token bit for bit with CSD_CHAIN_LAYERS_PLAIN, and within the trajectory tolerance in the default
+ * layout (whose folded blocks depend on a call's row count). */
+int csd_verify_bonus(csd_ctx *ctx, const csd_head *head_p, const csd_schedule *sched_p,
+                     const csd_schedule *sched_q, int B, int gamma, int cfg, float cfg_scale,
+                     const float *z_p, const float *x_T, const float *eps, const float *x0_q,
+                     const float *mu1_q, const float *u, const float *z_next, const float *x_T_next,
+                     const float *eps_next, float *logratio, int32_t *n_accept, uint32_t *accept_mask,
+                     float *mu1_p, float *x_bonus, uint32_t *taken);
+
 /* ---- Exact single-path criterion (Eq. 2; Table 1 "p(Y_q)/q(Y_q)") ------------------------------
  * Eq. 2 scores the DRAFT's own trajectory Y_q = (x_T, x^q_{T-1}, ..., x^q_0) under both models:
  *   log p(Y_q)/q(Y_q) = sum_{t=1..T} [ log N(x^q_{t-1}; mu^p_t(x^q_t), sigma_p,t^2 I)
@@ -326,6 +345,59 @@ int csd_round(csd_ctx *ctx, const csd_head *head_q, const csd_head *head_p,
               float *mu1_q, float *mu1_p, float *logratio, int32_t *n_accept,
               uint32_t *accept_mask, float *x_new, int32_t *n_prop, uint32_t *flags,
               int32_t *cap_hits);
+
+/* ---- Heads that predict their variances (the general transition of Eq. 3) -------------------------
+ * Eq. 3 writes the transition as N(x_{t-1}; mu_theta(x_t,t), Sigma_theta(x_t,t)) with both moments predicted by
+ * the network the paper cites for it.  A head created with var_out = 1 returns, next to eps_hat, a parameter w
+ * per coordinate; the transition's diagonal log-variance interpolates between two per-step bounds,
+ *   lv_{t,d} = lv_min[t-1] + (w_d + 1)/2 * (lv_max[t-1] - lv_min[t-1]),   x_{t-1} = mu_t + exp(lv_t / 2) * eps_t.
+ * With guidance eps_hat is guided and w is the conditional row's.  Sigma of Eq. 7 is then a per-token product:
+ * log Sigma[r] = half_logdet_q[r] - half_logdet_p[r], half_logdet = (1/2) sum_{t=2..T} sum_d lv_{t,d} of a chain;
+ * Eq. 8 and Corollary 1 use the diagonal final-step Gaussians N(mu1, diag(exp(lv1))).
+ * csd_schedule_lv: a, b, lv_min, lv_max HOST arrays [T]; tfeat DEVICE [T, F].
+ * csd_schedule_lv_ddpm (host only): a, b as csd_schedule_ddpm; lv_max = log beta_t, lv_min = log of the posterior
+ * variance beta_t (1 - abar_{t-1}) / (1 - abar_t) (its value at t = 2 also for t = 1, where it is zero), both
+ * plus 2 log tau. */
+typedef struct {
+  int T;
+  const float *a, *b, *lv_min, *lv_max;
+  const float *tfeat;
+} csd_schedule_lv;
+int csd_schedule_lv_ddpm(int T, const double *beta, double tau, float *a, float *b, float *lv_min, float *lv_max);
+/* As csd_draft_denoise; also returns lv1 device [R, C] (log-variance of the last step) and half_logdet device [R]. */
+int csd_draft_denoise_lv(csd_ctx *ctx, const csd_head *head, const csd_schedule_lv *sched, int R, int cfg,
+                         float cfg_scale, const float *z, const float *x_T, const float *eps, float *x0,
+                         float *mu1, float *lv1, float *half_logdet, float *x1);
+/* As csd_verify (shared x_T and eps: alignment); takes the draft's lv1_q, half_logdet_q and returns the target's
+ * mu1_p, lv1_p [R, C], half_logdet_p [R] and the per-token log_sigma_rows device [R] besides logratio, n_accept, mask. */
+int csd_verify_lv(csd_ctx *ctx, const csd_head *head_p, const csd_schedule_lv *sched_p, int B, int gamma, int cfg,
+                  float cfg_scale, const float *z_p, const float *x_T, const float *eps, const float *x0_q,
+                  const float *mu1_q, const float *lv1_q, const float *half_logdet_q, const float *u,
+                  float *logratio, int32_t *n_accept, uint32_t *accept_mask, float *mu1_p, float *lv1_p,
+                  float *half_logdet_p, float *log_sigma_rows);
+/* As csd_resample with x' = mu1_p + exp(lv1_p / 2) * xi and the rejected token's own log Sigma. */
+int csd_resample_lv(csd_ctx *ctx, int B, int gamma, int C, int cap, const float *log_sigma_rows,
+                    const int32_t *n_accept, const float *mu1_p, const float *lv1_p, const float *mu1_q,
+                    const float *lv1_q, const float *xi, const float *v, float *x_new, int32_t *n_prop,
+                    uint32_t *flags, int32_t *cap_hits);
+/* The three calls above as one round, the two chains concurrent, bit-identical results. */
+int csd_round_lv(csd_ctx *ctx, const csd_head *head_q, const csd_head *head_p, const csd_schedule_lv *sched_q,
+                 const csd_schedule_lv *sched_p, int B, int gamma, int cfg, float cfg_scale, int cap,
+                 const float *z_q, const float *z_p, const float *x_T, const float *eps, const float *u,
+                 const float *xi, const float *v, float *x0, float *mu1_q, float *lv1_q, float *half_logdet_q,
+                 float *mu1_p, float *lv1_p, float *half_logdet_p, float *log_sigma_rows, float *logratio,
+                 int32_t *n_accept, uint32_t *accept_mask, float *x_new, int32_t *n_prop, uint32_t *flags,
+                 int32_t *cap_hits);
+
+/* csd_round with the bonus token of the all-accepted branch of Alg. 1 (see csd_verify_bonus): the target chain
+ * runs R + B token rows. */
+int csd_round_bonus(csd_ctx *ctx, const csd_head *head_q, const csd_head *head_p, const csd_schedule *sched_q,
+                    const csd_schedule *sched_p, int B, int gamma, int cfg, float cfg_scale, int cap,
+                    const float *z_q, const float *z_p, const float *x_T, const float *eps, const float *u,
+                    const float *xi, const float *v, const float *z_next, const float *x_T_next,
+                    const float *eps_next, float *x0, float *mu1_q, float *mu1_p, float *logratio,
+                    int32_t *n_accept, uint32_t *accept_mask, float *x_new, int32_t *n_prop, uint32_t *flags,
+                    int32_t *cap_hits, float *x_bonus, uint32_t *taken);
 
 /* Same computation as csd_round, but every array is a HOST pointer: the call copies the inputs
  * to the device, runs the round, copies the outputs back and synchronises before returning. */

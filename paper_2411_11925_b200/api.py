@@ -24,10 +24,11 @@ DTYPES = {"f32": CSD_F32, "bf16": CSD_BF16, "f16": CSD_F16}
 
 EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launch_count",
            "csd_set_chain_mode", "csd_profile", "csd_profile_read", "csd_set_wait_limit", "csd_selftest_wait_timeout",
-           "csd_schedule_ddpm", "csd_schedule_ddim", "csd_log_sigma_term",
+           "csd_schedule_ddpm", "csd_schedule_ddim", "csd_log_sigma_term", "csd_schedule_lv_ddpm",
+           "csd_draft_denoise_lv", "csd_verify_lv", "csd_resample_lv", "csd_round_lv",
            "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_draft_denoise_static", "csd_verify",
            "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host", "csd_draft_denoise_traj",
-           "csd_verify_single_path", "csd_verify_unaligned", "csd_bonus_token")
+           "csd_verify_single_path", "csd_verify_unaligned", "csd_bonus_token", "csd_verify_bonus", "csd_round_bonus")
 
 WEIGHT_FIELDS = ("Wz", "bz", "Wt1", "bt1", "Wt2", "bt2", "Win", "bin", "Wada", "bada",
                  "W1", "b1", "W2", "b2", "Wfada", "bfada", "Wout", "bout")
@@ -40,7 +41,7 @@ class CsdError(RuntimeError):
 
 
 class _HeadDesc(C.Structure):
-    _fields_ = [(n, C.c_int) for n in ("C", "W", "L", "Dz", "F", "dtype")]
+    _fields_ = [(n, C.c_int) for n in ("C", "W", "L", "Dz", "F", "dtype", "var_out")]
 
 
 class _HeadWeights(C.Structure):
@@ -49,6 +50,11 @@ class _HeadWeights(C.Structure):
 
 class _Schedule(C.Structure):
     _fields_ = [("T", C.c_int), ("a", _c_float_p), ("b", _c_float_p), ("sigma", _c_float_p),
+                ("tfeat", C.c_void_p)]
+
+
+class _ScheduleLV(C.Structure):
+    _fields_ = [("T", C.c_int), ("a", _c_float_p), ("b", _c_float_p), ("lv_min", _c_float_p), ("lv_max", _c_float_p),
                 ("tfeat", C.c_void_p)]
 
 
@@ -71,6 +77,12 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_schedule_ddpm.argtypes = [i32, f64p, f64, _c_float_p, _c_float_p, _c_float_p]
     lib.csd_schedule_ddim.argtypes = [i32, f64p, i32, i32p, f64, _c_float_p, _c_float_p, _c_float_p]
     lib.csd_log_sigma_term.argtypes = [i32, _c_float_p, _c_float_p, i32, f64p]
+    lib.csd_schedule_lv_ddpm.argtypes = [i32, f64p, f64] + [_c_float_p] * 4
+    lib.csd_draft_denoise_lv.argtypes = [vp, vp, C.POINTER(_ScheduleLV), i32, i32, f32] + [vp] * 8
+    lib.csd_verify_lv.argtypes = [vp, vp, C.POINTER(_ScheduleLV), i32, i32, i32, f32] + [vp] * 15
+    lib.csd_resample_lv.argtypes = [vp, i32, i32, i32, i32] + [vp] * 12
+    lib.csd_round_lv.argtypes = ([vp, vp, vp, C.POINTER(_ScheduleLV), C.POINTER(_ScheduleLV), i32, i32, i32, f32, i32]
+                                 + [vp] * 22)
     lib.csd_profile.argtypes = [vp, i32]
     lib.csd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_int64), C.POINTER(f64), C.POINTER(f64)]
     lib.csd_head_create.argtypes = [vp, C.POINTER(_HeadDesc), C.POINTER(_HeadWeights), C.POINTER(vp)]
@@ -84,6 +96,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_verify_unaligned.argtypes = ([vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32]
                                          + [vp] * 11)
     lib.csd_bonus_token.argtypes = [vp, vp, C.POINTER(_Schedule), i32, i32, i32, f32] + [vp] * 6
+    lib.csd_verify_bonus.argtypes = [vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32] + [vp] * 15
+    lib.csd_round_bonus.argtypes = ([vp, vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32, i32]
+                                    + [vp] * 22)
     lib.csd_accept_scan.argtypes = [vp, i32, i32, i32, f64, f32, f32] + [vp] * 7
     lib.csd_resample.argtypes = [vp, i32, i32, i32, i32, f64, f32, f32] + [vp] * 9
     round_args = [vp, vp, vp, C.POINTER(_Schedule), C.POINTER(_Schedule), i32, i32, i32, f32, i32] + [vp] * 17
@@ -127,6 +142,17 @@ def ddim_coefficients(beta_full: np.ndarray, steps, eta: float) -> Dict[str, np.
     return out
 
 
+def lv_ddpm_coefficients(beta: np.ndarray, tau: float = 1.0) -> Dict[str, np.ndarray]:
+    """csd_schedule_lv_ddpm: {"a", "b", "lv_min", "lv_max"} of a DDPM whose head predicts its variances."""
+    beta = np.ascontiguousarray(beta, dtype=np.float64)
+    out = {k: np.zeros(beta.size, dtype=np.float32) for k in ("a", "b", "lv_min", "lv_max")}
+    rc = _LIB.csd_schedule_lv_ddpm(int(beta.size), beta.ctypes.data_as(C.POINTER(C.c_double)), float(tau),
+                                   *[out[k].ctypes.data_as(_c_float_p) for k in ("a", "b", "lv_min", "lv_max")])
+    if rc != 0:
+        raise CsdError(rc, "csd_schedule_lv_ddpm: beta must lie in (0, 1) and tau be positive")
+    return out
+
+
 def _ptr(t) -> Optional[int]:
     if t is None:
         return None
@@ -160,6 +186,18 @@ class Schedule:
         if rc != 0:
             raise CsdError(rc, "csd_log_sigma_term")
         return float(out.value)
+
+
+class ScheduleLV:
+    """csd_schedule_lv: keeps the host arrays and the device feature table alive."""
+
+    def __init__(self, a, b, lv_min, lv_max, tfeat: torch.Tensor):
+        self.a, self.b, self.lv_min, self.lv_max = (np.ascontiguousarray(x, dtype=np.float32) for x in (a, b, lv_min, lv_max))
+        assert tfeat.is_cuda and tfeat.dtype == torch.float32 and tfeat.is_contiguous()
+        self.tfeat = tfeat
+        self.T = int(self.a.shape[0])
+        self.c = _ScheduleLV(self.T, *[x.ctypes.data_as(_c_float_p) for x in (self.a, self.b, self.lv_min, self.lv_max)],
+                             tfeat.data_ptr())
 
 
 class Context:
@@ -263,6 +301,23 @@ class Context:
                                          _ptr(z_next), _ptr(x_T_next), _ptr(eps_next), _ptr(n_accept), _ptr(x_bonus),
                                          _ptr(taken)))
 
+    def csd_verify_bonus(self, head_p: "Head", sched_p: Schedule, sched_q: Schedule, B, gamma, cfg, cfg_scale, z_p, x_T,
+                         eps, x0_q, mu1_q, u, z_next, x_T_next, eps_next, logratio, n_accept, accept_mask, mu1_p,
+                         x_bonus, taken=None):
+        self._check(_LIB.csd_verify_bonus(self._h, head_p._h, C.byref(sched_p.c), C.byref(sched_q.c), B, gamma, int(cfg),
+                                          cfg_scale, *[_ptr(t) for t in (z_p, x_T, eps, x0_q, mu1_q, u, z_next, x_T_next,
+                                                                         eps_next, logratio, n_accept, accept_mask, mu1_p,
+                                                                         x_bonus, taken)]))
+
+    def csd_round_bonus(self, head_q, head_p, sched_q, sched_p, B, gamma, cfg, cfg_scale, cap, z_q, z_p, x_T, eps, u, xi,
+                        v, z_next, x_T_next, eps_next, x0, mu1_q, mu1_p, logratio, n_accept, accept_mask, x_new, n_prop,
+                        flags, cap_hits, x_bonus, taken=None):
+        self._check(_LIB.csd_round_bonus(self._h, head_q._h, head_p._h, C.byref(sched_q.c), C.byref(sched_p.c), B, gamma,
+                                         int(cfg), cfg_scale, cap,
+                                         *[_ptr(t) for t in (z_q, z_p, x_T, eps, u, xi, v, z_next, x_T_next, eps_next, x0,
+                                                             mu1_q, mu1_p, logratio, n_accept, accept_mask, x_new, n_prop,
+                                                             flags, cap_hits, x_bonus, taken)]))
+
     def csd_accept_scan(self, B, gamma, Cdim, log_sigma, sigma1_p, sigma1_q, x0_q, mu1_q, mu1_p, u, logratio,
                         n_accept, accept_mask=None):
         self._check(_LIB.csd_accept_scan(self._h, B, gamma, Cdim, log_sigma, sigma1_p, sigma1_q, _ptr(x0_q),
@@ -274,6 +329,34 @@ class Context:
         self._check(_LIB.csd_resample(self._h, B, gamma, Cdim, cap, log_sigma, sigma1_p, sigma1_q, _ptr(n_accept),
                                       _ptr(mu1_p), _ptr(mu1_q), _ptr(xi), _ptr(v), _ptr(x_new), _ptr(n_prop),
                                       _ptr(flags), _ptr(cap_hits)))
+
+    def csd_draft_denoise_lv(self, head: "Head", sched: ScheduleLV, R, cfg, cfg_scale, z, x_T, eps, x0, mu1, lv1,
+                             half_logdet, x1=None):
+        self._check(_LIB.csd_draft_denoise_lv(self._h, head._h, C.byref(sched.c), R, int(cfg), cfg_scale,
+                                              *[_ptr(t) for t in (z, x_T, eps, x0, mu1, lv1, half_logdet, x1)]))
+
+    def csd_verify_lv(self, head_p: "Head", sched_p: ScheduleLV, B, gamma, cfg, cfg_scale, z_p, x_T, eps, x0_q, mu1_q,
+                      lv1_q, half_logdet_q, u, logratio, n_accept, accept_mask, mu1_p, lv1_p, half_logdet_p,
+                      log_sigma_rows):
+        self._check(_LIB.csd_verify_lv(self._h, head_p._h, C.byref(sched_p.c), B, gamma, int(cfg), cfg_scale,
+                                       *[_ptr(t) for t in (z_p, x_T, eps, x0_q, mu1_q, lv1_q, half_logdet_q, u, logratio,
+                                                           n_accept, accept_mask, mu1_p, lv1_p, half_logdet_p,
+                                                           log_sigma_rows)]))
+
+    def csd_resample_lv(self, B, gamma, Cdim, cap, log_sigma_rows, n_accept, mu1_p, lv1_p, mu1_q, lv1_q, xi, v, x_new,
+                        n_prop, flags, cap_hits):
+        self._check(_LIB.csd_resample_lv(self._h, B, gamma, Cdim, cap,
+                                         *[_ptr(t) for t in (log_sigma_rows, n_accept, mu1_p, lv1_p, mu1_q, lv1_q, xi, v,
+                                                             x_new, n_prop, flags, cap_hits)]))
+
+    def csd_round_lv(self, head_q, head_p, sched_q: ScheduleLV, sched_p: ScheduleLV, B, gamma, cfg, cfg_scale, cap,
+                     z_q, z_p, x_T, eps, u, xi, v, x0, mu1_q, lv1_q, half_logdet_q, mu1_p, lv1_p, half_logdet_p,
+                     log_sigma_rows, logratio, n_accept, accept_mask, x_new, n_prop, flags, cap_hits):
+        self._check(_LIB.csd_round_lv(self._h, head_q._h, head_p._h, C.byref(sched_q.c), C.byref(sched_p.c), B, gamma,
+                                      int(cfg), cfg_scale, cap,
+                                      *[_ptr(t) for t in (z_q, z_p, x_T, eps, u, xi, v, x0, mu1_q, lv1_q, half_logdet_q,
+                                                          mu1_p, lv1_p, half_logdet_p, log_sigma_rows, logratio, n_accept,
+                                                          accept_mask, x_new, n_prop, flags, cap_hits)]))
 
     def _round(self, fn, head_q, head_p, sched_q, sched_p, B, gamma, cfg, cfg_scale, cap, z_q, z_p, x_T, eps, u,
                xi, v, x0, mu1_q, mu1_p, logratio, n_accept, accept_mask, x_new, n_prop, flags, cap_hits):
@@ -289,13 +372,14 @@ class Context:
 
 
 class Head:
-    def __init__(self, ctx: Context, weights: Dict[str, np.ndarray], operand: str):
-        """operand: "f32", "bf16" or "f16" = the GEMM operand format (see csd_head_desc)."""
+    def __init__(self, ctx: Context, weights: Dict[str, np.ndarray], operand: str, var_out: bool = False):
+        """operand: "f32", "bf16" or "f16" = the GEMM operand format; var_out: the head has 2C outputs, the second
+        half being the variance parameter (see csd_head_desc)."""
         Wd, Dz = weights["Wz"].shape
-        Cdim = weights["Wout"].shape[0]
+        Cdim = weights["Wout"].shape[0] // (2 if var_out else 1)
         L = weights["W1"].shape[0]
         F = weights["Wt1"].shape[1]
-        self.desc = _HeadDesc(Cdim, Wd, L, Dz, F, DTYPES[operand])
+        self.desc = _HeadDesc(Cdim, Wd, L, Dz, F, DTYPES[operand], int(var_out))
         keep = {k: np.ascontiguousarray(weights[k], dtype=np.float32) for k in WEIGHT_FIELDS}
         hw = _HeadWeights(*[keep[k].ctypes.data_as(_c_float_p) for k in WEIGHT_FIELDS])
         self._h = C.c_void_p()

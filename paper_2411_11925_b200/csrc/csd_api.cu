@@ -211,7 +211,7 @@ WsLayout ws_layout(const csd_head_desc& d, int Rh, int R, int T) {
   l.s = take(rh * W * asz); l.u = take(rh * W * asz); l.v = take(rh * W * asz);
   l.cz = take(rh * W * 4); l.te = take(static_cast<size_t>(T) * W * 4); l.h = take(rh * W * 4);
   l.stats = take(rh * (W / kStatCols) * 8);
-  l.epart = take(rh * (W / kStatCols) * kCPad * 4);   // room for 64-wide tiles
+  l.epart = take(rh * (W / kStatCols) * (d.var_out ? kCPad2 : kCPad) * 4);   // room for 64-wide tiles
   l.x = take(static_cast<size_t>(R) * kCPad * 4);
   l.ap = take(d.dtype == CSD_F32 ? 0 : rh * W * asz);
   l.hid = take(static_cast<size_t>(T) * W * 4);
@@ -261,7 +261,7 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
   const int units = tiles_n * (PAIR ? (row_tiles + 1) / 2 : row_tiles);
   const int max_units = PAIR ? ctx->num_sms / 2 : ctx->num_sms;
   dim3 grid((units < max_units ? units : max_units) * (PAIR ? 2 : 1));
-  ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * NMUL);
+  ProfScope ps(ctx, st, EPI == EPI_MODF2 ? EPI_MODF : EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * NMUL);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid; cfg.blockDim = dim3(TcWarps<EPI, TN>::kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute at[2];
@@ -307,7 +307,7 @@ template <int EPI, int NSEG, int MMA_N>
 int launch_simt(csd_ctx* ctx, cudaStream_t st, const float* A0, int lda0, const float* B0, int K0, const float* A1,
                 int lda1, const float* B1, int K1, int N, const EpiParams& ep) {
   dim3 grid(N / kTileN, (ep.M + kSimtRows - 1) / kSimtRows);
-  ProfScope ps(ctx, st, EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * ((NSEG == 1 && MMA_N == 256) ? 2.0 : 1.0));
+  ProfScope ps(ctx, st, EPI == EPI_MODF2 ? EPI_MODF : EPI, 2.0 * ep.M * static_cast<double>(N) * (K0 + K1) * ((NSEG == 1 && MMA_N == 256) ? 2.0 : 1.0));
   EpiParams e = ep;
   e.nt = N / kTileN;
   gemm_simt_kernel<EPI, NSEG, MMA_N><<<grid, 128, 0, st>>>(A0, lda0, B0, K0, K0, A1, lda1, B1, K1, K1, e);
@@ -367,6 +367,9 @@ struct Chain {
   StepParams sp{};
   // trajectory recording (csd_draft_denoise_traj): [T + 1, R, C] states and [T, R, C] means, or null
   float *traj_x = nullptr, *traj_mu = nullptr;
+  // learned-variance heads: host arrays [T] of the log-variance bounds, outputs lv1 [R, C] and half_logdet [R]
+  const float *lv_min = nullptr, *lv_max = nullptr;
+  float *lv1 = nullptr, *half_logdet = nullptr;
   // batched evaluation on a given trajectory (csd_verify_single_path): R = batch_steps * batch_Rin token rows,
   // one pass of the layers; slot batch_j0 of batch_traj is the first step of the pass
   int batch_Rin = 0, batch_j0 = 0, Ts = 0;
@@ -377,7 +380,8 @@ struct Chain {
 
   template <typename ACT>
   int launch_step_t(cudaLaunchConfig_t& cfg, bool rb4, int mode) {
-    if (traj_x) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<ACT, 4, true> : step_kernel<ACT, 1, true>, sp, mode));
+    if (lv_min) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<ACT, 4, false, true> : step_kernel<ACT, 1, false, true>, sp, mode));
+    else if (traj_x) CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<ACT, 4, true> : step_kernel<ACT, 1, true>, sp, mode));
     else CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, rb4 ? step_kernel<ACT, 4> : step_kernel<ACT, 1>, sp, mode));
     return CSD_OK;
   }
@@ -505,6 +509,7 @@ struct Chain {
     sbuf[0] = ws.s2; sbuf[1] = ws.s;
     if (batch_Rin) return launch_batch(0);   // a pass has one step (t = 1): its s is sbuf[1]
     sp.traj_x = traj_x; sp.traj_mu = nullptr; sp.status = ctx->d_err + 1;
+    sp.lv1 = lv1; sp.half_logdet = half_logdet; sp.lv_min = 0.0f; sp.lv_max = 0.0f;
     sp.R = R; sp.cfg = cfg; sp.C = d.C; sp.W = W; sp.NT = tc ? W / kStatCols : W / kTileN; sp.cfg_scale = cfg_scale;
     sp.sample_last = sample_last; sp.epart = ws.epart; sp.bout = hd->bout; sp.x_src = x_T; sp.x = ws.x;
     sp.x0 = x0; sp.mu1 = mu1; sp.x1 = x1; sp.win = hd->win; sp.bin = hd->bin; sp.cz = ws.cz; sp.h = ws.h;
@@ -616,7 +621,13 @@ struct Chain {
     }
     EpiParams e = ep;
     e.h = ws.h; e.stats = ws.stats; e.bias0 = hd->bfsh; e.bias1 = hd->bfsc; e.wout_t = hd->wout_t; e.epart = ws.epart;
-    if (tc && mod64) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wfss, tm_s, hd->tm[0].Wfss, tm_h, W, 0, W, W, e);
+    if (d.var_out) {   // 32 output columns: eps_hat | variance parameter
+      if (tc && mod64) rc = launch_tc<EPI_MODF2, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wfss, tm_s, hd->tm[0].Wfss, tm_h, W, 0, W, W, e);
+      else if (tc) rc = launch_tc<EPI_MODF2, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wfss, tm_s, tmw.Wfss, tm_h, W, 0, W, W, e);
+      else rc = launch_simt<EPI_MODF2, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
+                                               0, W, e);
+    }
+    else if (tc && mod64) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wfss, tm_s, hd->tm[0].Wfss, tm_h, W, 0, W, W, e);
     else if (tc) rc = launch_tc<EPI_MODF, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wfss, tm_s, tmw.Wfss, tm_h, W, 0, W, W, e);
     else rc = launch_simt<EPI_MODF, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wfss), W, nullptr, 0, nullptr,
                                             0, W, e);
@@ -626,7 +637,9 @@ struct Chain {
       sp.traj_x = traj_x + static_cast<size_t>(T - t + 1) * R * d.C;
       sp.traj_mu = traj_mu + static_cast<size_t>(T - t) * R * d.C;
     }
-    sp.a = sc->a[t - 1]; sp.b = sc->b[t - 1]; sp.sigma = sc->sigma[t - 1];
+    sp.a = sc->a[t - 1]; sp.b = sc->b[t - 1];
+    if (lv_min) { sp.sigma = 0.0f; sp.lv_min = lv_min[t - 1]; sp.lv_max = lv_max[t - 1]; }
+    else sp.sigma = sc->sigma[t - 1];
     sp.eps_t = eps + static_cast<size_t>(t - 1) * R * d.C;
     // this boundary prepares h of step t - 1 and s of step t - 2
     sp.s = t >= 3 ? sbuf[(t - 2) & 1] : nullptr;
@@ -649,11 +662,59 @@ int check_chain_args(csd_ctx* ctx, const csd_head* hd, const csd_schedule* sc, i
                      const void* x_T, const void* eps) {
   if (!hd) return fail(ctx, CSD_ERR_INVALID_ARG, "head is null");
   if (hd->ctx != ctx) return fail(ctx, CSD_ERR_INVALID_ARG, "head belongs to another context");
+  if (hd->d.var_out) return fail(ctx, CSD_ERR_UNSUPPORTED, "this head predicts its variances (var_out = 1): use the _lv calls");
   int rc = check_sched(ctx, sc, true);
   if (rc) return rc;
   if (R < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "row count %d must be >= 1", R);
   if (cfg != 0 && cfg != 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cfg must be 0 or 1");
   if (!z || !x_T || !eps) return fail(ctx, CSD_ERR_INVALID_ARG, "z / x_T / eps is null");
+  return CSD_OK;
+}
+
+int check_lv_args(csd_ctx* ctx, const csd_head* hd, const csd_schedule_lv* sc, int R, int cfg, const void* z,
+                  const void* x_T, const void* eps) {
+  if (!hd) return fail(ctx, CSD_ERR_INVALID_ARG, "head is null");
+  if (hd->ctx != ctx) return fail(ctx, CSD_ERR_INVALID_ARG, "head belongs to another context");
+  if (!hd->d.var_out) return fail(ctx, CSD_ERR_UNSUPPORTED, "this head has a fixed variance (var_out = 0): use the calls without _lv");
+  if (!sc) return fail(ctx, CSD_ERR_INVALID_ARG, "schedule is null");
+  if (sc->T < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "schedule T = %d must be >= 1", sc->T);
+  if (!sc->a || !sc->b || !sc->lv_min || !sc->lv_max || !sc->tfeat) return fail(ctx, CSD_ERR_INVALID_ARG, "schedule a / b / lv_min / lv_max / tfeat is null");
+  for (int t = 0; t < sc->T; ++t)
+    if (!(sc->lv_min[t] <= sc->lv_max[t]) || !std::isfinite(sc->lv_min[t]) || !std::isfinite(sc->lv_max[t]))
+      return fail(ctx, CSD_ERR_INVALID_ARG, "schedule needs finite lv_min[%d] <= lv_max[%d]", t, t);
+  if (R < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "row count %d must be >= 1", R);
+  if (cfg != 0 && cfg != 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cfg must be 0 or 1");
+  if (!z || !x_T || !eps) return fail(ctx, CSD_ERR_INVALID_ARG, "z / x_T / eps is null");
+  return CSD_OK;
+}
+
+// A learned-variance chain: the fixed-variance chain with the log-variance bounds in place of sigma.
+Chain make_lv_chain(csd_ctx* ctx, int slot, cudaStream_t st, const csd_head* hd, const csd_schedule* view,
+                    const csd_schedule_lv* sc, int R, int cfg, float cfg_scale, const float* z, const float* x_T,
+                    const float* eps, int sample_last, float* x0, float* mu1, float* lv1, float* half_logdet, float* x1) {
+  Chain c{ctx, slot, st, hd, view, R, cfg, cfg_scale, z, x_T, eps, sample_last, x0, mu1, x1};
+  c.lv_min = sc->lv_min; c.lv_max = sc->lv_max; c.lv1 = lv1; c.half_logdet = half_logdet;
+  return c;
+}
+
+int accept_scan_lv(csd_ctx* ctx, cudaStream_t st, int B, int gamma, int C, const float* x0, const float* mu_q,
+                   const float* lv_q, const float* hld_q, const float* mu_p, const float* lv_p, const float* hld_p,
+                   const float* u, float* logratio, float* log_sigma_rows, int32_t* n_accept, uint32_t* mask) {
+  accept_scan_lv_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, gamma, C, x0, mu_q, lv_q, hld_q, mu_p, lv_p, hld_p, u, logratio,
+                                                     log_sigma_rows, n_accept, mask);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+int resample_lv(csd_ctx* ctx, cudaStream_t st, int B, int gamma, int C, int cap, const float* log_sigma_rows,
+                const int32_t* n_accept, const float* mu_p, const float* lv_p, const float* mu_q, const float* lv_q,
+                const float* xi, const float* v, float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  CSD_CUDA(ctx, cudaMemsetAsync(cap_hits, 0, sizeof(int32_t), st));
+  resample_lv_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, gamma, C, cap, log_sigma_rows, n_accept, mu_p, lv_p, mu_q, lv_q, xi, v,
+                                                  x_new, n_prop, flags, cap_hits);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
   return CSD_OK;
 }
 
@@ -686,6 +747,55 @@ int resample(csd_ctx* ctx, cudaStream_t st, int B, int gamma, int C, int cap, do
                                                mu_q, xi, v, x_new, n_prop, flags, cap_hits);
   ctx->launches++;
   CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+// Target chain over the R = B gamma verified positions with the B rows of position gamma + 1 appended (Alg. 1
+// obtains p_{gamma+1} from the same parallel target pass): token rows [0, R) are the verified ones, [R, R + B) the
+// bonus ones; with guidance the unconditional twins follow in the same order.  The side buffer holds the gathered
+// inputs and the chain's last-step outputs for all R + B rows.
+struct BonusBuf {
+  float *z, *x_T, *eps, *mu1, *x0;
+};
+
+size_t bonus_buf_bytes(const csd_head_desc& d, int Rt, int cfg, int T) {
+  const size_t m = cfg ? 2 : 1, rt = static_cast<size_t>(Rt);
+  return align_up(rt * m * d.Dz * 4, 256) + align_up(rt * d.C * 4, 256) * 3 + align_up(static_cast<size_t>(T) * rt * d.C * 4, 256);
+}
+
+int ensure_side(csd_ctx* ctx, HostIo& io, size_t need, const char* what) {
+  if (need <= io.cap) return CSD_OK;
+  CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+  for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamSynchronize(ctx->side[i]));
+  if (io.base) CSD_CUDA(ctx, cudaFree(io.base));
+  io.base = nullptr; io.cap = 0;
+  if (cudaMalloc(&io.base, need) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes for %s", need, what);
+  }
+  io.cap = need;
+  return CSD_OK;
+}
+
+// Carves the (already large enough) side buffer and enqueues the gathering copies on `st`.
+int gather_bonus_inputs(csd_ctx* ctx, cudaStream_t st, const csd_head_desc& d, int R, int B, int cfg, int T,
+                        const float* z, const float* x_T, const float* eps, const float* z_next,
+                        const float* x_T_next, const float* eps_next, BonusBuf& bb) {
+  const size_t m = cfg ? 2 : 1, Rt = static_cast<size_t>(R) + B, C = d.C, Dz = d.Dz;
+  char* p = static_cast<char*>(ctx->bn.base);
+  bb.z = reinterpret_cast<float*>(p); p += align_up(Rt * m * Dz * 4, 256);
+  bb.x_T = reinterpret_cast<float*>(p); p += align_up(Rt * C * 4, 256);
+  bb.mu1 = reinterpret_cast<float*>(p); p += align_up(Rt * C * 4, 256);
+  bb.x0 = reinterpret_cast<float*>(p); p += align_up(Rt * C * 4, 256);
+  bb.eps = reinterpret_cast<float*>(p);
+  for (size_t h = 0; h < m; ++h) {
+    CSD_CUDA(ctx, cudaMemcpyAsync(bb.z + h * Rt * Dz, z + h * R * Dz, static_cast<size_t>(R) * Dz * 4, cudaMemcpyDeviceToDevice, st));
+    CSD_CUDA(ctx, cudaMemcpyAsync(bb.z + (h * Rt + R) * Dz, z_next + h * B * Dz, static_cast<size_t>(B) * Dz * 4, cudaMemcpyDeviceToDevice, st));
+  }
+  CSD_CUDA(ctx, cudaMemcpyAsync(bb.x_T, x_T, static_cast<size_t>(R) * C * 4, cudaMemcpyDeviceToDevice, st));
+  CSD_CUDA(ctx, cudaMemcpyAsync(bb.x_T + static_cast<size_t>(R) * C, x_T_next, static_cast<size_t>(B) * C * 4, cudaMemcpyDeviceToDevice, st));
+  CSD_CUDA(ctx, cudaMemcpy2DAsync(bb.eps, Rt * C * 4, eps, static_cast<size_t>(R) * C * 4, static_cast<size_t>(R) * C * 4, T, cudaMemcpyDeviceToDevice, st));
+  CSD_CUDA(ctx, cudaMemcpy2DAsync(bb.eps + static_cast<size_t>(R) * C, Rt * C * 4, eps_next, static_cast<size_t>(B) * C * 4, static_cast<size_t>(B) * C * 4, T, cudaMemcpyDeviceToDevice, st));
   return CSD_OK;
 }
 
@@ -903,6 +1013,7 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
   if (d.C < 1 || d.W < 1 || d.L < 1 || d.Dz < 1 || d.F < 1)
     return fail(ctx, CSD_ERR_INVALID_ARG, "head dims must be positive (C=%d W=%d L=%d Dz=%d F=%d)", d.C, d.W, d.L, d.Dz, d.F);
   if (d.C > kCPad) return fail(ctx, CSD_ERR_UNSUPPORTED, "token dim C = %d exceeds 16", d.C);
+  if (d.var_out != 0 && d.var_out != 1) return fail(ctx, CSD_ERR_INVALID_ARG, "var_out = %d must be 0 or 1", d.var_out);
   if (d.W % kTileN != 0) return fail(ctx, CSD_ERR_UNSUPPORTED, "width W = %d must be a multiple of 128", d.W);
   const int kmul = d.dtype != CSD_F32 ? kBlockK : kSimtBK;
   if (d.Dz % kmul != 0) return fail(ctx, CSD_ERR_UNSUPPORTED, "Dz = %d must be a multiple of %d", d.Dz, kmul);
@@ -963,12 +1074,19 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
   auto put = [&](const float* src, size_t n) { size_t o = fs.size(); fs.insert(fs.end(), src, src + n); while (fs.size() % 4) fs.push_back(0.0f); return o; };
   const size_t f_bz = put(w->bz, W), f_wt1 = put(w->Wt1, W * F), f_bt1 = put(w->bt1, W), f_wt2 = put(w->Wt2, W * W),
                f_bt2 = put(w->bt2, W), f_bin = put(w->bin, W);
-  std::vector<float> win_pad(W * kCPad, 0.0f), wout_t(W * kCPad, 0.0f), bout_pad(kCPad, 0.0f);
+  // Wout transposed to [W, 16] (or [W, 32] for a head that also predicts its variances: columns 16.. hold the
+  // variance rows C..2C of Wout), zero padded; the eps columns sit where they sit in a fixed-variance head
+  const size_t epw = d.var_out ? kCPad2 : kCPad;
+  std::vector<float> win_pad(W * kCPad, 0.0f), wout_t(W * epw, 0.0f), bout_pad(epw, 0.0f);
   for (size_t n = 0; n < W; ++n)
-    for (size_t c = 0; c < C; ++c) { win_pad[n * kCPad + c] = w->Win[n * C + c]; wout_t[n * kCPad + c] = w->Wout[c * W + n]; }
-  for (size_t c = 0; c < C; ++c) bout_pad[c] = w->bout[c];
+    for (size_t c = 0; c < C; ++c) {
+      win_pad[n * kCPad + c] = w->Win[n * C + c];
+      wout_t[n * epw + c] = w->Wout[c * W + n];
+      if (d.var_out) wout_t[n * epw + kCPad + c] = w->Wout[(C + c) * W + n];
+    }
+  for (size_t c = 0; c < C; ++c) { bout_pad[c] = w->bout[c]; if (d.var_out) bout_pad[kCPad + c] = w->bout[C + c]; }
   const size_t f_win = put(win_pad.data(), win_pad.size()), f_wout = put(wout_t.data(), wout_t.size()),
-               f_bout = put(bout_pad.data(), kCPad);
+               f_bout = put(bout_pad.data(), epw);
   std::vector<size_t> f_bsh(L), f_bsc(L), f_bg(L), f_b1(L), f_b2(L);
   for (size_t k = 0; k < L; ++k) {
     f_bsh[k] = put(w->bada + k * 3 * W, W); f_bsc[k] = put(w->bada + k * 3 * W + W, W);
@@ -1147,10 +1265,11 @@ int csd_accept_scan(csd_ctx* ctx, int B, int gamma, int C, double log_sigma_term
                      n_accept, accept_mask);
 }
 
-int csd_verify(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p, const csd_schedule* sched_q, int B,
-               int gamma, int cfg, float cfg_scale, const float* z_p, const float* x_T, const float* eps,
-               const float* x0_q, const float* mu1_q, const float* u, float* logratio, int32_t* n_accept,
-               uint32_t* accept_mask, float* mu1_p) {
+static int verify_impl(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p, const csd_schedule* sched_q,
+                       int B, int gamma, int cfg, float cfg_scale, const float* z_p, const float* x_T, const float* eps,
+                       const float* x0_q, const float* mu1_q, const float* u, float* logratio, int32_t* n_accept,
+                       uint32_t* accept_mask, float* mu1_p, bool bonus, const float* z_next, const float* x_T_next,
+                       const float* eps_next, float* x_bonus, uint32_t* taken) {
   if (!ctx) return CSD_ERR_INVALID_ARG;
   if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
   int rc = check_chain_args(ctx, head_p, sched_p, B * gamma, cfg, z_p, x_T, eps);
@@ -1159,12 +1278,45 @@ int csd_verify(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p
   if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
   if ((rc = check_verify_dims(ctx, B, gamma, head_p->d.C))) return rc;
   if (!x0_q || !mu1_q || !u || !logratio || !n_accept || !mu1_p) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  if (bonus && (!z_next || !x_T_next || !eps_next || !x_bonus)) return fail(ctx, CSD_ERR_INVALID_ARG, "z_next / x_T_next / eps_next / x_bonus is null");
   CSD_DEVICE(ctx);
-  rc = run_chain(ctx, 1, ctx->stream, head_p, sched_p, B * gamma, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr);
-  if (rc) return rc;
-  const int C = head_p->d.C;
-  return accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term(sched_q, sched_p, C), sched_p->sigma[0],
-                     sched_q->sigma[0], x0_q, mu1_q, mu1_p, u, logratio, n_accept, accept_mask);
+  const int R = B * gamma, C = head_p->d.C, T = sched_p->T;
+  BonusBuf bb{};
+  if (bonus) {
+    if ((rc = ensure_side(ctx, ctx->bn, bonus_buf_bytes(head_p->d, R + B, cfg, T), "the bonus rows"))) return rc;
+    if ((rc = gather_bonus_inputs(ctx, ctx->stream, head_p->d, R, B, cfg, T, z_p, x_T, eps, z_next, x_T_next, eps_next, bb))) return rc;
+    // every row samples at the last step; only the bonus rows' samples are used
+    rc = run_chain(ctx, 1, ctx->stream, head_p, sched_p, R + B, cfg, cfg_scale, bb.z, bb.x_T, bb.eps, 1, bb.x0, bb.mu1, nullptr);
+    if (rc) return rc;
+    CSD_CUDA(ctx, cudaMemcpyAsync(mu1_p, bb.mu1, static_cast<size_t>(R) * C * 4, cudaMemcpyDeviceToDevice, ctx->stream));
+  } else {
+    rc = run_chain(ctx, 1, ctx->stream, head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr);
+    if (rc) return rc;
+  }
+  rc = accept_scan(ctx, ctx->stream, B, gamma, C, log_sigma_term(sched_q, sched_p, C), sched_p->sigma[0],
+                   sched_q->sigma[0], x0_q, mu1_q, mu1_p, u, logratio, n_accept, accept_mask);
+  if (rc || !bonus) return rc;
+  bonus_select_kernel<<<(B * C + 255) / 256, 256, 0, ctx->stream>>>(B, C, gamma, n_accept, bb.x0 + static_cast<size_t>(R) * C, x_bonus, taken);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+int csd_verify(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p, const csd_schedule* sched_q, int B,
+               int gamma, int cfg, float cfg_scale, const float* z_p, const float* x_T, const float* eps,
+               const float* x0_q, const float* mu1_q, const float* u, float* logratio, int32_t* n_accept,
+               uint32_t* accept_mask, float* mu1_p) {
+  return verify_impl(ctx, head_p, sched_p, sched_q, B, gamma, cfg, cfg_scale, z_p, x_T, eps, x0_q, mu1_q, u, logratio,
+                     n_accept, accept_mask, mu1_p, false, nullptr, nullptr, nullptr, nullptr, nullptr);
+}
+
+int csd_verify_bonus(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p, const csd_schedule* sched_q, int B,
+                     int gamma, int cfg, float cfg_scale, const float* z_p, const float* x_T, const float* eps,
+                     const float* x0_q, const float* mu1_q, const float* u, const float* z_next, const float* x_T_next,
+                     const float* eps_next, float* logratio, int32_t* n_accept, uint32_t* accept_mask, float* mu1_p,
+                     float* x_bonus, uint32_t* taken) {
+  return verify_impl(ctx, head_p, sched_p, sched_q, B, gamma, cfg, cfg_scale, z_p, x_T, eps, x0_q, mu1_q, u, logratio,
+                     n_accept, accept_mask, mu1_p, true, z_next, x_T_next, eps_next, x_bonus, taken);
 }
 
 int csd_verify_unaligned(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sched_p, const csd_schedule* sched_q,
@@ -1212,17 +1364,7 @@ int csd_bonus_token(csd_ctx* ctx, const csd_head* head_p, const csd_schedule* sc
   if (!n_accept || !x_bonus) return fail(ctx, CSD_ERR_INVALID_ARG, "n_accept / x_bonus is null");
   CSD_DEVICE(ctx);
   const int C = head_p->d.C;
-  const size_t need = static_cast<size_t>(2) * B * C * 4;
-  if (need > ctx->bn.cap) {
-    CSD_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-    if (ctx->bn.base) CSD_CUDA(ctx, cudaFree(ctx->bn.base));
-    ctx->bn.base = nullptr; ctx->bn.cap = 0;
-    if (cudaMalloc(&ctx->bn.base, need) != cudaSuccess) {
-      cudaGetLastError();
-      return fail(ctx, CSD_ERR_WORKSPACE, "cannot allocate %zu bytes for the bonus samples", need);
-    }
-    ctx->bn.cap = need;
-  }
+  if ((rc = ensure_side(ctx, ctx->bn, static_cast<size_t>(2) * B * C * 4, "the bonus samples"))) return rc;
   float* d_x0 = static_cast<float*>(ctx->bn.base);
   float* d_mu = d_x0 + static_cast<size_t>(B) * C;
   // the masks live on the device, so every sequence is sampled and the selection is a kernel: no host round trip
@@ -1343,11 +1485,13 @@ int csd_resample(csd_ctx* ctx, int B, int gamma, int C, int cap, double log_sigm
                   x_new, n_prop, flags, cap_hits);
 }
 
-int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule* sched_q,
-              const csd_schedule* sched_p, int B, int gamma, int cfg, float cfg_scale, int cap, const float* z_q,
-              const float* z_p, const float* x_T, const float* eps, const float* u, const float* xi, const float* v,
-              float* x0, float* mu1_q, float* mu1_p, float* logratio, int32_t* n_accept, uint32_t* accept_mask,
-              float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+static int round_impl(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule* sched_q,
+                      const csd_schedule* sched_p, int B, int gamma, int cfg, float cfg_scale, int cap, const float* z_q,
+                      const float* z_p, const float* x_T, const float* eps, const float* u, const float* xi,
+                      const float* v, float* x0, float* mu1_q, float* mu1_p, float* logratio, int32_t* n_accept,
+                      uint32_t* accept_mask, float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits,
+                      bool bonus, const float* z_next, const float* x_T_next, const float* eps_next, float* x_bonus,
+                      uint32_t* taken) {
   if (!ctx) return CSD_ERR_INVALID_ARG;
   if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
   const int R = B * gamma;
@@ -1356,23 +1500,182 @@ int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, cons
   if ((rc = check_chain_args(ctx, head_p, sched_p, R, cfg, z_p, x_T, eps))) return rc;
   if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
   if (head_q->d.C != head_p->d.C) return fail(ctx, CSD_ERR_SHAPE, "draft C = %d and target C = %d differ", head_q->d.C, head_p->d.C);
-  const int C = head_p->d.C;
+  const int C = head_p->d.C, T = sched_p->T;
   if ((rc = check_verify_dims(ctx, B, gamma, C))) return rc;
   if (cap < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cap = %d must be >= 1", cap);
   if (!u || !xi || !v || !x0 || !mu1_q || !mu1_p || !logratio || !n_accept || !x_new || !n_prop || !flags || !cap_hits)
     return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  if (bonus && (!z_next || !x_T_next || !eps_next || !x_bonus)) return fail(ctx, CSD_ERR_INVALID_ARG, "z_next / x_T_next / eps_next / x_bonus is null");
   CSD_DEVICE(ctx);
+  const int Rp = bonus ? R + B : R;    // token rows of the target chain
   // workspaces first (growing one synchronises), then fork the two chains
   if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T))) return rc;
-  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, Rp * (cfg ? 2 : 1), Rp, sched_p->T))) return rc;
+  if (bonus && (rc = ensure_side(ctx, ctx->bn, bonus_buf_bytes(head_p->d, Rp, cfg, T), "the bonus rows"))) return rc;
   CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
   for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
   // the two chains' launches are interleaved step by step so that neither stream starves
   // the chain with more work per row goes to the higher-priority stream
   const double wq = static_cast<double>(head_q->d.L) * head_q->d.W * head_q->d.W, wp = static_cast<double>(head_p->d.L) * head_p->d.W * head_p->d.W;
   const int sq = wq > wp ? 1 : 0;
+  BonusBuf bb{};
+  if (bonus && (rc = gather_bonus_inputs(ctx, ctx->side[1 - sq], head_p->d, R, B, cfg, T, z_p, x_T, eps, z_next, x_T_next, eps_next, bb))) return rc;
   Chain cq{ctx, 0, ctx->side[sq], head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr};
-  Chain cp{ctx, 1, ctx->side[1 - sq], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr};
+  Chain cp = bonus ? Chain{ctx, 1, ctx->side[1 - sq], head_p, sched_p, Rp, cfg, cfg_scale, bb.z, bb.x_T, bb.eps, 1, bb.x0, bb.mu1, nullptr}
+                   : Chain{ctx, 1, ctx->side[1 - sq], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr};
+  cq.chains = cp.chains = 2;
+  rc = cp.begin();
+  int rc2 = cq.begin();
+  for (int t = sched_p->T; t >= 1 && !rc && !rc2; --t) {
+    rc = cp.step(t);
+    if (!rc) rc2 = cq.step(t);
+  }
+  if (bonus && !rc) CSD_CUDA(ctx, cudaMemcpyAsync(mu1_p, bb.mu1, static_cast<size_t>(R) * C * 4, cudaMemcpyDeviceToDevice, ctx->side[1 - sq]));
+  for (int i = 0; i < 2; ++i) {
+    CSD_CUDA(ctx, cudaEventRecord(ctx->ev_done[i], ctx->side[i]));
+    CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_done[i], 0));
+  }
+  if (rc) return rc;
+  if (rc2) return rc2;
+  const double ls = log_sigma_term(sched_q, sched_p, C);
+  rc = accept_scan(ctx, ctx->stream, B, gamma, C, ls, sched_p->sigma[0], sched_q->sigma[0], x0, mu1_q, mu1_p, u, logratio,
+                   n_accept, accept_mask);
+  if (rc) return rc;
+  if (bonus) {
+    bonus_select_kernel<<<(B * C + 255) / 256, 256, 0, ctx->stream>>>(B, C, gamma, n_accept, bb.x0 + static_cast<size_t>(R) * C, x_bonus, taken);
+    ctx->launches++;
+    CSD_CUDA(ctx, cudaGetLastError());
+  }
+  return resample(ctx, ctx->stream, B, gamma, C, cap, ls, sched_p->sigma[0], sched_q->sigma[0], n_accept, mu1_p, mu1_q, xi,
+                  v, x_new, n_prop, flags, cap_hits);
+}
+
+int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule* sched_q,
+              const csd_schedule* sched_p, int B, int gamma, int cfg, float cfg_scale, int cap, const float* z_q,
+              const float* z_p, const float* x_T, const float* eps, const float* u, const float* xi, const float* v,
+              float* x0, float* mu1_q, float* mu1_p, float* logratio, int32_t* n_accept, uint32_t* accept_mask,
+              float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  return round_impl(ctx, head_q, head_p, sched_q, sched_p, B, gamma, cfg, cfg_scale, cap, z_q, z_p, x_T, eps, u, xi, v, x0,
+                    mu1_q, mu1_p, logratio, n_accept, accept_mask, x_new, n_prop, flags, cap_hits, false, nullptr, nullptr,
+                    nullptr, nullptr, nullptr);
+}
+
+int csd_round_bonus(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule* sched_q,
+                    const csd_schedule* sched_p, int B, int gamma, int cfg, float cfg_scale, int cap, const float* z_q,
+                    const float* z_p, const float* x_T, const float* eps, const float* u, const float* xi, const float* v,
+                    const float* z_next, const float* x_T_next, const float* eps_next, float* x0, float* mu1_q,
+                    float* mu1_p, float* logratio, int32_t* n_accept, uint32_t* accept_mask, float* x_new,
+                    int32_t* n_prop, uint32_t* flags, int32_t* cap_hits, float* x_bonus, uint32_t* taken) {
+  return round_impl(ctx, head_q, head_p, sched_q, sched_p, B, gamma, cfg, cfg_scale, cap, z_q, z_p, x_T, eps, u, xi, v, x0,
+                    mu1_q, mu1_p, logratio, n_accept, accept_mask, x_new, n_prop, flags, cap_hits, true, z_next, x_T_next,
+                    eps_next, x_bonus, taken);
+}
+
+// ------------------------------------------------------------------ heads that predict their variances
+int csd_schedule_lv_ddpm(int T, const double* beta, double tau, float* a, float* b, float* lv_min, float* lv_max) {
+  if (T < 1 || !beta || !a || !b || !lv_min || !lv_max || !(tau > 0.0)) return CSD_ERR_INVALID_ARG;
+  double abar = 1.0, abar_prev = 1.0;
+  for (int t = 0; t < T; ++t) {
+    if (!(beta[t] > 0.0 && beta[t] < 1.0)) return CSD_ERR_INVALID_ARG;
+    const double alpha = 1.0 - beta[t];
+    abar_prev = abar;
+    abar *= alpha;
+    a[t] = static_cast<float>(1.0 / std::sqrt(alpha));
+    b[t] = static_cast<float>(beta[t] / (std::sqrt(alpha) * std::sqrt(1.0 - abar)));
+    lv_max[t] = static_cast<float>(std::log(beta[t]) + 2.0 * std::log(tau));
+    // posterior variance beta_t (1 - abar_{t-1}) / (1 - abar_t); zero at t = 1, which borrows the value of t = 2 below
+    if (t > 0) lv_min[t] = static_cast<float>(std::log(beta[t] * (1.0 - abar_prev) / (1.0 - abar)) + 2.0 * std::log(tau));
+  }
+  lv_min[0] = T > 1 ? lv_min[1] : lv_max[0];
+  return CSD_OK;
+}
+
+int csd_draft_denoise_lv(csd_ctx* ctx, const csd_head* head, const csd_schedule_lv* sched, int R, int cfg,
+                         float cfg_scale, const float* z, const float* x_T, const float* eps, float* x0, float* mu1,
+                         float* lv1, float* half_logdet, float* x1) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_lv_args(ctx, head, sched, R, cfg, z, x_T, eps);
+  if (rc) return rc;
+  if (!x0 || !mu1 || !lv1 || !half_logdet) return fail(ctx, CSD_ERR_INVALID_ARG, "x0 / mu1 / lv1 / half_logdet is null");
+  CSD_DEVICE(ctx);
+  csd_schedule view{sched->T, sched->a, sched->b, nullptr, sched->tfeat};
+  Chain c = make_lv_chain(ctx, 0, ctx->stream, head, &view, sched, R, cfg, cfg_scale, z, x_T, eps, 1, x0, mu1, lv1,
+                          half_logdet, x1);
+  rc = c.begin();
+  for (int t = sched->T; t >= 1 && !rc; --t) rc = c.step(t);
+  return rc;
+}
+
+int csd_verify_lv(csd_ctx* ctx, const csd_head* head_p, const csd_schedule_lv* sched_p, int B, int gamma, int cfg,
+                  float cfg_scale, const float* z_p, const float* x_T, const float* eps, const float* x0_q,
+                  const float* mu1_q, const float* lv1_q, const float* half_logdet_q, const float* u, float* logratio,
+                  int32_t* n_accept, uint32_t* accept_mask, float* mu1_p, float* lv1_p, float* half_logdet_p,
+                  float* log_sigma_rows) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
+  int rc = check_lv_args(ctx, head_p, sched_p, B * gamma, cfg, z_p, x_T, eps);
+  if (rc) return rc;
+  if ((rc = check_verify_dims(ctx, B, gamma, head_p->d.C))) return rc;
+  if (!x0_q || !mu1_q || !lv1_q || !half_logdet_q || !u || !logratio || !n_accept || !mu1_p || !lv1_p || !half_logdet_p ||
+      !log_sigma_rows)
+    return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_DEVICE(ctx);
+  csd_schedule view{sched_p->T, sched_p->a, sched_p->b, nullptr, sched_p->tfeat};
+  Chain c = make_lv_chain(ctx, 1, ctx->stream, head_p, &view, sched_p, B * gamma, cfg, cfg_scale, z_p, x_T, eps, 0,
+                          nullptr, mu1_p, lv1_p, half_logdet_p, nullptr);
+  rc = c.begin();
+  for (int t = sched_p->T; t >= 1 && !rc; --t) rc = c.step(t);
+  if (rc) return rc;
+  return accept_scan_lv(ctx, ctx->stream, B, gamma, head_p->d.C, x0_q, mu1_q, lv1_q, half_logdet_q, mu1_p, lv1_p,
+                        half_logdet_p, u, logratio, log_sigma_rows, n_accept, accept_mask);
+}
+
+int csd_resample_lv(csd_ctx* ctx, int B, int gamma, int C, int cap, const float* log_sigma_rows, const int32_t* n_accept,
+                    const float* mu1_p, const float* lv1_p, const float* mu1_q, const float* lv1_q, const float* xi,
+                    const float* v, float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_verify_dims(ctx, B, gamma, C);
+  if (rc) return rc;
+  if (cap < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cap = %d must be >= 1", cap);
+  if (!log_sigma_rows || !n_accept || !mu1_p || !lv1_p || !mu1_q || !lv1_q || !xi || !v || !x_new || !n_prop || !flags || !cap_hits)
+    return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_DEVICE(ctx);
+  return resample_lv(ctx, ctx->stream, B, gamma, C, cap, log_sigma_rows, n_accept, mu1_p, lv1_p, mu1_q, lv1_q, xi, v, x_new,
+                     n_prop, flags, cap_hits);
+}
+
+int csd_round_lv(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule_lv* sched_q,
+                 const csd_schedule_lv* sched_p, int B, int gamma, int cfg, float cfg_scale, int cap, const float* z_q,
+                 const float* z_p, const float* x_T, const float* eps, const float* u, const float* xi, const float* v,
+                 float* x0, float* mu1_q, float* lv1_q, float* half_logdet_q, float* mu1_p, float* lv1_p,
+                 float* half_logdet_p, float* log_sigma_rows, float* logratio, int32_t* n_accept, uint32_t* accept_mask,
+                 float* x_new, int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
+  const int R = B * gamma;
+  int rc = check_lv_args(ctx, head_q, sched_q, R, cfg, z_q, x_T, eps);
+  if (rc) return rc;
+  if ((rc = check_lv_args(ctx, head_p, sched_p, R, cfg, z_p, x_T, eps))) return rc;
+  if (sched_q->T != sched_p->T) return fail(ctx, CSD_ERR_SHAPE, "draft T = %d and target T = %d differ", sched_q->T, sched_p->T);
+  if (head_q->d.C != head_p->d.C) return fail(ctx, CSD_ERR_SHAPE, "draft C = %d and target C = %d differ", head_q->d.C, head_p->d.C);
+  const int C = head_p->d.C;
+  if ((rc = check_verify_dims(ctx, B, gamma, C))) return rc;
+  if (cap < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cap = %d must be >= 1", cap);
+  if (!u || !xi || !v || !x0 || !mu1_q || !lv1_q || !half_logdet_q || !mu1_p || !lv1_p || !half_logdet_p || !log_sigma_rows ||
+      !logratio || !n_accept || !x_new || !n_prop || !flags || !cap_hits)
+    return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_DEVICE(ctx);
+  if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T))) return rc;
+  if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, R * (cfg ? 2 : 1), R, sched_p->T))) return rc;
+  CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
+  for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
+  const double wq = static_cast<double>(head_q->d.L) * head_q->d.W * head_q->d.W, wp = static_cast<double>(head_p->d.L) * head_p->d.W * head_p->d.W;
+  const int sq = wq > wp ? 1 : 0;
+  csd_schedule vq{sched_q->T, sched_q->a, sched_q->b, nullptr, sched_q->tfeat}, vp{sched_p->T, sched_p->a, sched_p->b, nullptr, sched_p->tfeat};
+  Chain cq = make_lv_chain(ctx, 0, ctx->side[sq], head_q, &vq, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, lv1_q,
+                           half_logdet_q, nullptr);
+  Chain cp = make_lv_chain(ctx, 1, ctx->side[1 - sq], head_p, &vp, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p,
+                           lv1_p, half_logdet_p, nullptr);
   cq.chains = cp.chains = 2;
   rc = cp.begin();
   int rc2 = cq.begin();
@@ -1386,12 +1689,11 @@ int csd_round(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, cons
   }
   if (rc) return rc;
   if (rc2) return rc2;
-  const double ls = log_sigma_term(sched_q, sched_p, C);
-  rc = accept_scan(ctx, ctx->stream, B, gamma, C, ls, sched_p->sigma[0], sched_q->sigma[0], x0, mu1_q, mu1_p, u, logratio,
-                   n_accept, accept_mask);
+  rc = accept_scan_lv(ctx, ctx->stream, B, gamma, C, x0, mu1_q, lv1_q, half_logdet_q, mu1_p, lv1_p, half_logdet_p, u, logratio,
+                      log_sigma_rows, n_accept, accept_mask);
   if (rc) return rc;
-  return resample(ctx, ctx->stream, B, gamma, C, cap, ls, sched_p->sigma[0], sched_q->sigma[0], n_accept, mu1_p, mu1_q, xi,
-                  v, x_new, n_prop, flags, cap_hits);
+  return resample_lv(ctx, ctx->stream, B, gamma, C, cap, log_sigma_rows, n_accept, mu1_p, lv1_p, mu1_q, lv1_q, xi, v, x_new,
+                     n_prop, flags, cap_hits);
 }
 
 int csd_round_host(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule* sched_q,

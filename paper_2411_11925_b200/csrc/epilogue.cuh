@@ -21,8 +21,13 @@ enum Epi : int {
   EPI_SILU_ACT = 1,  // out_act = SiLU(acc0 + bias0)                             (block MLP, first layer)
   EPI_MOD = 2,       // out_act = LN(h)(1 + acc1 + bias1) + acc0 + bias0         (AdaLN modulate)
   EPI_GATE_RES = 3,  // h += (acc1 + bias1) * (acc0 + bias0); LayerNorm partials (second layer + gate)
-  EPI_MODF = 4       // eps partial = Wout^T-tile . [LN(h)(1 + acc1 + bias1) + acc0 + bias0]
+  EPI_MODF = 4,      // eps partial = Wout^T-tile . [LN(h)(1 + acc1 + bias1) + acc0 + bias0]
+  EPI_MODF2 = 5      // the same with 32 output columns: eps_hat | variance parameter (learned-variance heads)
 };
+constexpr int kCPad2 = 2 * kCPad;   // widest output projection
+template <int EPI> __host__ __device__ constexpr bool epi_is_modf() { return EPI == EPI_MODF || EPI == EPI_MODF2; }
+// output-projection columns per row (token dim padded to 16, once or twice)
+template <int EPI> __host__ __device__ constexpr int epi_out_width() { return EPI == EPI_MODF2 ? kCPad2 : kCPad; }
 
 struct EpiParams {
   int M;                 // valid rows
@@ -34,8 +39,8 @@ struct EpiParams {
   float* h;              // EPI_MOD / EPI_MODF (read), EPI_GATE_RES (read-modify-write)
   int nt;                // eps partials per row: N/64 (tensor-core kernel), N/128 (FMA kernel)
   float* stats;          // [M, ldo/64, 2] (mean, M2) per 64-column group of h
-  const float* wout_t;   // [N, 16] fp32, Wout transposed and zero padded (EPI_MODF)
-  float* epart;          // [M, nt, 16] (EPI_MODF)
+  const float* wout_t;   // [N, 16 or 32] fp32, Wout transposed and zero padded (EPI_MODF, EPI_MODF2)
+  float* epart;          // [M, nt, 16 or 32] (EPI_MODF, EPI_MODF2)
 };
 
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
@@ -103,7 +108,7 @@ __device__ __forceinline__ void load_chunk_f32(const float* src, float* v) {
 // Per-row state carried across the chunks of one tile.
 struct RowState {
   float mean, rstd;          // LayerNorm statistics of the row (EPI_MOD, EPI_MODF)
-  float eacc[kCPad];         // eps_hat partial sums (EPI_MODF)
+  float eacc[kCPad2];        // output-projection partial sums (EPI_MODF: the first 16; EPI_MODF2: all 32)
   float pm, pm2, pn;         // running (mean, M2, count) of the new h values (EPI_GATE_RES)
 };
 
@@ -158,15 +163,15 @@ __device__ __forceinline__ void row_stats(const float* stats, int m, int W, floa
 
 template <int EPI>
 __device__ __forceinline__ void epi_row_begin(const EpiParams& ep, int m, RowState& rs) {
-  if constexpr (EPI == EPI_MOD || EPI == EPI_MODF) row_stats<false>(ep.stats, m, ep.ldo, rs.mean, rs.rstd);
-  if constexpr (EPI == EPI_MODF) {
+  if constexpr (EPI == EPI_MOD || epi_is_modf<EPI>()) row_stats<false>(ep.stats, m, ep.ldo, rs.mean, rs.rstd);
+  if constexpr (epi_is_modf<EPI>()) {
 #pragma unroll
-    for (int c = 0; c < kCPad; ++c) rs.eacc[c] = 0.0f;
+    for (int c = 0; c < epi_out_width<EPI>(); ++c) rs.eacc[c] = 0.0f;
   }
   if constexpr (EPI == EPI_GATE_RES) { rs.pm = 0.0f; rs.pm2 = 0.0f; rs.pn = 0.0f; }
 }
 
-template <int EPI> __host__ __device__ constexpr bool epi_reads_h() { return EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES; }
+template <int EPI> __host__ __device__ constexpr bool epi_reads_h() { return EPI == EPI_MOD || epi_is_modf<EPI>() || EPI == EPI_GATE_RES; }
 
 // Residual update of one 32-column chunk, hv += (a1 + b1) (a0 + b0), and its (mean, M2) partial merged
 // into the row state (a thread owns one or two chunks of a 64-column group: the second is merged with
@@ -204,13 +209,14 @@ __device__ __forceinline__ void modulate_chunk(float* a0, const float* a1, const
   }
 }
 
-// eps_hat partial of one chunk: eacc[c] += sum_j a0[j] Wout^T[j][c]  (wout_c: [32][16]).
+// Output-projection partial of one chunk: eacc[c] += sum_j a0[j] Wout^T[j][c]  (wout_c: [32][EPW]).
+template <int EPW>
 __device__ __forceinline__ void outproj_chunk(const float* a0, const float* wout_c, RowState& rs) {
 #pragma unroll
   for (int j = 0; j < kChunk; ++j) {
-    const float4* w4 = reinterpret_cast<const float4*>(wout_c + j * kCPad);
+    const float4* w4 = reinterpret_cast<const float4*>(wout_c + j * EPW);
 #pragma unroll
-    for (int c4 = 0; c4 < kCPad / 4; ++c4) {
+    for (int c4 = 0; c4 < EPW / 4; ++c4) {
       const float4 w = w4[c4];
       rs.eacc[4 * c4 + 0] = fmaf(a0[j], w.x, rs.eacc[4 * c4 + 0]);
       rs.eacc[4 * c4 + 1] = fmaf(a0[j], w.y, rs.eacc[4 * c4 + 1]);
@@ -223,7 +229,7 @@ __device__ __forceinline__ void outproj_chunk(const float* a0, const float* wout
 // a0 / a1: accumulator chunk (32 columns) of the first / second accumulator; n0 = first global
 // output column of the chunk; b0 / b1: the chunk's 32 biases (shared or global memory); hv: the
 // chunk's 32 values of h, already loaded (EPI_MOD, EPI_MODF, EPI_GATE_RES); wout_c: the chunk's
-// [32][16] slice of Wout^T in shared memory (EPI_MODF).
+// [32][16 or 32] slice of Wout^T in shared memory (EPI_MODF, EPI_MODF2).
 template <int EPI, typename ACT, bool FAST>
 __device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, float* a0, const float* a1,
                                           const float* b0, const float* b1, float* hv, RowState& rs,
@@ -237,10 +243,10 @@ __device__ __forceinline__ void epi_chunk(const EpiParams& ep, int m, int n0, fl
 #pragma unroll
     for (int j = 0; j < kChunk; ++j) a0[j] = silu_t<FAST>(a0[j] + b0[j]);
     store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
-  } else if constexpr (EPI == EPI_MOD || EPI == EPI_MODF) {
+  } else if constexpr (EPI == EPI_MOD || epi_is_modf<EPI>()) {
     modulate_chunk(a0, a1, b0, b1, hv, rs);
     if constexpr (EPI == EPI_MOD) store_chunk<ACT>(reinterpret_cast<ACT*>(ep.out_act) + off, a0);
-    else outproj_chunk(a0, wout_c, rs);
+    else outproj_chunk<epi_out_width<EPI>()>(a0, wout_c, rs);
   } else if constexpr (EPI == EPI_GATE_RES) {
     gate_res_chunk(a0, a1, b0, b1, hv, rs);
     store_chunk<float>(ep.h + off, hv);
@@ -254,10 +260,11 @@ __device__ __forceinline__ void store_group_stats(const EpiParams& ep, int m, in
 
 template <int EPI>
 __device__ __forceinline__ void epi_row_end(const EpiParams& ep, int m, int part, const RowState& rs) {
-  if constexpr (EPI == EPI_MODF) {
-    float4* d = reinterpret_cast<float4*>(ep.epart + (static_cast<size_t>(m) * ep.nt + part) * kCPad);
+  if constexpr (epi_is_modf<EPI>()) {
+    constexpr int EPW = epi_out_width<EPI>();
+    float4* d = reinterpret_cast<float4*>(ep.epart + (static_cast<size_t>(m) * ep.nt + part) * EPW);
 #pragma unroll
-    for (int c = 0; c < kCPad / 4; ++c)
+    for (int c = 0; c < EPW / 4; ++c)
       d[c] = make_float4(rs.eacc[4 * c], rs.eacc[4 * c + 1], rs.eacc[4 * c + 2], rs.eacc[4 * c + 3]);
   }
 }

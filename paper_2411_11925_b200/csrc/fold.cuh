@@ -232,7 +232,6 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
 #pragma unroll
       for (int ci = 0; ci < 2; ++ci) {
         const int c = 2 * half + ci;                                  // 32-column chunk of the tile
-        const int n0 = n_base + c * kChunk;
         float a0[kChunk], a1[kChunk], am[kChunk];
         const uint32_t colp = kFoldAccPacked + (c >> 1) * 128 + (c & 1) * kChunk;
         tmem_ld32(trow + colp, a0);                                   // first packed product (P1 / gate)

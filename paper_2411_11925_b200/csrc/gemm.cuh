@@ -31,7 +31,7 @@ enum DevErr : int { DEV_OK = 0, DEV_ERR_TMA_WAIT = 1, DEV_ERR_MMA_WAIT = 2, DEV_
 // PAIR: two CTAs of a cluster share one MMA (cta_group::2, M = 256): each holds its own 128 rows of A
 // and half of the B rows, which cuts the shared-memory traffic per CTA and k-block.
 template <int EPI, int MMA_N, int TN, bool PAIR> struct TcCfg {
-  static constexpr bool kStageH = EPI == EPI_MOD || EPI == EPI_MODF || EPI == EPI_GATE_RES;
+  static constexpr bool kStageH = EPI == EPI_MOD || epi_is_modf<EPI>() || EPI == EPI_GATE_RES;
   // A stage holds kKps k-blocks of 64 elements (one TMA box per operand and k-block).  The kernels whose
   // MMAs are 128 wide use two: fewer barrier round trips per byte.
   static constexpr int kKps = ((EPI == EPI_SILU_ACT || EPI == EPI_GATE_RES) && MMA_N <= 128) ? 2 : 1;
@@ -43,7 +43,7 @@ template <int EPI, int MMA_N, int TN, bool PAIR> struct TcCfg {
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kHTileBytes = kTileM * TN * 4;        // fp32 h tile staged in shared memory
   static constexpr int kHBytes = kStageH ? kHTileBytes : 0;
-  static constexpr int kWoutBytes = kTileM * kCPad * 4;      // Wout^T tile [TN][16], reused for [128 rows][16] eps partials
+  static constexpr int kWoutBytes = kTileM * epi_out_width<EPI>() * 4;   // Wout^T tile [TN][16 or 32], reused for [128 rows][..] partials
   static constexpr int kMiscBytes = 2 * TN * 4 + kTileM * 16;   // two bias slices + per-row exchange
   static constexpr int kFixedBytes = 1024 + kHBytes + kWoutBytes + kMiscBytes + 256;
   static constexpr int kStagesMax = (227 * 1024 - kFixedBytes) / kStageBytes;
@@ -84,6 +84,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   constexpr int EW = TcWarps<EPI, TN>::kEpi, CPT = TcWarps<EPI, TN>::kChunksPerThread, kEpiThreads = EW * 32;
   constexpr int NC = TN / kChunk;               // column chunks per tile
   constexpr bool kPacked = (NSEG == 1) && (MMA_N == 2 * TN);
+  constexpr int EPW = epi_out_width<EPI>();   // output-projection columns (EPI_MODF, EPI_MODF2)
   constexpr bool kTwoAcc = kPacked || NSEG == 2;
   constexpr uint32_t kAccCols = NSEG * MMA_N;   // 64, 128 or 256 columns per accumulator buffer
   constexpr uint32_t kTmemCols = 2 * kAccCols;  // two buffers: a power of two in [128, 512]
@@ -252,11 +253,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         bias_s[et] = ep.bias0[tile_n * TN + et];
         bias_s[TN + et] = ep.bias1 ? ep.bias1[tile_n * TN + et] : 0.0f;
       }
-      if (EPI == EPI_MODF) {
-        const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * TN * kCPad);
+      if (epi_is_modf<EPI>()) {
+        const float4* src = reinterpret_cast<const float4*>(ep.wout_t + static_cast<size_t>(tile_n) * TN * EPW);
         float4* dst = reinterpret_cast<float4*>(wout_s);
 #pragma unroll
-        for (int j = 0; j < TN * kCPad / 4 / kEpiThreads; ++j) dst[et + j * kEpiThreads] = src[et + j * kEpiThreads];
+        for (int j = 0; j < TN * EPW / 4 / kEpiThreads; ++j) dst[et + j * kEpiThreads] = src[et + j * kEpiThreads];
       }
     };
     stage_consts(unit % tiles_n);
@@ -316,20 +317,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           if (kTwoAcc) tmem_ld32(trow + col0 + (kPacked ? kStatCols : TN), a1);
           if (Cfg::kStageH) load_swizzled_row32(h_s + c * (kTileM * 128), rloc, hv);
           tmem_ld_wait();
-          float efirst[kCPad];
-          if (EPI == EPI_MODF && ci == 1) {
+          float efirst[EPW];
+          if (epi_is_modf<EPI>() && ci == 1) {
 #pragma unroll
-            for (int e = 0; e < kCPad; ++e) { efirst[e] = rs.eacc[e]; rs.eacc[e] = 0.0f; }
+            for (int e = 0; e < EPW; ++e) { efirst[e] = rs.eacc[e]; rs.eacc[e] = 0.0f; }
           }
           if (EPI == EPI_GATE_RES) {
             gate_res_chunk(a0, a1, bias_s + c * kChunk, bias_s + TN + c * kChunk, hv, rs);
             store_swizzled_row32(h_s + c * (kTileM * 128), rloc, hv);   // in place; leaves by TMA store
           } else if (valid)
             epi_chunk<EPI, ACT, true>(ep, m, tile_n * TN + c * kChunk, a0, a1, bias_s + c * kChunk,
-                                      bias_s + TN + c * kChunk, hv, rs, wout_s + c * kChunk * kCPad);
-          if (EPI == EPI_MODF && ci == 1) {
+                                      bias_s + TN + c * kChunk, hv, rs, wout_s + c * kChunk * EPW);
+          if (epi_is_modf<EPI>() && ci == 1) {
 #pragma unroll
-            for (int e = 0; e < kCPad; ++e) rs.eacc[e] = efirst[e] + rs.eacc[e];
+            for (int e = 0; e < EPW; ++e) rs.eacc[e] = efirst[e] + rs.eacc[e];
           }
         }
         if (EPI == EPI_GATE_RES) fence_proxy_async_smem();
@@ -348,22 +349,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           }
         }
       }
-      if (EPI == EPI_MODF) {
+      if (epi_is_modf<EPI>()) {
         // one eps partial per row and 64-column group, always formed as (chunk sum) + (next chunk sum) so
         // that both tile widths give the same bits
         if (CPT == 2) {            // TN = 128: this thread's two chunks are one group
           if (ok && valid) epi_row_end<EPI>(ep, m, tile_n * 2 + half, rs);
         } else {                   // TN = 64: chunk 1 (warps 6..9) is added to chunk 0 (warps 2..5)
           asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread is done reading the Wout^T tile
-          float* part = wout_s;                            // [128 rows][16]
+          float* part = wout_s;                            // [128 rows][EPW]
           if (half == 1 && ok) {
 #pragma unroll
-            for (int c = 0; c < kCPad; ++c) part[rloc * kCPad + c] = rs.eacc[c];
+            for (int c = 0; c < EPW; ++c) part[rloc * EPW + c] = rs.eacc[c];
           }
           asm volatile("bar.sync 1, 256;" ::: "memory");
           if (half == 0 && ok && valid) {
 #pragma unroll
-            for (int c = 0; c < kCPad; ++c) rs.eacc[c] += part[rloc * kCPad + c];
+            for (int c = 0; c < EPW; ++c) rs.eacc[c] += part[rloc * EPW + c];
             epi_row_end<EPI>(ep, m, tile_n, rs);
           }
         }
@@ -399,13 +400,17 @@ gemm_simt_kernel(const float* __restrict__ A0, int lda0, const float* __restrict
                  EpiParams ep) {
   __shared__ float As[kSimtRows][kSimtBK + 1];
   __shared__ float Bs[MMA_N][kSimtBK + 1];
-  __shared__ float wout_s[(EPI == EPI_MODF) ? kTileN * kCPad : 1];
+  constexpr int EPW = epi_out_width<EPI>();
+  // the 16-column Wout^T tile is staged in shared memory; the 32-column one would not fit beside the operand tiles
+  // and is read through L1 instead
+  constexpr bool kStageWout = EPI == EPI_MODF;
+  __shared__ float wout_s[kStageWout ? kTileN * EPW : 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int tile_n = blockIdx.x, m0 = blockIdx.y * kSimtRows;
   const int m = m0 + lane;
-  if (EPI == EPI_MODF) {
-    const float* src = ep.wout_t + static_cast<size_t>(tile_n) * kTileN * kCPad;
-    for (int i = threadIdx.x; i < kTileN * kCPad; i += 128) wout_s[i] = src[i];
+  if (kStageWout) {
+    const float* src = ep.wout_t + static_cast<size_t>(tile_n) * kTileN * EPW;
+    for (int i = threadIdx.x; i < kTileN * EPW; i += 128) wout_s[i] = src[i];
   }
   float acc0[kChunk], acc1[kChunk];
 #pragma unroll
@@ -458,7 +463,8 @@ gemm_simt_kernel(const float* __restrict__ A0, int lda0, const float* __restrict
     epi_row_begin<EPI>(ep, m, rs);
     if (epi_reads_h<EPI>()) load_chunk_f32(ep.h + static_cast<size_t>(m) * ep.ldo + n0, hv);
     epi_chunk<EPI, float, false>(ep, m, n0, acc0, acc1, ep.bias0 + n0, ep.bias1 ? ep.bias1 + n0 : ep.bias0 + n0, hv, rs,
-                                 wout_s + warp * kChunk * kCPad);
+                                 kStageWout ? wout_s + warp * kChunk * EPW
+                                            : ep.wout_t + (static_cast<size_t>(tile_n) * kTileN + warp * kChunk) * EPW);
   }
   if constexpr (EPI == EPI_GATE_RES) {
     float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][4]: chunks (0,1) and (2,3) form the 64-column groups
@@ -471,19 +477,19 @@ gemm_simt_kernel(const float* __restrict__ A0, int lda0, const float* __restrict
       store_group_stats(ep, m, tile_n * 2 + (warp >> 1), rs.pm, rs.pm2);
     }
   }
-  if constexpr (EPI == EPI_MODF) {
-    float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][16]
+  if constexpr (epi_is_modf<EPI>()) {
+    float* scr = &Bs[0][0];  // reused as [4 chunks][32 rows][EPW]
     __syncthreads();
     if (m < ep.M) {
 #pragma unroll
-      for (int c = 0; c < kCPad; ++c) scr[(warp * kSimtRows + lane) * kCPad + c] = rs.eacc[c];
+      for (int c = 0; c < EPW; ++c) scr[(warp * kSimtRows + lane) * EPW + c] = rs.eacc[c];
     }
     __syncthreads();
     if (warp == 0 && m < ep.M) {
 #pragma unroll
-      for (int c = 0; c < kCPad; ++c) {
+      for (int c = 0; c < EPW; ++c) {
         float v = 0.0f;
-        for (int w = 0; w < 4; ++w) v += scr[(w * kSimtRows + lane) * kCPad + c];
+        for (int w = 0; w < 4; ++w) v += scr[(w * kSimtRows + lane) * EPW + c];
         rs.eacc[c] = v;
       }
       epi_row_end<EPI>(ep, m, tile_n, rs);

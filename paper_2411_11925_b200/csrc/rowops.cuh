@@ -102,7 +102,16 @@ struct StepParams {
   float* traj_x;                 // TRAJ kernels: where the state this boundary produces is recorded ([R, C])
   float* traj_mu;                // TRAJ kernels: where the mean of the step being finished is recorded ([R, C])
   int* status;                   // set to 1 when a mean or state of this step is not finite (csd_sync reports it)
+  // learned-variance heads (LV kernels): epart rows are 32 wide, [eps partials | variance-parameter partials]
+  float lv_min, lv_max;          // bounds of the log-variance at the step being finished
+  float* lv1;                    // STEP_LAST: [R, C] log-variance of the last step
+  float* half_logdet;            // [R]: (1/2) sum over steps t >= 2 and coordinates of the log-variance (zeroed by STEP_INIT)
 };
+
+// log-variance of one coordinate from the head's variance output w: lv_min + (w + 1)/2 (lv_max - lv_min)
+__device__ __forceinline__ float lv_interp(float w, float lv_min, float lv_max) {
+  return fmaf(__fmul_rn(0.5f, __fadd_rn(w, 1.0f)), __fsub_rn(lv_max, lv_min), lv_min);
+}
 
 // RB token rows per block.  Finishes step t (unless STEP_INIT) and prepares the next one:
 //   eps_hat = sum of tile partials + bout; guidance; mu = a x - b eps_hat; x <- mu + sigma eps_t
@@ -111,10 +120,14 @@ struct StepParams {
 // With one row per block the kernel is bound by re-reading Win (64 B per column and row) through L1; RB = 4 reads a
 // group's columns once for four rows.  The arithmetic of a row does not depend on RB.
 // TRAJ: also record the whole trajectory (every state and every mean), for the single-path ratio of Eq. 2.
-template <typename ACT, int RB, bool TRAJ = false>
+// LV: the head also predicts its transition's diagonal variance (Eq. 3 in its general form): the noise is scaled per
+// coordinate by exp(lv / 2), the row's half log-determinant is accumulated for Sigma of Eq. 7.
+template <typename ACT, int RB, bool TRAJ = false, bool LV = false>
 __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p, int mode) {
+  constexpr int EPW = LV ? kCPad2 : kCPad;
   __shared__ float xs[RB][kCPad];
   __shared__ float eh[RB][2][kCPad];
+  __shared__ float wv[LV ? RB : 1][kCPad];
   const int r0 = blockIdx.x * RB, tid = threadIdx.x;
   const int nrep = p.cfg ? 2 : 1;
   const int nrow = min(RB, p.R - r0);
@@ -128,6 +141,7 @@ __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p
         v = p.x_src[static_cast<size_t>(r0 + rr) * p.C + c];
         p.x[static_cast<size_t>(r0 + rr) * p.C + c] = v;
         if (TRAJ) p.traj_x[static_cast<size_t>(r0 + rr) * p.C + c] = v;
+        if (LV && c == 0) p.half_logdet[r0 + rr] = 0.0f;
       }
       xs[rr][c] = v;
     }
@@ -136,10 +150,15 @@ __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p
     if (tid < RB * 2 * kCPad) {
       const int c = tid % kCPad, rep = (tid / kCPad) & 1, rr = tid / (2 * kCPad);
       if (rr < nrow && rep < nrep) {
-        const float* e = p.epart + (static_cast<size_t>(r0 + rr + rep * p.R) * p.NT) * kCPad + c;
+        const float* e = p.epart + (static_cast<size_t>(r0 + rr + rep * p.R) * p.NT) * EPW + c;
         float acc = 0.0f;
-        for (int nt = 0; nt < p.NT; ++nt) acc += e[nt * kCPad];
+        for (int nt = 0; nt < p.NT; ++nt) acc += e[nt * EPW];
         eh[rr][rep][c] = acc + p.bout[c];
+        if (LV && rep == 0) {       // the variance parameter is the conditional row's own
+          float accv = 0.0f;
+          for (int nt = 0; nt < p.NT; ++nt) accv += e[nt * EPW + kCPad];
+          wv[rr][c] = accv + p.bout[kCPad + c];
+        }
       }
     }
     __syncthreads();
@@ -152,9 +171,12 @@ __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p
         if (p.cfg) e = cfg_combine(eh[rr][0][c], eh[rr][1][c], p.cfg_scale);
         const float xo = p.x[o];
         const float mu = ddpm_mean(p.a, xo, p.b, e);
-        xn = ddpm_sample(mu, p.sigma, p.eps_t[o]);
+        float sigma = p.sigma, lv = 0.0f;
+        if (LV) { lv = lv_interp(wv[rr][c], p.lv_min, p.lv_max); sigma = expf(0.5f * lv); }
+        xn = ddpm_sample(mu, sigma, p.eps_t[o]);
         // an activation beyond the 16-bit operand range became inf further up and arrives here as inf or NaN
         if (!(fabsf(xn) <= 3.0e38f)) *p.status = 1;
+        if (LV && mode == STEP_LAST) p.lv1[o] = lv;
         if (mode == STEP_LAST) {
           p.mu1[o] = mu;
           if (p.x1) p.x1[o] = xo;
@@ -165,6 +187,14 @@ __global__ void __launch_bounds__(256, RB == 4 ? 3 : 0) step_kernel(StepParams p
         }
       }
       xs[rr][c] = xn;
+      if (LV && mode != STEP_LAST) {
+        // (1/2) sum_d lv of this step, coordinates in order (lanes 0..15 of a half-warp hold one row)
+        float hsum = (rr < nrow && c < p.C) ? 0.5f * lv_interp(wv[rr][c], p.lv_min, p.lv_max) : 0.0f;
+        constexpr unsigned kRowLanes = RB * kCPad >= 32 ? 0xffffffffu : 0x0000ffffu;   // threads inside this branch
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) hsum += __shfl_xor_sync(kRowLanes, hsum, o);
+        if (rr < nrow && c == 0) p.half_logdet[r0 + rr] += hsum;
+      }
     }
     if (mode == STEP_LAST) return;
     __syncthreads();
@@ -456,6 +486,100 @@ bonus_select_kernel(int B, int C, int gamma, const int32_t* __restrict__ n_accep
   const bool all = n_accept[b] >= gamma;
   if (all) x_bonus[i] = x0[i];
   if (taken && i == b * C) taken[b] = all ? 1u : 0u;
+}
+
+// Verification with predicted diagonal variances.  Per token  log Sigma = half_logdet_q - half_logdet_p  (Eq. 7: the
+// product over t >= 2 of sqrt|Sigma_q,t| / sqrt|Sigma_p,t|, accumulated by the two chains), and
+//   logratio = log Sigma + log N(x0; mu_p, diag(exp(lv_p))) - log N(x0; mu_q, diag(exp(lv_q)))      (Eq. 8).
+// Each model's exponent-plus-normaliser sum is formed by the same instruction sequence, so identical draft and target
+// values give a difference of exactly zero.
+__device__ __forceinline__ float diag_neg_logpdf(const float* x, const float* mu, const float* lv, int C) {
+  float acc = 0.0f;     // sum_d [ lv_d / 2 + (x - mu)_d^2 / (2 exp(lv_d)) ]
+  for (int c = 0; c < C; ++c) {
+    const float e = x[c] - mu[c];
+    acc = __fadd_rn(acc, __fadd_rn(__fmul_rn(0.5f, lv[c]), __fmul_rn(__fmul_rn(0.5f, __fmul_rn(e, e)), expf(-lv[c]))));
+  }
+  return acc;
+}
+
+__global__ void __launch_bounds__(128)
+accept_scan_lv_kernel(int B, int gamma, int C, const float* __restrict__ x0, const float* __restrict__ mu_q,
+                      const float* __restrict__ lv_q, const float* __restrict__ hld_q, const float* __restrict__ mu_p,
+                      const float* __restrict__ lv_p, const float* __restrict__ hld_p, const float* __restrict__ u,
+                      float* __restrict__ logratio, float* __restrict__ log_sigma_rows, int32_t* __restrict__ n_accept,
+                      uint32_t* __restrict__ accept_mask) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  bool acc = true;
+  if (lane < gamma) {
+    const size_t row = static_cast<size_t>(b) * gamma + lane;
+    const float ls = __fsub_rn(hld_q[row], hld_p[row]);
+    const float nq = diag_neg_logpdf(x0 + row * C, mu_q + row * C, lv_q + row * C, C);
+    const float np = diag_neg_logpdf(x0 + row * C, mu_p + row * C, lv_p + row * C, C);
+    const float lr = __fadd_rn(ls, __fsub_rn(nq, np));
+    log_sigma_rows[row] = ls;
+    logratio[row] = lr;
+    acc = logf(u[row]) <= lr;
+  }
+  const uint32_t ballot = __ballot_sync(0xffffffffu, acc);
+  if (lane == 0) {
+    const uint32_t rej = ~ballot;
+    int n = rej ? (__ffs(rej) - 1) : gamma;
+    if (n > gamma) n = gamma;
+    n_accept[b] = n;
+    if (accept_mask) accept_mask[b] = (gamma >= 32) ? ballot : (ballot & ((1u << gamma) - 1u));
+  }
+}
+
+// Corollary 1 with diagonal final-step covariances: x' = mu_p + exp(lv_p / 2) xi, alpha_s = max(0, 1 - q(x') / (Sigma p(x')))
+// with the rejected token's own Sigma; one warp per sequence, lane c < C = coordinate.
+__global__ void __launch_bounds__(128)
+resample_lv_kernel(int B, int gamma, int C, int cap, const float* __restrict__ log_sigma_rows,
+                   const int32_t* __restrict__ n_accept, const float* __restrict__ mu_p, const float* __restrict__ lv_p,
+                   const float* __restrict__ mu_q, const float* __restrict__ lv_q, const float* __restrict__ xi,
+                   const float* __restrict__ v, float* __restrict__ x_new, int32_t* __restrict__ n_prop,
+                   uint32_t* __restrict__ flags, int32_t* __restrict__ cap_hits) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  const int n = n_accept[b];
+  if (n >= gamma) {
+    if (lane == 0) { n_prop[b] = 0; flags[b] = 0u; }
+    return;
+  }
+  const size_t row = static_cast<size_t>(b) * gamma + n;
+  const bool on = lane < C;
+  const float mp = on ? mu_p[row * C + lane] : 0.0f, mq = on ? mu_q[row * C + lane] : 0.0f;
+  const float lp_d = on ? lv_p[row * C + lane] : 0.0f, lq_d = on ? lv_q[row * C + lane] : 0.0f;
+  const float sp = expf(0.5f * lp_d), ivp = 0.5f * expf(-lp_d), ivq = 0.5f * expf(-lq_d);
+  const float ls = log_sigma_rows[row];
+  float hl = on ? 0.5f * (lq_d - lp_d) : 0.0f;      // (1/2) sum_d (lv_q - lv_p): the normalisers' part of lq - lp ... negated below
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) hl += __shfl_xor_sync(0xffffffffu, hl, o);
+  float xp = 0.0f;
+  int k = 0;
+  bool done = false;
+  for (; k < cap && !done; ++k) {
+    const float z = on ? xi[(static_cast<size_t>(b) * cap + k) * C + lane] : 0.0f;
+    xp = mp + sp * z;
+    float ep = on ? (xp - mp) : 0.0f, eq = on ? (xp - mq) : 0.0f;
+    ep = ep * ep * ivp; eq = eq * eq * ivq;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      ep += __shfl_xor_sync(0xffffffffu, ep, o);
+      eq += __shfl_xor_sync(0xffffffffu, eq, o);
+    }
+    // lq - lp = -(1/2) sum lv_q - eq + (1/2) sum lv_p + ep = -hl - eq + ep
+    const float alpha = fmaxf(0.0f, -expm1f(fminf(0.0f, (ep - eq) - hl - ls)));
+    done = v[static_cast<size_t>(b) * cap + k] <= alpha;
+  }
+  if (on) x_new[static_cast<size_t>(b) * C + lane] = xp;
+  if (lane == 0) {
+    n_prop[b] = k;
+    flags[b] = 1u | (done ? 0u : 2u);
+    if (!done) atomicAdd(cap_hits, 1);
+  }
 }
 
 // Self-test of the bounded waits: one thread waits on a barrier on which nobody ever arrives, so the wait runs

@@ -22,7 +22,8 @@ token dim C, timestep feature dim F); every matrix is row-major [out, in]:
     W1[L,W,W] b1[L,W]        per-block MLP, first layer
     W2[L,W,W] b2[L,W]        per-block MLP, second layer
     Wfada[2W,W] bfada[2W]    final AdaLN (shift | scale)
-    Wout[C,W] bout[C]        output projection
+    Wout[C,W] bout[C]        output projection ([2C,W], [2C] for a head that also predicts its
+                             transition's variance: rows C..2C give the variance parameter)
 """
 from __future__ import annotations
 
@@ -47,12 +48,14 @@ class HeadSpec:
     Dz: int
     C: int = 16
     F: int = 256
+    var_out: bool = False   # the head has 2C outputs: eps_hat and a variance parameter per coordinate
 
     def n_params(self) -> int:
         W, L, Dz, C, F = self.W, self.L, self.Dz, self.C, self.F
+        Co = 2 * C if self.var_out else C
         return (W * Dz + W + W * F + W + W * W + W + W * C + W
                 + L * (3 * W * W + 3 * W) + 2 * L * (W * W + W)
-                + 2 * W * W + 2 * W + C * W + C)
+                + 2 * W * W + 2 * W + Co * W + Co)
 
     def flops_per_row_step(self) -> float:
         """Algorithmic FLOPs of one head evaluation for one head row:
@@ -159,6 +162,7 @@ def make_head_weights(spec: HeadSpec, rng: np.random.Generator, bf16: bool = Fal
     matrices, N(0, 0.02^2) for Wz, Wt1, Wt2 and every bias.  No layer is
     zero-initialised (a zero gate would make every test vacuous)."""
     W, L, Dz, C, F = spec.W, spec.L, spec.Dz, spec.C, spec.F
+    Co = 2 * C if spec.var_out else C
     w = {
         "Wz": _normal(rng, 0.02, W, Dz), "bz": _normal(rng, 0.02, W),
         "Wt1": _normal(rng, 0.02, W, F), "bt1": _normal(rng, 0.02, W),
@@ -168,7 +172,7 @@ def make_head_weights(spec: HeadSpec, rng: np.random.Generator, bf16: bool = Fal
         "W1": _xavier(rng, L, W, W), "b1": _normal(rng, 0.02, L, W),
         "W2": _xavier(rng, L, W, W), "b2": _normal(rng, 0.02, L, W),
         "Wfada": _xavier(rng, 2 * W, W), "bfada": _normal(rng, 0.02, 2 * W),
-        "Wout": _xavier(rng, C, W), "bout": _normal(rng, 0.02, C),
+        "Wout": _xavier(rng, Co, W), "bout": _normal(rng, 0.02, Co),
     }
     if bf16:
         w = {k: (round_to_bf16(v) if v.ndim >= 2 and k.startswith("W") else v) for k, v in w.items()}

@@ -32,7 +32,7 @@ def test_binding_covers_the_header():
     from paper_2411_11925_b200 import api
     assert sorted(api.EXPORTS) == _declared()
     # struct layouts mirror the header
-    assert [f[0] for f in api._HeadDesc._fields_] == ["C", "W", "L", "Dz", "F", "dtype"]
+    assert [f[0] for f in api._HeadDesc._fields_] == ["C", "W", "L", "Dz", "F", "dtype", "var_out"]
     hdr = open(os.path.join(ROOT, "include", "csd.h")).read()
     block = hdr[hdr.index("typedef struct {\n  const float *Wz"):hdr.index("} csd_head_weights;")]
     assert re.findall(r"\*(\w+)", block) == list(api.WEIGHT_FIELDS)
