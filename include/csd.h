@@ -136,8 +136,19 @@ int64_t csd_launch_count(const csd_ctx *ctx);
  *                     bit for bit).
  *   CSD_CHAIN_LAYERS_PLAIN: as above without the folded blocks (three kernels per block everywhere); a
  *                     row's bits then do not depend on how many rows the call has.
+ *   CSD_CHAIN_SMALL_BATCH: as CSD_CHAIN_LAYERS, except that a chain of at most 128 head rows (R (1 + cfg) <= 128)
+ *                     on a 16-bit head with W in {512, 1024, 1536} and var_out = 0 runs as ONE persistent kernel
+ *                     that spreads every layer over the whole GPU (weights as the MMA's M operand, K split over
+ *                     a cluster of 8 CTAs with the partial sums reduced through distributed shared memory, the
+ *                     products of the condition vector computed a step ahead by the remaining SMs).  This is the
+ *                     calling pattern Alg. 1 forces on the draft model (x_i ~ q_i one position at a time), where
+ *                     the layer kernels are bound by kernel latency.  Every block is folded, so results agree
+ *                     with the other layouts within the parity tolerance.  The kernel needs the GPU to itself:
+ *                     csd_round then runs its two chains one after the other, and two contexts should not run
+ *                     such chains at the same time (the kernels would wait for each other's SMs until the wait
+ *                     limit and report CSD_ERR_TIMEOUT).
  * Takes effect for calls made after it returns. */
-enum { CSD_CHAIN_LAYERS = 0, CSD_CHAIN_LAYERS_PLAIN = 2 };
+enum { CSD_CHAIN_LAYERS = 0, CSD_CHAIN_SMALL_BATCH = 1, CSD_CHAIN_LAYERS_PLAIN = 2 };
 int csd_set_chain_mode(csd_ctx *ctx, int mode);
 
 /* Optional per-launch timing for benchmarks.  csd_profile(ctx, 1) synchronises, clears the records

@@ -19,6 +19,7 @@
 #include "fold.cuh"
 #include "gemm.cuh"
 #include "rowops.cuh"
+#include "smallbatch.cuh"
 
 using namespace csd;
 
@@ -67,6 +68,7 @@ struct csd_ctx {
   HostIo un;       // csd_verify_unaligned: per-row noise terms
   HostIo bn;       // csd_bonus_token: samples of every sequence before the selection
   HostIo sp;       // csd_verify_single_path: schedule constants, mu^p of one pass, running log-ratio
+  HostIo sb[2];    // small-batch chain kernel (per chain slot): s of all steps, early products, a', v, counters, schedule
   char err[512] = {0};
   // optional per-launch timing (csd_profile)
   bool prof_on = false;
@@ -99,6 +101,13 @@ struct csd_head {
   void* xblob = nullptr;
   std::vector<CUtensorMap> Wgs, Wf;
   std::vector<float*> c1, c2;   // first MLP layer with 256-row boxes (W a multiple of 256)
+  // small-batch chain kernel (smallbatch.cuh): usable for this head; device tables (tensor maps of W1_k, W2_k, then of
+  // the matrices multiplied by s: per block Wf_k, Wg_k, Wss_k, then Wfss, all in 128-row boxes; early tiles; biases)
+  bool sb_ready = false;
+  int sb_ntasks = 0;
+  CUtensorMap* d_sb_maps = nullptr;
+  SbTask* d_sb_tasks = nullptr;
+  const float** d_sb_bias = nullptr;
 };
 
 namespace {
@@ -345,6 +354,33 @@ bool fold_kernels_ready(const csd_ctx* ctx, const csd_head_desc& d) {
   return k == 1;
 }
 
+int ensure_side(csd_ctx* ctx, HostIo& io, size_t need, const char* what);
+
+// Whether the small-batch chain kernel can run on this device: its clusters of 8 CTAs (one per SM, ~213 KB of
+// shared memory each) must all be resident at once.  Returns the number of clusters the GPU holds (0: unusable).
+template <typename ACT, int FMT>
+int sb_clusters_of(csd_ctx* ctx) {
+  static int known[kMaxDevices] = {};   // 0 unknown, > 0 clusters, -1 unusable
+  int& k = known[ctx->device];
+  if (k == 0) {
+    k = -1;
+    auto kern = sb_chain_kernel<ACT, FMT>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSbSmemBytes) == cudaSuccess &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 0) == cudaSuccess) {
+      cudaLaunchConfig_t lc{};
+      lc.gridDim = dim3(kSbCluster); lc.blockDim = dim3(kSbThreads); lc.dynamicSmemBytes = kSbSmemBytes;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = kSbCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.attrs = at; lc.numAttrs = 1;
+      int ncl = 0;
+      if (cudaOccupancyMaxActiveClusters(&ncl, kern, &lc) == cudaSuccess && ncl >= 1) k = ncl;
+    }
+    cudaGetLastError();
+  }
+  return k > 0 ? k : 0;
+}
+
 // One head's denoising chain for R token rows on stream `st` with workspace slot `slot`:
 // begin() enqueues the per-call work (timestep embedding, condition projection, first boundary
 // kernel), step(t) enqueues the kernels of step t.  Two chains can be interleaved launch by launch.
@@ -353,6 +389,7 @@ struct Chain {
   int R, cfg; float cfg_scale; const float *z, *x_T, *eps; int sample_last; float *x0, *mu1, *x1;
   int chains = 1;   // chains that run concurrently with this one (itself included)
   int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
+  bool sbk = false;       // the whole chain runs in the small-batch kernel (smallbatch.cuh)
   bool fold = false;      // blocks 1.. run as two kernels (fold.cuh) instead of three
   CUtensorMap tm_ap{};
   bool mod64 = false;     // modulate kernels in 64-wide tiles although the others use 128
@@ -466,6 +503,12 @@ struct Chain {
       fold = tc && ctx->chain_mode == CSD_CHAIN_LAYERS && !pair && L >= 2 && !hd->Wf.empty() &&
              8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && fold_kernels_ready(ctx, d);
     }
+    // Few rows: one persistent kernel for the whole chain (opt-in per context).  It needs the GPU to itself, so a
+    // round that uses it runs its two chains one after the other (chains == 1 here).
+    sbk = tc && ctx->chain_mode == CSD_CHAIN_SMALL_BATCH && Rh <= kSbRows && hd->sb_ready && chains == 1 && slot != 2 &&
+          !traj_x && !batch_Rin && !lv_min && !ctx->prof_on &&
+          (d.dtype == CSD_F16 ? sb_clusters_of<__half, 0>(ctx) : sb_clusters_of<__nv_bfloat16, 1>(ctx)) > kSbRows / kSbGroup;
+    if (sbk) { fold = false; pair = false; }
     ChainWs& ws = ctx->ws[slot];
     int rc = batch_Rin ? ensure_ws(ctx, ws, d, ws_steps * batch_Rin * (cfg ? 2 : 1), ws_steps * batch_Rin, Ts)
                        : ensure_ws(ctx, ws, d, Rh, R, Ts);
@@ -507,6 +550,7 @@ struct Chain {
                                                 nullptr, 0, W, e);
     if (rc) return rc;
     sbuf[0] = ws.s2; sbuf[1] = ws.s;
+    if (sbk) return launch_small_batch();
     if (batch_Rin) return launch_batch(0);   // a pass has one step (t = 1): its s is sbuf[1]
     sp.traj_x = traj_x; sp.traj_mu = nullptr; sp.status = ctx->d_err + 1;
     sp.lv1 = lv1; sp.half_logdet = half_logdet; sp.lv_min = 0.0f; sp.lv_max = 0.0f;
@@ -556,7 +600,59 @@ struct Chain {
     return CSD_OK;
   }
 
+  // The persistent small-batch kernel: s of every step, zeroed counters, the schedule on the device, one launch.
+  int launch_small_batch() {
+    const csd_head_desc& d = hd->d;
+    ChainWs& ws = ctx->ws[slot];
+    const size_t asz = 2, nm = static_cast<size_t>(5 * L + 2) * W;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+    const size_t o_s = take(static_cast<size_t>(Ts) * kSbRows * W * asz), o_mods = take(2 * kSbRows * nm * 4),
+                 o_ap = take(static_cast<size_t>(kSbRows) * W * asz), o_v = take(static_cast<size_t>(kSbRows) * W * asz),
+                 o_sync = take(static_cast<size_t>(Ts + 2) * 4), o_sched = take(static_cast<size_t>(3) * Ts * 4),
+                 o_h = take(static_cast<size_t>(kSbRows) * W * 4), o_st = take(static_cast<size_t>(kSbRows) * (W / kStatCols) * 8);
+    int rc = ensure_side(ctx, ctx->sb[slot], off, "the small-batch chain buffers");
+    if (rc) return rc;
+    char* b = static_cast<char*>(ctx->sb[slot].base);
+    CUtensorMap tm_a{}, tm_vv{}, tm_sa{};
+    if ((rc = make_tmap(ctx, &tm_a, d.dtype, b + o_ap, kSbRows, W, W, kSbGroup))) return rc;     // boxes of one row group
+    if ((rc = make_tmap(ctx, &tm_vv, d.dtype, b + o_v, kSbRows, W, W, kSbGroup))) return rc;
+    if ((rc = make_tmap(ctx, &tm_sa, d.dtype, b + o_s, static_cast<uint64_t>(Ts) * kSbRows, W, W, kTileM))) return rc;
+    CSD_CUDA(ctx, cudaMemsetAsync(b + o_sync, 0, static_cast<size_t>(Ts + 2) * 4, st));
+    // small pageable sources: staged by the runtime before the calls return
+    float* d_sched = reinterpret_cast<float*>(b + o_sched);
+    CSD_CUDA(ctx, cudaMemcpyAsync(d_sched, sc->a, Ts * sizeof(float), cudaMemcpyHostToDevice, st));
+    CSD_CUDA(ctx, cudaMemcpyAsync(d_sched + Ts, sc->b, Ts * sizeof(float), cudaMemcpyHostToDevice, st));
+    CSD_CUDA(ctx, cudaMemcpyAsync(d_sched + 2 * Ts, sc->sigma, Ts * sizeof(float), cudaMemcpyHostToDevice, st));
+    const dim3 sgrid(static_cast<unsigned>(kSbRows), static_cast<unsigned>(Ts));
+    if (d.dtype == CSD_F16) sb_cond_all_kernel<__half><<<sgrid, 256, 0, st>>>(ws.cz, ws.te, reinterpret_cast<__half*>(b + o_s), R, cfg, W, Ts);
+    else sb_cond_all_kernel<__nv_bfloat16><<<sgrid, 256, 0, st>>>(ws.cz, ws.te, reinterpret_cast<__nv_bfloat16*>(b + o_s), R, cfg, W, Ts);
+    ctx->launches++;
+    CSD_CUDA(ctx, cudaGetLastError());
+    const int ncl = d.dtype == CSD_F16 ? sb_clusters_of<__half, 0>(ctx) : sb_clusters_of<__nv_bfloat16, 1>(ctx);
+    SbParams p{};
+    p.R = R; p.Rh = Rh; p.cfg = cfg; p.W = W; p.L = L; p.T = Ts; p.C = d.C; p.sample_last = sample_last; p.cfg_scale = cfg_scale;
+    const int per = cfg ? 8 : 16;                 // tokens per row group
+    p.nd = (R + per - 1) / per; p.ne = ncl - p.nd; p.ntasks = hd->sb_ntasks; p.nm = static_cast<int>(nm);
+    p.maps = hd->d_sb_maps; p.tasks = hd->d_sb_tasks; p.sched = d_sched; p.bias = hd->d_sb_bias;
+    p.mods = reinterpret_cast<float*>(b + o_mods); p.h = reinterpret_cast<float*>(b + o_h); p.stats = reinterpret_cast<float*>(b + o_st);
+    p.ap = b + o_ap; p.v = b + o_v; p.x = ws.x;
+    p.win = hd->win; p.bin = hd->bin; p.wout_t = hd->wout_t; p.bout = hd->bout; p.x_T = x_T; p.eps = eps;
+    p.x0 = x0; p.mu1 = mu1; p.x1 = x1; p.sync = reinterpret_cast<int*>(b + o_sync); p.err = ctx->d_err; p.status = ctx->d_err + 1;
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((p.nd + p.ne) * kSbCluster); lc.blockDim = dim3(kSbThreads); lc.dynamicSmemBytes = kSbSmemBytes; lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = kSbCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, sb_chain_kernel<__half, 0>, tm_a, tm_vv, tm_sa, p));
+    else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, sb_chain_kernel<__nv_bfloat16, 1>, tm_a, tm_vv, tm_sa, p));
+    ctx->launches++;
+    return CSD_OK;
+  }
+
   int step(int t) {
+    if (sbk) return CSD_OK;   // already enqueued by begin()
     const csd_head_desc& d = hd->d;
     ChainWs& ws = ctx->ws[slot];
     cur_t = t;
@@ -872,6 +968,7 @@ int csd_destroy(csd_ctx* c) {
   if (c->sp.base) cudaFree(c->sp.base);
   if (c->un.base) cudaFree(c->un.base);
   if (c->bn.base) cudaFree(c->bn.base);
+  for (HostIo& b : c->sb) if (b.base) cudaFree(b.base);
   if (c->d_err) cudaFree(c->d_err);
   cudaGetLastError();
   delete c;
@@ -922,7 +1019,7 @@ int csd_selftest_wait_timeout(csd_ctx* c) {
 
 int csd_set_chain_mode(csd_ctx* c, int mode) {
   if (!c) return CSD_ERR_INVALID_ARG;
-  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_LAYERS_PLAIN) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
+  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_LAYERS_PLAIN && mode != CSD_CHAIN_SMALL_BATCH) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
   c->chain_mode = mode;
   return CSD_OK;
 }
@@ -1096,10 +1193,13 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
   const size_t f_bfsh = put(w->bfada, W), f_bfsc = put(w->bfada + W, W);
   // folded blocks: c1_k = W1_k (1 + bscale_k), c2_k = W1_k bshift_k + b1_k  (double accumulation, rounded once)
   const bool folded = d.dtype != CSD_F32 && L >= 2;
+  // the small-batch chain kernel folds every block, the first included
+  const bool sbk = d.dtype != CSD_F32 && W % 512 == 0 && W <= static_cast<size_t>(kSbMaxW) && !d.var_out;
+  const size_t kfold0 = sbk ? 0 : 1;      // first block that has folded weights
   std::vector<size_t> f_c1(L, 0), f_c2(L, 0);
-  if (folded) {
+  if (folded || sbk) {
     std::vector<float> v1(W), v2(W);
-    for (size_t k = 1; k < L; ++k) {
+    for (size_t k = kfold0; k < L; ++k) {
       const float* W1k = w->W1 + k * W * W;
       const float* bsh = w->bada + k * 3 * W;
       const float* bsc = bsh + W;
@@ -1118,7 +1218,7 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
   h->win = fb + f_win; h->bin = fb + f_bin; h->wout_t = fb + f_wout; h->bout = fb + f_bout;
   h->bfsh = fb + f_bfsh; h->bfsc = fb + f_bfsc;
   h->c1.assign(L, nullptr); h->c2.assign(L, nullptr);
-  if (folded) for (size_t k = 1; k < L; ++k) { h->c1[k] = fb + f_c1[k]; h->c2[k] = fb + f_c2[k]; }
+  if (folded || sbk) for (size_t k = kfold0; k < L; ++k) { h->c1[k] = fb + f_c1[k]; h->c2[k] = fb + f_c2[k]; }
   h->bsh.resize(L); h->bsc.resize(L); h->bg.resize(L); h->b1.resize(L); h->b2.resize(L);
   for (size_t k = 0; k < L; ++k) { h->bsh[k] = fb + f_bsh[k]; h->bsc[k] = fb + f_bsc[k]; h->bg[k] = fb + f_bg[k]; h->b1[k] = fb + f_b1[k]; h->b2[k] = fb + f_b2[k]; }
 
@@ -1137,9 +1237,11 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
       }
       if (!rc) rc = make_tmap(ctx, &tm.Wfss, d.dtype, h->Wfss, 2 * W, W, W, 2 * tn);
     }
-    if (!rc && folded) {
-      // xblob: Wgs_0 .. Wgs_{L-2} | Wf_1 .. Wf_{L-1}, each [2 W, W] in operand format
-      const size_t per = 2 * W * W, nx = 2 * (L - 1) * per;
+    std::vector<CUtensorMap> wf128(L);
+    if (!rc && (folded || sbk)) {
+      // xblob: Wgs_0 .. Wgs_{L-2} | Wf_1 .. Wf_{L-1} | Wf_0 (small-batch kernel only), each [2 W, W] in operand format
+      const size_t per = 2 * W * W, nx = (2 * (L - 1) + (sbk ? 1 : 0)) * per;
+      auto wf_slot = [&](size_t k) { return k == 0 ? 2 * (L - 1) : L - 1 + k - 1; };
       std::vector<float> xs;
       try { xs.resize(nx); } catch (...) { return bail(CSD_ERR_WORKSPACE, "out of host memory"); }
       float *dA = nullptr, *dB = nullptr, *dC = nullptr;
@@ -1147,7 +1249,7 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
       bool okx = cudaMalloc(&dA, W * W * 4) == cudaSuccess && cudaMalloc(&dB, W * W * 4) == cudaSuccess && cudaMalloc(&dC, W * W * 4) == cudaSuccess;
       for (size_t k = 0; k + 1 < L && okx; ++k)     // gate of block k | scale of block k + 1
         interleave(w->Wada + k * 3 * W * W + 2 * W * W, w->Wada + (k + 1) * 3 * W * W + W * W, &xs[k * per]);
-      for (size_t k = 1; k < L && okx; ++k) {       // W1_k Wscale_k | W1_k Wshift_k
+      for (size_t k = kfold0; k < L && okx; ++k) {  // W1_k Wscale_k | W1_k Wshift_k
         const float* ada = w->Wada + k * 3 * W * W;
         const dim3 grid(static_cast<unsigned>(W / 32), static_cast<unsigned>(W / 32));
         okx = okx && cudaMemcpy(dA, w->W1 + k * W * W, W * W * 4, cudaMemcpyHostToDevice) == cudaSuccess;
@@ -1157,7 +1259,7 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
         okx = okx && cudaMemcpy(dB, ada, W * W * 4, cudaMemcpyHostToDevice) == cudaSuccess;
         if (okx) square_matmul_kernel<<<grid, 256>>>(dA, dB, dC, static_cast<int>(W));
         okx = okx && cudaMemcpy(f2.data(), dC, W * W * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
-        if (okx) interleave(f1.data(), f2.data(), &xs[(L - 1 + k - 1) * per]);
+        if (okx) interleave(f1.data(), f2.data(), &xs[wf_slot(k) * per]);
       }
       if (dA) cudaFree(dA);
       if (dB) cudaFree(dB);
@@ -1172,13 +1274,42 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
       h->Wgs.resize(L); h->Wf.resize(L);
       char* xbase = static_cast<char*>(h->xblob);
       for (size_t k = 0; k + 1 < L && !rc; ++k) rc = make_tmap(ctx, &h->Wgs[k], d.dtype, xbase + k * per * 2, 2 * W, W, W, 256);
-      for (size_t k = 1; k < L && !rc; ++k) rc = make_tmap(ctx, &h->Wf[k], d.dtype, xbase + (L - 1 + k - 1) * per * 2, 2 * W, W, W, 256);
+      for (size_t k = 1; k < L && !rc; ++k) rc = make_tmap(ctx, &h->Wf[k], d.dtype, xbase + wf_slot(k) * per * 2, 2 * W, W, W, 256);
+      for (size_t k = kfold0; k < L && !rc && sbk; ++k) rc = make_tmap(ctx, &wf128[k], d.dtype, xbase + wf_slot(k) * per * 2, 2 * W, W, W, 128);
     }
     if (!rc && W % 256 == 0) {
       h->W1_wide.resize(L);
       for (size_t k = 0; k < L && !rc; ++k) rc = make_tmap(ctx, &h->W1_wide[k], d.dtype, h->W1[k], W, W, W, 256);
     }
     if (rc) { csd_head_destroy(h); return rc; }
+    if (sbk) {
+      // tables of the small-batch chain kernel
+      std::vector<CUtensorMap> maps;
+      for (size_t k = 0; k < L; ++k) { maps.push_back(h->tm[1].W1[k]); maps.push_back(h->tm[1].W2[k]); }
+      std::vector<SbTask> tasks;
+      auto add = [&](const CUtensorMap& m, size_t rows, size_t col0) {
+        const int mi = static_cast<int>(maps.size());
+        maps.push_back(m);
+        for (size_t r = 0; r < rows; r += 128) tasks.push_back(SbTask{mi, static_cast<int>(r), static_cast<int>(col0 + r), 0});
+      };
+      for (size_t k = 0; k < L; ++k) {           // mods columns of block k: [P1 | P2 : 2 W][gate : W][shift | scale : 2 W]
+        add(wf128[k], 2 * W, 5 * k * W);
+        add(h->tm[1].Wg[k], W, 5 * k * W + 2 * W);
+        add(h->tm[0].Wss[k], 2 * W, 5 * k * W + 3 * W);
+      }
+      add(h->tm[0].Wfss, 2 * W, 5 * L * W);
+      std::vector<const float*> bt;
+      for (size_t k = 0; k < L; ++k) { bt.push_back(h->c1[k]); bt.push_back(h->c2[k]); bt.push_back(h->bg[k]); bt.push_back(h->b2[k]); bt.push_back(h->bsc[k]); }
+      bt.push_back(h->bfsh); bt.push_back(h->bfsc);
+      if (cudaMalloc(&h->d_sb_maps, maps.size() * sizeof(CUtensorMap)) != cudaSuccess ||
+          cudaMalloc(&h->d_sb_tasks, tasks.size() * sizeof(SbTask)) != cudaSuccess ||
+          cudaMalloc(&h->d_sb_bias, bt.size() * sizeof(float*)) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the small-batch tables"); }
+      if (cudaMemcpy(h->d_sb_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemcpy(h->d_sb_tasks, tasks.data(), tasks.size() * sizeof(SbTask), cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemcpy(h->d_sb_bias, bt.data(), bt.size() * sizeof(float*), cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "small-batch table upload failed");
+      h->sb_ntasks = static_cast<int>(tasks.size());
+      h->sb_ready = true;
+    }
   }
   *out = h;
   return CSD_OK;
@@ -1194,6 +1325,9 @@ int csd_head_destroy(csd_head* h) {
   if (h->wblob) cudaFree(h->wblob);
   if (h->fblob) cudaFree(h->fblob);
   if (h->xblob) cudaFree(h->xblob);
+  if (h->d_sb_maps) cudaFree(h->d_sb_maps);
+  if (h->d_sb_tasks) cudaFree(h->d_sb_tasks);
+  if (h->d_sb_bias) cudaFree(h->d_sb_bias);
   cudaGetLastError();
   delete h;
   return CSD_OK;
@@ -1512,26 +1646,32 @@ static int round_impl(csd_ctx* ctx, const csd_head* head_q, const csd_head* head
   if ((rc = ensure_ws(ctx, ctx->ws[0], head_q->d, R * (cfg ? 2 : 1), R, sched_q->T))) return rc;
   if ((rc = ensure_ws(ctx, ctx->ws[1], head_p->d, Rp * (cfg ? 2 : 1), Rp, sched_p->T))) return rc;
   if (bonus && (rc = ensure_side(ctx, ctx->bn, bonus_buf_bytes(head_p->d, Rp, cfg, T), "the bonus rows"))) return rc;
-  CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
-  for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
+  // Few rows in small-batch mode: each chain is one persistent kernel that wants the whole GPU, so the two run one
+  // after the other on the context's stream (the same kernels, hence the same bits, as the separate calls).
+  const bool seq = ctx->chain_mode == CSD_CHAIN_SMALL_BATCH && Rp * (cfg ? 2 : 1) <= kSbRows && head_q->sb_ready && head_p->sb_ready;
+  if (!seq) {
+    CSD_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
+    for (int i = 0; i < 2; ++i) CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->side[i], ctx->ev_fork, 0));
+  }
   // the two chains' launches are interleaved step by step so that neither stream starves
   // the chain with more work per row goes to the higher-priority stream
   const double wq = static_cast<double>(head_q->d.L) * head_q->d.W * head_q->d.W, wp = static_cast<double>(head_p->d.L) * head_p->d.W * head_p->d.W;
   const int sq = wq > wp ? 1 : 0;
+  cudaStream_t st_q = seq ? ctx->stream : ctx->side[sq], st_p = seq ? ctx->stream : ctx->side[1 - sq];
   BonusBuf bb{};
-  if (bonus && (rc = gather_bonus_inputs(ctx, ctx->side[1 - sq], head_p->d, R, B, cfg, T, z_p, x_T, eps, z_next, x_T_next, eps_next, bb))) return rc;
-  Chain cq{ctx, 0, ctx->side[sq], head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr};
-  Chain cp = bonus ? Chain{ctx, 1, ctx->side[1 - sq], head_p, sched_p, Rp, cfg, cfg_scale, bb.z, bb.x_T, bb.eps, 1, bb.x0, bb.mu1, nullptr}
-                   : Chain{ctx, 1, ctx->side[1 - sq], head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr};
-  cq.chains = cp.chains = 2;
+  if (bonus && (rc = gather_bonus_inputs(ctx, st_p, head_p->d, R, B, cfg, T, z_p, x_T, eps, z_next, x_T_next, eps_next, bb))) return rc;
+  Chain cq{ctx, 0, st_q, head_q, sched_q, R, cfg, cfg_scale, z_q, x_T, eps, 1, x0, mu1_q, nullptr};
+  Chain cp = bonus ? Chain{ctx, 1, st_p, head_p, sched_p, Rp, cfg, cfg_scale, bb.z, bb.x_T, bb.eps, 1, bb.x0, bb.mu1, nullptr}
+                   : Chain{ctx, 1, st_p, head_p, sched_p, R, cfg, cfg_scale, z_p, x_T, eps, 0, nullptr, mu1_p, nullptr};
+  cq.chains = cp.chains = seq ? 1 : 2;
   rc = cp.begin();
   int rc2 = cq.begin();
   for (int t = sched_p->T; t >= 1 && !rc && !rc2; --t) {
     rc = cp.step(t);
     if (!rc) rc2 = cq.step(t);
   }
-  if (bonus && !rc) CSD_CUDA(ctx, cudaMemcpyAsync(mu1_p, bb.mu1, static_cast<size_t>(R) * C * 4, cudaMemcpyDeviceToDevice, ctx->side[1 - sq]));
-  for (int i = 0; i < 2; ++i) {
+  if (bonus && !rc) CSD_CUDA(ctx, cudaMemcpyAsync(mu1_p, bb.mu1, static_cast<size_t>(R) * C * 4, cudaMemcpyDeviceToDevice, st_p));
+  for (int i = 0; i < 2 && !seq; ++i) {
     CSD_CUDA(ctx, cudaEventRecord(ctx->ev_done[i], ctx->side[i]));
     CSD_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_done[i], 0));
   }

@@ -42,12 +42,19 @@ def test_ddim_round_matches_checker(op, kw, eta_q, eta_p):
 
 
 @pytest.mark.parametrize("eta", [1.0, 0.5])
-def test_ddim_100_of_1000_steps_at_mar256_size_sampled_sequences(eta):
-    # The sampler setting of the paper's DDIM table: 100 DDIM steps out of a 1000-step linear-beta ladder, at the
-    # size and launch configuration of the benchmark's 256x256-shaped workload; the checker evaluates four sequences
-    # (first, last, both sides of a 128-row tile boundary).
+def test_ddim_100_of_1000_steps_at_mar256_size_every_step_of_sampled_sequences(eta):
+    # The sampler setting of the paper's DDIM table: 100 DDIM steps out of a 1000-step linear-beta ladder, at the size
+    # and launch configuration of the benchmark's 256x256-shaped workload.  On that ladder prod_t a_t = 1 / sqrt(abar_1000)
+    # is about 158 (1.65 for the 100-step DDPM ladder), and a random untrained head does not pull a perturbed state
+    # back, so any per-step rounding is amplified a hundredfold by the end: an end-to-end comparison of x_0 says
+    # nothing about the kernels.  Every step is therefore checked on its own: the checker evaluates each of the 100
+    # transitions from the GPU's OWN recorded state x_t (four sequences: first, last, both sides of a 128-row tile
+    # boundary) and must reproduce the GPU's mean mu_t and next state; then the round's ratio, scan and resampling are
+    # checked on the GPU's own final-step arrays.
+    import torch
     from paper_2411_11925_b200 import api
     from paper_2411_11925_b200.runner import DeviceRound
+    from _parity import F32_EPS, TOL_LOGR, eq8_float64
     wl = gen.WORKLOADS["mar256"]
     inp = gen.make_round_inputs(wl)
     N = 1000
@@ -56,18 +63,42 @@ def test_ddim_100_of_1000_steps_at_mar256_size_sampled_sequences(eta):
     inp.tfeat = np.ascontiguousarray(gen.timestep_features(N, wl.draft.F)[steps - 1])
     co = api.ddim_coefficients(beta_full, steps, eta)
     dr = DeviceRound(inp, coeffs_q=co, coeffs_p=co)
-    dr.fused_round()
-    out = dr.results()
-    assert np.all(np.isfinite(out["x0"])) and np.all(np.isfinite(out["logratio"]))
+    T, R, C = wl.T, wl.R, dr.C
+    dr.draft_traj()
+    tx_p = torch.zeros(T + 1, R, C, device=dr.dev)
+    tm_p = torch.zeros(T, R, C, device=dr.dev)
+    dr.ctx.csd_draft_denoise_traj(dr.head_p, dr.sched_p, R, wl.cfg, wl.cfg_scale, dr.z_p, dr.x_T, dr.eps, tx_p, tm_p)
+    dr.ctx.sync()
     seqs = [0, 15, 16, 63]
     sub = gen.select_sequences(inp, seqs)
-    sched = orc.ddim_schedule(beta_full, steps, eta)
-    eq = orc.make_mlp_head(sub.w_q, sub.z_q, sub.tfeat, wl.cfg, wl.cfg_scale)
-    ep = orc.make_mlp_head(sub.w_p, sub.z_p, sub.tfeat, wl.cfg, wl.cfg_scale)
-    ref = orc.csd_round(eq, ep, sched, sched, sub.x_T, sub.eps, sub.u, sub.xi, sub.v, len(seqs), wl.gamma, wl.cap)
     rows = sub.extras["rows"]
-    gsub = {k: (out[k][rows] if out[k].shape[0] == wl.R else out[k][seqs]) for k in out if k != "cap_hits"}
-    gsub["cap_hits"] = out["cap_hits"]
-    st = compare_round(gsub, ref, sub.wl, sched["sigma"][0], sched["sigma"][0], sub.u, sub.v, f"ddim-100 eta {eta}", xi=sub.xi)
-    print("ddim-100", eta, st)
+    sched = orc.ddim_schedule(beta_full, steps, eta)
+    worst = {}
+    for name, w, z, tx, tm in (("draft", sub.w_q, sub.z_q, dr.traj_x, dr.traj_mu), ("target", sub.w_p, sub.z_p, tx_p, tm_p)):
+        fn = orc.make_mlp_head(w, z, sub.tfeat, wl.cfg, wl.cfg_scale)
+        gx, gm = tx.cpu().numpy()[:, rows].astype(np.float64), tm.cpu().numpy()[:, rows].astype(np.float64)
+        err_mu = err_x = 0.0
+        for j in range(T):
+            t = T - j
+            mu = sched["a"][t - 1] * gx[j] - sched["b"][t - 1] * fn(gx[j], t)        # one checker step from the GPU's state
+            err_mu = max(err_mu, float(np.max(np.abs(gm[j] - mu))))
+            err_x = max(err_x, float(np.max(np.abs(gx[j + 1] - (gm[j] + sched["sigma"][t - 1] * sub.eps[t - 1])))))
+        worst[name] = (err_mu, err_x)
+        assert err_mu <= 5e-3, (name, err_mu)          # fp16 operands: a single head evaluation, |b_t| <= 1.6
+        assert err_x <= 2e-6 * max(1.0, float(np.abs(gx).max())), (name, err_x)   # x_{t-1} = mu_t + sigma_t eps_t in fp32
+    dr.fused_round()
+    out = dr.results()
+    np.testing.assert_array_equal(out["x0"], dr.traj_x[-1].cpu().numpy())       # the round runs the same chains
+    np.testing.assert_array_equal(out["mu1_p"], tm_p[-1].cpu().numpy())
+    s1 = float(sched["sigma"][0])
+    own, qp, qq = eq8_float64(out["x0"], out["mu1_q"], out["mu1_p"], s1, s1, 0.0)
+    assert np.all(np.abs(out["logratio"].reshape(-1) - own) <= TOL_LOGR + 8 * F32_EPS * (qp + qq))
+    logu32 = np.log(inp.u.astype(np.float32)).astype(np.float32)
+    gm_ = out["accept_mask"].astype(np.int64) & 0xFFFFFFFF
+    acc = ((gm_[:, None] >> np.arange(wl.gamma)[None, :]) & 1).astype(bool)
+    knife = np.abs(logu32.astype(np.float64) - out["logratio"]) < 1e-5
+    assert np.array_equal(acc | knife, (logu32 <= out["logratio"]) | knife)
+    np.testing.assert_array_equal(out["n_accept"], [(list(r) + [False]).index(False) for r in acc])
+    np.testing.assert_array_equal(out["flags"] & 1, (out["n_accept"] < wl.gamma).astype(out["flags"].dtype))
+    print("ddim-100 eta", eta, "worst per-step (mu, x) errors", worst, "amplification", float(np.prod(sched["a"])))
     dr.ctx.close()

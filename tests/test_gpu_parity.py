@@ -326,5 +326,5 @@ def test_chain_layouts_agree(op):
         for k in ("x0", "mu1_q", "mu1_p"):
             assert float(np.max(np.abs(d[k] - a[k]))) <= TOL_X[op] / 4, (kw, k)
         with pytest.raises(api.CsdError):
-            dr.ctx.set_chain_mode(1)          # no such layout
+            dr.ctx.set_chain_mode(7)          # no such layout
         dr.ctx.close()
