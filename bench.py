@@ -316,15 +316,23 @@ def measure(name, args, peaks, steps, warmup, rounds_per_step, full):
         r1 = DeviceRound(inp1, ctx=ctx, device=local, heads=(rounds[0].head_q, rounds[0].head_p))
         seq_step = lambda i: [r1.draft() for _ in range(wl.gamma)]
         timed(seq_step, 3)
+        layers_secs = timed(seq_step, few)
+        # the persistent small-batch kernel (csd_set_chain_mode): chains of at most 128 head rows
+        ctx.set_chain_mode(api.Context.CHAIN_SMALL_BATCH)
+        timed(seq_step, 3)
         l1 = ctx.launch_count()
         seq_secs = timed(seq_step, few)
+        launches_per_call = int((ctx.launch_count() - l1) // (few * wl.gamma))
+        ctx.set_chain_mode(api.Context.CHAIN_LAYERS)
         d = wl.draft
         wbytes = 2.0 * (d.W * d.Dz + d.L * 5 * d.W * d.W + 2 * d.W * d.W)     # 16-bit GEMM weights of the draft head
         per_call = seq_secs / (few * wl.gamma)
         out["sequential_draft"] = {
             "calls_per_round": wl.gamma, "head_rows_per_call": wl.B * (2 if wl.cfg else 1),
+            "chain_mode": "CSD_CHAIN_SMALL_BATCH" if launches_per_call < 50 else "CSD_CHAIN_LAYERS (small-batch kernel not eligible)",
             "ms_per_call": 1e3 * per_call, "us_per_denoising_step": 1e6 * per_call / wl.T,
-            "launches_per_call": int((ctx.launch_count() - l1) // (few * wl.gamma)),
+            "layer_kernels_ms_per_call": 1e3 * layers_secs / (few * wl.gamma),
+            "launches_per_call": launches_per_call,
             "value": wl.B * wl.gamma * few / seq_secs, "unit": UNIT,
             "bound": "hbm", "weight_bytes_per_step": wbytes, "achieved": wbytes * wl.T / per_call / 1e9,
             "peak": peaks["hbm_gbs"], "roofline_unit": "GB/s", "frac": wbytes * wl.T / per_call / 1e9 / peaks["hbm_gbs"],

@@ -28,6 +28,10 @@ What pins each function (see tests/test_oracle_pins.py):
                            heads against scipy's normal densities over the whole pair of paths; posterior
                            variance against the textbook closed form; KS of the resampler with different
                            per-dimension variances against the numerically integrated max(0, Sigma p - q)
+  gmm_logpdf, gmm_sample, gmm_resample, gmm_round (explicit mixture heads)
+                           scipy's multivariate-normal densities and logsumexp; one component reduces to the
+                           diagonal Gaussian; KS of the draws against the mixture CDF and of the resampled tokens
+                           against the numerically integrated max(0, p - q); acceptance rate = 1 - TV(p, q)
   accept_prefix            brute force over all accept masks (Alg. 1)
   resample                 KS test against the numerically integrated
                            max(0, Sigma*p - q) (Eq. 5, Eq. 11, Cor. 1); textbook
@@ -516,3 +520,79 @@ def csd_round_lv(fn_q, fn_p, sched_q, sched_p, x_T, noise, u, xi, v, B, gamma, c
     if keep:
         out["dq"], out["dp"] = dq, dp
     return out
+
+
+# --------------------------------------------------------------------------
+# Gaussian-mixture output heads (Appendix "More Variants of Diffusion Model"): the AR model emits, per token, an
+# explicit mixture p(x) = sum_k pi_k N(x; mu_k, diag(sigma_k^2)) instead of a diffusion head.  Both densities are
+# then available in closed form, so the accept test is the plain rule of Sec. 3.1 (accept iff u <= p(x)/q(x)) and the
+# modified distribution max(0, p - q)/Z (Eq. 5) is sampled by the same acceptance-rejection loop (Eq. 9-11) with
+# proposals from p itself: alpha_s = max(0, p(x') - q(x')) / p(x').
+# A mixture is (logw [N,K] unnormalised log-weights, mu [N,K,C], log_sigma [N,K,C]).
+# --------------------------------------------------------------------------
+def _logsumexp(a: np.ndarray, axis: int) -> np.ndarray:
+    m = np.max(a, axis=axis, keepdims=True)
+    return np.squeeze(m, axis=axis) + np.log(np.sum(np.exp(a - m), axis=axis))
+
+
+def gmm_logpdf(x: np.ndarray, logw: np.ndarray, mu: np.ndarray, log_sigma: np.ndarray) -> np.ndarray:
+    x, logw, mu, log_sigma = (np.asarray(a, dtype=f64) for a in (x, logw, mu, log_sigma))
+    C = x.shape[-1]
+    lw = logw - _logsumexp(logw, axis=-1)[..., None]
+    t = (x[:, None, :] - mu) * np.exp(-log_sigma)
+    comp = lw - np.sum(log_sigma, axis=-1) - 0.5 * np.sum(t * t, axis=-1) - 0.5 * C * np.log(2.0 * np.pi)
+    return _logsumexp(comp, axis=-1)
+
+
+def gmm_sample(logw, mu, log_sigma, u_comp, noise) -> Tuple[np.ndarray, np.ndarray]:
+    """x = mu_k + sigma_k * noise with k drawn by inverting the weights' CDF at u_comp: the first k whose cumulative
+    weight reaches u_comp (the last component if rounding leaves the total short of it)."""
+    logw, mu, log_sigma = (np.asarray(a, dtype=f64) for a in (logw, mu, log_sigma))
+    w = np.exp(logw - _logsumexp(logw, axis=-1)[..., None])
+    cum = np.cumsum(w, axis=-1)
+    K = w.shape[-1]
+    comp = np.minimum((cum < np.asarray(u_comp, dtype=f64)[:, None]).sum(axis=-1), K - 1).astype(np.int32)
+    rows = np.arange(len(comp))
+    x = mu[rows, comp] + np.exp(log_sigma[rows, comp]) * np.asarray(noise, dtype=f64)
+    return x, comp
+
+
+def gmm_resample(n_accept, q, p, w, xi, v, gamma, cap):
+    """q, p: mixtures (logw, mu, log_sigma) over the R = B gamma token rows; proposals x' ~ p of the first rejected
+    row (component from w[b,k], Gaussian draw xi[b,k]), consumed in order, accepted iff v <= max(0, 1 - q(x')/p(x'))."""
+    B = len(n_accept)
+    C = p[1].shape[-1]
+    x_new = np.zeros((B, C), dtype=f64)
+    n_prop = np.zeros(B, dtype=np.int32)
+    flags = np.zeros(B, dtype=np.uint32)
+    for b in range(B):
+        n = int(n_accept[b])
+        if n >= gamma:
+            continue
+        j = b * gamma + n
+        flags[b] |= 1
+        done = False
+        pj = tuple(a[j:j + 1] for a in p)
+        qj = tuple(a[j:j + 1] for a in q)
+        for k in range(cap):
+            xp, _ = gmm_sample(pj[0], pj[1], pj[2], np.array([w[b, k]]), xi[b, k][None, :])
+            lp, lq = gmm_logpdf(xp, *pj)[0], gmm_logpdf(xp, *qj)[0]
+            alpha_s = max(0.0, -np.expm1(min(0.0, lq - lp)))
+            x_new[b] = xp[0]
+            n_prop[b] = k + 1
+            if float(v[b, k]) <= alpha_s:
+                done = True
+                break
+        if not done:
+            flags[b] |= 2
+    return {"x_new": x_new, "n_prop": n_prop, "flags": flags, "cap_hits": int(np.sum((flags & 2) != 0))}
+
+
+def gmm_round(q, p, u_comp, noise, u, w, xi, v, B, gamma, cap) -> Dict[str, np.ndarray]:
+    """One round of Alg. 1 with explicit mixture heads: drafts x_i ~ q_i, ratio p_i(x_i)/q_i(x_i), accepted prefix,
+    resampling of the first rejected position from max(0, p - q)/Z."""
+    x, comp = gmm_sample(q[0], q[1], q[2], u_comp, noise)
+    logr = gmm_logpdf(x, *p) - gmm_logpdf(x, *q)
+    n, acc = accept_prefix(logr.reshape(B, gamma), u)
+    rs = gmm_resample(n, q, p, w, xi, v, gamma, cap)
+    return {"x": x, "comp": comp, "logratio": logr.reshape(B, gamma), "n_accept": n, "accept": acc, **rs}
