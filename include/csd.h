@@ -410,6 +410,31 @@ int csd_round_bonus(csd_ctx *ctx, const csd_head *head_q, const csd_head *head_p
                     int32_t *n_accept, uint32_t *accept_mask, float *x_new, int32_t *n_prop, uint32_t *flags,
                     int32_t *cap_hits, float *x_bonus, uint32_t *taken);
 
+/* ---- Explicit Gaussian-mixture heads (appendix "More Variants of Diffusion Model", GMM paragraph) ----------
+ * With a mixture output head the token distribution p(x) = sum_k pi_k N(x; mu_k, diag(sigma_k^2)) is explicit, so
+ * the method needs no diffusion chain: drafts are samples of q, the ratio is p(x)/q(x) itself (accept rule of
+ * Sec. 3.1 / Alg. 1), and the modified distribution max(0, p - q)/Z (Eq. 5) is sampled by the same
+ * acceptance-rejection loop (Eq. 9-11) with proposals from p: alpha_s = max(0, 1 - q(x')/p(x')).
+ * A mixture holds, per token row, K components: logw [rows, K] (unnormalised log-weights, normalised inside),
+ * mu and log_sigma [rows, K, C]; all DEVICE arrays, C <= 32.
+ *   csd_gmm_draft_sample: x[r] = mu_k + sigma_k * noise[r] with k the first component whose cumulative weight
+ *     reaches u_comp[r] in (0,1); comp int32 [R] out or NULL.
+ *   csd_gmm_verify: logratio[b,i] = log p(x) - log q(x); accept iff log u <= logratio; n_accept, accept_mask as
+ *     csd_verify.  Identical mixtures give exactly 0.
+ *   csd_gmm_resample: for sequences with n_accept < gamma, proposals for row b*gamma + n_accept[b]: component from
+ *     w[b,k], x' = mu_k + sigma_k * xi[b,k]; outputs as csd_resample (capped loop, flags, cap_hits). */
+typedef struct {
+  int K;
+  const float *logw, *mu, *log_sigma;
+} csd_gmm;
+int csd_gmm_draft_sample(csd_ctx *ctx, int R, int C, const csd_gmm *q, const float *u_comp, const float *noise,
+                         float *x, int32_t *comp);
+int csd_gmm_verify(csd_ctx *ctx, int B, int gamma, int C, const csd_gmm *q, const csd_gmm *p, const float *x,
+                   const float *u, float *logratio, int32_t *n_accept, uint32_t *accept_mask);
+int csd_gmm_resample(csd_ctx *ctx, int B, int gamma, int C, int cap, const csd_gmm *q, const csd_gmm *p,
+                     const int32_t *n_accept, const float *w, const float *xi, const float *v, float *x_new,
+                     int32_t *n_prop, uint32_t *flags, int32_t *cap_hits);
+
 /* Same computation as csd_round, but every array is a HOST pointer: the call copies the inputs
  * to the device, runs the round, copies the outputs back and synchronises before returning. */
 int csd_round_host(csd_ctx *ctx, const csd_head *head_q, const csd_head *head_p,

@@ -28,7 +28,8 @@ EXPORTS = ("csd_create", "csd_destroy", "csd_last_error", "csd_sync", "csd_launc
            "csd_draft_denoise_lv", "csd_verify_lv", "csd_resample_lv", "csd_round_lv",
            "csd_head_create", "csd_head_destroy", "csd_draft_denoise", "csd_draft_denoise_static", "csd_verify",
            "csd_accept_scan", "csd_resample", "csd_round", "csd_round_host", "csd_draft_denoise_traj",
-           "csd_verify_single_path", "csd_verify_unaligned", "csd_bonus_token", "csd_verify_bonus", "csd_round_bonus")
+           "csd_verify_single_path", "csd_verify_unaligned", "csd_bonus_token", "csd_verify_bonus", "csd_round_bonus",
+           "csd_gmm_draft_sample", "csd_gmm_verify", "csd_gmm_resample")
 
 WEIGHT_FIELDS = ("Wz", "bz", "Wt1", "bt1", "Wt2", "bt2", "Win", "bin", "Wada", "bada",
                  "W1", "b1", "W2", "b2", "Wfada", "bfada", "Wout", "bout")
@@ -51,6 +52,10 @@ class _HeadWeights(C.Structure):
 class _Schedule(C.Structure):
     _fields_ = [("T", C.c_int), ("a", _c_float_p), ("b", _c_float_p), ("sigma", _c_float_p),
                 ("tfeat", C.c_void_p)]
+
+
+class _Gmm(C.Structure):
+    _fields_ = [("K", C.c_int), ("logw", C.c_void_p), ("mu", C.c_void_p), ("log_sigma", C.c_void_p)]
 
 
 class _ScheduleLV(C.Structure):
@@ -83,6 +88,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.csd_resample_lv.argtypes = [vp, i32, i32, i32, i32] + [vp] * 12
     lib.csd_round_lv.argtypes = ([vp, vp, vp, C.POINTER(_ScheduleLV), C.POINTER(_ScheduleLV), i32, i32, i32, f32, i32]
                                  + [vp] * 22)
+    gp = C.POINTER(_Gmm)
+    lib.csd_gmm_draft_sample.argtypes = [vp, i32, i32, gp] + [vp] * 4
+    lib.csd_gmm_verify.argtypes = [vp, i32, i32, i32, gp, gp] + [vp] * 5
+    lib.csd_gmm_resample.argtypes = [vp, i32, i32, i32, i32, gp, gp] + [vp] * 8
     lib.csd_profile.argtypes = [vp, i32]
     lib.csd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_int64), C.POINTER(f64), C.POINTER(f64)]
     lib.csd_head_create.argtypes = [vp, C.POINTER(_HeadDesc), C.POINTER(_HeadWeights), C.POINTER(vp)]
@@ -358,6 +367,26 @@ class Context:
                                       *[_ptr(t) for t in (z_q, z_p, x_T, eps, u, xi, v, x0, mu1_q, lv1_q, half_logdet_q,
                                                           mu1_p, lv1_p, half_logdet_p, log_sigma_rows, logratio, n_accept,
                                                           accept_mask, x_new, n_prop, flags, cap_hits)]))
+
+    @staticmethod
+    def _gmm(m):
+        """m: (logw [rows,K], mu [rows,K,C], log_sigma [rows,K,C]) device tensors."""
+        logw, mu, ls = m
+        return _Gmm(int(logw.shape[1]), _ptr(logw), _ptr(mu), _ptr(ls))
+
+    def csd_gmm_draft_sample(self, R, Cdim, q, u_comp, noise, x, comp=None):
+        g = self._gmm(q)
+        self._check(_LIB.csd_gmm_draft_sample(self._h, R, Cdim, C.byref(g), _ptr(u_comp), _ptr(noise), _ptr(x), _ptr(comp)))
+
+    def csd_gmm_verify(self, B, gamma, Cdim, q, p, x, u, logratio, n_accept, accept_mask=None):
+        gq, gp_ = self._gmm(q), self._gmm(p)
+        self._check(_LIB.csd_gmm_verify(self._h, B, gamma, Cdim, C.byref(gq), C.byref(gp_), _ptr(x), _ptr(u), _ptr(logratio),
+                                        _ptr(n_accept), _ptr(accept_mask)))
+
+    def csd_gmm_resample(self, B, gamma, Cdim, cap, q, p, n_accept, w, xi, v, x_new, n_prop, flags, cap_hits):
+        gq, gp_ = self._gmm(q), self._gmm(p)
+        self._check(_LIB.csd_gmm_resample(self._h, B, gamma, Cdim, cap, C.byref(gq), C.byref(gp_), _ptr(n_accept), _ptr(w),
+                                          _ptr(xi), _ptr(v), _ptr(x_new), _ptr(n_prop), _ptr(flags), _ptr(cap_hits)))
 
     def _round(self, fn, head_q, head_p, sched_q, sched_p, B, gamma, cfg, cfg_scale, cap, z_q, z_p, x_T, eps, u,
                xi, v, x0, mu1_q, mu1_p, logratio, n_accept, accept_mask, x_new, n_prop, flags, cap_hits):

@@ -18,6 +18,7 @@
 #include "../../include/csd.h"
 #include "fold.cuh"
 #include "gemm.cuh"
+#include "gmm.cuh"
 #include "rowops.cuh"
 #include "smallbatch.cuh"
 
@@ -1834,6 +1835,64 @@ int csd_round_lv(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, c
   if (rc) return rc;
   return resample_lv(ctx, ctx->stream, B, gamma, C, cap, log_sigma_rows, n_accept, mu1_p, lv1_p, mu1_q, lv1_q, xi, v, x_new,
                      n_prop, flags, cap_hits);
+}
+
+// ------------------------------------------------------------------ explicit Gaussian-mixture heads
+static int check_gmm(csd_ctx* ctx, const csd_gmm* m, const char* what) {
+  if (!m || !m->logw || !m->mu || !m->log_sigma) return fail(ctx, CSD_ERR_INVALID_ARG, "%s mixture or one of its arrays is null", what);
+  if (m->K < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "%s mixture has K = %d components", what, m->K);
+  return CSD_OK;
+}
+static GmmView gmm_view(const csd_gmm* m) { return GmmView{m->K, m->logw, m->mu, m->log_sigma}; }
+
+int csd_gmm_draft_sample(csd_ctx* ctx, int R, int C, const csd_gmm* q, const float* u_comp, const float* noise, float* x,
+                         int32_t* comp) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_gmm(ctx, q, "draft");
+  if (rc) return rc;
+  if (R < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "row count %d must be >= 1", R);
+  if (C < 1 || C > 32) return fail(ctx, CSD_ERR_UNSUPPORTED, "token dim C = %d must be in [1, 32]", C);
+  if (!u_comp || !noise || !x) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_DEVICE(ctx);
+  gmm_sample_kernel<<<(R + 3) / 4, 128, 0, ctx->stream>>>(R, C, gmm_view(q), u_comp, noise, x, comp);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+int csd_gmm_verify(csd_ctx* ctx, int B, int gamma, int C, const csd_gmm* q, const csd_gmm* p, const float* x,
+                   const float* u, float* logratio, int32_t* n_accept, uint32_t* accept_mask) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_gmm(ctx, q, "draft");
+  if (rc || (rc = check_gmm(ctx, p, "target"))) return rc;
+  if (B < 1 || gamma < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "B = %d and gamma = %d must be >= 1", B, gamma);
+  if (gamma > 32) return fail(ctx, CSD_ERR_UNSUPPORTED, "gamma = %d exceeds 32", gamma);
+  if (C < 1 || C > 32) return fail(ctx, CSD_ERR_UNSUPPORTED, "token dim C = %d must be in [1, 32]", C);
+  if (!x || !u || !logratio || !n_accept) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_DEVICE(ctx);
+  gmm_verify_kernel<<<B, 32 * gamma, 0, ctx->stream>>>(B, gamma, C, gmm_view(q), gmm_view(p), x, u, logratio, n_accept, accept_mask);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
+}
+
+int csd_gmm_resample(csd_ctx* ctx, int B, int gamma, int C, int cap, const csd_gmm* q, const csd_gmm* p,
+                     const int32_t* n_accept, const float* w, const float* xi, const float* v, float* x_new,
+                     int32_t* n_prop, uint32_t* flags, int32_t* cap_hits) {
+  if (!ctx) return CSD_ERR_INVALID_ARG;
+  int rc = check_gmm(ctx, q, "draft");
+  if (rc || (rc = check_gmm(ctx, p, "target"))) return rc;
+  if (B < 1 || gamma < 1 || gamma > 32) return fail(ctx, B < 1 || gamma < 1 ? CSD_ERR_INVALID_ARG : CSD_ERR_UNSUPPORTED, "B = %d, gamma = %d: need B >= 1 and 1 <= gamma <= 32", B, gamma);
+  if (C < 1 || C > 32) return fail(ctx, CSD_ERR_UNSUPPORTED, "token dim C = %d must be in [1, 32]", C);
+  if (cap < 1) return fail(ctx, CSD_ERR_INVALID_ARG, "cap = %d must be >= 1", cap);
+  if (!n_accept || !w || !xi || !v || !x_new || !n_prop || !flags || !cap_hits) return fail(ctx, CSD_ERR_INVALID_ARG, "null array argument");
+  CSD_DEVICE(ctx);
+  CSD_CUDA(ctx, cudaMemsetAsync(cap_hits, 0, sizeof(int32_t), ctx->stream));
+  gmm_resample_kernel<<<(B + 3) / 4, 128, 0, ctx->stream>>>(B, gamma, C, cap, gmm_view(q), gmm_view(p), n_accept, w, xi, v, x_new,
+                                                            n_prop, flags, cap_hits);
+  ctx->launches++;
+  CSD_CUDA(ctx, cudaGetLastError());
+  return CSD_OK;
 }
 
 int csd_round_host(csd_ctx* ctx, const csd_head* head_q, const csd_head* head_p, const csd_schedule* sched_q,
