@@ -369,6 +369,38 @@ def measure(name, args, peaks, steps, warmup, rounds_per_step, full):
                               "bound": "tensor", "achieved": fl * few / sp_secs / 1e12, "peak": peaks["tflops_sustained"],
                               "roofline_unit": "TFLOP/s", "frac": fl * few / sp_secs / 1e12 / peaks["tflops_sustained"]}
 
+    # Bonus token of the all-accepted branch of Alg. 1 folded into the round (the target chain runs R + B rows), against
+    # the plain round on the same inputs; and a round under the DDIM-100 sampler of the paper's sampler table (100 of
+    # 1000 linear-beta steps, eta = 1: same kernels, other coefficients and feature rows).
+    if full and world == 1 and not args.no_seq:
+        r0 = rounds[0]
+        nxt = gen.make_round_inputs(gen.Workload(**{**wl.__dict__, "gamma": 1}), seed_offset=321, weights=False)
+        zn, xn, en = (torch.from_numpy(a).to(dev) for a in (nxt.z_p, nxt.x_T, nxt.eps))
+        xb = torch.zeros(wl.B, r0.C, dtype=torch.float32, device=dev)
+        tk = torch.zeros(wl.B, dtype=torch.int32, device=dev)
+        bonus_step = lambda i: ctx.csd_round_bonus(r0.head_q, r0.head_p, r0.sched_q, r0.sched_p, wl.B, wl.gamma, wl.cfg,
+                                                   wl.cfg_scale, wl.cap, r0.z_q, r0.z_p, r0.x_T, r0.eps, r0.u, r0.xi, r0.v,
+                                                   zn, xn, en, r0.x0, r0.mu1_q, r0.mu1_p, r0.logratio, r0.n_accept,
+                                                   r0.accept_mask, r0.x_new, r0.n_prop, r0.flags, r0.cap_hits, xb, tk)
+        plain_step = lambda i: r0.fused_round()
+        timed(bonus_step, 3); b_secs = timed(bonus_step, few)
+        timed(plain_step, 3); p_secs = timed(plain_step, few)
+        out["bonus_fused_tail"] = {"call": "csd_round_bonus", "ms_per_round": 1e3 * b_secs / few,
+                                   "plain_round_ms": 1e3 * p_secs / few, "extra_frac": b_secs / p_secs - 1.0,
+                                   "extra_rows": f"{wl.B} of {wl.R} token rows"}
+        if wl.T == 100:
+            N = 1000
+            steps_d = np.linspace(N // wl.T, N, wl.T).astype(np.int64)
+            inp_d = gen.make_round_inputs(wl, seed_offset=777, weights=False)
+            inp_d.w_q, inp_d.w_p = inp0.w_q, inp0.w_p
+            inp_d.tfeat = np.ascontiguousarray(gen.timestep_features(N, wl.draft.F)[steps_d - 1])
+            co = api.ddim_coefficients(gen.beta_linear(N), steps_d, 1.0)
+            rd = DeviceRound(inp_d, ctx=ctx, device=local, heads=(r0.head_q, r0.head_p), coeffs_q=co, coeffs_p=co)
+            ddim_step = lambda i: rd.fused_round()
+            timed(ddim_step, 3); d_secs = timed(ddim_step, few)
+            out["ddim100"] = {"sampler": "DDIM, 100 of 1000 linear-beta steps, eta = 1", "ms_per_round": 1e3 * d_secs / few,
+                              "value": wl.R * few / d_secs, "unit": UNIT}
+
     # per-kernel-class device time (events around every launch: separate pass).  The three calls one after the
     # other: the same kernels and grids as csd_round, but the draft and the target chain do not share the GPU,
     # so a launch's duration is the kernel's own
@@ -468,7 +500,7 @@ def run_ours(args):
                                                   "share": round(v["ms"] / tot_ms, 4),
                                                   "tflops": (v["flops"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0)}
                                               for k, v in prof.items()}}
-        for k in ("sequential_draft", "prefill", "single_path"):
+        for k in ("sequential_draft", "prefill", "single_path", "bonus_fused_tail", "ddim100"):
             if k in m:
                 line[k] = m[k]
         if others:

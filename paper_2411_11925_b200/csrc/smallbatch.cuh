@@ -195,10 +195,10 @@ sb_chain_kernel(const __grid_constant__ CUtensorMap tmAp, const __grid_constant_
 
     // Ends a phase: this CTA's global writes are published to the cluster, then the group's eight CTAs meet.
     auto cluster_sync_all = [&]() {
-      fence_proxy_async_all();                   // generic-proxy writes, for the peers' TMA loads
+      if (warp >= 2) fence_proxy_async_all();    // the workers' generic-proxy writes, for the peers' TMA loads
       cluster_arrive();
       cluster_wait();
-      fence_proxy_async_all();
+      if (warp == 0) fence_proxy_async_all();    // ... which this warp issues
     };
 
     // Step boundary, first half (token-parallel: one or two tokens of the group per CTA).  finish_t > 0: finish step
