@@ -26,7 +26,10 @@ import numpy as np  # noqa: E402
 
 # dram__bytes_read + dram__bytes_write per launch of a kernel class, from the ncu capture summarised under
 # profiles/ for (workload, class); absent = no capture of the kernel as it stands (reported as null)
-NCU_DRAM_BYTES_PER_LAUNCH = {}
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    # profiles/mar256_sequential_draft_sb_chain_kernel_ncu.md: 99.4 MB read + 51.8 MB written per launch
+    ("mar256", "sb_chain"): 151.2e6,
+}
 
 # Sequences of each workload that the float64 checker evaluates when it is timed (the first n of the batch): the
 # CPU-baseline leg and the reference arm time the very same sample.
@@ -336,6 +339,7 @@ def measure(name, args, peaks, steps, warmup, rounds_per_step, full):
             "value": wl.B * wl.gamma * few / seq_secs, "unit": UNIT,
             "bound": "hbm", "weight_bytes_per_step": wbytes, "achieved": wbytes * wl.T / per_call / 1e9,
             "peak": peaks["hbm_gbs"], "roofline_unit": "GB/s", "frac": wbytes * wl.T / per_call / 1e9 / peaks["hbm_gbs"],
+            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, "sb_chain")) if launches_per_call < 50 else None,
             "note": "algorithmic bytes = draft weight bytes x T per call; the weights fit L2 (126 MB), so the "
                     "fraction says how far the call is from streaming them from HBM once per step"}
 
