@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libcsd.so")
 SOURCES = ["csd_api.cu"]
-HEADERS = ["ptx.cuh", "epilogue.cuh", "gemm.cuh", "rowops.cuh", "fold.cuh", "smallbatch.cuh", "gmm.cuh"]
+HEADERS = ["ptx.cuh", "epilogue.cuh", "gemm.cuh", "rowops.cuh", "fold.cuh", "smallbatch.cuh", "pchain.cuh", "gmm.cuh"]
 
 
 def _nvcc() -> str:

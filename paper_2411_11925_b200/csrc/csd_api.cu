@@ -21,6 +21,7 @@
 #include "gmm.cuh"
 #include "rowops.cuh"
 #include "smallbatch.cuh"
+#include "pchain.cuh"
 
 using namespace csd;
 
@@ -69,6 +70,7 @@ struct csd_ctx {
   HostIo un;       // csd_verify_unaligned: per-row noise terms
   HostIo bn;       // csd_bonus_token: samples of every sequence before the selection
   HostIo sp;       // csd_verify_single_path: schedule constants, mu^p of one pass, running log-ratio
+  HostIo pc[3];    // persistent chain kernel (per chain slot): s of all steps, a', v, partials, counters, schedule
   HostIo sb[2];    // small-batch chain kernel (per chain slot): s of all steps, early products, a', v, counters, schedule
   char err[512] = {0};
   // optional per-launch timing (csd_profile)
@@ -101,10 +103,15 @@ struct csd_head {
   // 256-row boxes; c1_k = W1_k (1 + bscale_k), c2_k = W1_k bshift_k + b1_k
   void* xblob = nullptr;
   std::vector<CUtensorMap> Wgs, Wf;
+  std::vector<CUtensorMap> Wgs_half, Wf_half;   // the same matrices in 128-row boxes: what one CTA of a pair loads
   std::vector<float*> c1, c2;   // first MLP layer with 256-row boxes (W a multiple of 256)
   // small-batch chain kernel (smallbatch.cuh): usable for this head; device tables (tensor maps of W1_k, W2_k, then of
   // the matrices multiplied by s: per block Wf_k, Wg_k, Wss_k, then Wfss, all in 128-row boxes; early tiles; biases)
   bool sb_ready = false;
+  // persistent chain kernel (pchain.cuh): per phase the early and the dependent weight maps; per phase three bias rows
+  bool pc_ready = false;
+  CUtensorMap* d_pc_maps = nullptr;
+  const float** d_pc_bias = nullptr;
   int sb_ntasks = 0;
   CUtensorMap* d_sb_maps = nullptr;
   SbTask* d_sb_tasks = nullptr;
@@ -336,6 +343,18 @@ int check_sched(csd_ctx* ctx, const csd_schedule* s, bool full) {
   return CSD_OK;
 }
 
+// Chains whose layers are one wave of tiles run as one persistent kernel (pchain.cuh) where it applies.
+#ifndef CSD_PERSISTENT_CHAINS
+#define CSD_PERSISTENT_CHAINS 1
+#endif
+constexpr bool kPersistentChains = CSD_PERSISTENT_CHAINS != 0;
+
+// Folded blocks run as CTA pairs when a layer's row tiles pair up.
+#ifndef CSD_FOLD_PAIRS
+#define CSD_FOLD_PAIRS 1
+#endif
+constexpr bool kFoldPairs = CSD_FOLD_PAIRS != 0;
+
 // Shared-memory opt-in of the folded block kernels, once per device and operand type.
 bool fold_kernels_ready(const csd_ctx* ctx, const csd_head_desc& d) {
   static int known[kMaxDevices][2] = {};
@@ -343,11 +362,15 @@ bool fold_kernels_ready(const csd_ctx* ctx, const csd_head_desc& d) {
   if (k == 0) {
     bool ok = true;
     if (d.dtype == CSD_F16) {
-      ok = ok && cudaFuncSetAttribute(fold_kernel<__half, 0, FOLD_W1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_W1>::kSmemBytes) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(fold_kernel<__half, 0, FOLD_GATE>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_GATE>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__half, 0, FOLD_W1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_W1>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__half, 0, FOLD_GATE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_GATE>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__half, 0, FOLD_W1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_W1>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__half, 0, FOLD_GATE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_GATE>::kSmemBytes) == cudaSuccess;
     } else {
-      ok = ok && cudaFuncSetAttribute(fold_kernel<__nv_bfloat16, 1, FOLD_W1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_W1>::kSmemBytes) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(fold_kernel<__nv_bfloat16, 1, FOLD_GATE>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_GATE>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__nv_bfloat16, 1, FOLD_W1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_W1>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__nv_bfloat16, 1, FOLD_GATE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_GATE>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__nv_bfloat16, 1, FOLD_W1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_W1>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(fold_kernel<__nv_bfloat16, 1, FOLD_GATE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FoldCfg<FOLD_GATE>::kSmemBytes) == cudaSuccess;
     }
     cudaGetLastError();
     k = ok ? 1 : -1;
@@ -356,6 +379,20 @@ bool fold_kernels_ready(const csd_ctx* ctx, const csd_head_desc& d) {
 }
 
 int ensure_side(csd_ctx* ctx, HostIo& io, size_t need, const char* what);
+
+// Shared-memory opt-in of the persistent chain kernel, once per device and operand type.
+bool pchain_kernel_ready(const csd_ctx* ctx, int dtype) {
+  static int known[kMaxDevices][2] = {};
+  int& k = known[ctx->device][dtype == CSD_F16 ? 0 : 1];
+  if (k == 0) {
+    const bool ok = dtype == CSD_F16
+        ? cudaFuncSetAttribute(pchain_kernel<__half, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPcSmemBytes) == cudaSuccess
+        : cudaFuncSetAttribute(pchain_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPcSmemBytes) == cudaSuccess;
+    cudaGetLastError();
+    k = ok ? 1 : -1;
+  }
+  return k == 1;
+}
 
 // Whether the small-batch chain kernel can run on this device: its clusters of 8 CTAs (one per SM, ~213 KB of
 // shared memory each) must all be resident at once.  Returns the number of clusters the GPU holds (0: unusable).
@@ -391,6 +428,7 @@ struct Chain {
   int chains = 1;   // chains that run concurrently with this one (itself included)
   int Rh = 0, W = 0, L = 0, T = 0, tn = kTileN;
   bool sbk = false;       // the whole chain runs in the small-batch kernel (smallbatch.cuh)
+  bool pck = false;       // the whole chain runs in the persistent chain kernel (pchain.cuh)
   bool fold = false;      // blocks 1.. run as two kernels (fold.cuh) instead of three
   CUtensorMap tm_ap{};
   bool mod64 = false;     // modulate kernels in 64-wide tiles although the others use 128
@@ -510,6 +548,14 @@ struct Chain {
           !traj_x && !batch_Rin && !lv_min && !ctx->prof_on &&
           (d.dtype == CSD_F16 ? sb_clusters_of<__half, 0>(ctx) : sb_clusters_of<__nv_bfloat16, 1>(ctx)) > kSbRows / kSbGroup;
     if (sbk) { fold = false; pair = false; }
+    // One wave of 128 x 128 tiles per layer and W = 1024: one persistent kernel per chain (pchain.cuh).  Row blocks are
+    // paired, so their number must be even.
+    {
+      const int row_tiles = (Rh + kTileM - 1) / kTileM, nb = cfg ? (R + 63) / 64 : (R + 127) / 128;
+      pck = kPersistentChains && fold && !sbk && hd->pc_ready && W / kTileN == kPcColTiles && nb % 2 == 0 && nb * kTileM >= Rh &&
+            row_tiles == nb && !batch_Rin && !lv_min && !ctx->prof_on && d.C <= kCPad && pchain_kernel_ready(ctx, d.dtype);
+      if (pck) { fold = false; pair = false; }
+    }
     ChainWs& ws = ctx->ws[slot];
     int rc = batch_Rin ? ensure_ws(ctx, ws, d, ws_steps * batch_Rin * (cfg ? 2 : 1), ws_steps * batch_Rin, Ts)
                        : ensure_ws(ctx, ws, d, Rh, R, Ts);
@@ -552,6 +598,7 @@ struct Chain {
     if (rc) return rc;
     sbuf[0] = ws.s2; sbuf[1] = ws.s;
     if (sbk) return launch_small_batch();
+    if (pck) return launch_pchain();
     if (batch_Rin) return launch_batch(0);   // a pass has one step (t = 1): its s is sbuf[1]
     sp.traj_x = traj_x; sp.traj_mu = nullptr; sp.status = ctx->d_err + 1;
     sp.lv1 = lv1; sp.half_logdet = half_logdet; sp.lv_min = 0.0f; sp.lv_max = 0.0f;
@@ -571,32 +618,87 @@ struct Chain {
     ChainWs& ws = ctx->ws[slot];
     FoldParams p{};
     p.M = Rh; p.W = W; p.err = ctx->d_err;
+    const int tiles_n = W / kTileN, row_tiles = (Rh + kTileM - 1) / kTileM;
+    // CTA pairs (two row tiles per MMA) whenever the row tiles pair up
+    const bool fp = kFoldPairs && row_tiles % 2 == 0;
     const CUtensorMap *tp, *ta, *tw, *tout;
     if (kind == FOLD_W1) {
       p.c0 = hd->c1[k]; p.c1 = hd->c2[k]; p.c2 = nullptr; p.stats_in = ws.stats; p.out = ws.v;
-      tp = &hd->Wf[k]; ta = &tm_ap; tw = &hd->tm[1].W1[k]; tout = &tm_v;
+      tp = fp ? &hd->Wf_half[k] : &hd->Wf[k]; ta = &tm_ap; tw = &hd->tm[fp ? 0 : 1].W1[k]; tout = &tm_v;
     } else {
       p.c0 = hd->bg[k]; p.c1 = hd->b2[k]; p.c2 = hd->bsc[k + 1]; p.stats_out = ws.stats; p.h = ws.h; p.out = ws.ap;
-      tp = &hd->Wgs[k]; ta = &tm_v; tw = &hd->tm[1].W2[k]; tout = &tm_ap;
+      tp = fp ? &hd->Wgs_half[k] : &hd->Wgs[k]; ta = &tm_v; tw = &hd->tm[fp ? 0 : 1].W2[k]; tout = &tm_ap;
     }
-    const int tiles_n = W / kTileN, row_tiles = (Rh + kTileM - 1) / kTileM;
     // algorithmic FLOPs: the block's five W x W products are split 2 (first layer and the modulation folded into
     // it; the kernel executes three products) + 3 (gate, next scale, second layer)
     ProfScope ps(ctx, st, kind == FOLD_W1 ? 1 : 3, 2.0 * Rh * static_cast<double>(W) * W * (kind == FOLD_W1 ? 2.0 : 3.0));
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(tiles_n * row_tiles); lc.blockDim = dim3(kFoldThreads); lc.stream = st;
     lc.dynamicSmemBytes = kind == FOLD_W1 ? FoldCfg<FOLD_W1>::kSmemBytes : FoldCfg<FOLD_GATE>::kSmemBytes;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
-    lc.attrs = at; lc.numAttrs = ctx->prof_on ? 0 : 1;
+    cudaLaunchAttribute at[2];
+    int na = 0;
+    if (fp) { at[na].id = cudaLaunchAttributeClusterDimension; at[na].val.clusterDim.x = 2; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1; ++na; }
+    if (!ctx->prof_on) { at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization; at[na].val.programmaticStreamSerializationAllowed = 1; ++na; }
+    lc.attrs = at; lc.numAttrs = na;
+    const CUtensorMap& ts = tm_sb[cur_t & 1];
+#define CSD_FOLD_LAUNCH(ACT, FMT, KIND, PAIR) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<ACT, FMT, KIND, PAIR>, ts, *tp, *ta, *tw, *tout, tm_h, tiles_n, p))
     if (d.dtype == CSD_F16) {
-      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_W1>, tm_sb[cur_t & 1], *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
-      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__half, 0, FOLD_GATE>, tm_sb[cur_t & 1], *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
+      if (kind == FOLD_W1) { if (fp) CSD_FOLD_LAUNCH(__half, 0, FOLD_W1, true); else CSD_FOLD_LAUNCH(__half, 0, FOLD_W1, false); }
+      else { if (fp) CSD_FOLD_LAUNCH(__half, 0, FOLD_GATE, true); else CSD_FOLD_LAUNCH(__half, 0, FOLD_GATE, false); }
     } else {
-      if (kind == FOLD_W1) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_W1>, tm_sb[cur_t & 1], *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
-      else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, fold_kernel<__nv_bfloat16, 1, FOLD_GATE>, tm_sb[cur_t & 1], *tp, *ta, *tw, *tout, tm_h, tiles_n, p));
+      if (kind == FOLD_W1) { if (fp) CSD_FOLD_LAUNCH(__nv_bfloat16, 1, FOLD_W1, true); else CSD_FOLD_LAUNCH(__nv_bfloat16, 1, FOLD_W1, false); }
+      else { if (fp) CSD_FOLD_LAUNCH(__nv_bfloat16, 1, FOLD_GATE, true); else CSD_FOLD_LAUNCH(__nv_bfloat16, 1, FOLD_GATE, false); }
     }
+#undef CSD_FOLD_LAUNCH
+    ctx->launches++;
+    return CSD_OK;
+  }
+
+  // The persistent chain kernel: s of every step in the kernel's row order, zeroed counters, the schedule on the
+  // device, one launch of CTA pairs.
+  int launch_pchain() {
+    const csd_head_desc& d = hd->d;
+    ChainWs& ws = ctx->ws[slot];
+    const size_t asz = 2;
+    const int nb = cfg ? (R + 63) / 64 : (R + 127) / 128;
+    const size_t rows = static_cast<size_t>(nb) * kTileM, G = W / kStatCols;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+    const size_t o_s = take(static_cast<size_t>(Ts) * rows * W * asz), o_ap = take(rows * W * asz), o_v = take(rows * W * asz),
+                 o_st = take(rows * G * 8), o_ep = take(rows * G * kCPad * 4), o_sync = take(static_cast<size_t>(nb / 2) * 4),
+                 o_sched = take(static_cast<size_t>(3) * Ts * 4);
+    int rc = ensure_side(ctx, ctx->pc[slot], off, "the persistent chain buffers");
+    if (rc) return rc;
+    char* b = static_cast<char*>(ctx->pc[slot].base);
+    CUtensorMap tm_s{}, tm_a{}, tm_vv{};
+    if ((rc = make_tmap(ctx, &tm_s, d.dtype, b + o_s, static_cast<uint64_t>(Ts) * rows, W, W, kTileM))) return rc;
+    if ((rc = make_tmap(ctx, &tm_a, d.dtype, b + o_ap, rows, W, W, kTileM))) return rc;
+    if ((rc = make_tmap(ctx, &tm_vv, d.dtype, b + o_v, rows, W, W, kTileM))) return rc;
+    CSD_CUDA(ctx, cudaMemsetAsync(b + o_sync, 0, static_cast<size_t>(nb / 2) * 4, st));
+    float* d_sched = reinterpret_cast<float*>(b + o_sched);
+    CSD_CUDA(ctx, cudaMemcpyAsync(d_sched, sc->a, Ts * sizeof(float), cudaMemcpyHostToDevice, st));
+    CSD_CUDA(ctx, cudaMemcpyAsync(d_sched + Ts, sc->b, Ts * sizeof(float), cudaMemcpyHostToDevice, st));
+    CSD_CUDA(ctx, cudaMemcpyAsync(d_sched + 2 * Ts, sc->sigma, Ts * sizeof(float), cudaMemcpyHostToDevice, st));
+    const dim3 sgrid(static_cast<unsigned>(rows), static_cast<unsigned>(Ts));
+    if (d.dtype == CSD_F16) pc_cond_all_kernel<__half><<<sgrid, 256, 0, st>>>(ws.cz, ws.te, reinterpret_cast<__half*>(b + o_s), R, cfg, W, static_cast<int>(rows));
+    else pc_cond_all_kernel<__nv_bfloat16><<<sgrid, 256, 0, st>>>(ws.cz, ws.te, reinterpret_cast<__nv_bfloat16*>(b + o_s), R, cfg, W, static_cast<int>(rows));
+    ctx->launches++;
+    CSD_CUDA(ctx, cudaGetLastError());
+    PcParams p{};
+    p.R = R; p.cfg = cfg; p.W = W; p.L = L; p.T = Ts; p.C = d.C; p.sample_last = sample_last; p.nblk = nb; p.cfg_scale = cfg_scale;
+    p.maps = hd->d_pc_maps; p.bias = hd->d_pc_bias; p.sched = d_sched;
+    p.win = hd->win; p.bin = hd->bin; p.wout_t = hd->wout_t; p.bout = hd->bout; p.x_T = x_T; p.eps = eps;
+    p.x0 = x0; p.mu1 = mu1; p.x1 = x1; p.x = ws.x; p.traj_x = traj_x; p.traj_mu = traj_mu;
+    p.stats = reinterpret_cast<float*>(b + o_st); p.epart = reinterpret_cast<float*>(b + o_ep);
+    p.sync = reinterpret_cast<unsigned*>(b + o_sync); p.err = ctx->d_err; p.status = ctx->d_err + 1;
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(static_cast<unsigned>(nb) * kPcColTiles); lc.blockDim = dim3(kPcThreads); lc.dynamicSmemBytes = kPcSmemBytes; lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    if (d.dtype == CSD_F16) CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, pchain_kernel<__half, 0>, tm_s, tm_a, tm_vv, p));
+    else CSD_CUDA(ctx, cudaLaunchKernelEx(&lc, pchain_kernel<__nv_bfloat16, 1>, tm_s, tm_a, tm_vv, p));
     ctx->launches++;
     return CSD_OK;
   }
@@ -653,7 +755,7 @@ struct Chain {
   }
 
   int step(int t) {
-    if (sbk) return CSD_OK;   // already enqueued by begin()
+    if (sbk || pck) return CSD_OK;   // already enqueued by begin()
     const csd_head_desc& d = hd->d;
     ChainWs& ws = ctx->ws[slot];
     cur_t = t;
@@ -970,6 +1072,7 @@ int csd_destroy(csd_ctx* c) {
   if (c->un.base) cudaFree(c->un.base);
   if (c->bn.base) cudaFree(c->bn.base);
   for (HostIo& b : c->sb) if (b.base) cudaFree(b.base);
+  for (HostIo& b : c->pc) if (b.base) cudaFree(b.base);
   if (c->d_err) cudaFree(c->d_err);
   cudaGetLastError();
   delete c;
@@ -1272,10 +1375,12 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
       else { for (size_t i = 0; i < nx; ++i) { const __half hv = __float2half_rn(xs[i]); memcpy(&xb[i], &hv, 2); } }
       if (cudaMalloc(&h->xblob, nx * 2) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the fused weights"); }
       if (cudaMemcpy(h->xblob, xb.data(), nx * 2, cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "fused weight upload failed");
-      h->Wgs.resize(L); h->Wf.resize(L);
+      h->Wgs.resize(L); h->Wf.resize(L); h->Wgs_half.resize(L); h->Wf_half.resize(L);
       char* xbase = static_cast<char*>(h->xblob);
       for (size_t k = 0; k + 1 < L && !rc; ++k) rc = make_tmap(ctx, &h->Wgs[k], d.dtype, xbase + k * per * 2, 2 * W, W, W, 256);
       for (size_t k = 1; k < L && !rc; ++k) rc = make_tmap(ctx, &h->Wf[k], d.dtype, xbase + wf_slot(k) * per * 2, 2 * W, W, W, 256);
+      for (size_t k = 0; k + 1 < L && !rc; ++k) rc = make_tmap(ctx, &h->Wgs_half[k], d.dtype, xbase + k * per * 2, 2 * W, W, W, 128);
+      for (size_t k = kfold0; k < L && !rc; ++k) rc = make_tmap(ctx, &h->Wf_half[k], d.dtype, xbase + wf_slot(k) * per * 2, 2 * W, W, W, 128);
       for (size_t k = kfold0; k < L && !rc && sbk; ++k) rc = make_tmap(ctx, &wf128[k], d.dtype, xbase + wf_slot(k) * per * 2, 2 * W, W, W, 128);
     }
     if (!rc && W % 256 == 0) {
@@ -1311,6 +1416,26 @@ int csd_head_create(csd_ctx* ctx, const csd_head_desc* desc, const csd_head_weig
       h->sb_ntasks = static_cast<int>(tasks.size());
       h->sb_ready = true;
     }
+    if (sbk && W / kTileN == static_cast<size_t>(kPcColTiles)) {
+      // tables of the persistent chain kernel: phases B, (W1_k, GATE_k) for every block, F
+      const size_t NP = 2 * L + 2;
+      std::vector<CUtensorMap> maps(2 * NP);
+      std::vector<const float*> bt(3 * NP, nullptr);
+      maps[0] = h->tm[0].Wss[0]; bt[0] = h->bsc[0];
+      for (size_t k = 0; k < L; ++k) {
+        const size_t w1 = 1 + 2 * k, gt = 2 + 2 * k;
+        maps[w1] = h->Wf_half[k]; maps[NP + w1] = h->tm[0].W1[k]; bt[3 * w1] = h->c1[k]; bt[3 * w1 + 1] = h->c2[k];
+        maps[gt] = k + 1 < L ? h->Wgs_half[k] : h->tm[0].Wg[k]; maps[NP + gt] = h->tm[0].W2[k];
+        bt[3 * gt] = h->bg[k]; bt[3 * gt + 1] = h->b2[k]; bt[3 * gt + 2] = k + 1 < L ? h->bsc[k + 1] : nullptr;
+      }
+      maps[NP - 1] = h->tm[0].Wfss; bt[3 * (NP - 1)] = h->bfsh; bt[3 * (NP - 1) + 1] = h->bfsc;
+      maps[NP] = h->tm[0].W1[0]; maps[2 * NP - 1] = h->tm[0].W1[0];   // unused entries: any valid map
+      if (cudaMalloc(&h->d_pc_maps, maps.size() * sizeof(CUtensorMap)) != cudaSuccess ||
+          cudaMalloc(&h->d_pc_bias, bt.size() * sizeof(float*)) != cudaSuccess) { cudaGetLastError(); return bail(CSD_ERR_WORKSPACE, "cannot allocate device memory for the persistent-chain tables"); }
+      if (cudaMemcpy(h->d_pc_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemcpy(h->d_pc_bias, bt.data(), bt.size() * sizeof(float*), cudaMemcpyHostToDevice) != cudaSuccess) return bail(CSD_ERR_CUDA, "persistent-chain table upload failed");
+      h->pc_ready = true;
+    }
   }
   *out = h;
   return CSD_OK;
@@ -1326,6 +1451,8 @@ int csd_head_destroy(csd_head* h) {
   if (h->wblob) cudaFree(h->wblob);
   if (h->fblob) cudaFree(h->fblob);
   if (h->xblob) cudaFree(h->xblob);
+  if (h->d_pc_maps) cudaFree(h->d_pc_maps);
+  if (h->d_pc_bias) cudaFree(h->d_pc_bias);
   if (h->d_sb_maps) cudaFree(h->d_sb_maps);
   if (h->d_sb_tasks) cudaFree(h->d_sb_tasks);
   if (h->d_sb_bias) cudaFree(h->d_sb_bias);

@@ -15,8 +15,12 @@
 //   fold_kernel<KIND_W1>   : acc(P1 | P2) = s [W1 Wscale | W1 Wshift]^T          (early, N = 256 packed),
 //                            acc_main = a' W1_k^T;  v = SiLU(rstd (acc_main - mean (P1 + c1)) + P2 + c2)
 // The early products depend only on s and overlap the preceding kernel (programmatic dependent launch).
-// One tile per CTA (128 x 128), a TMA ring of three 64 KB slot pairs, three TMEM accumulators, two TMA warps, one MMA warp,
+// One tile per CTA (128 x 128), a 192 KB TMA ring, three TMEM accumulators, three TMA warps, one MMA warp,
 // eight epilogue warps (one row x 64 columns per thread).
+// PAIR: two CTAs of a cluster (row tiles 2p and 2p + 1 of one column tile) share every MMA (cta_group::2, M = 256):
+// each loads its own rows of the activations and half of the weight rows, so a k-block of the dependent product
+// costs a CTA 24 KB of shared-memory traffic instead of 32 KB and the ring holds four two-k-block stages instead of
+// three: the product that the preceding kernel gates is bound by what the ring keeps in flight, not by the MMAs.
 #pragma once
 #include "gemm.cuh"
 #include "rowops.cuh"
@@ -47,14 +51,21 @@ struct FoldParams {
   int* err;
 };
 
-template <typename ACT, int AB_FMT, int KIND>
+template <typename ACT, int AB_FMT, int KIND, bool PAIR>
 __global__ void __launch_bounds__(kFoldThreads, 1)
 fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmWp,
             const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
             const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmHst, int tiles_n,
             const FoldParams p) {
   using Cfg = FoldCfg<KIND>;
-  constexpr int S = Cfg::kSlots, SP = S / 2, kPairBytes = 2 * kChSlotBytes;
+  // Ring stages.  Alone: three of 64 KB; early product [A 16 KB | packed 256-row weight tile 32 KB], dependent product two
+  // k-blocks [A 16 KB | B 16 KB] each.  PAIR: four of 48 KB; early [A 16 KB | this CTA's 128 packed weight rows 16 KB],
+  // dependent [A, A | this CTA's 64 weight rows 8 KB, 8 KB].
+  constexpr int S = Cfg::kSlots, SP = PAIR ? 4 : 3, kPairBytes = PAIR ? 49152 : 2 * kChSlotBytes;
+  constexpr int kDepA = PAIR ? 16384 : kChSlotBytes;          // dependent stage: distance between the two A boxes
+  constexpr int kDepB0 = PAIR ? 32768 : 16384;                // first B box
+  constexpr int kDepB = PAIR ? 8192 : kChSlotBytes;           // distance between the two B boxes
+  static_assert(SP * kPairBytes == S * kChSlotBytes, "the ring is 192 KB either way");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* ring = smem;
@@ -66,7 +77,9 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int W = p.W, nkb = W / kBlockK;
-  const int tile_n = static_cast<int>(blockIdx.x) % tiles_n, tile_m = static_cast<int>(blockIdx.x) / tiles_n;
+  const int rank = PAIR ? static_cast<int>(cluster_ctarank()) : 0;
+  const int unit = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int tile_n = unit % tiles_n, tile_m = PAIR ? 2 * (unit / tiles_n) + rank : unit / tiles_n;
   const int n_base = tile_n * kTileN, row0 = tile_m * kTileM;
 
   const bool run = *reinterpret_cast<const volatile int*>(p.err) == 0;
@@ -78,9 +91,13 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
     mbar_init(&acc_full[0], 1); mbar_init(&acc_full[1], 1);
     fence_mbar_init();
   }
-  if (warp == 1) { tmem_alloc(tmem_base_s, 512); tmem_relinquish(); }
+  if (warp == 1) {
+    if (PAIR) { tmem_alloc_pair(tmem_base_s, 512); tmem_relinquish_pair(); }
+    else { tmem_alloc(tmem_base_s, 512); tmem_relinquish(); }
+  }
   tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) { cluster_arrive(); cluster_wait(); }   // the peer's barriers exist before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_base_s;
 
@@ -97,43 +114,53 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
     auto pair_free = [&](int c) {   // c: pair counter
       if (ok && c >= SP) { ok = ch_wait<false>(&empty_bar[c % SP], ((c / SP) & 1) ^ 1, p.err); if (!ok && leader) ch_fail(p.err, DEV_ERR_TMA_WAIT, 2, c); }
     };
-    // early product: [A 16 KB | packed 256-row weight tile 32 KB]
+    // A pair's loads are all credited to the leader's barrier, which only the leader's producers arm (with the bytes
+    // of both CTAs); the peer's producers only request.
+    auto arm = [&](uint64_t* bar, uint32_t bytes) { if (!PAIR) mbar_arrive_expect_tx(bar, bytes); else if (rank == 0) mbar_arrive_expect_tx(bar, 2 * bytes); };
+    auto load = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int x, int y) {
+      if (PAIR) tma_load_2d_pair(dst, tm, mapa_shared(smem_u32(bar), 0), x, y); else tma_load_2d(dst, tm, bar, x, y);
+    };
+    // early product
     for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
       pair_free(it);
       if (ok && leader) {
         const int s = it % SP;
-        if (second) mbar_arrive(&full_bar[s]);
+        if (second) { if (rank == 0) mbar_arrive(&full_bar[s]); }
         else {
-          mbar_arrive_expect_tx(&full_bar[s], is_a ? 16384 : 32768);
-          tma_load_2d(ring + s * kPairBytes + (is_a ? 0 : 16384), is_a ? &tmS : &tmWp, &full_bar[s], kb * kBlockK,
-                      is_a ? row0 : 2 * n_base);
+          arm(&full_bar[s], is_a ? 16384 : (PAIR ? 16384 : 32768));
+          load(ring + s * kPairBytes + (is_a ? 0 : 16384), is_a ? &tmS : &tmWp, &full_bar[s], kb * kBlockK,
+               is_a ? row0 : 2 * n_base + rank * 128);
         }
       }
       __syncwarp();
     }
     if (is_a) griddep_wait();            // the dependent operand is written by the preceding kernel
-    // dependent product: two k-blocks per pair, each [A 16 KB | B 16 KB]
+    // dependent product: two k-blocks per stage
     for (int kb = 0; kb < nkb && ok; kb += 2, ++it) {
       pair_free(it);
       if (ok && leader) {
         const int s = it % SP;
         if (is_a) {
           const int jj = second ? 1 : 0;
-          mbar_arrive_expect_tx(&full_bar[s], 16384);
-          tma_load_2d(ring + s * kPairBytes + jj * kChSlotBytes, &tmA, &full_bar[s], (kb + jj) * kBlockK, row0);
+          arm(&full_bar[s], 16384);
+          load(ring + s * kPairBytes + jj * kDepA, &tmA, &full_bar[s], (kb + jj) * kBlockK, row0);
         } else {
-          mbar_arrive_expect_tx(&full_bar[s], 32768);
+          arm(&full_bar[s], PAIR ? 16384 : 32768);
 #pragma unroll
           for (int jj = 0; jj < 2; ++jj)
-            tma_load_2d(ring + s * kPairBytes + jj * kChSlotBytes + 16384, &tmW, &full_bar[s], (kb + jj) * kBlockK, n_base);
+            load(ring + s * kPairBytes + kDepB0 + jj * kDepB, &tmW, &full_bar[s], (kb + jj) * kBlockK, n_base + rank * 64);
         }
       }
       __syncwarp();
     }
-  } else if (run && warp == 1) {
-    // ------------------------------------------------------------------ MMA issue
+  } else if (run && warp == 1 && rank == 0) {
+    // ------------------------------------------------------------------ MMA issue (of a pair, the leader's)
     const bool leader = elect_one();
-    constexpr uint32_t idesc128 = umma_idesc_f16(128, AB_FMT), idesc256 = umma_idesc_f16(256, AB_FMT);
+    constexpr uint32_t idesc128 = umma_idesc_f16(128, AB_FMT, PAIR ? 256 : 128), idesc256 = umma_idesc_f16(256, AB_FMT, PAIR ? 256 : 128);
+    auto mma = [&](uint32_t d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+      if (PAIR) umma_f16_pair(d, da, db, idesc, acc); else umma_f16(d, da, db, idesc, acc);
+    };
+    auto commit = [&](uint64_t* bar) { if (PAIR) umma_commit_pair(bar); else umma_commit(bar); };
     bool ok = true;
     int it = 0;
     for (int kb = 0; kb < nkb && ok; ++kb, ++it) {
@@ -145,14 +172,14 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
         const uint32_t sa = smem_u32(ring + s * kPairBytes);
         const uint64_t da = umma_smem_desc_sw128(sa), db = umma_smem_desc_sw128(sa + 16384);
 #pragma unroll
-        for (int k = 0; k < kBlockK / 16; ++k) umma_f16(tmem_base + kFoldAccPacked, da + 2 * k, db + 2 * k, idesc256, (kb > 0 || k > 0) ? 1u : 0u);
-        umma_commit(&empty_bar[s]);
+        for (int k = 0; k < kBlockK / 16; ++k) mma(tmem_base + kFoldAccPacked, da + 2 * k, db + 2 * k, idesc256, (kb > 0 || k > 0) ? 1u : 0u);
+        commit(&empty_bar[s]);
       }
       __syncwarp();
     }
-    if (ok && leader) umma_commit(&acc_full[0]);
+    if (ok && leader) commit(&acc_full[0]);
     __syncwarp();
-    // dependent product: two k-blocks (slots) per barrier round trip
+    // dependent product: two k-blocks per barrier round trip
     for (int kb = 0; kb < nkb && ok; kb += 2, ++it) {
       const int s = it % SP;
       ok = ch_wait<false>(&full_bar[s], (it / SP) & 1, p.err);
@@ -161,16 +188,16 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
       if (leader) {
 #pragma unroll
         for (int jj = 0; jj < 2; ++jj) {
-          const uint32_t sa = smem_u32(ring + s * kPairBytes + jj * kChSlotBytes);
-          const uint64_t da = umma_smem_desc_sw128(sa), db = umma_smem_desc_sw128(sa + 16384);
+          const uint32_t sa = smem_u32(ring + s * kPairBytes);
+          const uint64_t da = umma_smem_desc_sw128(sa + jj * kDepA), db = umma_smem_desc_sw128(sa + kDepB0 + jj * kDepB);
 #pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k) umma_f16(tmem_base + kFoldAccMain, da + 2 * k, db + 2 * k, idesc128, (kb > 0 || jj > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < kBlockK / 16; ++k) mma(tmem_base + kFoldAccMain, da + 2 * k, db + 2 * k, idesc128, (kb > 0 || jj > 0 || k > 0) ? 1u : 0u);
         }
-        umma_commit(&empty_bar[s]);
+        commit(&empty_bar[s]);
       }
       __syncwarp();
     }
-    if (ok && leader) umma_commit(&acc_full[1]);
+    if (ok && leader) commit(&acc_full[1]);
     __syncwarp();
   } else if (run && warp >= 2 && warp < kFoldEpiWarps + 2) {
     // ------------------------------------------------------------------ epilogue: one row, two 32-column chunks of one 64-column group per thread
@@ -275,7 +302,8 @@ fold_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUt
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, 512);
+  if (PAIR) { cluster_arrive(); cluster_wait(); }   // neither CTA leaves while the pair's MMAs or signals may touch it
+  if (warp == 1) { if (PAIR) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512); }
 }
 
 // C[n, i] = sum_j A[n, j] B[j, i], all [W, W] fp32 row-major: the once-per-head products W1 Wscale, W1 Wshift.
