@@ -103,6 +103,29 @@ __device__ __forceinline__ bool pc_wait_count(const unsigned* p, unsigned target
   }
 }
 
+__device__ __forceinline__ void pc_flag_set(uint32_t* smem_word, uint32_t v) {
+  asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(smem_word)), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t pc_flag_get(const uint32_t* smem_word) {
+  uint32_t v;
+  asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(smem_word)) : "memory");
+  return v;
+}
+// One thread waits until this CTA's flag word has reached target (bounded).
+__device__ __forceinline__ bool pc_wait_flag(const uint32_t* smem_word, uint32_t target, const int* err) {
+  long long t0 = 0;
+  uint32_t spins = 0;
+  for (;;) {
+    if (pc_flag_get(smem_word) >= target) return true;
+    if ((++spins & 1023u) == 0u) {
+      if (*reinterpret_cast<const volatile int*>(err) != 0) return false;
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > *reinterpret_cast<volatile long long*>(&g_wait_limit_cycles)) return false;
+    }
+  }
+}
+
 // Token and guidance row (0 conditional, 1 unconditional) of kernel row rho.
 __host__ __device__ __forceinline__ int pc_row_token(int rho, int cfg, int* rep) {
   const int blk = rho >> 7, r = rho & 127;
@@ -131,6 +154,7 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
   uint64_t* acc_empty = acc_full + 2;           // the epilogues of both CTAs have read the accumulators
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(acc_empty + 1);
   volatile int* epi_ok_s = reinterpret_cast<volatile int*>(tmem_base_s + 1);
+  uint32_t* meet_seen_s = tmem_base_s + 2;      // meeting points this CTA's epilogue has seen complete (count)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int W = p.W, L = p.L, T = p.T, nkb = W / kBlockK;
@@ -146,8 +170,9 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmS); tma_prefetch_desc(&tmAp); tma_prefetch_desc(&tmV);
     for (int s = 0; s < kPcBars; ++s) { mbar_init(&full_bar[s], 3); mbar_init(&empty_bar[s], 1); }
-    mbar_init(&acc_full[0], 1); mbar_init(&acc_full[1], 1); mbar_init(acc_empty, 2);
+    mbar_init(&acc_full[0], 1); mbar_init(&acc_full[1], 1); mbar_init(acc_empty, 16);   // 8 epilogue warps of each CTA
     *epi_ok_s = 1;
+    *meet_seen_s = 0;
     fence_mbar_init();
   }
   if (warp == 1) { tmem_alloc_pair(tmem_base_s, 512); tmem_relinquish_pair(); }
@@ -200,9 +225,15 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
       for (int ph = 0; ph < NP && ok; ++ph) {
         const CUtensorMap* tmE = p.maps + ph;
         const bool n128 = early_n128(ph);
+        // A dependent operand is complete once every CTA of the group has finished the preceding phase; this CTA's
+        // epilogue watches the group's counter and raises a flag in shared memory.  The proxy fence that must follow
+        // is taken between early stages as soon as the flag is up, off the path of the first dependent load.
+        const uint32_t meet_target = static_cast<uint32_t>(si * NS + ph + 1);
+        bool fenced = !(is_a && has_dep(ph));
         for (int kb = 0; kb < nkb && ok; ++kb) {
           acquire(2);
           if (ok && leader) {
+            if (!fenced && kb >= nkb - 6 && pc_flag_get(meet_seen_s) >= meet_target) { fence_proxy_async_all(); fenced = true; }
             uint64_t* fb = &full_bar[n & (kPcBars - 1)];
             if (second) { if (rank == 0) mbar_arrive(fb); }
             else if (is_a) { arm(fb, 16384); load(gran(0), &tmS, fb, kb * kBlockK, srow); }
@@ -216,9 +247,8 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
         }
         if (!has_dep(ph)) continue;
         if (is_a && ok) {
-          // the dependent operand is complete once every CTA of the group has finished the preceding phase
-          if (leader) {
-            if (!pc_wait_count(ctr, static_cast<unsigned>(kPcGroup) * static_cast<unsigned>(si * NS + ph + 1), p.err)) { ch_fail(p.err, DEV_ERR_TMA_WAIT, 3, ph); ok = false; }
+          if (leader && !fenced) {
+            if (!pc_wait_flag(meet_seen_s, meet_target, p.err)) { ch_fail(p.err, DEV_ERR_TMA_WAIT, 3, ph); ok = false; }
             fence_proxy_async_all();
           }
           ok = __all_sync(0xffffffffu, ok);
@@ -317,11 +347,21 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
     auto publish = [&](bool mine) { if (et == 0 && !mine) *epi_ok_s = 0; epi_sync(); ok = *epi_ok_s != 0; };
     auto meet_wait = [&](int idx) {      // every CTA of the group has passed meeting point idx
       bool w = true;
-      if (et == 0 && ok) { w = pc_wait_count(ctr, static_cast<unsigned>(kPcGroup) * static_cast<unsigned>(idx + 1), p.err); if (!w) ch_fail(p.err, DEV_ERR_EPI_WAIT, 8, idx); }
+      if (et == 0 && ok) {
+        w = pc_wait_count(ctr, static_cast<unsigned>(kPcGroup) * static_cast<unsigned>(idx + 1), p.err);
+        if (w) pc_flag_set(meet_seen_s, static_cast<uint32_t>(idx + 1)); else ch_fail(p.err, DEV_ERR_EPI_WAIT, 8, idx);
+      }
       publish(w);
     };
     auto meet_arrive = [&]() {           // after a barrier among the epilogue threads: their global writes are ordered before
       if (et == 0) pc_arrive(ctr);   // release: cumulative over the writes the barrier ordered before it
+    };
+    // The accumulators may be overwritten once every epilogue warp of the pair has read its part: each warp says so
+    // right after its last read, before the arithmetic on what it read.
+    auto release_acc = [&]() {
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(acc_empty), 0));
     };
     auto stage_act = [&](int c, const float* v) {
       uint8_t* row = stage_out + (c >> 1) * (kTileM * 128) + rloc * 128;
@@ -402,7 +442,29 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
         meet_wait(si * NS + ph);
         if (!ok) break;
         float mean = 0.0f, rstd = 0.0f;
-        if (is_w1 || is_f) row_stats<true>(p.stats, m, W, mean, rstd);
+        if (is_w1 || is_f) {
+          // LayerNorm statistics of the row from its 16 partials.  The row block's partials (16 KB, contiguous) come in
+          // with coalesced loads through the idle output buffer: row-per-thread loads (32 lines per instruction) held up
+          // the SM's TMA traffic for about 3 k cycles.
+          const float4* src = reinterpret_cast<const float4*>(p.stats) + static_cast<size_t>(row0) * (G / 2);
+          float4* st4 = reinterpret_cast<float4*>(stage_out);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int idx = et + kEpiThreads * k, r = idx >> 3, j = idx & 7;
+            st4[r * 8 + (j ^ (r & 7))] = __ldcg(src + idx);
+          }
+          epi_sync();
+          float4 b[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) b[j] = st4[rloc * 8 + (j ^ (rloc & 7))];
+          float sum = 0.0f, m2 = 0.0f, qq = 0.0f;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) { sum += b[j].x; sum += b[j].z; m2 += b[j].y; m2 += b[j].w; }
+          mean = sum / static_cast<float>(G);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) { const float d0 = b[j].x - mean, d1 = b[j].z - mean; qq = fmaf(d0, d0, qq); qq = fmaf(d1, d1, qq); }
+          rstd = 1.0f / sqrtf(fmaf(static_cast<float>(kStatCols), qq, m2) / static_cast<float>(W) + 1e-6f);
+        }
         if (is_b) {
           for (int e = et; e < per * kCPad; e += kEpiThreads) {
             const int i = tile_m * per + (e >> 4), cc = e & 15;
@@ -433,6 +495,7 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
             tmem_ld32(trow + colp + kStatCols, a1);                       // P2
             tmem_ld32(trow + kPcAccM + c * kChunk, am);
             tmem_ld_wait();
+            if (ci == 1) release_acc();
             const float* k0 = bias_s + c * kChunk;
             const float* k1 = bias_s + 128 + c * kChunk;
 #pragma unroll
@@ -448,20 +511,20 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
 #pragma unroll
           for (int ci = 0; ci < 2; ++ci) {
             const int c = 2 * half + ci;
-            float a0[kChunk], am[kChunk], hv[kChunk];
+            float a0[kChunk], a1[kChunk], am[kChunk], hv[kChunk];
             const uint32_t colp = kPcAccP + (last_gate ? c * kChunk : (c >> 1) * 128 + (c & 1) * kChunk);
             tmem_ld32(trow + colp, a0);                                   // gate
+            if (!last_gate) tmem_ld32(trow + colp + kStatCols, a1);       // next block's scale
             tmem_ld32(trow + kPcAccM + c * kChunk, am);
             tmem_ld32(trow + kPcAccH + c * kChunk, hv);
             tmem_ld_wait();
+            if (ci == 1) release_acc();
             gate_res_chunk(a0, am, bias_s + c * kChunk, bias_s + 128 + c * kChunk, hv, rs);
             tmem_st32(trow + kPcAccH + c * kChunk, hv);
             if (!last_gate) {
-              tmem_ld32(trow + colp + kStatCols, a0);                     // next block's scale
-              tmem_ld_wait();
               const float* k2 = bias_s + 256 + c * kChunk;
 #pragma unroll
-              for (int j = 0; j < kChunk; ++j) hv[j] = __fmul_rn(hv[j], __fadd_rn(1.0f, __fadd_rn(a0[j], k2[j])));
+              for (int j = 0; j < kChunk; ++j) hv[j] = __fmul_rn(hv[j], __fadd_rn(1.0f, __fadd_rn(a1[j], k2[j])));
               stage_act(c, hv);
             }
           }
@@ -480,6 +543,7 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
             tmem_ld32(trow + colp + kStatCols, a1);                       // scale
             tmem_ld32(trow + kPcAccH + c * kChunk, hv);
             tmem_ld_wait();
+            if (ci == 1) release_acc();
             const float* k0 = bias_s + c * kChunk;
             const float* k1 = bias_s + 128 + c * kChunk;
             const float* wc = wout_s + c * kChunk * kCPad;
@@ -512,18 +576,24 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
             const int c = 2 * half + ci;
             float a1[kChunk], hv[kChunk];
             tmem_ld32(trow + kPcAccP + (c >> 1) * 128 + (c & 1) * kChunk + kStatCols, a1);   // scale of block 0
+            if (ci == 1) { tmem_ld_wait(); release_acc(); }
             float sum = 0.0f;
 #pragma unroll
-            for (int j = 0; j < kChunk; ++j) {
-              const float4* w4 = reinterpret_cast<const float4*>(win_s + (c * kChunk + j) * kCPad);
-              float a = bin_s[c * kChunk + j];
+            for (int j0 = 0; j0 < kChunk; j0 += 4) {          // four independent chains
+              float acc4[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) acc4[u] = bin_s[c * kChunk + j0 + u];
 #pragma unroll
               for (int c4 = 0; c4 < kCPad / 4; ++c4) {
-                const float4 w = w4[c4];
-                a = fmaf(w.x, xr[4 * c4], a); a = fmaf(w.y, xr[4 * c4 + 1], a); a = fmaf(w.z, xr[4 * c4 + 2], a); a = fmaf(w.w, xr[4 * c4 + 3], a);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                  const float4 w = reinterpret_cast<const float4*>(win_s + (c * kChunk + j0 + u) * kCPad)[c4];
+                  acc4[u] = fmaf(w.x, xr[4 * c4], acc4[u]); acc4[u] = fmaf(w.y, xr[4 * c4 + 1], acc4[u]);
+                  acc4[u] = fmaf(w.z, xr[4 * c4 + 2], acc4[u]); acc4[u] = fmaf(w.w, xr[4 * c4 + 3], acc4[u]);
+                }
               }
-              hv[j] = a;
-              sum += a;
+#pragma unroll
+              for (int u = 0; u < 4; ++u) { hv[j0 + u] = acc4[u]; sum += acc4[u]; }
             }
             const float mu = sum * (1.0f / kChunk);
             float m2 = 0.0f;
@@ -545,14 +615,12 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
         tc_fence_before_sync();   // orders the TMEM reads before the barrier that releases the accumulators
         epi_sync();
         if (et == 0) {
-          mbar_arrive_cluster(mapa_shared(smem_u32(acc_empty), 0));
           if (stores) {
             const CUtensorMap* tmo = is_w1 ? &tmV : &tmAp;
             tma_store_2d(tmo, stage_out, n_base, row0);
             tma_store_2d(tmo, stage_out + kTileM * 128, n_base + 64, row0);
             tma_store_commit();
-            tma_store_wait_all();
-            fence_proxy_async_all();
+            tma_store_wait_all();   // complete before the release below; the readers fence before their TMA loads
           }
         }
         meet_arrive();
