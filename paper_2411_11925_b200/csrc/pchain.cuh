@@ -94,6 +94,7 @@ __device__ __forceinline__ bool pc_wait_count(const unsigned* p, unsigned target
   uint32_t spins = 0;
   for (;;) {
     if (pc_ld_acquire(p) >= target) return true;
+    __nanosleep(40);   // the poll is a round trip to L2 anyway; idle issue slots instead of a hot loop (the GPU runs at its power cap)
     if ((++spins & 255u) == 0u) {
       if (*reinterpret_cast<const volatile int*>(err) != 0) return false;
       const long long now = clock64();
