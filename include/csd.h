@@ -128,27 +128,36 @@ int csd_selftest_wait_timeout(csd_ctx *ctx);
 int64_t csd_launch_count(const csd_ctx *ctx);
 
 /* How the blocks of a denoising chain (the T steps of Eq. 3 for one head) are split into kernels.
- *   CSD_CHAIN_LAYERS  (default): one kernel per layer, chained with programmatic dependent launch; a
- *                     layer's independent part overlaps its predecessor on otherwise idle SMs.  For 16-bit
- *                     heads on grids of one wave, blocks 2..L run as two kernels instead of three: LayerNorm
- *                     is folded into the first layer's epilogue (algebraically the same function, rounded
- *                     differently: results agree with the plain layout within the parity tolerance, not
- *                     bit for bit).
- *   CSD_CHAIN_LAYERS_PLAIN: as above without the folded blocks (three kernels per block everywhere); a
+ *   CSD_CHAIN_LAYERS  (default): the library picks by size.
+ *                     - Layers of one wave of 128 x 128 tiles on a 16-bit head with W = 1024, var_out = 0 and an
+ *                       even number of row blocks (128 head rows each: 64 tokens with guidance, 128 without; a few
+ *                       hundred to about a thousand head rows) run as ONE persistent kernel per chain: a pair of
+ *                       CTAs owns its output tiles for every layer and step, the residual stream stays in tensor
+ *                       memory, the CTAs that share rows meet at a counter once per layer.  Draft and target chain
+ *                       of csd_round then run side by side without competing for SMs.  Its buffers grow with T
+ *                       (the condition vectors of all steps: T x rows x W 16-bit values).
+ *                     - Otherwise one kernel per layer, chained with programmatic dependent launch; a layer's
+ *                       independent part overlaps its predecessor on otherwise idle SMs.  For 16-bit heads on
+ *                       grids of one wave, blocks 2..L run as two kernels instead of three: LayerNorm is folded
+ *                       into the first layer's epilogue.
+ *                     Folding is algebraically the same function, rounded differently: the layouts agree within
+ *                     the parity tolerance, not bit for bit, and which one runs depends on the call's row count.
+ *   CSD_CHAIN_LAYER_KERNELS: as CSD_CHAIN_LAYERS without the persistent kernel (layer kernels, folded where
+ *                     that applies): what csd_draft_denoise_static always runs.
+ *   CSD_CHAIN_LAYERS_PLAIN: layer kernels without the folded blocks (three kernels per block everywhere); a
  *                     row's bits then do not depend on how many rows the call has.
  *   CSD_CHAIN_SMALL_BATCH: as CSD_CHAIN_LAYERS, except that a chain of at most 128 head rows (R (1 + cfg) <= 128)
  *                     on a 16-bit head with W in {512, 1024, 1536} and var_out = 0 runs as ONE persistent kernel
- *                     that spreads every layer over the whole GPU (weights as the MMA's M operand, K split over
- *                     a cluster of 8 CTAs with the partial sums reduced through distributed shared memory, the
- *                     products of the condition vector computed a step ahead by the remaining SMs).  This is the
- *                     calling pattern Alg. 1 forces on the draft model (x_i ~ q_i one position at a time), where
- *                     the layer kernels are bound by kernel latency.  Every block is folded, so results agree
- *                     with the other layouts within the parity tolerance.  The kernel needs the GPU to itself:
- *                     csd_round then runs its two chains one after the other, and two contexts should not run
- *                     such chains at the same time (the kernels would wait for each other's SMs until the wait
- *                     limit and report CSD_ERR_TIMEOUT).
+ *                     that spreads every layer over the whole GPU (weights as the MMA's M operand, a cluster of 8
+ *                     CTAs per group of 16 rows, the products of the condition vector computed a step ahead by the
+ *                     remaining SMs).  This is the calling pattern Alg. 1 forces on the draft model (x_i ~ q_i one
+ *                     position at a time), where the layer kernels are bound by kernel latency.  Every block is
+ *                     folded, so results agree with the other layouts within the parity tolerance.  The kernel
+ *                     needs the GPU to itself: csd_round then runs its two chains one after the other, and two
+ *                     contexts should not run such chains at the same time (the kernels would wait for each
+ *                     other's SMs until the wait limit and report CSD_ERR_TIMEOUT).
  * Takes effect for calls made after it returns. */
-enum { CSD_CHAIN_LAYERS = 0, CSD_CHAIN_SMALL_BATCH = 1, CSD_CHAIN_LAYERS_PLAIN = 2 };
+enum { CSD_CHAIN_LAYERS = 0, CSD_CHAIN_SMALL_BATCH = 1, CSD_CHAIN_LAYERS_PLAIN = 2, CSD_CHAIN_LAYER_KERNELS = 3 };
 int csd_set_chain_mode(csd_ctx *ctx, int mode);
 
 /* Optional per-launch timing for benchmarks.  csd_profile(ctx, 1) synchronises, clears the records
@@ -202,7 +211,10 @@ int csd_draft_denoise(csd_ctx *ctx, const csd_head *head, const csd_schedule *sc
                       float *x0, float *mu1, float *x1);
 
 /* csd_draft_denoise without any allocation (the paper has no counterpart: this is a deployment
- * variant of the call above, same arguments, same kernels, bit-identical results).
+ * variant of the call above with the same arguments; it runs the layer kernels, so its results are
+ * bit-identical to csd_draft_denoise in the modes CSD_CHAIN_LAYER_KERNELS and CSD_CHAIN_LAYERS_PLAIN, and
+ * in the default mode whenever that call does not take the persistent chain kernel, whose buffers
+ * grow with T and cannot live in a fixed array; otherwise the two agree within the parity tolerance).
  * Who needs it: code that must not, or cannot, reach the CUDA allocator when the call is made -
  * a serving process whose framework has handed all free device memory to its own pool so that
  * cudaMalloc fails, a latency-critical loop where cudaMalloc's implicit device synchronisation is

@@ -230,10 +230,11 @@ class Context:
     def launch_count(self) -> int:
         return int(_LIB.csd_launch_count(self._h))
 
-    CHAIN_LAYERS, CHAIN_SMALL_BATCH, CHAIN_LAYERS_PLAIN = 0, 1, 2
+    CHAIN_LAYERS, CHAIN_SMALL_BATCH, CHAIN_LAYERS_PLAIN, CHAIN_LAYER_KERNELS = 0, 1, 2, 3
 
     def set_chain_mode(self, mode: int):
-        """csd_set_chain_mode: CHAIN_LAYERS (default: one kernel per layer, folded blocks where they apply),
+        """csd_set_chain_mode: CHAIN_LAYERS (default: the persistent chain kernel where it applies, else one kernel per
+        layer with folded blocks where they apply), CHAIN_LAYER_KERNELS (never the persistent chain kernel),
         CHAIN_LAYERS_PLAIN (three kernels per block everywhere) or CHAIN_SMALL_BATCH (chains of at most 128 head rows
         run as one persistent kernel over the whole GPU)."""
         self._check(_LIB.csd_set_chain_mode(self._h, int(mode)))

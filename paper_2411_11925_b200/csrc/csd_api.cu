@@ -539,7 +539,7 @@ struct Chain {
     // (the rule looks at this chain alone, so that csd_round and the three separate calls take the same path).
     {
       const int t128 = (W / kTileN) * ((Rh + kTileM - 1) / kTileM);
-      fold = tc && ctx->chain_mode == CSD_CHAIN_LAYERS && !pair && L >= 2 && !hd->Wf.empty() &&
+      fold = tc && (ctx->chain_mode == CSD_CHAIN_LAYERS || ctx->chain_mode == CSD_CHAIN_LAYER_KERNELS) && !pair && L >= 2 && !hd->Wf.empty() &&
              8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && fold_kernels_ready(ctx, d);
     }
     // Few rows: one persistent kernel for the whole chain (opt-in per context).  It needs the GPU to itself, so a
@@ -552,8 +552,10 @@ struct Chain {
     // paired, so their number must be even.
     {
       const int row_tiles = (Rh + kTileM - 1) / kTileM, nb = cfg ? (R + 63) / 64 : (R + 127) / 128;
-      pck = kPersistentChains && fold && !sbk && hd->pc_ready && W / kTileN == kPcColTiles && nb % 2 == 0 && nb * kTileM >= Rh &&
-            row_tiles == nb && !batch_Rin && !lv_min && !ctx->prof_on && d.C <= kCPad && pchain_kernel_ready(ctx, d.dtype);
+      const int t128 = (W / kTileN) * row_tiles;
+      pck = kPersistentChains && tc && ctx->chain_mode == CSD_CHAIN_LAYERS && !pair && !sbk && slot != 2 && hd->pc_ready &&
+            8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && W / kTileN == kPcColTiles && nb % 2 == 0 && row_tiles == nb &&
+            !batch_Rin && !lv_min && !ctx->prof_on && d.C <= kCPad && pchain_kernel_ready(ctx, d.dtype);
       if (pck) { fold = false; pair = false; }
     }
     ChainWs& ws = ctx->ws[slot];
@@ -1123,7 +1125,7 @@ int csd_selftest_wait_timeout(csd_ctx* c) {
 
 int csd_set_chain_mode(csd_ctx* c, int mode) {
   if (!c) return CSD_ERR_INVALID_ARG;
-  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_LAYERS_PLAIN && mode != CSD_CHAIN_SMALL_BATCH) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
+  if (mode != CSD_CHAIN_LAYERS && mode != CSD_CHAIN_LAYERS_PLAIN && mode != CSD_CHAIN_SMALL_BATCH && mode != CSD_CHAIN_LAYER_KERNELS) return fail(c, CSD_ERR_INVALID_ARG, "chain mode %d unknown", mode);
   c->chain_mode = mode;
   return CSD_OK;
 }

@@ -91,7 +91,10 @@ def test_static_scratch_near_the_limit_runs_the_folded_blocks():
     from paper_2411_11925_b200.runner import DeviceRound
     wl = gen.Workload(**{**gen.WORKLOADS["tiny_fp32"].__dict__, "B": 41, "gamma": 5, "T": 3, "bf16": True,
                          "cfg": True, "cfg_scale": 3.0, "draft": gen.HeadSpec(2, 1024, 128)})
+    from paper_2411_11925_b200 import api
     dr = DeviceRound(gen.make_round_inputs(wl))
+    # the static call runs the layer kernels: the allocating call's bits in that mode ...
+    dr.ctx.set_chain_mode(api.Context.CHAIN_LAYER_KERNELS)
     dr.draft()
     dr.ctx.sync()
     want = dr.x0.clone(), dr.mu1_q.clone()
@@ -100,6 +103,19 @@ def test_static_scratch_near_the_limit_runs_the_folded_blocks():
                                     got[0], got[1], None)
     dr.ctx.sync()
     assert torch.equal(got[0], want[0]) and torch.equal(got[1], want[1])
+    # ... and in the default mode, where this shape (4 row blocks, W = 1024) takes the persistent chain kernel, the same
+    # function within the rounding of the two layouts
+    dr.ctx.set_chain_mode(api.Context.CHAIN_LAYERS)
+    l0 = dr.ctx.launch_count()
+    dr.draft()
+    dr.ctx.sync()
+    assert dr.ctx.launch_count() - l0 < 10
+    assert float((dr.x0 - got[0]).abs().max()) <= 5e-3 and float((dr.mu1_q - got[1]).abs().max()) <= 5e-3
+    got2 = torch.full_like(dr.x0, float("nan")), torch.full_like(dr.x0, float("nan"))
+    dr.ctx.csd_draft_denoise_static(dr.head_q, dr.sched_q, wl.R, wl.cfg, wl.cfg_scale, dr.z_q, dr.x_T, dr.eps,
+                                    got2[0], got2[1], None)
+    dr.ctx.sync()
+    assert torch.equal(got2[0], got[0]) and torch.equal(got2[1], got[1])      # the static call does not change with the mode
     dr.ctx.close()
 
 
