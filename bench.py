@@ -309,6 +309,24 @@ def measure(name, args, peaks, steps, warmup, rounds_per_step, full):
         out["e2e_secs"] = float("nan")
 
     few = max(3, min(steps, 5))
+    # The two chains of a round on their own (csd_draft_denoise, csd_verify): with the persistent chain kernel a call
+    # is one launch, so this is the kernel's duration; and the same round from the layer kernels only.
+    if full:
+        l1 = ctx.launch_count()
+        timed(lambda i: rounds[i % nsets].draft(), 2)
+        d_launches = (ctx.launch_count() - l1) // 2
+        d_secs = timed(lambda i: rounds[i % nsets].draft(), few)
+        timed(lambda i: rounds[i % nsets].verify(), 2)
+        v_secs = timed(lambda i: rounds[i % nsets].verify(), few)
+        ctx.set_chain_mode(api.Context.CHAIN_LAYER_KERNELS)
+        timed(lambda i: rounds[i % nsets].fused_round(), 3)
+        lk_secs = timed(lambda i: rounds[i % nsets].fused_round(), few)
+        ctx.set_chain_mode(api.Context.CHAIN_LAYERS)
+        out["chains"] = {"draft_ms": 1e3 * d_secs / few, "verify_ms": 1e3 * v_secs / few,
+                         "draft_launches_per_call": int(d_launches),
+                         "persistent_chain_kernel": bool(d_launches < 50),
+                         "layer_kernels_ms_per_round": 1e3 * lk_secs / few}
+
     # Sequential-draft variant: how an autoregressive loop has to call the draft head, one position at a time
     # (gamma calls of csd_draft_denoise with B tokens = B (1 + cfg) head rows each).  Few rows per call: the
     # binding resource is streaming the draft head's weights once per denoising step.
@@ -490,7 +508,23 @@ def run_ours(args):
         line["path_frac_of_tensor_peak"] = tf / peaks["tflops_sustained"]
         line["decisions"] = m["decisions"]
         prof = m.get("prof")
-        if prof:
+        ch = m.get("chains")
+        if ch and ch["persistent_chain_kernel"] and wl.operand_format != "f32":
+            # the dominant kernel of the timed region is the target chain's persistent kernel: one launch per csd_verify
+            # call, timed by events around the call on the library's stream (the other kernels of the call take microseconds)
+            fl = wl.Rh * wl.T * wl.target.flops_per_row_step()
+            ach = fl / (ch["verify_ms"] * 1e-3) / 1e12
+            line["roofline"] = {"bound": "tensor", "kernel": "pchain_kernel (target chain, one launch per call)",
+                                "achieved": ach, "peak": peaks["tflops_sustained"], "unit": "TFLOP/s",
+                                "frac": ach / peaks["tflops_sustained"],
+                                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, "pchain_target")),
+                                "peak_source": f"{peaks['source']} bf16 sustained (fp16 has the same nominal rate)",
+                                "avg_launch_us": 1e3 * ch["verify_ms"], "flops_per_launch": fl,
+                                "sms_used": "64 of 148 (the draft chain's kernel runs beside it on 64 others)",
+                                "draft_chain": {"avg_launch_us": 1e3 * ch["draft_ms"],
+                                                "achieved": wl.Rh * wl.T * wl.draft.flops_per_row_step() / (ch["draft_ms"] * 1e-3) / 1e12}}
+            line["chains"] = ch
+        elif prof:
             gemm = {k: v for k, v in prof.items() if k != "step" and v["launches"] > 0}
             top = max(gemm, key=lambda k: gemm[k]["ms"])
             tot_ms = sum(v["ms"] for v in prof.values())
@@ -504,6 +538,11 @@ def run_ours(args):
                                                   "share": round(v["ms"] / tot_ms, 4),
                                                   "tflops": (v["flops"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0)}
                                               for k, v in prof.items()}}
+        if prof and "roofline" in line and "per_class" not in line["roofline"]:
+            tot_ms = sum(v["ms"] for v in prof.values())
+            line["layer_kernels_per_class"] = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / tot_ms, 4),
+                                                    "tflops": (v["flops"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0)}
+                                               for k, v in prof.items()}
         for k in ("sequential_draft", "prefill", "single_path", "bonus_fused_tail", "ddim100"):
             if k in m:
                 line[k] = m[k]

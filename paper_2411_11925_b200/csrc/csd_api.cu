@@ -549,12 +549,12 @@ struct Chain {
           (d.dtype == CSD_F16 ? sb_clusters_of<__half, 0>(ctx) : sb_clusters_of<__nv_bfloat16, 1>(ctx)) > kSbRows / kSbGroup;
     if (sbk) { fold = false; pair = false; }
     // One wave of 128 x 128 tiles per layer and W = 1024: one persistent kernel per chain (pchain.cuh).  Row blocks are
-    // paired, so their number must be even.
+    // paired: an odd number is rounded up with a block of rows that belong to no token.
     {
       const int row_tiles = (Rh + kTileM - 1) / kTileM, nb = cfg ? (R + 63) / 64 : (R + 127) / 128;
       const int t128 = (W / kTileN) * row_tiles;
       pck = kPersistentChains && tc && ctx->chain_mode == CSD_CHAIN_LAYERS && !pair && !sbk && slot != 2 && hd->pc_ready &&
-            8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && W / kTileN == kPcColTiles && nb % 2 == 0 && row_tiles == nb &&
+            8 * t128 > ctx->num_sms && 2 * t128 <= ctx->num_sms && W / kTileN == kPcColTiles && row_tiles == nb &&
             !batch_Rin && !lv_min && !ctx->prof_on && d.C <= kCPad && pchain_kernel_ready(ctx, d.dtype);
       if (pck) { fold = false; pair = false; }
     }
@@ -662,7 +662,7 @@ struct Chain {
     const csd_head_desc& d = hd->d;
     ChainWs& ws = ctx->ws[slot];
     const size_t asz = 2;
-    const int nb = cfg ? (R + 63) / 64 : (R + 127) / 128;
+    const int nb0 = cfg ? (R + 63) / 64 : (R + 127) / 128, nb = nb0 + (nb0 & 1);   // row blocks, paired
     const size_t rows = static_cast<size_t>(nb) * kTileM, G = W / kStatCols;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
