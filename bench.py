@@ -29,6 +29,8 @@ import numpy as np  # noqa: E402
 NCU_DRAM_BYTES_PER_LAUNCH = {
     # profiles/mar256_sequential_draft_sb_chain_kernel_ncu.md: 99.4 MB read + 51.8 MB written per launch
     ("mar256", "sb_chain"): 151.2e6,
+    # profiles/mar256_persistent_chain_kernel_ncu.md: 6.02 GB read + 43.6 MB written per launch of the target chain
+    ("mar256", "pchain_target"): 6.062e9,
 }
 
 # Sequences of each workload that the float64 checker evaluates when it is timed (the first n of the batch): the

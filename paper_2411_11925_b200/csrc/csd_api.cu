@@ -682,8 +682,8 @@ struct Chain {
     CSD_CUDA(ctx, cudaMemcpyAsync(d_sched + Ts, sc->b, Ts * sizeof(float), cudaMemcpyHostToDevice, st));
     CSD_CUDA(ctx, cudaMemcpyAsync(d_sched + 2 * Ts, sc->sigma, Ts * sizeof(float), cudaMemcpyHostToDevice, st));
     const dim3 sgrid(static_cast<unsigned>(rows), static_cast<unsigned>(Ts));
-    if (d.dtype == CSD_F16) pc_cond_all_kernel<__half><<<sgrid, 256, 0, st>>>(ws.cz, ws.te, reinterpret_cast<__half*>(b + o_s), R, cfg, W, static_cast<int>(rows));
-    else pc_cond_all_kernel<__nv_bfloat16><<<sgrid, 256, 0, st>>>(ws.cz, ws.te, reinterpret_cast<__nv_bfloat16*>(b + o_s), R, cfg, W, static_cast<int>(rows));
+    if (d.dtype == CSD_F16) pc_cond_all_kernel<__half><<<sgrid, 128, 0, st>>>(ws.cz, ws.te, reinterpret_cast<__half*>(b + o_s), R, cfg, W, static_cast<int>(rows));
+    else pc_cond_all_kernel<__nv_bfloat16><<<sgrid, 128, 0, st>>>(ws.cz, ws.te, reinterpret_cast<__nv_bfloat16*>(b + o_s), R, cfg, W, static_cast<int>(rows));
     ctx->launches++;
     CSD_CUDA(ctx, cudaGetLastError());
     PcParams p{};

@@ -640,18 +640,27 @@ pchain_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ C
 // s_t = SiLU(cz + te_t) of every step, in the kernel's row order and operand format: s_all[(t - 1) rows + rho][col];
 // rows of tokens beyond R are zero.
 template <typename ACT>
-__global__ void __launch_bounds__(256) pc_cond_all_kernel(const float* __restrict__ cz, const float* __restrict__ te,
+__global__ void __launch_bounds__(128) pc_cond_all_kernel(const float* __restrict__ cz, const float* __restrict__ te,
                                                           ACT* __restrict__ s_all, int R, int cfg, int W, int rows) {
   const int t = blockIdx.y, rho = blockIdx.x;
   int rep;
   const int i = pc_row_token(rho, cfg, &rep);
-  ACT* dst = s_all + (static_cast<size_t>(t) * rows + rho) * W;
+  uint4* dst = reinterpret_cast<uint4*>(s_all + (static_cast<size_t>(t) * rows + rho) * W);     // 8 values per store
   if (i >= R) {
-    for (int j = threadIdx.x; j < W; j += blockDim.x) dst[j] = to_act<ACT>(0.0f);
+    for (int j = threadIdx.x; j < W / 8; j += blockDim.x) dst[j] = make_uint4(0u, 0u, 0u, 0u);
     return;
   }
-  const size_t src = static_cast<size_t>(rep) * R + i;
-  for (int j = threadIdx.x; j < W; j += blockDim.x) dst[j] = to_act<ACT>(silu_f(cz[src * W + j] + te[static_cast<size_t>(t) * W + j]));
+  const float4* c4 = reinterpret_cast<const float4*>(cz + (static_cast<size_t>(rep) * R + i) * W);
+  const float4* t4 = reinterpret_cast<const float4*>(te + static_cast<size_t>(t) * W);
+  for (int j = threadIdx.x; j < W / 8; j += blockDim.x) {
+    const float4 a = c4[2 * j], b = c4[2 * j + 1], ta = __ldg(t4 + 2 * j), tb = __ldg(t4 + 2 * j + 1);
+    __align__(16) ACT o[8];
+    o[0] = to_act<ACT>(silu_f(a.x + ta.x)); o[1] = to_act<ACT>(silu_f(a.y + ta.y));
+    o[2] = to_act<ACT>(silu_f(a.z + ta.z)); o[3] = to_act<ACT>(silu_f(a.w + ta.w));
+    o[4] = to_act<ACT>(silu_f(b.x + tb.x)); o[5] = to_act<ACT>(silu_f(b.y + tb.y));
+    o[6] = to_act<ACT>(silu_f(b.z + tb.z)); o[7] = to_act<ACT>(silu_f(b.w + tb.w));
+    dst[j] = *reinterpret_cast<const uint4*>(o);
+  }
 }
 
 }  // namespace csd
