@@ -33,6 +33,7 @@ def _ref(inp):
                   draft=gen.HeadSpec(2, 1024, 128), target=gen.HeadSpec(2, 1024, 128))),
     ("f16", dict(B=47, gamma=8, T=3)),                                        # 376 tokens: 6 row blocks, the last one ragged
     ("f16", dict(B=40, gamma=8, T=3)),                                        # 320 tokens: 5 row blocks, paired with an empty sixth
+    ("f16", dict(T=1)),                                                       # a single denoising step
     ("f16", dict(B=121, gamma=4, T=2, cfg=False, cfg_scale=1.0,               # 484 tokens without guidance: ragged last block
                  draft=gen.HeadSpec(1, 1024, 128), target=gen.HeadSpec(3, 1024, 128))),
 ])
