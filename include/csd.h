@@ -135,7 +135,10 @@ int64_t csd_launch_count(const csd_ctx *ctx);
  *                       CTAs owns its output tiles for every layer and step, the residual stream stays in tensor
  *                       memory, the CTAs that share rows meet at a counter once per layer.  Draft and target chain
  *                       of csd_round then run side by side without competing for SMs.  Its buffers grow with T
- *                       (the condition vectors of all steps: T x rows x W 16-bit values).
+ *                       (the condition vectors of all steps: T x rows x W 16-bit values).  A chain that has the GPU
+ *                       to itself (csd_draft_denoise or csd_verify called alone) is about a tenth faster with
+ *                       CSD_CHAIN_LAYER_KERNELS, whose kernels spread over the idle SMs; the default is chosen
+ *                       per chain, not per call, so that csd_round and the three separate calls give the same bits.
  *                     - Otherwise one kernel per layer, chained with programmatic dependent launch; a layer's
  *                       independent part overlaps its predecessor on otherwise idle SMs.  For 16-bit heads on
  *                       grids of one wave, blocks 2..L run as two kernels instead of three: LayerNorm is folded
