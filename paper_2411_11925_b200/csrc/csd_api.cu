@@ -264,7 +264,8 @@ int ensure_ws(csd_ctx* ctx, ChainWs& ws, const csd_head_desc& d, int Rh, int R, 
 
 template <int EPI, int NSEG, int NMUL, int TN, typename ACT, bool PAIR>
 int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0, const CUtensorMap& a1,
-                const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k, int N, const EpiParams& ep) {
+                const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k, int N, const EpiParams& ep,
+                const CUtensorMap* tout = nullptr) {
   constexpr int MMA_N = NMUL * TN;
   auto kern = gemm_tc_kernel<EPI, ACT, NSEG, MMA_N, TN, std::is_same<ACT, __half>::value ? 0 : 1, PAIR>;
   static bool attr_done[kMaxDevices] = {};   // function attributes are per device
@@ -296,7 +297,7 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
   cfg.attrs = at; cfg.numAttrs = na;
   EpiParams e = ep;
   e.nt = N / kStatCols;   // eps partials are per 64-column group for both tile widths
-  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, tiles_n, units, e,
+  CSD_CUDA(ctx, cudaLaunchKernelEx(&cfg, kern, a0, b0, a1, b1, th, tout ? *tout : th, K0 / kBlockK, K1 / kBlockK, dep_k / kBlockK, tiles_n, units, e,
                                    ctx->d_err));
   ctx->launches++;
   return CSD_OK;
@@ -309,15 +310,15 @@ int launch_tc_t(csd_ctx* ctx, cudaStream_t st, const CUtensorMap& a0, const CUte
 template <int EPI, int NSEG, int NMUL>
 int launch_tc(csd_ctx* ctx, int dtype, int tn, bool pair, cudaStream_t st, const CUtensorMap& a0, const CUtensorMap& b0,
               const CUtensorMap& a1, const CUtensorMap& b1, const CUtensorMap& th, int K0, int K1, int dep_k,
-              int N, const EpiParams& ep) {
+              int N, const EpiParams& ep, const CUtensorMap* tout = nullptr) {
   if (dtype == CSD_F16) {
-    if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __half, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
-    if (pair) return launch_tc_t<EPI, NSEG, NMUL, 128, __half, true>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
-    return launch_tc_t<EPI, NSEG, NMUL, 128, __half, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+    if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __half, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep, tout);
+    if (pair) return launch_tc_t<EPI, NSEG, NMUL, 128, __half, true>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep, tout);
+    return launch_tc_t<EPI, NSEG, NMUL, 128, __half, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep, tout);
   }
-  if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __nv_bfloat16, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
-  if (pair) return launch_tc_t<EPI, NSEG, NMUL, 128, __nv_bfloat16, true>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
-  return launch_tc_t<EPI, NSEG, NMUL, 128, __nv_bfloat16, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep);
+  if (tn == 64) return launch_tc_t<EPI, NSEG, NMUL, 64, __nv_bfloat16, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep, tout);
+  if (pair) return launch_tc_t<EPI, NSEG, NMUL, 128, __nv_bfloat16, true>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep, tout);
+  return launch_tc_t<EPI, NSEG, NMUL, 128, __nv_bfloat16, false>(ctx, st, a0, b0, a1, b1, th, K0, K1, dep_k, N, ep, tout);
 }
 
 template <int EPI, int NSEG, int MMA_N>
@@ -783,8 +784,8 @@ struct Chain {
       // s of the first step is written by the kernel right before the first modulate kernel; every later s is older
       const int dep_mod = (k == 0 && t == T) ? 0 : W;
       if (folded_in) rc = CSD_OK;
-      else if (tc && mod64) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wss[k], tm_s, hd->tm[0].Wss[k], tm_h, W, 0, dep_mod, W, e);
-      else if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, dep_mod, W, e);
+      else if (tc && mod64) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, 64, false, st, tm_s, hd->tm[0].Wss[k], tm_s, hd->tm[0].Wss[k], tm_h, W, 0, dep_mod, W, e, &tm_u);
+      else if (tc) rc = launch_tc<EPI_MOD, 1, 2>(ctx, d.dtype, tn, pair, st, tm_s, tmw.Wss[k], tm_s, tmw.Wss[k], tm_h, W, 0, dep_mod, W, e, &tm_u);
       else rc = launch_simt<EPI_MOD, 1, 256>(ctx, st, sf, W, static_cast<const float*>(hd->Wss[k]), W, nullptr, 0,
                                              nullptr, 0, W, e);
       if (rc) return rc;
@@ -795,15 +796,15 @@ struct Chain {
         // CTA pairs over 256 x 256 tiles: per MMA byte the pair loads half as many operand bytes as with 256 x 128
         // tiles, and the first layer (one accumulator, K = W) is the kernel bound by that feed
         const CUtensorMap& w1 = hd->tm[1].W1[k];   // 128-row boxes: each CTA of the pair loads half of the 256 rows
-        rc = d.dtype == CSD_F16 ? launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __half, true>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e)
-                                : launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __nv_bfloat16, true>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e);
+        rc = d.dtype == CSD_F16 ? launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __half, true>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e, &tm_v)
+                                : launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __nv_bfloat16, true>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e, &tm_v);
       }
       else if (tc && w1_wide) {
         const CUtensorMap& w1 = hd->W1_wide[k];
-        rc = d.dtype == CSD_F16 ? launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __half, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e)
-                                : launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __nv_bfloat16, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e);
+        rc = d.dtype == CSD_F16 ? launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __half, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e, &tm_v)
+                                : launch_tc_t<EPI_SILU_ACT, 1, 1, 256, __nv_bfloat16, false>(ctx, st, tm_u, w1, tm_u, w1, tm_h, W, 0, 0, W, e, &tm_v);
       }
-      else if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 1>(ctx, d.dtype, tn, pair, st, tm_u, tmw.W1[k], tm_u, tmw.W1[k], tm_h, W, 0, 0, W, e);
+      else if (tc) rc = launch_tc<EPI_SILU_ACT, 1, 1>(ctx, d.dtype, tn, pair, st, tm_u, tmw.W1[k], tm_u, tmw.W1[k], tm_h, W, 0, 0, W, e, &tm_v);
       else rc = launch_simt<EPI_SILU_ACT, 1, 128>(ctx, st, uf, W, static_cast<const float*>(hd->W1[k]), W, nullptr, 0,
                                                   nullptr, 0, W, e);
       if (rc) return rc;

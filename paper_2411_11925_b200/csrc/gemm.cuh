@@ -43,9 +43,15 @@ template <int EPI, int MMA_N, int TN, bool PAIR> struct TcCfg {
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kHTileBytes = kTileM * TN * 4;        // fp32 h tile staged in shared memory
   static constexpr int kHBytes = kStageH ? kHTileBytes : 0;
-  static constexpr int kWoutBytes = kTileM * epi_out_width<EPI>() * 4;   // Wout^T tile [TN][16 or 32], reused for [128 rows][..] partials
-  static constexpr int kMiscBytes = 2 * TN * 4 + kTileM * 16;   // two bias slices + per-row exchange
-  static constexpr int kFixedBytes = 1024 + kHBytes + kWoutBytes + kMiscBytes + 256;
+  // 16-bit output tiles (SiLU and modulate epilogues) leave through shared memory and TMA stores: a thread owns a row,
+  // so direct stores touch 32 lines per instruction, and such bursts hold up the TMA loads of the next tile's
+  // mainloop.  The modulate epilogue reuses the h tile it has just read; the SiLU epilogue gets a buffer of its own.
+  static constexpr bool kStagedOut = EPI == EPI_SILU_ACT || EPI == EPI_MOD;
+  static constexpr int kOutBytes = EPI == EPI_SILU_ACT ? kTileM * TN * 2 : 0;
+  static constexpr int kWoutBytes = epi_is_modf<EPI>() ? kTileM * epi_out_width<EPI>() * 4 : 0;   // Wout^T tile [TN][16 or 32], reused for [128 rows][..] partials
+  static constexpr int kXchBytes = (EPI == EPI_GATE_RES || epi_is_modf<EPI>()) ? kTileM * 16 : 0;   // per-row exchange between column halves
+  static constexpr int kMiscBytes = 2 * TN * 4 + kXchBytes;     // two bias slices + exchange
+  static constexpr int kFixedBytes = 1024 + kHBytes + kOutBytes + kWoutBytes + kMiscBytes + 256;
   static constexpr int kStagesMax = (227 * 1024 - kFixedBytes) / kStageBytes;
   static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
   static constexpr int kSmemBytes = kFixedBytes + kStages * kStageBytes;
@@ -77,7 +83,8 @@ template <int EPI, typename ACT, int NSEG, int MMA_N, int TN, int AB_FMT, bool P
 __global__ void __launch_bounds__(TcWarps<EPI, TN>::kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
-               const __grid_constant__ CUtensorMap tmH, int nkb0, int nkb1, int dep_kb, int tiles_n, int tiles_total,
+               const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmOut, int nkb0, int nkb1, int dep_kb,
+               int tiles_n, int tiles_total,
                EpiParams ep, int* err) {
   using Cfg = TcCfg<EPI, MMA_N, TN, PAIR>;
   constexpr int S = Cfg::kStages;
@@ -93,10 +100,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stage_base = smem;
   uint8_t* h_s = smem + S * Cfg::kStageBytes;                    // NC chunks of [128 rows][128 B], swizzled
-  float* wout_s = reinterpret_cast<float*>(h_s + Cfg::kHBytes);
-  float* bias_s = reinterpret_cast<float*>(h_s + Cfg::kHBytes + Cfg::kWoutBytes);
+  uint8_t* out_s = h_s + Cfg::kHBytes;                           // SiLU epilogue: outgoing 16-bit tile, boxes of 64 columns
+  float* wout_s = reinterpret_cast<float*>(out_s + Cfg::kOutBytes);
+  float* bias_s = reinterpret_cast<float*>(out_s + Cfg::kOutBytes + Cfg::kWoutBytes);
   float* xch_s = bias_s + 2 * TN;                            // [128 rows][4] exchange between column halves
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(h_s + Cfg::kHBytes + Cfg::kWoutBytes + Cfg::kMiscBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(out_s + Cfg::kOutBytes + Cfg::kWoutBytes + Cfg::kMiscBytes);
   uint64_t* empty_bar = full_bar + S;
   uint64_t* tmem_full_bar = empty_bar + S;      // [2]
   uint64_t* tmem_empty_bar = tmem_full_bar + 2; // [2]
@@ -139,6 +147,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     tma_prefetch_desc(&tmB0);
     if (NSEG == 2) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
     if (Cfg::kStageH) tma_prefetch_desc(&tmH);
+    if (Cfg::kStagedOut) tma_prefetch_desc(&tmOut);
     for (int s = 0; s < S; ++s) { mbar_init(&full_bar[s], 2); mbar_init(&empty_bar[s], 1); }
     // a pair's accumulator buffer is released by the epilogues of both CTAs (to the leader's barrier)
     for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full_bar[i], 1); mbar_init(&tmem_empty_bar[i], PAIR ? 2 : 1); }
@@ -278,6 +287,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           if (PAIR) mbar_arrive_cluster(mapa_shared(smem_u32(&tmem_empty_bar[ab ^ 1]), 0));
           else mbar_arrive(&tmem_empty_bar[ab ^ 1]);
         }
+        if (Cfg::kStagedOut && i >= 1) {
+          // the previous tile's 16-bit output sits in shared memory (the modulate epilogue wrote it over the h tile)
+          const int tp = unit + (i - 1) * nunits;
+          const int pn = tp % tiles_n, pm = PAIR ? 2 * (tp / tiles_n) + rank : tp / tiles_n;
+#pragma unroll
+          for (int b = 0; b < TN / 64; ++b)
+            tma_store_2d(&tmOut, (EPI == EPI_MOD ? h_s + 2 * b * (kTileM * 128) : out_s + b * (kTileM * 128)), pn * TN + b * 64, pm * kTileM);
+          tma_store_commit();
+          tma_store_wait_read();   // before this tile's h lands on it / the epilogue writes the next tile
+        }
         if (EPI == EPI_GATE_RES && i >= 1) {
           // the previous tile's new h sits in the h tile (the threads that own its rows wrote it in place): TMA
           // stores instead of row-per-thread stores, which touch 32 rows per instruction
@@ -325,6 +344,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           if (EPI == EPI_GATE_RES) {
             gate_res_chunk(a0, a1, bias_s + c * kChunk, bias_s + TN + c * kChunk, hv, rs);
             store_swizzled_row32(h_s + c * (kTileM * 128), rloc, hv);   // in place; leaves by TMA store
+          } else if (Cfg::kStagedOut) {
+            if (EPI == EPI_SILU_ACT) {
+#pragma unroll
+              for (int j = 0; j < kChunk; ++j) a0[j] = silu_t<true>(a0[j] + bias_s[c * kChunk + j]);
+            } else
+              modulate_chunk(a0, a1, bias_s + c * kChunk, bias_s + TN + c * kChunk, hv, rs);
+            // 64 bytes of row rloc in box c / 2 (TMA's 128-byte swizzle); the modulate epilogue writes over the h it read
+            uint8_t* row = (EPI == EPI_MOD ? h_s + 2 * (c >> 1) * (kTileM * 128) : out_s + (c >> 1) * (kTileM * 128)) + rloc * 128;
+            __align__(16) ACT o[kChunk];
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) o[j] = to_act<ACT>(a0[j]);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              *reinterpret_cast<uint4*>(row + ((((c & 1) * 4 + u) ^ (rloc & 7)) << 4)) = reinterpret_cast<const uint4*>(o)[u];
           } else if (valid)
             epi_chunk<EPI, ACT, true>(ep, m, tile_n * TN + c * kChunk, a0, a1, bias_s + c * kChunk,
                                       bias_s + TN + c * kChunk, hv, rs, wout_s + c * kChunk * EPW);
@@ -333,7 +366,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             for (int e = 0; e < EPW; ++e) rs.eacc[e] = efirst[e] + rs.eacc[e];
           }
         }
-        if (EPI == EPI_GATE_RES) fence_proxy_async_smem();
+        if (EPI == EPI_GATE_RES || Cfg::kStagedOut) fence_proxy_async_smem();
         tc_fence_before_sync();   // orders the TMEM reads before the barrier that releases the buffer
       }
       if (EPI == EPI_GATE_RES) {
@@ -369,6 +402,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           }
         }
       }
+    }
+    if (Cfg::kStagedOut) {
+      // the last tile's output
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+      if (et == 0 && ok) {
+        const int tp = unit + (my_tiles - 1) * nunits;
+        const int pn = tp % tiles_n, pm = PAIR ? 2 * (tp / tiles_n) + rank : tp / tiles_n;
+#pragma unroll
+        for (int b = 0; b < TN / 64; ++b)
+          tma_store_2d(&tmOut, (EPI == EPI_MOD ? h_s + 2 * b * (kTileM * 128) : out_s + b * (kTileM * 128)), pn * TN + b * 64, pm * kTileM);
+        tma_store_commit();
+      }
+      if (et == 0) tma_store_wait_all();
     }
     if (EPI == EPI_GATE_RES) {
       // the last tile's new h
