@@ -514,6 +514,8 @@ def run_ours(args):
         if ch and ch["persistent_chain_kernel"] and wl.operand_format != "f32":
             # the dominant kernel of the timed region is the target chain's persistent kernel: one launch per csd_verify
             # call, timed by events around the call on the library's stream (the other kernels of the call take microseconds)
+            nb0 = -(-wl.R // (64 if wl.cfg else 128))
+            ctas = 8 * (nb0 + (nb0 & 1))            # one CTA per 128 x 128 tile of a layer, row blocks paired
             fl = wl.Rh * wl.T * wl.target.flops_per_row_step()
             ach = fl / (ch["verify_ms"] * 1e-3) / 1e12
             line["roofline"] = {"bound": "tensor", "kernel": "pchain_kernel (target chain, one launch per call)",
@@ -522,8 +524,8 @@ def run_ours(args):
                                 "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, "pchain_target")),
                                 "peak_source": f"{peaks['source']} bf16 sustained (fp16 has the same nominal rate)",
                                 "avg_launch_us": 1e3 * ch["verify_ms"], "flops_per_launch": fl,
-                                "sms_used": "64 of 148 (the draft chain's kernel runs beside it on 64 others)",
-                                "frac_of_the_peak_of_the_sms_used": ach / (peaks["tflops_sustained"] * 64.0 / 148.0),
+                                "sms_used": f"{ctas} of 148 (the draft chain's kernel runs beside it on others)",
+                                "frac_of_the_peak_of_the_sms_used": ach / (peaks["tflops_sustained"] * ctas / 148.0),
                                 "draft_chain": {"avg_launch_us": 1e3 * ch["draft_ms"],
                                                 "achieved": wl.Rh * wl.T * wl.draft.flops_per_row_step() / (ch["draft_ms"] * 1e-3) / 1e12}}
             line["chains"] = ch
