@@ -525,7 +525,6 @@ def run_ours(args):
                                 "peak_source": f"{peaks['source']} bf16 sustained (fp16 has the same nominal rate)",
                                 "avg_launch_us": 1e3 * ch["verify_ms"], "flops_per_launch": fl,
                                 "sms_used": f"{ctas} of 148 (the draft chain's kernel runs beside it on others)",
-                                "frac_of_the_peak_of_the_sms_used": ach / (peaks["tflops_sustained"] * ctas / 148.0),
                                 "draft_chain": {"avg_launch_us": 1e3 * ch["draft_ms"],
                                                 "achieved": wl.Rh * wl.T * wl.draft.flops_per_row_step() / (ch["draft_ms"] * 1e-3) / 1e12}}
             line["chains"] = ch
